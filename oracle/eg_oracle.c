@@ -1,0 +1,397 @@
+/*
+ * CPU oracle for the EventGraD per-iteration communication step.
+ *
+ * TEST INFRASTRUCTURE ONLY.  Plain, slow, step-by-step restatement of the method of
+ * "EventGraD: Event-Triggered Communication in Parallel Machine Learning"
+ * (Algorithm B, the trigger condition of Section 4, Eq. (dist_sgd_event), Eq. (thres),
+ * the history-averaged slope of Section 7 and the Top-K paragraph of Section 7).
+ * It shares no code with the CUDA library and must never be reachable from it.
+ *
+ * State is stored in fp32 exactly as the method stores it; every arithmetic step is
+ * fp64 unless stated.  Build with -ffp-contract=off so that no multiply-add is fused
+ * except where fma() is written out.
+ *
+ * Data layout: packed, x[i*N + off[t] + e] is element e of tensor t of replica (PE) i,
+ * off[t] = numel[0] + ... + numel[t-1], N = sum of numel.
+ *
+ * Pins (tests/test_oracle_pins.py): threshold 0 == regular D-PSGD X W - gamma G
+ * (Section 5 remark after Corollary 1; Eq. (dist_sgd_neigh)); infinite threshold == no
+ * messages and independent SGD; doubly-stochastic W preserves the replica mean and the
+ * ring's circulant eigen-modes decay as ((1+2cos(2 pi m/P))/3)^s (Section 3, Assumption
+ * 2.2); error bound ||x_hat - x|| < delta (Section 5); forced event at k = 0 (Section 4);
+ * a hand-worked threshold sequence from Eq. (thres) with and without history
+ * (tests/golden/threshold_sequence.txt); Top-K against a brute-force sort, K = n == dense,
+ * payload = 2K percent (Section 7).
+ * Parity unpinned: the paper prints no worked numeric trigger sequence, so the readings
+ * listed below are pinned by consistency with its equations, not by printed values.
+ *
+ * Readings where the paper is silent (kept in one place so they can be checked by eye):
+ *  - the tested quantity is the L2 norm of the element-wise difference x - x_hat
+ *    (the displayed trigger condition), not the difference of norms;
+ *  - inside one iteration: test current x, then communicate, then average + SGD, and a
+ *    message is visible to the neighbours in the same iteration (the only order for
+ *    which threshold 0 gives exactly Eq. (dist_sgd_neigh));
+ *  - the replica's own term in the average is its current x; neighbours contribute the
+ *    last value they sent;
+ *  - the first event of a tensor has no previous event, hence no slope: the threshold
+ *    stays at delta_init until the second event;
+ *  - history of H slopes: slope of an event = its norm / iterations since the previous
+ *    event; threshold = horizon * mean of the slopes kept (H = 1 is Eq. (thres));
+ *  - a mailbox that never received anything is left out of the average and the weight is
+ *    1/(1 + number of neighbours heard from); with the forced first event this never
+ *    happens and the weight is 1/3 on a ring;
+ *  - Top-K ranks by |x - x_hat| (fp32 difference), sends the parameter values x[e] with
+ *    their indices, ties go to the lower index, the message is in ascending index order,
+ *    K_t = max(1, ceil(n_t * k_num / k_den)); the first message of a tensor is dense.
+ */
+#include <float.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#if FLT_EVAL_METHOD != 0
+#error "the oracle needs float expressions evaluated in float (FLT_EVAL_METHOD == 0)"
+#endif
+
+#define EGO_ADAPTIVE 0
+#define EGO_FIXED 1
+
+typedef struct {
+    uint32_t key;
+    int32_t idx;
+} ego_keyidx;
+
+typedef struct ego_ctx {
+    int P, T;
+    int64_t N;
+    int64_t *numel, *off;
+    int mode;
+    double horizon;
+    int H;
+    double delta_init, delta_fixed;
+    int force_first;
+    int topk;
+    uint32_t k_num, k_den;
+    int64_t *Kt;      /* [T] */
+    int64_t *out_off; /* [T+1] prefix of Kt */
+    int64_t k;        /* iteration counter */
+    float *xhat;      /* [P][N] last communicated values */
+    double *delta;    /* [P*T] current threshold */
+    int64_t *khat;    /* [P*T] iteration of the last event */
+    double *hist;     /* [P*T][H] slopes, oldest first */
+    int *hist_len;    /* [P*T] */
+    uint8_t *valid;   /* [P*T] something has been sent */
+    uint8_t *flag;    /* [P*T] decisions of the last step */
+    double *norm;     /* [P*T] ||x - x_hat|| seen by the last step */
+    double *thr_used; /* [P*T] threshold the last step compared against */
+    int32_t *out_idx; /* [P][sum Kt] */
+    float *out_val;
+    int32_t *out_count; /* [P*T] entries of the last step's sparse message, 0 if none */
+    uint64_t *seg_events;
+    uint64_t *seg_payload; /* scratch: payload bytes of this step's event, 0 if none */
+    uint64_t messages, bytes, events;
+    int threads;
+} ego_ctx;
+
+void ego_destroy(ego_ctx *c) {
+    if (!c) return;
+    free(c->numel); free(c->off); free(c->Kt); free(c->out_off); free(c->xhat);
+    free(c->delta); free(c->khat); free(c->hist); free(c->hist_len); free(c->valid);
+    free(c->flag); free(c->norm); free(c->thr_used); free(c->out_idx); free(c->out_val);
+    free(c->out_count); free(c->seg_events); free(c->seg_payload);
+    free(c);
+}
+
+void ego_reset(ego_ctx *c) {
+    int64_t S = (int64_t)c->P * c->T;
+    c->k = 0;
+    c->messages = c->bytes = c->events = 0;
+    memset(c->xhat, 0, sizeof(float) * (size_t)c->P * (size_t)c->N); /* X_0 = 0, Assumption 2.4 */
+    for (int64_t s = 0; s < S; ++s) {
+        c->delta[s] = (c->mode == EGO_FIXED) ? c->delta_fixed : c->delta_init;
+        c->khat[s] = 0;
+        c->hist_len[s] = 0;
+        c->valid[s] = 0;
+        c->flag[s] = 0;
+        c->norm[s] = 0.0;
+        c->thr_used[s] = c->delta[s];
+        c->out_count[s] = 0;
+        c->seg_events[s] = 0;
+    }
+    memset(c->hist, 0, sizeof(double) * (size_t)S * (size_t)c->H);
+}
+
+/* Number of elements of the sparse message of a tensor with n elements. */
+static int64_t topk_count(int64_t n, uint32_t k_num, uint32_t k_den) {
+    /* ceil(n*k_num/k_den) in integers, at least 1, at most n */
+    uint64_t prod = (uint64_t)n * (uint64_t)k_num;
+    uint64_t q = (prod + (uint64_t)k_den - 1u) / (uint64_t)k_den;
+    if (q < 1) q = 1;
+    if (q > (uint64_t)n) q = (uint64_t)n;
+    return (int64_t)q;
+}
+
+ego_ctx *ego_create(int P, int T, const int64_t *numel, int mode, double horizon, int H,
+                    double delta_init, double delta_fixed, int force_first, int topk,
+                    uint32_t k_num, uint32_t k_den) {
+    if (P < 1 || T < 1 || H < 1 || (topk && (k_den == 0 || k_num == 0))) return NULL;
+    ego_ctx *c = (ego_ctx *)calloc(1, sizeof(ego_ctx));
+    if (!c) return NULL;
+    c->P = P; c->T = T; c->mode = mode; c->horizon = horizon; c->H = H;
+    c->delta_init = delta_init; c->delta_fixed = delta_fixed; c->force_first = force_first;
+    c->topk = topk; c->k_num = k_num; c->k_den = k_den; c->threads = 1;
+    c->numel = (int64_t *)malloc(sizeof(int64_t) * T);
+    c->off = (int64_t *)malloc(sizeof(int64_t) * T);
+    c->Kt = (int64_t *)malloc(sizeof(int64_t) * T);
+    c->out_off = (int64_t *)malloc(sizeof(int64_t) * (T + 1));
+    int64_t N = 0, KS = 0;
+    for (int t = 0; t < T; ++t) {
+        if (numel[t] < 1) { ego_destroy(c); return NULL; }
+        c->numel[t] = numel[t];
+        c->off[t] = N;
+        N += numel[t];
+        c->Kt[t] = topk ? topk_count(numel[t], k_num, k_den) : 0;
+        c->out_off[t] = KS;
+        KS += c->Kt[t];
+    }
+    c->out_off[T] = KS;
+    c->N = N;
+    int64_t S = (int64_t)P * T;
+    c->xhat = (float *)malloc(sizeof(float) * (size_t)P * (size_t)N);
+    c->delta = (double *)malloc(sizeof(double) * S);
+    c->khat = (int64_t *)malloc(sizeof(int64_t) * S);
+    c->hist = (double *)malloc(sizeof(double) * S * H);
+    c->hist_len = (int *)malloc(sizeof(int) * S);
+    c->valid = (uint8_t *)malloc(S);
+    c->flag = (uint8_t *)malloc(S);
+    c->norm = (double *)malloc(sizeof(double) * S);
+    c->thr_used = (double *)malloc(sizeof(double) * S);
+    c->out_idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(P * (KS > 0 ? KS : 1)));
+    c->out_val = (float *)malloc(sizeof(float) * (size_t)(P * (KS > 0 ? KS : 1)));
+    c->out_count = (int32_t *)malloc(sizeof(int32_t) * S);
+    c->seg_events = (uint64_t *)malloc(sizeof(uint64_t) * S);
+    c->seg_payload = (uint64_t *)malloc(sizeof(uint64_t) * S);
+    ego_reset(c);
+    return c;
+}
+
+void ego_set_threads(ego_ctx *c, int threads) { c->threads = threads < 1 ? 1 : threads; }
+
+int ego_threads_available(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+static uint32_t f32_bits(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return u;
+}
+
+/* order of the Top-K ranking: larger |delta| first, then lower index */
+static int cmp_rank(const void *a, const void *b) {
+    const ego_keyidx *p = (const ego_keyidx *)a, *q = (const ego_keyidx *)b;
+    if (p->key != q->key) return (p->key > q->key) ? -1 : 1;
+    if (p->idx != q->idx) return (p->idx < q->idx) ? -1 : 1;
+    return 0;
+}
+
+static int cmp_idx(const void *a, const void *b) {
+    const ego_keyidx *p = (const ego_keyidx *)a, *q = (const ego_keyidx *)b;
+    return (p->idx < q->idx) ? -1 : (p->idx > q->idx);
+}
+
+/* Number of distinct ring neighbours of replica i and their ids (left first). */
+static int ring_neighbours(int P, int i, int nbr[2]) {
+    if (P <= 1) return 0;
+    int left = (i - 1 + P) % P, right = (i + 1) % P;
+    nbr[0] = left;
+    if (right == left) return 1;
+    nbr[1] = right;
+    return 2;
+}
+
+/* Phase A for one (replica i, tensor t): norm of the change, trigger test, threshold
+ * update, communication into the mailbox x_hat (Algorithm B inner loop; trigger
+ * condition of Section 4; Eq. (thres); history paragraph and Top-K paragraph of
+ * Section 7). */
+static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
+    const int64_t s = (int64_t)i * c->T + t;
+    const int64_t n = c->numel[t];
+    const float *xs = x + (int64_t)i * c->N + c->off[t];
+    float *hs = c->xhat + (int64_t)i * c->N + c->off[t];
+
+    /* 1-2: d = || x - x_hat ||_2 with fp32 differences, exact fp64 squares, fp64 sum */
+    double acc = 0.0;
+    for (int64_t e = 0; e < n; ++e) {
+        const float d32 = xs[e] - hs[e]; /* one fp32 subtraction (FLT_EVAL_METHOD 0) */
+        double dd = (double)d32;
+        acc = acc + dd * dd;
+    }
+    const double d = sqrt(acc);
+    const double thr = c->delta[s];
+    c->norm[s] = d;
+    c->thr_used[s] = thr;
+
+    /* 3: the event test; the first event is forced at k = 0 (Section 4) */
+    const int fire = (c->force_first && c->k == 0) || (d >= thr);
+    c->flag[s] = (uint8_t)fire;
+    c->out_count[s] = 0;
+    c->seg_payload[s] = 0;
+    if (!fire) return;
+
+    /* 4a: new threshold from the slope between this event and the previous one */
+    if (c->mode == EGO_ADAPTIVE && c->valid[s]) {
+        const double slope = d / (double)(c->k - c->khat[s]);
+        double *h = c->hist + s * c->H;
+        if (c->hist_len[s] == c->H) {
+            for (int q = 1; q < c->H; ++q) h[q - 1] = h[q];
+            c->hist_len[s] = c->H - 1;
+        }
+        h[c->hist_len[s]++] = slope;
+        double sum = 0.0;
+        for (int q = 0; q < c->hist_len[s]; ++q) sum = sum + h[q];
+        c->delta[s] = c->horizon * (sum / (double)c->hist_len[s]);
+    }
+
+    /* 4b: the message */
+    uint64_t payload;
+    if (!c->topk || !c->valid[s]) {
+        for (int64_t e = 0; e < n; ++e) hs[e] = xs[e];
+        payload = 4u * (uint64_t)n;
+    } else {
+        const int64_t K = c->Kt[t];
+        ego_keyidx *r = (ego_keyidx *)malloc(sizeof(ego_keyidx) * (size_t)n);
+        for (int64_t e = 0; e < n; ++e) {
+            const float d32 = xs[e] - hs[e];
+            r[e].key = f32_bits(d32) & 0x7FFFFFFFu; /* bits of |delta| order like |delta| */
+            r[e].idx = (int32_t)e;
+        }
+        qsort(r, (size_t)n, sizeof(ego_keyidx), cmp_rank);
+        qsort(r, (size_t)K, sizeof(ego_keyidx), cmp_idx);
+        int32_t *oi = c->out_idx + (int64_t)i * c->out_off[c->T] + c->out_off[t];
+        float *ov = c->out_val + (int64_t)i * c->out_off[c->T] + c->out_off[t];
+        for (int64_t q = 0; q < K; ++q) { /* pack (index, value) */
+            oi[q] = r[q].idx;
+            ov[q] = xs[r[q].idx];
+        }
+        for (int64_t q = 0; q < K; ++q) hs[oi[q]] = ov[q]; /* scatter on receipt */
+        c->out_count[s] = (int32_t)K;
+        payload = 8u * (uint64_t)K;
+        free(r);
+    }
+    c->seg_payload[s] = payload;
+
+    /* 4c: bookkeeping */
+    c->khat[s] = c->k;
+    c->valid[s] = 1;
+    c->seg_events[s] += 1;
+}
+
+/* Phase B for one (replica i, tensor t): average with the neighbours' last received
+ * values and apply the gradient (Eq. (dist_sgd_event) with W_ij = 1/(N_i + 1)). */
+static void phase_b_segment(ego_ctx *c, float *x, const float *g, float lr, int i, int t) {
+    int nbr[2];
+    const int deg = ring_neighbours(c->P, i, nbr);
+    const float *hn[2];
+    int cnt = 0;
+    for (int q = 0; q < deg; ++q)
+        if (c->valid[(int64_t)nbr[q] * c->T + t])
+            hn[cnt++] = c->xhat + (int64_t)nbr[q] * c->N + c->off[t];
+    const double w = 1.0 / (double)(1 + cnt);
+    float *xs = x + (int64_t)i * c->N + c->off[t];
+    const float *gs = g + (int64_t)i * c->N + c->off[t];
+    const double neg_lr = -(double)lr;
+    for (int64_t e = 0; e < c->numel[t]; ++e) {
+        double sum = (double)xs[e];
+        for (int q = 0; q < cnt; ++q) sum = sum + (double)hn[q][e];
+        const double avg = sum * w;
+        const double r = fma(neg_lr, (double)gs[e], avg);
+        xs[e] = (float)r;
+    }
+}
+
+/* One iteration of Algorithm B for all replicas.  x is updated in place. */
+void ego_step(ego_ctx *c, float *x, const float *g, float lr) {
+    const int64_t S = (int64_t)c->P * c->T;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) num_threads(c->threads)
+#endif
+    for (int64_t s = 0; s < S; ++s) phase_a_segment(c, x, (int)(s / c->T), (int)(s % c->T));
+
+    /* message accounting: one message per (event, neighbour) */
+    for (int64_t s = 0; s < S; ++s) {
+        if (!c->flag[s]) continue;
+        int nbr[2];
+        const uint64_t deg = (uint64_t)ring_neighbours(c->P, (int)(s / c->T), nbr);
+        c->events += 1;
+        c->messages += deg;
+        c->bytes += deg * c->seg_payload[s];
+    }
+
+    /* every mailbox is final before anybody averages */
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) num_threads(c->threads)
+#endif
+    for (int64_t s = 0; s < S; ++s)
+        phase_b_segment(c, x, g, lr, (int)(s / c->T), (int)(s % c->T));
+
+    c->k += 1;
+}
+
+/* ---- readers ---------------------------------------------------------------------- */
+void ego_stats(const ego_ctx *c, uint64_t *messages, uint64_t *bytes, uint64_t *events) {
+    if (messages) *messages = c->messages;
+    if (bytes) *bytes = c->bytes;
+    if (events) *events = c->events;
+}
+int64_t ego_iteration(const ego_ctx *c) { return c->k; }
+int64_t ego_total_numel(const ego_ctx *c) { return c->N; }
+const uint8_t *ego_flags(const ego_ctx *c) { return c->flag; }
+const double *ego_norms(const ego_ctx *c) { return c->norm; }
+const double *ego_thresholds_used(const ego_ctx *c) { return c->thr_used; }
+const double *ego_thresholds(const ego_ctx *c) { return c->delta; }
+const uint8_t *ego_valid(const ego_ctx *c) { return c->valid; }
+const int64_t *ego_last_event_iteration(const ego_ctx *c) { return c->khat; }
+const uint64_t *ego_segment_events(const ego_ctx *c) { return c->seg_events; }
+float *ego_xhat(ego_ctx *c) { return c->xhat; }
+int64_t ego_topk_count(const ego_ctx *c, int t) { return c->Kt[t]; }
+int32_t ego_outbox(const ego_ctx *c, int i, int t, const int32_t **idx, const float **val) {
+    const int64_t o = (int64_t)i * c->out_off[c->T] + c->out_off[t];
+    *idx = c->out_idx + o;
+    *val = c->out_val + o;
+    return c->out_count[(int64_t)i * c->T + t];
+}
+
+/* Model obtained after training by averaging all replicas (last line of Algorithms A and
+ * B): out[e] = (1/P) sum_i x_i[e], fp64 sum in ascending i, rounded once to fp32. */
+void ego_average_model(const ego_ctx *c, const float *x, float *out) {
+    for (int64_t e = 0; e < c->N; ++e) {
+        double s = 0.0;
+        for (int i = 0; i < c->P; ++i) s = s + (double)x[(int64_t)i * c->N + e];
+        out[e] = (float)(s / (double)c->P);
+    }
+}
+
+/* Consensus distance sum_i || x_i - mean ||^2 (the quantity bounded by Lemma 2 of the
+ * appendix), fp64 throughout, mean unrounded. */
+double ego_consensus_distance(const ego_ctx *c, const float *x) {
+    double total = 0.0;
+    for (int64_t e = 0; e < c->N; ++e) {
+        double s = 0.0;
+        for (int i = 0; i < c->P; ++i) s = s + (double)x[(int64_t)i * c->N + e];
+        const double m = s / (double)c->P;
+        for (int i = 0; i < c->P; ++i) {
+            const double d = (double)x[(int64_t)i * c->N + e] - m;
+            total = total + d * d;
+        }
+    }
+    return total;
+}

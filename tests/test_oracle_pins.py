@@ -1,0 +1,388 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests re-types the oracle's own loop: each compares it with a closed form, a
+dense matrix product, a brute-force sort, an invariant, or a sequence worked by hand and
+stored under tests/golden/.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import eg_oracle as eo
+from paper_2103_07454_b200 import workload as W
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+INF = float("inf")
+
+
+def ring_matrix(P):
+    """Mixing matrix of Section 3: W_ij = 1/(N_i + 1) over the PE itself and its distinct
+    ring neighbours."""
+    Wm = np.zeros((P, P))
+    for i in range(P):
+        nb = {i, (i - 1) % P, (i + 1) % P}
+        for j in nb:
+            Wm[i, j] = 1.0 / len(nb)
+    return Wm
+
+
+def ulp32(a):
+    return np.spacing(np.abs(a).astype(np.float32)).astype(np.float64)
+
+
+def small(P=5, numel=(7, 1, 33, 128, 5), **kw):
+    return W.synthetic(P, numel, **kw)
+
+
+# ---------------------------------------------------------------------------------------
+# delta = 0  ==  regular D-PSGD,  X_{k+1} = X_k W - gamma G   (Eq. (dist_sgd_neigh); remark
+# after Corollary 1: "a threshold of 0 reduces to the regular algorithm")
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 7])
+def test_zero_threshold_is_dpsgd(P):
+    wl = small(P=P, steps=6, lr=0.1, grad_sigma=0.01)
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=0.0, force_first_event=False)
+    x = W.distinct_init_params(wl).numpy().copy()
+    Wm = ring_matrix(P)
+    deg = 0 if P == 1 else (1 if P == 2 else 2)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        ref = Wm @ x.astype(np.float64) - np.float64(np.float32(wl.lr)) * g.astype(np.float64)
+        o.step(x, g, wl.lr)
+        assert o.flags().all()
+        assert np.all(np.abs(x.astype(np.float64) - ref) <= 0.5000001 * ulp32(ref) + 1e-300)
+        st = o.stats()
+        assert st["messages"] == P * wl.T * deg * (k + 1)
+        assert st["bytes"] == 4 * wl.N * P * deg * (k + 1)
+        assert st["events"] == P * wl.T * (k + 1)
+
+
+# ---------------------------------------------------------------------------------------
+# delta = infinity: no messages, every replica runs plain SGD on its own
+# ---------------------------------------------------------------------------------------
+def test_infinite_threshold_is_independent_sgd():
+    wl = small(P=4, steps=5, lr=0.25, grad_sigma=0.02)
+    o = eo.Oracle(4, wl.numel, mode=eo.FIXED, delta_fixed=INF, force_first_event=False)
+    x0 = W.distinct_init_params(wl).numpy().copy()
+    x = x0.copy()
+    ref = x0.astype(np.float64)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        o.step(x, g, wl.lr)
+        ref = (ref - np.float64(np.float32(wl.lr)) * g.astype(np.float64)).astype(np.float32).astype(np.float64)
+        assert not o.flags().any()
+        assert np.all(np.abs(x - ref) <= ulp32(ref))
+    assert o.stats() == {"messages": 0, "bytes": 0, "events": 0}
+    assert not o.valid().any()
+    assert np.all(o.xhat() == 0)
+
+
+def test_only_forced_event_then_frozen_mailboxes():
+    """With an infinite threshold but the forced event at k = 0 (Section 4), neighbours keep
+    averaging with the value received at k = 0 ("the last received version") while the own
+    term follows the replica's current parameters."""
+    P = 5
+    wl = small(P=P, steps=4, lr=0.1, grad_sigma=0.05)
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=INF, force_first_event=True)
+    x0 = W.distinct_init_params(wl).numpy().copy()
+    x = x0.copy()
+    frozen = x0.astype(np.float64)
+    ref = x0.astype(np.float64)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        o.step(x, g, wl.lr)
+        assert o.flags().all() == (k == 0) and o.flags().any() == (k == 0)
+        left, right = np.roll(frozen, 1, axis=0), np.roll(frozen, -1, axis=0)
+        ref = (ref + left + right) / 3.0 - np.float64(np.float32(wl.lr)) * g.astype(np.float64)
+        ref = ref.astype(np.float32).astype(np.float64)
+        assert np.all(np.abs(x - ref) <= ulp32(ref))
+    assert np.array_equal(o.xhat(), x0)
+    assert o.stats()["messages"] == P * wl.T * 2
+
+
+# ---------------------------------------------------------------------------------------
+# W doubly stochastic: replica mean preserved; circulant eigen-modes of the ring
+# ---------------------------------------------------------------------------------------
+def test_mean_preserved_with_zero_gradients():
+    P = 6
+    wl = small(P=P, steps=25)
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=0.0)
+    x = W.distinct_init_params(wl).numpy().copy()
+    mean0 = x.astype(np.float64).mean(axis=0)
+    g = np.zeros_like(x)
+    d_prev = o.consensus_distance(x)
+    for _ in range(wl.steps):
+        o.step(x, g, 0.1)
+        mean = x.astype(np.float64).mean(axis=0)
+        assert np.all(np.abs(mean - mean0) <= 4 * wl.steps * ulp32(np.abs(x).max(axis=0)))
+        d = o.consensus_distance(x)
+        assert d < d_prev  # contraction towards the mean on a connected ring
+        d_prev = d
+    assert d_prev < 1e-6 * o.consensus_distance(W.distinct_init_params(wl).numpy())
+
+
+@pytest.mark.parametrize("P,m", [(4, 1), (5, 1), (5, 2), (8, 3), (16, 1)])
+def test_ring_eigenmode_decay(P, m):
+    """The ring W is circulant with eigenvalues (1 + 2 cos(2 pi m / P)) / 3 (all of modulus
+    < 1 for m != 0: the spectral-gap assumption); a cosine mode decays geometrically."""
+    n = 4
+    steps = 12
+    o = eo.Oracle(P, [n], mode=eo.FIXED, delta_fixed=0.0)
+    mode = np.cos(2 * np.pi * m * np.arange(P) / P)
+    amp = np.array([1.0, -2.5, 0.125, 3.0])
+    x = (mode[:, None] * amp[None, :]).astype(np.float32)
+    x_init = x.astype(np.float64)
+    lam = (1 + 2 * math.cos(2 * math.pi * m / P)) / 3
+    g = np.zeros_like(x)
+    for s in range(1, steps + 1):
+        o.step(x, g, 0.3)
+        ref = lam ** s * x_init
+        assert np.all(np.abs(x - ref) <= 2e-7 * np.abs(amp)[None, :] * s + 1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# forced first event, error bound, accounting
+# ---------------------------------------------------------------------------------------
+def seg_norms(a, b, numel):
+    """||a - b|| per (replica, tensor) with fp32 differences, computed by numpy."""
+    P = a.shape[0]
+    out = np.zeros((P, len(numel)))
+    off = 0
+    for t, n in enumerate(numel):
+        d = (a[:, off:off + n] - b[:, off:off + n]).astype(np.float32).astype(np.float64)
+        out[:, t] = np.sqrt((d * d).sum(axis=1))
+        off += n
+    return out
+
+
+@pytest.mark.parametrize("hist", [1, 3])
+def test_error_bound_and_forced_first_event(hist):
+    P = 4
+    wl = small(P=P, steps=30, lr=0.1, grad_sigma=0.01, history_len=hist)
+    o = eo.from_workload(wl)
+    x = W.distinct_init_params(wl).numpy().copy()
+    total_events = 0
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        x_pre = x.copy()
+        xhat_pre = o.xhat()
+        o.step(x, g, wl.lr)
+        f = o.flags().astype(bool)
+        if k == 0:
+            assert f.all()                      # forced event at k = 0
+            assert np.all(o.thresholds_used() == 0.0)
+        d_np = seg_norms(x_pre, xhat_pre, wl.numel)
+        assert np.allclose(o.norms(), d_np, rtol=1e-13, atol=0)
+        # the decision is the displayed inequality
+        if k > 0:
+            differs = f != (d_np >= o.thresholds_used())
+            assert np.all(np.abs(d_np - o.thresholds_used())[differs] <= 1e-12 * d_np[differs])
+        # error bound of Section 5: after communicating, ||x_hat - x|| is 0 for the tensors
+        # sent and stays below the threshold for the others
+        e_post = seg_norms(x_pre, o.xhat(), wl.numel)
+        assert np.all(e_post[f] == 0.0)
+        assert np.all(e_post[~f] < o.thresholds_used()[~f])
+        total_events += int(f.sum())
+        assert np.array_equal(o.last_event_iteration()[f], np.full(f.sum(), k))
+    st = o.stats()
+    assert st["events"] == total_events
+    assert st["messages"] == 2 * total_events
+    assert 0 < total_events < P * wl.T * wl.steps  # some, not all: the trigger does select
+    assert o.segment_events().sum() == total_events
+
+
+@pytest.mark.parametrize("P,deg", [(1, 0), (2, 1), (3, 2)])
+def test_message_accounting_and_neighbour_dedup(P, deg):
+    numel = [3, 10]
+    o = eo.Oracle(P, numel, mode=eo.FIXED, delta_fixed=0.0)
+    x = np.arange(P * 13, dtype=np.float32).reshape(P, 13) / 8
+    x0 = x.astype(np.float64)
+    o.step(x, np.zeros_like(x), 0.0)
+    st = o.stats()
+    assert st["events"] == 2 * P and st["messages"] == 2 * P * deg
+    assert st["bytes"] == deg * P * 4 * 13
+    assert np.allclose(x, ring_matrix(P) @ x0, rtol=0, atol=1e-6)
+
+
+# ---------------------------------------------------------------------------------------
+# adaptive threshold: hand-worked sequences
+# ---------------------------------------------------------------------------------------
+def load_threshold_cases():
+    cases, cur = [], None
+    with open(os.path.join(GOLDEN, "threshold_sequence.txt")) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            if line.startswith("case"):
+                _, name, H, h = line.split()
+                cur = {"name": name, "H": int(H[2:]), "h": float(h[2:]), "rows": []}
+                cases.append(cur)
+            else:
+                cur["rows"].append([float(v) for v in line.split()])
+    return cases
+
+
+@pytest.mark.parametrize("case", load_threshold_cases(), ids=lambda c: c["name"])
+def test_hand_worked_threshold_sequence(case):
+    rows = case["rows"]
+    o = eo.Oracle(1, [2], horizon=case["h"], history_len=case["H"], delta_init=0.0)
+    x = np.array([[rows[0][1], rows[0][2]]], dtype=np.float32)
+    for r, row in enumerate(rows):
+        k, x0, x1, flag, d, thr_tested, thr_after = row
+        assert o.iteration == int(k)
+        assert x[0, 0] == x0 and x[0, 1] == x1
+        nxt = rows[r + 1] if r + 1 < len(rows) else row
+        g = np.array([[x0 - nxt[1], x1 - nxt[2]]], dtype=np.float32)
+        o.step(x, g, 1.0)
+        assert int(o.flags()[0, 0]) == int(flag), f"k={k}"
+        assert o.norms()[0, 0] == pytest.approx(d, rel=1e-15, abs=0)
+        assert o.thresholds_used()[0, 0] == pytest.approx(thr_tested, rel=1e-15, abs=0)
+        assert o.thresholds()[0, 0] == pytest.approx(thr_after, rel=1e-15, abs=0)
+
+
+def test_fixed_threshold_never_adapts():
+    o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=2.0, force_first_event=False)
+    x = np.zeros((1, 2), np.float32)
+    fired = []
+    for k in range(6):
+        o.step(x, np.array([[-0.6, -0.8]], np.float32), 1.0)  # |x| grows by 1 per step
+        fired.append(int(o.flags()[0, 0]))
+        assert o.thresholds()[0, 0] == 2.0
+    # x_k = k*(0.6,0.8): k=0,1 below 2; k=2 fires (d~2, x_hat<-x_2); k=3 d~1; k=4 fires; ...
+    assert fired[:2] == [0, 0] and sum(fired) >= 1
+
+
+# ---------------------------------------------------------------------------------------
+# Top-K
+# ---------------------------------------------------------------------------------------
+def brute_force_topk(x_row, xhat_row, K):
+    d = (x_row - xhat_row).astype(np.float32)
+    key = np.abs(d).view(np.uint32).astype(np.int64)
+    order = np.lexsort((np.arange(len(d)), -key))  # key descending, index ascending
+    return np.sort(order[:K]).astype(np.int32)
+
+
+@pytest.mark.parametrize("frac", [(1, 100), (10, 100), (1, 3), (1, 1)])
+def test_topk_against_brute_force(frac):
+    P = 3
+    numel = [1, 2, 17, 100, 1000, 4097]
+    wl = W.synthetic(P, numel, steps=24, lr=0.1, grad_sigma=0.01, topk=frac)
+    o = eo.from_workload(wl)
+    x = W.distinct_init_params(wl).numpy().copy()
+    rng = np.random.default_rng(5)
+    sparse_seen = 0
+    bytes_expected = 0
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy().copy()
+        # engineered ties: quantise some gradients so many |delta| coincide, and zero some
+        g[:, 1200:1600] = np.round(g[:, 1200:1600] * 64) / 64
+        g[:, 3000:3100] = 0.0
+        x_pre = x.copy()
+        xhat_pre = o.xhat()
+        valid_pre = o.valid().astype(bool)
+        o.step(x, g, wl.lr)
+        f = o.flags().astype(bool)
+        xhat_post = o.xhat()
+        off = 0
+        for t, n in enumerate(numel):
+            K = max(1, -(-n * frac[0] // frac[1]))
+            assert o.topk_count(t) == K
+            for i in range(P):
+                idx, val = o.outbox(i, t)
+                seg_pre = xhat_pre[i, off:off + n]
+                seg_post = xhat_post[i, off:off + n]
+                if f[i, t] and valid_pre[i, t]:
+                    want = brute_force_topk(x_pre[i, off:off + n], seg_pre, K)
+                    assert np.array_equal(idx, want)
+                    assert np.array_equal(val, x_pre[i, off:off + n][want])
+                    expect = seg_pre.copy()
+                    expect[want] = x_pre[i, off:off + n][want]
+                    assert np.array_equal(seg_post, expect)
+                    sparse_seen += 1
+                    bytes_expected += 2 * 8 * K          # "2K percent" of a dense message
+                elif f[i, t]:
+                    assert len(idx) == 0                    # first message of a tensor is dense
+                    assert np.array_equal(seg_post, x_pre[i, off:off + n])
+                    bytes_expected += 2 * 4 * n
+                else:
+                    assert len(idx) == 0
+                    assert np.array_equal(seg_post, seg_pre)
+            off += n
+    assert sparse_seen > 12
+    assert o.stats()["bytes"] == bytes_expected
+
+
+def test_topk_tie_break_prefers_lower_index():
+    o = eo.Oracle(1, [8], mode=eo.FIXED, delta_fixed=0.0, topk=(3, 8))
+    x = np.zeros((1, 8), np.float32)
+    z = np.zeros_like(x)
+    o.step(x, z, 0.0)                                   # first message: dense
+    x[0] = [1, -2, 2, 0.5, -2, 2, -0.0, 1]              # |delta| = 1 2 2 .5 2 2 0 1
+    o.step(x, z, 0.0)
+    idx, val = o.outbox(0, 0)
+    assert idx.tolist() == [1, 2, 4]                    # four ties at 2: lowest three indices
+    assert val.tolist() == [-2.0, 2.0, -2.0]
+    assert o.xhat()[0].tolist() == [0, -2, 2, 0, -2, 0, 0, 0]
+
+
+def test_topk_with_k_equal_n_is_dense():
+    P = 4
+    wl_d = small(P=P, steps=15, lr=0.1, grad_sigma=0.01)
+    wl_s = small(P=P, steps=15, lr=0.1, grad_sigma=0.01, topk=(1, 1))
+    od, os_ = eo.from_workload(wl_d), eo.from_workload(wl_s)
+    xd = W.distinct_init_params(wl_d).numpy().copy()
+    xs = xd.copy()
+    for k in range(wl_d.steps):
+        g = wl_d.grads(k).numpy()
+        od.step(xd, g, wl_d.lr)
+        os_.step(xs, g, wl_s.lr)
+        assert np.array_equal(od.flags(), os_.flags())
+        assert np.array_equal(xd, xs)
+        assert np.array_equal(od.xhat(), os_.xhat())
+    sd, ss = od.stats(), os_.stats()
+    assert sd["messages"] == ss["messages"]
+    first = 2 * 4 * wl_d.N * P                         # the dense first messages
+    assert ss["bytes"] - first == 2 * (sd["bytes"] - first)  # index + value: twice the size
+
+
+def test_topk_counts_of_the_resnet18_tensors():
+    o = eo.Oracle(1, [10, 64, 1728, 2359296], topk=(1, 100))
+    assert [o.topk_count(t) for t in range(4)] == [1, 1, 18, 23593]
+    o = eo.Oracle(1, [10, 64, 1728, 2359296], topk=(10, 100))
+    assert [o.topk_count(t) for t in range(4)] == [1, 7, 173, 235930]
+
+
+# ---------------------------------------------------------------------------------------
+# after training: averaged model (last line of Algorithms A and B)
+# ---------------------------------------------------------------------------------------
+def test_average_model_and_consensus_distance():
+    wl = small(P=5)
+    o = eo.from_workload(wl)
+    x = W.distinct_init_params(wl).numpy()
+    x64 = x.astype(np.float64)
+    mean = x64.mean(axis=0)
+    assert np.all(np.abs(o.average_model(x) - mean) <= ulp32(mean))
+    assert o.consensus_distance(x) == pytest.approx(((x64 - mean) ** 2).sum(), rel=1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# the input generator (shared by both sides): tensor form == pure-Python definition
+# ---------------------------------------------------------------------------------------
+def test_generator_matches_python_definition():
+    base = W.stream_base(W.MASTER_SEED, W.STREAM_GRAD, 3, 1)
+    t = W.ih8_integers(base, 5, 50, "cpu").tolist()
+    assert t == [W.ih8_integers_py(base, e) for e in range(5, 55)]
+    z = W.ih8_integers(base, 0, 200000, "cpu").double()
+    assert abs(z.mean().item()) < 4 * W.IH8_STD / math.sqrt(200000)
+    assert z.std().item() == pytest.approx(W.IH8_STD, rel=0.01)
+
+
+def test_workload_sizes():
+    sizes = {1: (4, 6, 52650), 2: (8, 59, 269722), 3: (16, 62, 11173962),
+             4: (8, 62, 11173962), 5: (64, 161, 25557032)}
+    for idx, (P, T, N) in sizes.items():
+        for wl in W.config(idx):
+            assert (wl.P, wl.T, wl.N) == (P, T, N)
