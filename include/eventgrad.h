@@ -1,0 +1,171 @@
+/*
+ * eventgrad.h — C ABI of the B200 (sm_100a) library for EventGraD's per-iteration
+ * event-triggered communication step.
+ *
+ * One context simulates a ring of P data-parallel replicas ("PEs" in the paper) that all
+ * live in one GPU's memory.  One eg_step is one pass of the inner part of Algorithm B of
+ * "EventGraD: Event-Triggered Communication in Parallel Machine Learning":
+ *   for every replica i and every layer tensor I ("parameter" in the paper):
+ *     d = || x - x_hat ||_2                         (trigger condition, Section 4)
+ *     event  <=>  d >= delta  (or k == 0, forced)   (Section 4; Fig. 1 discussion)
+ *     on an event: delta = horizon * mean of the last H slopes d / (k - k_hat)
+ *                                                    (Eq. (thres); history: Section 7)
+ *                  x_hat <- x   (dense message, the one-sided put into the neighbours'
+ *                  windows of Section 6) or, with Top-K, the K_t entries of largest
+ *                  |x - x_hat| packed as (index, value) and scattered into x_hat on
+ *                  receipt (Top-K paragraph of Section 7)
+ *   then  x_i <- w * (x_i + sum over ring neighbours j of x_hat_j) - lr * g_i,
+ *         w = 1/(N_i + 1) = 1/3 on a ring            (Eq. (dist_sgd_event), Section 3)
+ *
+ * Conventions
+ *  - All pointers named params / grads / *_dev are DEVICE pointers owned by the caller.
+ *    Pointers named *_host (and all out-parameters of eg_stats, eg_layout,
+ *    eg_last_decisions, eg_last_outbox, eg_export_state) are HOST pointers owned by the
+ *    caller.  The context owns everything else and frees it in eg_destroy.
+ *  - Parameter layout: fp32, [P][replica_stride]; tensor t of replica i starts at element
+ *    i*replica_stride + tensor_offset[t].  The library chooses the offsets (each tensor
+ *    starts on a 128-byte boundary; read them with eg_layout).  Padding elements between
+ *    tensors are never written and their content is ignored.
+ *  - params and grads must be 16-byte aligned device allocations of at least
+ *    P*replica_stride floats.
+ *  - eg_step only enqueues work on `stream` (a cudaStream_t passed as void*; NULL is the
+ *    legacy default stream).  It never synchronises and never copies to the host.  The
+ *    calls that read results back (eg_stats, eg_last_*, eg_export_state, eg_step_host)
+ *    synchronise that stream.
+ *  - One context belongs to one device (the one current at eg_create) and is used from one
+ *    stream at a time.
+ *  - Every function returns an eg_status; nothing throws, aborts or traps.  A device-side
+ *    problem (an index outside its table) sets an error word that the next synchronising
+ *    call returns as EG_ERR_INTERNAL.
+ *  - Counters: an event of tensor t at replica i adds deg(i) to messages_sent (deg = number
+ *    of distinct ring neighbours: 2, or 1 for P = 2, or 0 for P = 1) and deg(i)*payload to
+ *    bytes_sent; payload = 4*n_t for a dense message, 8*K_t for a Top-K message
+ *    ("2K percent", Section 7).  The paper's "percentage of messages" (Table 1) is
+ *    messages_sent / (P * T * 2 * steps).
+ */
+#ifndef EVENTGRAD_H
+#define EVENTGRAD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct eg_ctx eg_ctx; /* opaque */
+
+typedef enum {
+    EG_OK = 0,
+    EG_ERR_INVALID = 1,  /* bad argument */
+    EG_ERR_OOM = 2,      /* host or device allocation failed */
+    EG_ERR_CUDA = 3,     /* a CUDA runtime call failed; see eg_last_cuda_error */
+    EG_ERR_STATE = 4,    /* call not allowed in the context's current state */
+    EG_ERR_TIMEOUT = 5,  /* reserved */
+    EG_ERR_INTERNAL = 6  /* device-side consistency check failed */
+} eg_status;
+
+enum { EG_TOPO_RING = 0 }; /* the topology the paper fixes (Section 3) */
+enum { EG_THRESH_ADAPTIVE = 0, /* Eq. (thres) with a history of H slopes */
+       EG_THRESH_FIXED = 1 };  /* one static threshold for all tensors (Section 4 calls it
+                                  the simplest option); 0 gives regular D-PSGD, +inf none */
+
+typedef struct {
+    int mode;              /* EG_THRESH_ADAPTIVE or EG_THRESH_FIXED */
+    double horizon;        /* h of Eq. (thres); the paper's experiments use 1 */
+    int history_len;       /* H >= 1 slopes averaged; 1 is Eq. (thres) literally */
+    double delta_init;     /* threshold in force until the second event of a tensor */
+    double delta_fixed;    /* the threshold of EG_THRESH_FIXED */
+    int force_first_event; /* 1: every tensor communicates at k = 0 (Section 4) */
+} eg_threshold_params;
+
+typedef struct {
+    int enabled;           /* 0: dense messages */
+    uint32_t k_num, k_den; /* K_t = max(1, ceil(n_t * k_num / k_den)) entries per message;
+                              the first message of every tensor is dense */
+} eg_topk_params;
+
+/* Creates a context on the current device for P replicas of T tensors with layer_numel[t]
+ * elements each (host array).  topk may be NULL (dense).  Allocates the mailboxes x_hat
+ * (zero: X_0 = 0 of Assumption 2), the per-(replica, tensor) trigger state, scratch for the
+ * norm partial sums, the Top-K outboxes and the counters.  *out is NULL on failure. */
+eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_numel, int T,
+                    const eg_threshold_params* thr, const eg_topk_params* topk);
+
+/* Layout chosen by the library: tensor_offset_host[T] (elements, within one replica) and
+ * *replica_stride_host (elements).  Either pointer may be NULL. */
+eg_status eg_layout(const eg_ctx* ctx, int64_t* tensor_offset_host, int64_t* replica_stride_host);
+
+/* One iteration of Algorithm B (see the top of this file) on `stream`.  params (device,
+ * [P][replica_stride] fp32) is updated in place; grads has the same layout and is only read.
+ * Errors: EG_ERR_INVALID for NULL or misaligned pointers, EG_ERR_CUDA if a launch fails. */
+eg_status eg_step(eg_ctx* ctx, float* params, const float* grads, float lr, void* stream);
+
+/* Same iteration for callers whose data lives in HOST memory: copies params_host and
+ * grads_host ([P][replica_stride] fp32, ideally pinned) to device staging buffers owned by
+ * the context (allocated on first use), runs eg_step, copies the updated parameters back
+ * and synchronises. */
+eg_status eg_step_host(eg_ctx* ctx, float* params_host, const float* grads_host, float lr);
+
+/* Carried-norm mode (off by default).  When on, the fused average/update kernel of step k
+ * also accumulates || x_{k+1} - x_hat ||^2 of every tensor, so step k+1 skips its separate
+ * norm pass (16 instead of 24 bytes of memory traffic per element).  Only valid while the
+ * caller leaves params untouched between consecutive eg_step calls on the same buffer;
+ * turning it on, eg_reset and eg_import_state make the next step recompute the norms. */
+eg_status eg_set_carry_norm(eg_ctx* ctx, int enabled);
+
+/* Totals since creation / eg_reset (Table 1 and Table 2 report ratios of these).
+ * Synchronises.  Pointers may be NULL. */
+eg_status eg_stats(eg_ctx* ctx, uint64_t* messages_sent_host, uint64_t* bytes_sent_host);
+eg_status eg_event_count(eg_ctx* ctx, uint64_t* events_host);
+
+/* Decisions of the most recent step, host arrays of P*T entries indexed [i*T + t]:
+ * flags (1 = event), norms (d), thresholds (the delta that d was compared with).
+ * Any pointer may be NULL.  Synchronises. */
+eg_status eg_last_decisions(eg_ctx* ctx, uint8_t* flags_host, double* norms_host,
+                            double* thresholds_host);
+
+/* Threshold in force after the most recent step and number of events so far, per
+ * (replica, tensor); host arrays of P*T entries.  Synchronises. */
+eg_status eg_thresholds(eg_ctx* ctx, double* delta_host, uint64_t* events_host);
+
+/* The Top-K message replica i sent for tensor t in the most recent step: *count_host entries
+ * (0 if it sent none or sent a dense message), ascending indices in idx_host and the
+ * parameter values in val_host (capacity: eg_topk_count(t) entries each). */
+eg_status eg_last_outbox(eg_ctx* ctx, int i, int t, int32_t* idx_host, float* val_host,
+                         int32_t* count_host);
+eg_status eg_topk_count(const eg_ctx* ctx, int t, int64_t* k_t_host);
+
+/* Copies the mailboxes x_hat ([P][replica_stride] fp32) into a host buffer. Synchronises. */
+eg_status eg_read_mailboxes(eg_ctx* ctx, float* xhat_host);
+
+/* After training: the model averaged over all replicas ("Obtain averaged model from all
+ * PEs", last line of Algorithms A and B): avg_dev[e] = (1/P) sum_i params[i][e] for every
+ * element of the replica layout (device buffer of replica_stride floats), fp64 sum in
+ * ascending i, rounded once.  consensus_host, if not NULL, receives
+ * sum_i || x_i - mean ||^2 (the consensus distance bounded in the appendix) and makes the
+ * call synchronise. */
+eg_status eg_average_model(eg_ctx* ctx, const float* params, float* avg_dev,
+                           double* consensus_host, void* stream);
+
+/* Checkpoint: eg_export_state with host_buf == NULL stores the needed size in *bytes;
+ * otherwise writes the state (iteration counter, counters, trigger state, mailboxes) and
+ * the size.  eg_import_state restores it into a context created with the same arguments
+ * (EG_ERR_INVALID otherwise). */
+eg_status eg_export_state(eg_ctx* ctx, void* host_buf, size_t* bytes);
+eg_status eg_import_state(eg_ctx* ctx, const void* host_buf, size_t bytes);
+
+/* Back to iteration 0 with empty mailboxes, initial thresholds and zero counters. */
+eg_status eg_reset(eg_ctx* ctx);
+void eg_destroy(eg_ctx* ctx);
+
+const char* eg_strerror(eg_status s);
+/* cudaError_t of the most recent failed CUDA call of this context (0 if none). */
+int eg_last_cuda_error(const eg_ctx* ctx);
+/* Kernels launched by the most recent eg_step of this context. */
+int eg_last_launch_count(const eg_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EVENTGRAD_H */

@@ -361,6 +361,8 @@ const double *ego_thresholds(const ego_ctx *c) { return c->delta; }
 const uint8_t *ego_valid(const ego_ctx *c) { return c->valid; }
 const int64_t *ego_last_event_iteration(const ego_ctx *c) { return c->khat; }
 const uint64_t *ego_segment_events(const ego_ctx *c) { return c->seg_events; }
+const double *ego_history(const ego_ctx *c) { return c->hist; }
+const int *ego_history_len(const ego_ctx *c) { return c->hist_len; }
 float *ego_xhat(ego_ctx *c) { return c->xhat; }
 int64_t ego_topk_count(const ego_ctx *c, int t) { return c->Kt[t]; }
 int32_t ego_outbox(const ego_ctx *c, int i, int t, const int32_t **idx, const float **val) {

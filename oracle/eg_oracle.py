@@ -50,7 +50,8 @@ def _load():
         lib.ego_iteration.restype = C.c_int64
         lib.ego_iteration.argtypes = [C.c_void_p]
         for name in ("ego_flags", "ego_norms", "ego_thresholds_used", "ego_thresholds",
-                     "ego_valid", "ego_last_event_iteration", "ego_segment_events", "ego_xhat"):
+                     "ego_valid", "ego_last_event_iteration", "ego_segment_events", "ego_xhat",
+                     "ego_history", "ego_history_len"):
             getattr(lib, name).restype = C.c_void_p
             getattr(lib, name).argtypes = [C.c_void_p]
         lib.ego_topk_count.restype = C.c_int64
@@ -98,6 +99,7 @@ class Oracle:
             raise ValueError("ego_create rejected the arguments")
         lib.ego_set_threads(self._h, int(threads))
         self.S = self.P * self.T
+        self.history_len = int(history_len)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -152,6 +154,13 @@ class Oracle:
 
     def segment_events(self):
         return self._seg("ego_segment_events", np.uint64)
+
+    def history(self):
+        """(slopes [P, T, H] oldest first, number of slopes kept [P, T])."""
+        H = self.history_len
+        h = _view(self._lib.ego_history(self._h), np.float64, self.S * H).reshape(
+            self.P, self.T, H).copy()
+        return h, self._seg("ego_history_len", np.int32)
 
     def xhat(self) -> np.ndarray:
         """Copy of the mailboxes (last communicated values), packed ``[P, N]``."""

@@ -1,0 +1,69 @@
+// Shared device-side declarations of the EventGraD step library (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace eg {
+
+constexpr int kThreads = 256;          // threads per CTA in every streaming kernel
+constexpr int kWarps = kThreads / 32;
+constexpr int kNormTile = 4096;        // elements per CTA of the norm / Top-K kernels
+constexpr int kMaxReplicas = 1024;     // P limit (shared-memory tables are sized by P)
+constexpr int kMaxHistory = 64;
+
+// Top-K radix select: the 31-bit key bits(|x - x_hat|) is resolved in three digits.
+constexpr int kDigitBits0 = 11, kDigitBits1 = 10, kDigitBits2 = 10;
+constexpr int kMaxBins = 1 << kDigitBits0;
+
+// Tile table: a tile is a run of at most `tile` consecutive elements of one tensor.
+struct TileTable {
+    const int* tensor;           // [n_tiles] tensor id
+    const long long* offset;     // [n_tiles] element offset inside one replica
+    const int* length;           // [n_tiles] elements in the tile
+    const int* seg_begin;        // [T+1] first tile of every tensor
+    int n_tiles;
+};
+
+// Per-(replica, tensor) trigger state and the decisions of the current step, all [P*T].
+struct SegState {
+    double* delta;               // threshold in force
+    long long* khat;             // iteration of the last event
+    double* hist;                // [P*T][H] slopes, oldest first
+    int* hist_len;
+    uint8_t* valid;              // the tensor has been sent at least once
+    uint8_t* flag;               // event in this step
+    uint8_t* snap;               // event whose message is dense (x_hat <- x in the fused kernel)
+    uint8_t* sparse;             // event whose message is a Top-K message
+    double* norm;                // d of this step
+    double* thr_used;            // delta that d was compared with
+    unsigned long long* events;  // events so far
+};
+
+struct Counters {                // device-resident, 64-bit
+    unsigned long long messages, bytes, events, pad;
+};
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+    return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st_stream(float* p, float4 v) {
+    __stcs(reinterpret_cast<float4*>(p), v);
+}
+
+// Sum over the CTA in a fixed order (lane tree, then warps in ascending order); the result
+// is valid in thread 0.
+__device__ __forceinline__ double block_sum(double v, double* s_warp) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_down_sync(0xffffffffu, v, o));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) s_warp[warp] = v;
+    __syncthreads();
+    double r = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) r = __dadd_rn(r, s_warp[w]);
+    }
+    return r;
+}
+
+}  // namespace eg

@@ -1,0 +1,130 @@
+// Segmented change-norm and the device-side trigger decision.
+//
+// k_norm_partial: || x - x_hat ||^2 of every (replica, tensor), as one fp64 partial sum per
+//                 tile (trigger condition of Section 4: the tested quantity).
+// k_decide:       sums the partials of a segment in a fixed order, takes the square root,
+//                 tests it against the threshold and, on an event, recomputes the threshold
+//                 from the slope history (Eq. (thres); history: Section 7) — all on device.
+#pragma once
+#include "eg_common.cuh"
+
+namespace eg {
+
+__device__ __forceinline__ double sq_diff4(float4 a, float4 b, int nel, double acc) {
+    // fp32 difference, exact fp64 square, fp64 accumulation (a product of two fp32 values
+    // is exact in fp64, so the fused multiply-add rounds exactly like multiply-then-add)
+    const float d0 = __fsub_rn(a.x, b.x), d1 = __fsub_rn(a.y, b.y);
+    const float d2 = __fsub_rn(a.z, b.z), d3 = __fsub_rn(a.w, b.w);
+    if (nel > 0) acc = __fma_rn((double)d0, (double)d0, acc);
+    if (nel > 1) acc = __fma_rn((double)d1, (double)d1, acc);
+    if (nel > 2) acc = __fma_rn((double)d2, (double)d2, acc);
+    if (nel > 3) acc = __fma_rn((double)d3, (double)d3, acc);
+    return acc;
+}
+
+// grid (n_tiles, P).  partials[i * n_tiles + tile].
+__global__ void __launch_bounds__(kThreads)
+k_norm_partial(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt,
+               long long stride, double* __restrict__ partials) {
+    __shared__ double s_warp[kWarps];
+    const int tile = blockIdx.x, i = blockIdx.y;
+    const int len = tt.length[tile];
+    const long long base = (long long)i * stride + tt.offset[tile];
+    constexpr int kIter = kNormTile / (kThreads * 4);
+    float4 a[kIter], b[kIter];
+    int nel[kIter];
+#pragma unroll
+    for (int q = 0; q < kIter; ++q) {
+        const int local = (q * kThreads + threadIdx.x) * 4;
+        nel[q] = min(4, max(0, len - local));
+        if (nel[q] > 0) {
+            a[q] = ld_stream(x + base + local);
+            b[q] = ld_stream(xhat + base + local);
+        } else {
+            a[q] = b[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+    double acc = 0.0;
+#pragma unroll
+    for (int q = 0; q < kIter; ++q) acc = sq_diff4(a[q], b[q], nel[q], acc);
+    const double total = block_sum(acc, s_warp);
+    if (threadIdx.x == 0) partials[(long long)i * tt.n_tiles + tile] = total;
+}
+
+struct DecideParams {
+    int P, T, H;
+    int mode;                 // 0 adaptive, 1 fixed
+    double horizon;
+    int force_first;
+    int topk;                 // Top-K messages enabled
+    int degree;               // distinct ring neighbours of every replica
+};
+
+// One warp per (replica, tensor).  grid ceil(P*T / kWarps).
+__global__ void __launch_bounds__(kThreads)
+k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin, int n_tiles,
+         DecideParams dp, SegState st, const long long* __restrict__ numel,
+         const long long* __restrict__ topk_count, int* __restrict__ outbox_count,
+         Counters* ctr, const long long* __restrict__ step_k) {
+    const int lane = threadIdx.x & 31;
+    const long long s = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (s >= (long long)dp.P * dp.T) return;
+    const int i = (int)(s / dp.T), t = (int)(s % dp.T);
+    const int q0 = seg_begin[t], q1 = seg_begin[t + 1];
+    const double* p = partials + (long long)i * n_tiles;
+    double acc = 0.0;
+    for (int q = q0 + lane; q < q1; q += 32) acc = __dadd_rn(acc, p[q]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc = __dadd_rn(acc, __shfl_down_sync(0xffffffffu, acc, o));
+    if (lane != 0) return;
+
+    const long long k = *step_k;
+    const double d = __dsqrt_rn(acc);
+    const double thr = st.delta[s];
+    st.norm[s] = d;
+    st.thr_used[s] = thr;
+    const bool fire = (dp.force_first && k == 0) || (d >= thr);
+    const bool was_valid = st.valid[s] != 0;
+    uint8_t snap = 0, sparse = 0;
+    int out_count = 0;
+    if (fire) {
+        if (dp.mode == 0 && was_valid) {
+            // slope between this event and the previous one, pushed into the history
+            const double slope = __ddiv_rn(d, (double)(k - st.khat[s]));
+            double* h = st.hist + s * dp.H;
+            int n = st.hist_len[s];
+            if (n == dp.H) {
+                for (int q = 1; q < dp.H; ++q) h[q - 1] = h[q];
+                n = dp.H - 1;
+            }
+            h[n++] = slope;
+            st.hist_len[s] = n;
+            double sum = 0.0;
+            for (int q = 0; q < n; ++q) sum = __dadd_rn(sum, h[q]);
+            st.delta[s] = __dmul_rn(dp.horizon, __ddiv_rn(sum, (double)n));
+        }
+        unsigned long long payload;
+        if (!dp.topk || !was_valid) {   // the first message of a tensor is always dense
+            snap = 1;
+            payload = 4ull * (unsigned long long)numel[t];
+        } else {
+            sparse = 1;
+            out_count = (int)topk_count[t];
+            payload = 8ull * (unsigned long long)topk_count[t];
+        }
+        st.khat[s] = k;
+        st.valid[s] = 1;
+        st.events[s] += 1ull;
+        atomicAdd(&ctr->events, 1ull);
+        if (dp.degree > 0) {
+            atomicAdd(&ctr->messages, (unsigned long long)dp.degree);
+            atomicAdd(&ctr->bytes, (unsigned long long)dp.degree * payload);
+        }
+    }
+    st.flag[s] = fire ? 1 : 0;
+    st.snap[s] = snap;
+    st.sparse[s] = sparse;
+    if (outbox_count) outbox_count[s] = out_count;
+}
+
+}  // namespace eg

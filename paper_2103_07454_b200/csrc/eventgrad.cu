@@ -1,0 +1,629 @@
+// Host side of the C ABI declared in include/eventgrad.h: context, layout, tile tables,
+// stream-ordered launches.  No decision of the step is taken on the host.
+#include "../../include/eventgrad.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "eg_common.cuh"
+#include "eg_fused.cuh"
+#include "eg_norm.cuh"
+#include "eg_topk.cuh"
+
+using namespace eg;
+
+namespace {
+
+constexpr int kFusedVpt = EG_FUSED_VPT;               // float4 columns per thread
+constexpr int kFusedTile = kThreads * 4 * kFusedVpt;  // elements per CTA of the fused kernel
+constexpr uint64_t kStateMagic = 0x4547535441544531ull;  // "EGSTATE1"
+
+struct HostTiles {
+    std::vector<int> tensor, length, seg_begin;
+    std::vector<long long> offset;
+};
+
+struct DeviceTiles {
+    int *tensor = nullptr, *length = nullptr, *seg_begin = nullptr;
+    long long* offset = nullptr;
+    int n_tiles = 0;
+    TileTable view() const { return TileTable{tensor, offset, length, seg_begin, n_tiles}; }
+};
+
+}  // namespace
+
+struct eg_ctx {
+    int device = 0;
+    int P = 0, T = 0, H = 1;
+    eg_threshold_params thr{};
+    eg_topk_params topk{};
+    std::vector<int64_t> numel, offset, kcount, out_off;
+    int64_t stride = 0, n_total = 0, out_stride = 0;
+    int degree = 0;
+    DeviceTiles tiles_norm, tiles_fused;
+    // device state
+    float* xhat = nullptr;
+    double *partials_norm = nullptr, *partials_fused = nullptr;
+    SegState st{};
+    Counters* ctr = nullptr;
+    long long* step_k = nullptr;
+    unsigned int* err = nullptr;
+    long long *d_numel = nullptr, *d_kcount = nullptr, *d_out_off = nullptr;
+    int* outbox_count = nullptr;
+    TopkState tk{};
+    double* cons_partials = nullptr;
+    // host staging for eg_step_host
+    float *stage_x = nullptr, *stage_g = nullptr;
+    // bookkeeping
+    std::vector<void*> allocs;
+    bool carry = false, carried_valid = false;
+    const float* carried_params = nullptr;
+    cudaStream_t last_stream = nullptr;
+    int last_cuda_error = 0;
+    int last_launches = 0;
+    size_t fused_smem = 0;
+};
+
+namespace {
+
+#define EG_CUDA(ctx, call)                                   \
+    do {                                                     \
+        cudaError_t e_ = (call);                             \
+        if (e_ != cudaSuccess) {                             \
+            (ctx)->last_cuda_error = (int)e_;                \
+            return e_ == cudaErrorMemoryAllocation ? EG_ERR_OOM : EG_ERR_CUDA; \
+        }                                                    \
+    } while (0)
+
+template <typename Tp>
+eg_status dev_alloc(eg_ctx* c, Tp** out, size_t count, bool zero = true) {
+    void* p = nullptr;
+    const size_t bytes = (count ? count : 1) * sizeof(Tp);
+    EG_CUDA(c, cudaMalloc(&p, bytes));
+    c->allocs.push_back(p);
+    if (zero) EG_CUDA(c, cudaMemset(p, 0, bytes));
+    *out = static_cast<Tp*>(p);
+    return EG_OK;
+}
+
+template <typename Tp>
+eg_status upload(eg_ctx* c, Tp** out, const std::vector<Tp>& v) {
+    eg_status s = dev_alloc(c, out, v.size(), false);
+    if (s != EG_OK) return s;
+    if (!v.empty()) EG_CUDA(c, cudaMemcpy(*out, v.data(), v.size() * sizeof(Tp), cudaMemcpyHostToDevice));
+    return EG_OK;
+}
+
+HostTiles build_tiles(const std::vector<int64_t>& numel, const std::vector<int64_t>& offset, int tile) {
+    HostTiles h;
+    for (size_t t = 0; t < numel.size(); ++t) {
+        h.seg_begin.push_back((int)h.tensor.size());
+        for (int64_t b = 0; b < numel[t]; b += tile) {
+            h.tensor.push_back((int)t);
+            h.offset.push_back((long long)(offset[t] + b));
+            h.length.push_back((int)std::min<int64_t>(tile, numel[t] - b));
+        }
+    }
+    h.seg_begin.push_back((int)h.tensor.size());
+    return h;
+}
+
+eg_status upload_tiles(eg_ctx* c, const HostTiles& h, DeviceTiles* d) {
+    eg_status s;
+    if ((s = upload(c, &d->tensor, h.tensor)) != EG_OK) return s;
+    if ((s = upload(c, &d->length, h.length)) != EG_OK) return s;
+    if ((s = upload(c, &d->seg_begin, h.seg_begin)) != EG_OK) return s;
+    if ((s = upload(c, &d->offset, h.offset)) != EG_OK) return s;
+    d->n_tiles = (int)h.tensor.size();
+    return EG_OK;
+}
+
+int64_t topk_entries(int64_t n, uint32_t num, uint32_t den) {
+    const unsigned long long prod = (unsigned long long)n * num;
+    unsigned long long q = (prod + den - 1ull) / den;
+    if (q < 1) q = 1;
+    if (q > (unsigned long long)n) q = (unsigned long long)n;
+    return (int64_t)q;
+}
+
+eg_status init_state(eg_ctx* c) {
+    const size_t S = (size_t)c->P * c->T;
+    std::vector<double> delta(S, c->thr.mode == EG_THRESH_FIXED ? c->thr.delta_fixed : c->thr.delta_init);
+    EG_CUDA(c, cudaMemcpy(c->st.delta, delta.data(), S * sizeof(double), cudaMemcpyHostToDevice));
+    EG_CUDA(c, cudaMemcpy(c->st.thr_used, delta.data(), S * sizeof(double), cudaMemcpyHostToDevice));
+    EG_CUDA(c, cudaMemset(c->st.khat, 0, S * sizeof(long long)));
+    EG_CUDA(c, cudaMemset(c->st.hist, 0, S * c->H * sizeof(double)));
+    EG_CUDA(c, cudaMemset(c->st.hist_len, 0, S * sizeof(int)));
+    EG_CUDA(c, cudaMemset(c->st.valid, 0, S));
+    EG_CUDA(c, cudaMemset(c->st.flag, 0, S));
+    EG_CUDA(c, cudaMemset(c->st.snap, 0, S));
+    EG_CUDA(c, cudaMemset(c->st.sparse, 0, S));
+    EG_CUDA(c, cudaMemset(c->st.norm, 0, S * sizeof(double)));
+    EG_CUDA(c, cudaMemset(c->st.events, 0, S * sizeof(unsigned long long)));
+    EG_CUDA(c, cudaMemset(c->ctr, 0, sizeof(Counters)));
+    EG_CUDA(c, cudaMemset(c->step_k, 0, sizeof(long long)));
+    EG_CUDA(c, cudaMemset(c->err, 0, sizeof(unsigned int)));
+    EG_CUDA(c, cudaMemset(c->outbox_count, 0, S * sizeof(int)));
+    EG_CUDA(c, cudaMemset(c->xhat, 0, (size_t)c->P * c->stride * sizeof(float)));
+    if (c->topk.enabled) {
+        EG_CUDA(c, cudaMemset(c->tk.hist, 0, S * kMaxBins * sizeof(unsigned int)));
+        EG_CUDA(c, cudaMemset(c->tk.prefix, 0, S * sizeof(unsigned int)));
+        EG_CUDA(c, cudaMemset(c->tk.remaining, 0, S * sizeof(unsigned int)));
+    }
+    c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status sync_and_check(eg_ctx* c) {
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    unsigned int e = 0;
+    EG_CUDA(c, cudaMemcpy(&e, c->err, sizeof(e), cudaMemcpyDeviceToHost));
+    return e ? EG_ERR_INTERNAL : EG_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* eg_strerror(eg_status s) {
+    switch (s) {
+        case EG_OK: return "ok";
+        case EG_ERR_INVALID: return "invalid argument";
+        case EG_ERR_OOM: return "out of memory";
+        case EG_ERR_CUDA: return "CUDA runtime error";
+        case EG_ERR_STATE: return "call not allowed in this state";
+        case EG_ERR_TIMEOUT: return "timeout";
+        case EG_ERR_INTERNAL: return "device-side consistency check failed";
+    }
+    return "unknown status";
+}
+
+int eg_last_cuda_error(const eg_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+int eg_last_launch_count(const eg_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+void eg_destroy(eg_ctx* c) {
+    if (!c) return;
+    {
+        DeviceGuard guard(c->device);
+        cudaDeviceSynchronize();
+        for (void* p : c->allocs) cudaFree(p);
+    }
+    delete c;
+}
+
+eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_numel, int T,
+                    const eg_threshold_params* thr, const eg_topk_params* topk) {
+    if (!out) return EG_ERR_INVALID;
+    *out = nullptr;
+    if (topology != EG_TOPO_RING || P < 1 || P > kMaxReplicas || T < 1 || !layer_numel || !thr)
+        return EG_ERR_INVALID;
+    if (thr->mode != EG_THRESH_ADAPTIVE && thr->mode != EG_THRESH_FIXED) return EG_ERR_INVALID;
+    if (thr->history_len < 1 || thr->history_len > kMaxHistory) return EG_ERR_INVALID;
+    if (std::isnan(thr->horizon) || std::isnan(thr->delta_init) || std::isnan(thr->delta_fixed))
+        return EG_ERR_INVALID;
+    if (topk && topk->enabled && (topk->k_num == 0 || topk->k_den == 0)) return EG_ERR_INVALID;
+    for (int t = 0; t < T; ++t)
+        if (layer_numel[t] < 1 || layer_numel[t] > 0x7fffffffll) return EG_ERR_INVALID;
+
+    eg_ctx* c = new (std::nothrow) eg_ctx();
+    if (!c) return EG_ERR_OOM;
+    eg_status s = EG_OK;
+    auto fail = [&](eg_status code) { eg_destroy(c); return code; };
+    if (cudaGetDevice(&c->device) != cudaSuccess) return fail(EG_ERR_CUDA);
+    c->P = P; c->T = T; c->H = thr->history_len; c->thr = *thr;
+    if (topk) c->topk = *topk;
+    c->degree = P == 1 ? 0 : (P == 2 ? 1 : 2);
+    // layout: every tensor starts on a 128-byte boundary
+    int64_t off = 0, koff = 0;
+    for (int t = 0; t < T; ++t) {
+        c->numel.push_back(layer_numel[t]);
+        c->offset.push_back(off);
+        off += (layer_numel[t] + 31) / 32 * 32;
+        c->n_total += layer_numel[t];
+        const int64_t kt = c->topk.enabled ? topk_entries(layer_numel[t], c->topk.k_num, c->topk.k_den) : 0;
+        c->kcount.push_back(kt);
+        c->out_off.push_back(koff);
+        koff += kt;
+    }
+    c->stride = off;
+    c->out_stride = koff;
+
+    const size_t S = (size_t)P * T;
+    if ((s = upload_tiles(c, build_tiles(c->numel, c->offset, kNormTile), &c->tiles_norm)) != EG_OK) return fail(s);
+    if ((s = upload_tiles(c, build_tiles(c->numel, c->offset, kFusedTile), &c->tiles_fused)) != EG_OK) return fail(s);
+    std::vector<long long> numel_ll(c->numel.begin(), c->numel.end());
+    std::vector<long long> kcount_ll(c->kcount.begin(), c->kcount.end());
+    std::vector<long long> out_off_ll(c->out_off.begin(), c->out_off.end());
+    if ((s = upload(c, &c->d_numel, numel_ll)) != EG_OK) return fail(s);
+    if ((s = upload(c, &c->d_kcount, kcount_ll)) != EG_OK) return fail(s);
+    if ((s = upload(c, &c->d_out_off, out_off_ll)) != EG_OK) return fail(s);
+#define EG_ALLOC(ptr, count)                                              \
+    if ((s = dev_alloc(c, &(ptr), (size_t)(count))) != EG_OK) return fail(s)
+    EG_ALLOC(c->xhat, (size_t)P * c->stride);
+    EG_ALLOC(c->partials_norm, (size_t)P * c->tiles_norm.n_tiles);
+    EG_ALLOC(c->partials_fused, (size_t)P * c->tiles_fused.n_tiles);
+    EG_ALLOC(c->st.delta, S); EG_ALLOC(c->st.khat, S); EG_ALLOC(c->st.hist, S * c->H);
+    EG_ALLOC(c->st.hist_len, S); EG_ALLOC(c->st.valid, S); EG_ALLOC(c->st.flag, S);
+    EG_ALLOC(c->st.snap, S); EG_ALLOC(c->st.sparse, S); EG_ALLOC(c->st.norm, S);
+    EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S);
+    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 1);
+    EG_ALLOC(c->outbox_count, S);
+    EG_ALLOC(c->cons_partials, (size_t)c->tiles_fused.n_tiles + 1);
+    if (c->topk.enabled) {
+        EG_ALLOC(c->tk.hist, S * kMaxBins);
+        EG_ALLOC(c->tk.prefix, S); EG_ALLOC(c->tk.remaining, S);
+        EG_ALLOC(c->tk.tile_count, (size_t)P * c->tiles_norm.n_tiles);
+        EG_ALLOC(c->tk.outbox, (size_t)P * c->out_stride);
+        c->tk.out_off = c->d_out_off;
+        c->tk.count = c->d_kcount;
+        c->tk.out_stride = c->out_stride;
+    }
+#undef EG_ALLOC
+    c->fused_smem = ((2 * (size_t)P + 15) & ~(size_t)15) + (size_t)P * kWarps * sizeof(double);
+    if (c->fused_smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(k_fused<kFusedVpt, true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fused_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_fused<kFusedVpt, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fused_smem);
+        if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
+    }
+    if ((s = init_state(c)) != EG_OK) return fail(s);
+    if (cudaDeviceSynchronize() != cudaSuccess) return fail(EG_ERR_CUDA);
+    *out = c;
+    return EG_OK;
+}
+
+eg_status eg_layout(const eg_ctx* c, int64_t* tensor_offset_host, int64_t* replica_stride_host) {
+    if (!c) return EG_ERR_INVALID;
+    if (tensor_offset_host) memcpy(tensor_offset_host, c->offset.data(), c->T * sizeof(int64_t));
+    if (replica_stride_host) *replica_stride_host = c->stride;
+    return EG_OK;
+}
+
+eg_status eg_topk_count(const eg_ctx* c, int t, int64_t* k_t_host) {
+    if (!c || t < 0 || t >= c->T || !k_t_host) return EG_ERR_INVALID;
+    *k_t_host = c->kcount[t];
+    return EG_OK;
+}
+
+eg_status eg_set_carry_norm(eg_ctx* c, int enabled) {
+    if (!c) return EG_ERR_INVALID;
+    c->carry = enabled != 0;
+    c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* stream_v) {
+    if (!c || !params || !grads) return EG_ERR_INVALID;
+    if (((uintptr_t)params & 15u) || ((uintptr_t)grads & 15u)) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return EG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    c->last_stream = stream;
+    int launches = 0;
+    const TileTable tn = c->tiles_norm.view(), tf = c->tiles_fused.view();
+    const dim3 grid_norm(tn.n_tiles, c->P);
+    const int S = c->P * c->T;
+
+    // a1: || x - x_hat || partial sums, unless the previous step carried them over
+    const bool use_carried = c->carry && c->carried_valid && c->carried_params == params;
+    if (!use_carried) {
+        k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, c->partials_norm);
+        ++launches;
+    }
+    // a2 + a6: decision, threshold update, counters
+    DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
+                    c->topk.enabled, c->degree};
+    const double* partials = use_carried ? c->partials_fused : c->partials_norm;
+    const TileTable& tp = use_carried ? tf : tn;
+    k_decide<<<(S + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
+        partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
+        c->ctr, c->step_k);
+    ++launches;
+    // a4: Top-K select / pack / scatter for the segments that send a sparse message
+    if (c->topk.enabled) {
+        for (int digit = 0; digit < 3; ++digit) {
+            k_topk_hist<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
+                                                           c->st.sparse, c->tk, digit);
+            k_topk_pick<<<S, kThreads, 0, stream>>>(c->T, c->st.sparse, c->tk, digit);
+            launches += 2;
+        }
+        k_topk_count<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
+                                                        c->st.sparse, c->tk);
+        k_topk_scan<<<S, kThreads, 0, stream>>>(tn, c->T, c->st.sparse, c->tk);
+        k_topk_write<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
+                                                        c->st.sparse, c->tk, c->err);
+        k_topk_scatter<<<grid_norm, kThreads, 0, stream>>>(c->xhat, tn, c->T, c->stride,
+                                                          c->st.sparse, c->tk, c->d_numel, c->err);
+        launches += 4;
+    }
+    // a3 + a5: dense snapshot, consensus average, SGD
+    if (c->carry)
+        k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+            params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+            c->partials_fused, c->step_k);
+    else
+        k_fused<kFusedVpt, false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+            params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+            c->partials_fused, c->step_k);
+    ++launches;
+    c->carried_valid = c->carry;
+    c->carried_params = params;
+    c->last_launches = launches;
+    EG_CUDA(c, cudaGetLastError());
+    return EG_OK;
+}
+
+eg_status eg_step_host(eg_ctx* c, float* params_host, const float* grads_host, float lr) {
+    if (!c || !params_host || !grads_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return EG_ERR_CUDA;
+    const size_t bytes = (size_t)c->P * c->stride * sizeof(float);
+    if (!c->stage_x) {
+        eg_status s = dev_alloc(c, &c->stage_x, (size_t)c->P * c->stride, false);
+        if (s != EG_OK) return s;
+        if ((s = dev_alloc(c, &c->stage_g, (size_t)c->P * c->stride, false)) != EG_OK) return s;
+    }
+    cudaStream_t stream = c->last_stream;
+    EG_CUDA(c, cudaMemcpyAsync(c->stage_x, params_host, bytes, cudaMemcpyHostToDevice, stream));
+    EG_CUDA(c, cudaMemcpyAsync(c->stage_g, grads_host, bytes, cudaMemcpyHostToDevice, stream));
+    c->carried_valid = false;  // the parameters came from outside
+    eg_status s = eg_step(c, c->stage_x, c->stage_g, lr, stream);
+    if (s != EG_OK) return s;
+    EG_CUDA(c, cudaMemcpyAsync(params_host, c->stage_x, bytes, cudaMemcpyDeviceToHost, stream));
+    EG_CUDA(c, cudaStreamSynchronize(stream));
+    c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status eg_stats(eg_ctx* c, uint64_t* messages_sent_host, uint64_t* bytes_sent_host) {
+    if (!c) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    Counters h{};
+    EG_CUDA(c, cudaMemcpy(&h, c->ctr, sizeof(h), cudaMemcpyDeviceToHost));
+    if (messages_sent_host) *messages_sent_host = h.messages;
+    if (bytes_sent_host) *bytes_sent_host = h.bytes;
+    return EG_OK;
+}
+
+eg_status eg_event_count(eg_ctx* c, uint64_t* events_host) {
+    if (!c || !events_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    Counters h{};
+    EG_CUDA(c, cudaMemcpy(&h, c->ctr, sizeof(h), cudaMemcpyDeviceToHost));
+    *events_host = h.events;
+    return EG_OK;
+}
+
+eg_status eg_last_decisions(eg_ctx* c, uint8_t* flags_host, double* norms_host, double* thresholds_host) {
+    if (!c) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    const size_t S = (size_t)c->P * c->T;
+    if (flags_host) EG_CUDA(c, cudaMemcpy(flags_host, c->st.flag, S, cudaMemcpyDeviceToHost));
+    if (norms_host) EG_CUDA(c, cudaMemcpy(norms_host, c->st.norm, S * sizeof(double), cudaMemcpyDeviceToHost));
+    if (thresholds_host)
+        EG_CUDA(c, cudaMemcpy(thresholds_host, c->st.thr_used, S * sizeof(double), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_thresholds(eg_ctx* c, double* delta_host, uint64_t* events_host) {
+    if (!c) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    const size_t S = (size_t)c->P * c->T;
+    if (delta_host) EG_CUDA(c, cudaMemcpy(delta_host, c->st.delta, S * sizeof(double), cudaMemcpyDeviceToHost));
+    if (events_host)
+        EG_CUDA(c, cudaMemcpy(events_host, c->st.events, S * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_last_outbox(eg_ctx* c, int i, int t, int32_t* idx_host, float* val_host, int32_t* count_host) {
+    if (!c || i < 0 || i >= c->P || t < 0 || t >= c->T || !count_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    int n = 0;
+    EG_CUDA(c, cudaMemcpy(&n, c->outbox_count + (size_t)i * c->T + t, sizeof(int), cudaMemcpyDeviceToHost));
+    *count_host = n;
+    if (n <= 0 || !c->topk.enabled) { *count_host = 0; return EG_OK; }
+    std::vector<int2> buf((size_t)n);
+    EG_CUDA(c, cudaMemcpy(buf.data(), c->tk.outbox + (size_t)i * c->out_stride + c->out_off[t],
+                          (size_t)n * sizeof(int2), cudaMemcpyDeviceToHost));
+    for (int q = 0; q < n; ++q) {
+        if (idx_host) idx_host[q] = buf[q].x;
+        if (val_host) memcpy(&val_host[q], &buf[q].y, 4);
+    }
+    return EG_OK;
+}
+
+eg_status eg_read_mailboxes(eg_ctx* c, float* xhat_host) {
+    if (!c || !xhat_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    EG_CUDA(c, cudaMemcpy(xhat_host, c->xhat, (size_t)c->P * c->stride * sizeof(float), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_reset(eg_ctx* c) {
+    if (!c) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    eg_status s = init_state(c);
+    if (s != EG_OK) return s;
+    EG_CUDA(c, cudaDeviceSynchronize());
+    return EG_OK;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// averaged model and consensus distance
+// ---------------------------------------------------------------------------------------
+namespace eg {
+
+// grid n_tiles (fused tile table).  avg[e] = (1/P) sum_i x_i[e]; cons[tile] = sum over the
+// tile and all replicas of (x_i[e] - mean)^2 with the mean kept in fp64.
+__global__ void __launch_bounds__(kThreads)
+k_average_model(const float* __restrict__ x, float* __restrict__ avg, TileTable tt, int P,
+                long long stride, double* __restrict__ cons) {
+    __shared__ double s_warp[kWarps];
+    const int tile = blockIdx.x;
+    const int len = tt.length[tile];
+    const long long off = tt.offset[tile];
+    double acc = 0.0;
+    for (int local = threadIdx.x; local < len; local += kThreads) {
+        double s = 0.0;
+        for (int i = 0; i < P; ++i) s = __dadd_rn(s, (double)x[(long long)i * stride + off + local]);
+        const double m = __ddiv_rn(s, (double)P);
+        avg[off + local] = __double2float_rn(m);
+        if (cons) {
+            for (int i = 0; i < P; ++i) {
+                const double d = __dsub_rn((double)x[(long long)i * stride + off + local], m);
+                acc = __fma_rn(d, d, acc);
+            }
+        }
+    }
+    if (cons) {
+        const double total = block_sum(acc, s_warp);
+        if (threadIdx.x == 0) cons[tile] = total;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_sum_partials(const double* __restrict__ in, int n, double* __restrict__ out) {
+    __shared__ double s_warp[kWarps];
+    double acc = 0.0;
+    for (int q = threadIdx.x; q < n; q += kThreads) acc = __dadd_rn(acc, in[q]);
+    const double total = block_sum(acc, s_warp);
+    if (threadIdx.x == 0) *out = total;
+}
+
+}  // namespace eg
+
+extern "C" {
+
+eg_status eg_average_model(eg_ctx* c, const float* params, float* avg_dev, double* consensus_host,
+                           void* stream_v) {
+    if (!c || !params || !avg_dev) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const TileTable tf = c->tiles_fused.view();
+    k_average_model<<<tf.n_tiles, kThreads, 0, stream>>>(params, avg_dev, tf, c->P, c->stride,
+                                                        consensus_host ? c->cons_partials : nullptr);
+    if (consensus_host) {
+        k_sum_partials<<<1, kThreads, 0, stream>>>(c->cons_partials, tf.n_tiles, c->cons_partials + tf.n_tiles);
+        EG_CUDA(c, cudaMemcpyAsync(consensus_host, c->cons_partials + tf.n_tiles, sizeof(double),
+                                   cudaMemcpyDeviceToHost, stream));
+        EG_CUDA(c, cudaStreamSynchronize(stream));
+    }
+    EG_CUDA(c, cudaGetLastError());
+    return EG_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// checkpoint
+// ---------------------------------------------------------------------------------------
+struct StateHeader {
+    uint64_t magic;
+    int64_t P, T, H, stride, n_total, topk, k_num, k_den;
+    int64_t step;
+    uint64_t messages, bytes, events;
+};
+
+static size_t state_bytes(const eg_ctx* c) {
+    const size_t S = (size_t)c->P * c->T;
+    return sizeof(StateHeader) + S * (sizeof(double) + sizeof(long long) + sizeof(int) + 1 +
+                                      sizeof(unsigned long long)) +
+           S * c->H * sizeof(double) + (size_t)c->P * c->stride * sizeof(float);
+}
+
+eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
+    if (!c || !bytes) return EG_ERR_INVALID;
+    const size_t need = state_bytes(c);
+    if (!host_buf) { *bytes = need; return EG_OK; }
+    if (*bytes < need) { *bytes = need; return EG_ERR_INVALID; }
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    const size_t S = (size_t)c->P * c->T;
+    StateHeader h{};
+    Counters ctr{};
+    long long k = 0;
+    EG_CUDA(c, cudaMemcpy(&ctr, c->ctr, sizeof(ctr), cudaMemcpyDeviceToHost));
+    EG_CUDA(c, cudaMemcpy(&k, c->step_k, sizeof(k), cudaMemcpyDeviceToHost));
+    h.magic = kStateMagic; h.P = c->P; h.T = c->T; h.H = c->H; h.stride = c->stride;
+    h.n_total = c->n_total; h.topk = c->topk.enabled; h.k_num = c->topk.k_num; h.k_den = c->topk.k_den;
+    h.step = k; h.messages = ctr.messages; h.bytes = ctr.bytes; h.events = ctr.events;
+    char* p = static_cast<char*>(host_buf);
+    memcpy(p, &h, sizeof(h)); p += sizeof(h);
+#define EG_PULL(ptr, nbytes)                                                     \
+    EG_CUDA(c, cudaMemcpy(p, (ptr), (nbytes), cudaMemcpyDeviceToHost)); p += (nbytes)
+    EG_PULL(c->st.delta, S * sizeof(double));
+    EG_PULL(c->st.khat, S * sizeof(long long));
+    EG_PULL(c->st.hist_len, S * sizeof(int));
+    EG_PULL(c->st.valid, S);
+    EG_PULL(c->st.events, S * sizeof(unsigned long long));
+    EG_PULL(c->st.hist, S * c->H * sizeof(double));
+    EG_PULL(c->xhat, (size_t)c->P * c->stride * sizeof(float));
+#undef EG_PULL
+    *bytes = need;
+    return EG_OK;
+}
+
+eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
+    if (!c || !host_buf || bytes < state_bytes(c)) return EG_ERR_INVALID;
+    StateHeader h;
+    memcpy(&h, host_buf, sizeof(h));
+    if (h.magic != kStateMagic || h.P != c->P || h.T != c->T || h.H != c->H || h.stride != c->stride ||
+        h.n_total != c->n_total || h.topk != c->topk.enabled ||
+        (h.topk && (h.k_num != c->topk.k_num || h.k_den != c->topk.k_den)))
+        return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    eg_status s = init_state(c);
+    if (s != EG_OK) return s;
+    const size_t S = (size_t)c->P * c->T;
+    Counters ctr{h.messages, h.bytes, h.events, 0};
+    long long k = h.step;
+    EG_CUDA(c, cudaMemcpy(c->ctr, &ctr, sizeof(ctr), cudaMemcpyHostToDevice));
+    EG_CUDA(c, cudaMemcpy(c->step_k, &k, sizeof(k), cudaMemcpyHostToDevice));
+    const char* p = static_cast<const char*>(host_buf) + sizeof(h);
+#define EG_PUSH(ptr, nbytes)                                                     \
+    EG_CUDA(c, cudaMemcpy((ptr), p, (nbytes), cudaMemcpyHostToDevice)); p += (nbytes)
+    EG_PUSH(c->st.delta, S * sizeof(double));
+    EG_PUSH(c->st.khat, S * sizeof(long long));
+    EG_PUSH(c->st.hist_len, S * sizeof(int));
+    EG_PUSH(c->st.valid, S);
+    EG_PUSH(c->st.events, S * sizeof(unsigned long long));
+    EG_PUSH(c->st.hist, S * c->H * sizeof(double));
+    EG_PUSH(c->xhat, (size_t)c->P * c->stride * sizeof(float));
+#undef EG_PUSH
+    EG_CUDA(c, cudaDeviceSynchronize());
+    c->carried_valid = false;
+    return EG_OK;
+}
+
+}  // extern "C"

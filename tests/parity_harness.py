@@ -1,0 +1,183 @@
+"""Lock-step comparison of the CUDA library (through its C ABI) with the CPU oracle.
+
+Both sides are fed the same seeded inputs, step by step.  Compared every step:
+trigger flags (bit-exact, except decisions whose norm lies within 1e-6 relative of the
+threshold, which are reported and followed by a re-synchronisation), change norms and
+thresholds (1e-12 relative: only the summation order differs), message / byte / event
+counters (exact), Top-K messages (exact index sets and values), mailboxes and parameters.
+
+Tensors never interact with each other in the method, so at sizes where the oracle would be
+too slow it is run on a subset of the tensors (``tensors=[...]``) while the CUDA library runs
+the whole configuration.
+"""
+from __future__ import annotations
+
+import os
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from oracle import eg_oracle as eo
+from paper_2103_07454_b200 import binding as B
+from paper_2103_07454_b200 import workload as W
+
+PARAM_RTOL = 1e-5      # parameters: 1e-5 relative in fp32
+NEAR_BAND = 1e-6       # decisions this close to the threshold are reported, not failed
+NORM_RTOL = 1e-12      # fp64 sums that differ only in summation order
+
+
+@dataclass
+class Report:
+    steps: int = 0
+    events: int = 0
+    sparse_checked: int = 0
+    near_threshold: List[tuple] = field(default_factory=list)
+    max_param_rel: float = 0.0
+    params_bit_exact: bool = True
+    launches: int = 0
+
+
+def oracle_threads() -> int:
+    return max(1, min(eo.threads_available(), int(os.environ.get("EG_ORACLE_THREADS", "64"))))
+
+
+def _columns(numel: Sequence[int], tensors: Sequence[int]) -> np.ndarray:
+    off = np.concatenate([[0], np.cumsum(numel)])
+    return np.concatenate([np.arange(off[t], off[t] + numel[t]) for t in tensors])
+
+
+HEADER_WORDS = 13  # checkpoint header: magic, P, T, H, stride, N, topk, k_num, k_den, step, 3 counters
+
+
+def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np.ndarray):
+    """After a reported near-threshold disagreement: overwrite the CUDA context's state and
+    parameters with the oracle's (through the checkpoint interface) so the comparison of the
+    following steps stays meaningful."""
+    blob = bytearray(eg.export_state())
+    S, H = eg.P * eg.T, o.history_len
+    head = np.frombuffer(blob, dtype=np.int64, count=HEADER_WORDS)
+    st = o.stats()
+    head[9] = o.iteration
+    head[10:13] = [st["messages"], st["bytes"], st["events"]]
+    pos = HEADER_WORDS * 8
+
+    def put(arr, dtype):
+        nonlocal pos
+        raw = np.ascontiguousarray(arr, dtype=dtype).tobytes()
+        blob[pos:pos + len(raw)] = raw
+        pos += len(raw)
+
+    hist, hist_len = o.history()
+    put(o.thresholds(), np.float64)
+    put(o.last_event_iteration(), np.int64)
+    put(hist_len, np.int32)
+    put(o.valid(), np.uint8)
+    put(o.segment_events(), np.uint64)
+    put(hist, np.float64)
+    xhat = torch.zeros((eg.P, eg.replica_stride), dtype=torch.float32)
+    eg.pack_into(xhat, torch.from_numpy(o.xhat()))
+    put(xhat.numpy(), np.float32)
+    assert pos == len(blob)
+    eg.import_state(bytes(blob))
+    eg.pack_into(x_dev, torch.from_numpy(x_host).to(x_dev.device))
+
+
+def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "workload",
+             gen_device: str = "cuda", tensors: Optional[Sequence[int]] = None,
+             carry: bool = False, check_every: int = 1, oracle_kw: Optional[dict] = None,
+             eg_kw: Optional[dict] = None, outbox_samples: int = 8, grad_hook=None) -> Report:
+    steps = wl.steps if steps is None else steps
+    dev = torch.device("cuda")
+    full = tensors is None
+    tensors = list(range(wl.T)) if full else list(tensors)
+    sub_numel = [wl.numel[t] for t in tensors]
+    cols = None if full else torch.from_numpy(_columns(wl.numel, tensors)).to(gen_device)
+
+    okw = dict(horizon=wl.horizon, history_len=wl.history_len, delta_init=wl.delta_init,
+               topk=wl.topk, threads=oracle_threads())
+    okw.update(oracle_kw or {})
+    o = eo.Oracle(wl.P, sub_numel, **okw)
+    ekw = dict(eg_kw or {})
+    for key in ("mode", "delta_fixed", "force_first_event", "horizon", "history_len", "delta_init"):
+        if key in okw and key not in ekw:
+            ekw[key] = okw[key]
+    eg = B.from_workload(wl, **ekw)
+    eg.set_carry_norm(carry)
+
+    x0 = W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)
+    x_dev = eg.to_layout(x0)
+    x_host = (x0 if full else x0[:, cols]).cpu().numpy().copy()
+    g_dev = eg.empty_params()
+    del x0
+    rep = Report()
+    sub_off = np.concatenate([[0], np.cumsum(sub_numel)])
+    rng = np.random.default_rng(7)
+
+    def gpu_sub(padded: torch.Tensor) -> np.ndarray:
+        parts = [padded[:, eg.tensor_offset[t]:eg.tensor_offset[t] + wl.numel[t]] for t in tensors]
+        return torch.cat(parts, dim=1).cpu().numpy()
+
+    for k in range(steps):
+        g = wl.grads(k, gen_device)
+        if grad_hook is not None:
+            g = grad_hook(k, g)
+        eg.pack_into(g_dev, g.to(dev))
+        g_host = (g if full else g[:, cols]).cpu().numpy()
+        del g
+        x_pre = x_host.copy() if wl.topk else None
+        o.step(x_host, np.ascontiguousarray(g_host), wl.lr)
+        eg.step(x_dev, g_dev, wl.lr)
+        rep.launches += eg.last_launch_count
+        rep.steps += 1
+        if (k % check_every) and k != steps - 1:
+            continue
+
+        f_g, d_g, thr_g = eg.last_decisions()
+        f_g, d_g, thr_g = f_g[:, tensors], d_g[:, tensors], thr_g[:, tensors]
+        f_o, d_o, thr_o = o.flags(), o.norms(), o.thresholds_used()
+        assert np.allclose(thr_g, thr_o, rtol=NORM_RTOL, atol=0, equal_nan=True), f"thresholds, step {k}"
+        assert np.allclose(d_g, d_o, rtol=NORM_RTOL, atol=1e-300), f"norms, step {k}"
+        bad = f_g != f_o
+        if bad.any():
+            near = np.abs(d_o - thr_o) <= NEAR_BAND * np.abs(thr_o)
+            assert near[bad].all(), f"trigger flags differ away from the threshold, step {k}"
+            rep.near_threshold += [(k, int(i), int(tensors[t])) for i, t in zip(*np.nonzero(bad))]
+            assert full, "near-threshold disagreement in a tensor-subset run cannot be re-synchronised"
+            resynchronise(eg, o, x_dev, x_host)
+            continue
+        rep.events += int(f_o.sum())
+
+        if full:
+            so, sg = o.stats(), eg.stats()
+            assert so == sg, f"counters, step {k}: oracle {so} cuda {sg}"
+        _, ev_g = eg.thresholds()
+        assert np.array_equal(ev_g[:, tensors], o.segment_events()), f"per-tensor events, step {k}"
+        dl_g, _ = eg.thresholds()
+        assert np.allclose(dl_g[:, tensors], o.thresholds(), rtol=NORM_RTOL, atol=0), f"delta, step {k}"
+
+        if wl.topk:
+            valid_events = np.argwhere(f_o.astype(bool))
+            if len(valid_events) > outbox_samples:
+                valid_events = valid_events[rng.choice(len(valid_events), outbox_samples, replace=False)]
+            for i, ts in valid_events:
+                idx_o, val_o = o.outbox(int(i), int(ts))
+                idx_g, val_g = eg.last_outbox(int(i), int(tensors[ts]))
+                assert np.array_equal(idx_o, idx_g), f"Top-K index set, step {k}, replica {i}, tensor {tensors[ts]}"
+                assert np.array_equal(val_o.view(np.uint32), val_g.view(np.uint32)), "Top-K values"
+                rep.sparse_checked += int(len(idx_o) > 0)
+
+        x_g = gpu_sub(x_dev)
+        same = np.array_equal(x_g.view(np.uint32), x_host.view(np.uint32))
+        rep.params_bit_exact &= bool(same)
+        if not same:
+            err = np.abs(x_g.astype(np.float64) - x_host) / np.maximum(np.abs(x_host), 1e-30)
+            rep.max_param_rel = max(rep.max_param_rel, float(err.max()))
+            assert rep.max_param_rel <= PARAM_RTOL, f"parameters, step {k}: rel err {rep.max_param_rel}"
+        xh_g = gpu_sub(eg.mailboxes().to(dev))
+        assert np.array_equal(xh_g.view(np.uint32), o.xhat().view(np.uint32)), f"mailboxes, step {k}"
+
+    eg.close()
+    o.close()
+    return rep

@@ -1,0 +1,198 @@
+"""CUDA library (through the C ABI) against the CPU oracle, element by element."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2103_07454_b200 import binding as B
+from paper_2103_07454_b200 import workload as W
+
+pytestmark = pytest.mark.gpu
+
+from parity_harness import lockstep  # noqa: E402
+
+RAGGED = [1, 3, 4, 5, 31, 32, 33, 1023, 1024, 1025, 4095, 4096, 4097, 10000, (1 << 20) + 1]
+INF = float("inf")
+
+
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 64])
+@pytest.mark.parametrize("carry", [False, True])
+def test_ragged_dense(P, carry):
+    numel = RAGGED if P <= 4 else RAGGED[:-1]
+    wl = W.synthetic(P, numel, steps=12, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=carry)
+    assert rep.params_bit_exact and not rep.near_threshold
+    assert 0 < rep.events < P * wl.T * wl.steps
+
+
+@pytest.mark.parametrize("hist,horizon", [(1, 1.0), (4, 1.0), (2, 0.5)])
+def test_history_and_horizon(hist, horizon):
+    wl = W.synthetic(5, RAGGED[:-1], steps=25, lr=0.1, grad_sigma=0.01, history_len=hist,
+                     horizon=horizon)
+    rep = lockstep(wl, init="distinct")
+    assert rep.params_bit_exact and not rep.near_threshold
+
+
+@pytest.mark.parametrize("delta,force", [(0.0, False), (INF, False), (INF, True), (0.02, True)])
+def test_fixed_threshold_modes(delta, force):
+    wl = W.synthetic(4, RAGGED[:-1], steps=6, lr=0.1, grad_sigma=0.01)
+    kw = dict(mode=1, delta_fixed=delta, force_first_event=force)
+    rep = lockstep(wl, init="distinct", oracle_kw=kw)
+    assert rep.params_bit_exact
+    if delta == 0.0:
+        assert rep.events == 4 * wl.T * wl.steps
+    if delta == INF:
+        assert rep.events == (4 * wl.T if force else 0)
+
+
+@pytest.mark.parametrize("frac", [(1, 100), (10, 100), (1, 1)])
+@pytest.mark.parametrize("P", [1, 3, 8])
+def test_ragged_topk(P, frac):
+    wl = W.synthetic(P, RAGGED, steps=14, lr=0.1, grad_sigma=0.01, topk=frac)
+
+    def ties(k, g):  # engineered ties: many equal |delta|, and exact zeros
+        g[:, 3000:9000] = torch.round(g[:, 3000:9000] * 256) / 256
+        g[:, 12000:12500] = 0.0
+        return g
+
+    rep = lockstep(wl, init="distinct", outbox_samples=10 ** 6, grad_hook=ties)
+    assert rep.params_bit_exact and rep.sparse_checked > 10
+
+
+def test_topk_carry_norm():
+    wl = W.synthetic(4, RAGGED, steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
+    rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64)
+    assert rep.params_bit_exact and rep.sparse_checked > 10
+
+
+def test_config1_mlp():
+    (wl,) = W.config(1)
+    rep = lockstep(wl)
+    assert rep.params_bit_exact and not rep.near_threshold
+
+
+def test_config2_resnet20():
+    (wl,) = W.config(2)
+    rep = lockstep(wl)
+    assert rep.params_bit_exact and not rep.near_threshold
+
+
+@pytest.mark.parametrize("carry", [False, True])
+def test_config3_resnet18_p16(carry):
+    (wl,) = W.config(3)
+    steps = wl.steps if (carry or os.environ.get("EG_FULL")) else 30
+    rep = lockstep(wl, steps=steps, carry=carry, check_every=5)
+    assert rep.params_bit_exact and not rep.near_threshold
+    assert rep.launches == (steps * 2 + 1 if carry else steps * 3)
+
+
+def _sample_tensors(wl, n_small=6, n_mid=3, n_big=2):
+    order = np.argsort(wl.numel)
+    mid = len(order) // 2
+    pick = list(order[:n_small]) + list(order[mid:mid + n_mid]) + list(order[-n_big:])
+    return sorted(set(int(t) for t in pick))
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_config4_resnet18_topk(which):
+    wl = W.config(4)[which]
+    steps = wl.steps if os.environ.get("EG_FULL") else 40
+    rep = lockstep(wl, steps=steps, tensors=_sample_tensors(wl), check_every=4, outbox_samples=12)
+    assert rep.params_bit_exact and rep.sparse_checked > 20
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_config5_resnet50_p64(which):
+    wl = W.config(5)[which]
+    steps = wl.steps if os.environ.get("EG_FULL") else 12
+    rep = lockstep(wl, steps=steps, tensors=_sample_tensors(wl, 6, 3, 1), check_every=4,
+                   outbox_samples=12, carry=(which == 0))
+    assert rep.params_bit_exact
+
+
+def test_checkpoint_roundtrip_and_reset():
+    wl = W.synthetic(3, [5, 1000, 4097], steps=8, lr=0.1, grad_sigma=0.01, history_len=3)
+    eg = B.from_workload(wl)
+    x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+    g = [eg.to_layout(wl.grads(k, "cuda")) for k in range(wl.steps)]
+    for k in range(4):
+        eg.step(x, g[k], wl.lr)
+    blob, x_mid = eg.export_state(), x.clone()
+    for k in range(4, 8):
+        eg.step(x, g[k], wl.lr)
+    ref_x, ref_stats, ref_dec = x.clone(), eg.stats(), eg.last_decisions()
+    eg.reset()
+    assert eg.stats() == {"messages": 0, "bytes": 0, "events": 0}
+    assert float(eg.mailboxes().abs().max()) == 0.0
+    eg.import_state(blob)
+    x.copy_(x_mid)
+    for k in range(4, 8):
+        eg.step(x, g[k], wl.lr)
+    assert torch.equal(x, ref_x) and eg.stats() == ref_stats
+    for a, b in zip(eg.last_decisions(), ref_dec):
+        assert np.array_equal(a, b)
+    with pytest.raises(B.EventGradError):
+        eg.import_state(blob[:100])
+    eg.close()
+
+
+def test_host_buffer_entry_point():
+    wl = W.synthetic(3, [7, 3000], steps=3, lr=0.1, grad_sigma=0.01)
+    a, b = B.from_workload(wl), B.from_workload(wl)
+    x0 = a.to_layout(W.distinct_init_params(wl, "cuda"))
+    xa, xb = x0.clone(), x0.cpu().pin_memory()
+    for k in range(wl.steps):
+        g = a.to_layout(wl.grads(k, "cuda"))
+        a.step(xa, g, wl.lr)
+        b.step_host(xb, g.cpu().pin_memory(), wl.lr)
+    assert torch.equal(xa.cpu(), xb) and a.stats() == b.stats()
+
+
+def test_run_twice_is_deterministic():
+    wl = W.synthetic(6, RAGGED, steps=6, lr=0.1, grad_sigma=0.01, topk=(3, 100))
+    outs = []
+    for _ in range(2):
+        eg = B.from_workload(wl)
+        x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+        for k in range(wl.steps):
+            eg.step(x, eg.to_layout(wl.grads(k, "cuda")), wl.lr)
+        outs.append((x.clone(), eg.last_decisions(), eg.stats(), eg.mailboxes()))
+        eg.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][3], outs[1][3])
+    assert outs[0][2] == outs[1][2]
+    assert all(np.array_equal(a, b) for a, b in zip(outs[0][1], outs[1][1]))
+
+
+def test_average_model_and_consensus():
+    from oracle import eg_oracle as eo
+    wl = W.synthetic(5, [3, 1000, 4097])
+    eg = B.from_workload(wl)
+    xp = W.distinct_init_params(wl, "cuda")
+    x = eg.to_layout(xp)
+    avg, cons = eg.average_model(x, consensus=True)
+    o = eo.from_workload(wl)
+    xn = xp.cpu().numpy()
+    assert np.array_equal(eg.from_layout(avg.unsqueeze(0))[0].cpu().numpy(), o.average_model(xn))
+    assert cons == pytest.approx(o.consensus_distance(xn), rel=1e-12)
+
+
+def test_generator_is_device_independent():
+    base = W.stream_base(W.MASTER_SEED, W.STREAM_GRAD, 7, 2)
+    a = W.ih8_integers(base, 0, 1 << 16, "cpu")
+    b = W.ih8_integers(base, 0, 1 << 16, "cuda").cpu()
+    assert torch.equal(a, b)
+    (wl,) = W.config(1)
+    assert torch.equal(wl.grads(3, "cpu"), wl.grads(3, "cuda").cpu())
+    assert torch.equal(wl.init_params("cpu"), wl.init_params("cuda").cpu())
+
+
+def test_invalid_arguments_are_reported():
+    wl = W.synthetic(2, [8])
+    eg = B.from_workload(wl)
+    x = eg.empty_params()
+    lib = B.load_library()
+    assert lib.eg_step(eg._h, None, x.data_ptr(), 0.1, None) == 1
+    assert lib.eg_step(eg._h, x.data_ptr() + 4, x.data_ptr(), 0.1, None) == 1   # misaligned
+    with pytest.raises(B.EventGradError):
+        B.EventGrad(2000, [8])                                                  # P over the limit
