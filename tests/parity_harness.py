@@ -25,7 +25,15 @@ from paper_2103_07454_b200 import workload as W
 
 PARAM_RTOL = 1e-5      # parameters: 1e-5 relative in fp32
 NEAR_BAND = 1e-6       # decisions this close to the threshold are reported, not failed
-NORM_RTOL = 1e-12      # fp64 sums that differ only in summation order
+UNIT_ROUNDOFF = 2.0 ** -53
+
+
+def norm_rtol(numel) -> np.ndarray:
+    """Tolerance on || x - x_hat ||: the oracle adds the n squares one after the other, the
+    kernels add them as a tree; each is within (n-1)*u relative of the exact sum of these
+    non-negative terms (standard bound for recursive summation), so the two norms (square
+    roots halve the error) agree within n*u.  Floor: a few roundings."""
+    return np.maximum(np.asarray(numel, dtype=np.float64) * UNIT_ROUNDOFF, 8 * UNIT_ROUNDOFF)
 
 
 @dataclass
@@ -35,6 +43,7 @@ class Report:
     sparse_checked: int = 0
     near_threshold: List[tuple] = field(default_factory=list)
     max_param_rel: float = 0.0
+    max_norm_rel: float = 0.0
     params_bit_exact: bool = True
     launches: int = 0
 
@@ -131,14 +140,22 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
         eg.step(x_dev, g_dev, wl.lr)
         rep.launches += eg.last_launch_count
         rep.steps += 1
-        if (k % check_every) and k != steps - 1:
-            continue
+        if (k % check_every) and k != steps - 1 and k >= 8:
+            continue        # the first steps (where most events happen) are always checked
 
         f_g, d_g, thr_g = eg.last_decisions()
         f_g, d_g, thr_g = f_g[:, tensors], d_g[:, tensors], thr_g[:, tensors]
         f_o, d_o, thr_o = o.flags(), o.norms(), o.thresholds_used()
-        assert np.allclose(thr_g, thr_o, rtol=NORM_RTOL, atol=0, equal_nan=True), f"thresholds, step {k}"
-        assert np.allclose(d_g, d_o, rtol=NORM_RTOL, atol=1e-300), f"norms, step {k}"
+        tol = 2 * norm_rtol(sub_numel)[None, :]     # thresholds are norms divided by integers
+        fin = np.isfinite(thr_o)
+        assert np.array_equal(fin, np.isfinite(thr_g)) and np.array_equal(thr_g[~fin], thr_o[~fin])
+        tol = np.broadcast_to(tol, thr_o.shape)
+        assert np.all(np.abs(thr_g[fin] - thr_o[fin]) <= tol[fin] * np.abs(thr_o[fin])), f"thresholds, step {k}"
+        rel = np.abs(d_g - d_o) / np.maximum(np.abs(d_o), 1e-300) / norm_rtol(sub_numel)[None, :]
+        rep.max_norm_rel = max(rep.max_norm_rel, float(rel.max()))
+        assert rel.max() <= 1.0, (
+            f"norms, step {k}: {rel.max():.3e} x tolerance at {np.unravel_index(rel.argmax(), rel.shape)} "
+            f"cuda {d_g.flat[rel.argmax()]!r} oracle {d_o.flat[rel.argmax()]!r}")
         bad = f_g != f_o
         if bad.any():
             near = np.abs(d_o - thr_o) <= NEAR_BAND * np.abs(thr_o)
@@ -155,7 +172,9 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
         _, ev_g = eg.thresholds()
         assert np.array_equal(ev_g[:, tensors], o.segment_events()), f"per-tensor events, step {k}"
         dl_g, _ = eg.thresholds()
-        assert np.allclose(dl_g[:, tensors], o.thresholds(), rtol=NORM_RTOL, atol=0), f"delta, step {k}"
+        dl_g, dl_o = dl_g[:, tensors], o.thresholds()
+        fin = np.isfinite(dl_o)
+        assert np.all(np.abs(dl_g[fin] - dl_o[fin]) <= tol[fin] * np.abs(dl_o[fin])), f"delta, step {k}"
 
         if wl.topk:
             valid_events = np.argwhere(f_o.astype(bool))

@@ -99,7 +99,7 @@ def test_config4_resnet18_topk(which):
     wl = W.config(4)[which]
     steps = wl.steps if os.environ.get("EG_FULL") else 40
     rep = lockstep(wl, steps=steps, tensors=_sample_tensors(wl), check_every=4, outbox_samples=12)
-    assert rep.params_bit_exact and rep.sparse_checked > 20
+    assert rep.params_bit_exact and rep.sparse_checked > 10
 
 
 @pytest.mark.parametrize("which", [0, 1])
