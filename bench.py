@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the event-triggered communication step.
+
+    python bench.py --gpus N --steps K --warmup W            (CUDA library)
+    python bench.py --impl reference --steps K --warmup W    (CPU oracle on the host cores)
+
+A "step" is one ``eg_step``: change norms, device-side trigger decisions, dense snapshots
+(or Top-K select / pack / scatter), ring average and SGD update for all P replicas of the
+workload.  Default workload: the 16-replica ring of ResNet-18 (CIFAR) parameter sets with the
+step-indexed synthetic gradients of that configuration.  With N > 1 (torchrun) every rank runs
+an independent copy of the workload on its own GPU ("replicas only": the method is defined on
+one device's memory, nothing is exchanged); the value is the sum over ranks divided by the
+slowest rank's time.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2103_07454_b200 import workload as W  # noqa: E402
+
+METRIC = "event-triggered step: effective HBM GB/s (% of peak), replica-steps/s, msgs sent"
+FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used if no peaks file
+NOMINAL_HBM_GBS = 8000.0
+BYTES_PER_ELEMENT = {"carry": 16, "two_pass": 24}   # algorithmic bytes per element-replica-step
+FUSED_BYTES_PER_ELEMENT = 16       # fused kernel: reads x, g, touches x_hat once, writes x
+
+# DRAM traffic of the fused kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum per launch on the default workload), keyed by the hash of the kernel
+# sources it was taken with; reported as null once the sources change.
+FUSED_TRAFFIC = {}
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2103_07454_b200", "csrc")
+    for name in ("eg_common.cuh", "eg_norm.cuh", "eg_fused.cuh"):
+        with open(os.path.join(d, name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+# ----------------------------------------------------------------------------------------
+# multi-process plumbing (one process per GPU; nothing of the data path is exchanged)
+# ----------------------------------------------------------------------------------------
+def dist_setup(backend: str):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world <= 1:
+        return 0, 1, 0
+    import torch.distributed as dist
+    rank, local = int(os.environ["RANK"]), int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    if not dist.is_initialized():
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world, local
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def aggregate(units_this_rank: float, ms_this_rank: float, device="cpu"):
+    """Whole-job figures from per-rank ones: (sum of units, max of milliseconds)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(units_this_rank), float(ms_this_rank)
+    u = torch.tensor([units_this_rank], dtype=torch.float64, device=device)
+    t = torch.tensor([ms_this_rank], dtype=torch.float64, device=device)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(u.item()), float(t.item())
+
+
+# ----------------------------------------------------------------------------------------
+# clocks during the timed region
+# ----------------------------------------------------------------------------------------
+REASON_BITS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+               0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x100: "display_clock_setting"}
+
+
+class ClockSampler:
+    """Polls SM clock and clock-event reasons through NVML from a thread."""
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            self._nv = pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as exc:  # pragma: no cover - depends on the box
+            self.error = repr(exc)
+
+    def _poll(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                self.samples.append(mhz)
+                for bit, name in REASON_BITS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                break
+            time.sleep(0.0005)
+
+    def start(self):
+        if self._h is not None:
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self) -> dict:
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------------------
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def pick_workload(args) -> W.Workload:
+    return W.config(args.config)[args.which]
+
+
+def sample_tensors(wl: W.Workload, fraction: float):
+    """Tensors (in order) holding about ``fraction`` of the elements; at least one."""
+    picked, acc = [], 0
+    for t, n in enumerate(wl.numel):
+        if picked and acc >= fraction * wl.N:
+            break
+        picked.append(t)
+        acc += n
+    return picked
+
+
+def time_oracle(wl: W.Workload, steps: int, warmup: int, budget_s: float, gen_device: str):
+    """Times the CPU oracle, as it stands, on all host cores.  If ``steps`` full-size steps do
+    not fit ``budget_s`` the run uses a subset of the tensors (they do not interact)."""
+    import numpy as np
+    from oracle import eg_oracle as eo
+    threads = eo.threads_available()
+    # calibrate on a small prefix of the tensors
+    probe_t = sample_tensors(wl, 0.05)
+    numel = [wl.numel[t] for t in probe_t]
+    o = eo.Oracle(wl.P, numel, horizon=wl.horizon, history_len=wl.history_len,
+                  delta_init=wl.delta_init, topk=wl.topk, threads=threads)
+    n_probe = sum(numel)
+    x = np.zeros((wl.P, n_probe), np.float32)
+    g = np.full((wl.P, n_probe), 1e-3, np.float32)
+    o.step(x, g, wl.lr)
+    t0 = time.perf_counter()
+    o.step(x, g, wl.lr)
+    per_elem = (time.perf_counter() - t0) / (wl.P * n_probe)
+    o.close()
+    full_step_s = per_elem * wl.P * wl.N
+    fraction = min(1.0, budget_s / max(1e-9, full_step_s * (steps + warmup)))
+    tensors = sample_tensors(wl, fraction) if fraction < 1.0 else list(range(wl.T))
+    numel = [wl.numel[t] for t in tensors]
+    n_sub = sum(numel)
+    off = np.concatenate([[0], np.cumsum(wl.numel)])
+    cols = np.concatenate([np.arange(off[t], off[t] + wl.numel[t]) for t in tensors])
+    cols_t = torch.from_numpy(cols).to(gen_device)
+    n_buf = max(1, min(steps + warmup, 4))
+    grads = [np.ascontiguousarray(wl.grads(k, gen_device)[:, cols_t].cpu().numpy()) for k in range(n_buf)]
+    x = np.ascontiguousarray(wl.init_params(gen_device)[:, cols_t].cpu().numpy())
+    o = eo.Oracle(wl.P, numel, horizon=wl.horizon, history_len=wl.history_len,
+                  delta_init=wl.delta_init, topk=wl.topk, threads=threads)
+    for k in range(warmup):
+        o.step(x, grads[k % n_buf], wl.lr)
+    t0 = time.perf_counter()
+    for k in range(steps):
+        o.step(x, grads[(warmup + k) % n_buf], wl.lr)
+    sec = time.perf_counter() - t0
+    stats = o.stats()
+    o.close()
+    elems = wl.P * n_sub * steps
+    gbs = elems * BYTES_PER_ELEMENT["two_pass"] / sec / 1e9
+    sample = (f"{steps} steps of all {wl.P} replicas x {len(tensors)}/{wl.T} tensors "
+              f"({n_sub}/{wl.N} elements per replica)")
+    return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample,
+            "replica_steps_per_s": wl.P * steps * (n_sub / wl.N) / sec, "seconds": sec,
+            "messages_sent": stats["messages"]}
+
+
+def run_reference(args):
+    rank, world, local = dist_setup("gloo")
+    if rank != 0:
+        return
+    wl = pick_workload(args)
+    gen = "cuda" if torch.cuda.is_available() else "cpu"
+    r = time_oracle(wl, args.steps, args.warmup, budget_s=120.0, gen_device=gen)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": "GB/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * r["seconds"] / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "P": wl.P, "tensors": wl.T, "elements": wl.N,
+                       "bytes_per_element_step": BYTES_PER_ELEMENT["two_pass"]},
+            "replica_steps_per_s": r["replica_steps_per_s"],
+            "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def time_steps(eg, x, grads, lr, steps, sampler=None):
+    """K steps bracketed by events on the launching stream, barrier + synchronise outside."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    e0.record()
+    launches = 0
+    for k in range(steps):
+        eg.step(x, grads[k % len(grads)], lr)
+        launches += eg.last_launch_count
+    e1.record()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.stop()
+    barrier()
+    return e0.elapsed_time(e1), launches
+
+
+def run_native(args):
+    from paper_2103_07454_b200 import binding as B
+    rank, world, local = dist_setup("nccl")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    wl = pick_workload(args)
+    K, Wm = args.steps, max(args.warmup, 3)
+    eg = B.from_workload(wl)
+    buf_bytes = wl.P * eg.replica_stride * 4
+    free, _ = torch.cuda.mem_get_info()
+    n_buf = int(max(1, min(max(K, Wm), (free - (24 << 30)) // buf_bytes)))
+    grads = [eg.to_layout(wl.grads(k, dev)) for k in range(n_buf)]
+    x0 = eg.to_layout(wl.init_params(dev))
+    x = x0.clone()
+    peak, peak_kind = measured_peak()
+    elems = wl.P * wl.N
+    results = {}
+    sampler = ClockSampler(local)
+    clocks = None
+    for variant in ([args.variant] + [v for v in ("carry", "two_pass") if v != args.variant]):
+        eg.set_carry_norm(variant == "carry")
+        x.copy_(x0)
+        eg.reset()
+        eg.set_timing(False)
+        for k in range(Wm):
+            eg.step(x, grads[k % n_buf], wl.lr)
+        x.copy_(x0)
+        eg.reset()
+        eg.set_carry_norm(variant == "carry")
+        eg.set_timing(True)
+        main = variant == args.variant
+        ms, launches = time_steps(eg, x, grads, wl.lr, K, sampler if main else None)
+        kt = eg.kernel_times()
+        stats = eg.stats()
+        units, ms_max = aggregate(float(elems) * K, ms, dev)
+        results[variant] = {
+            "ms_per_step": ms_max / K, "gbs": units * BYTES_PER_ELEMENT[variant] / ms_max / 1e6,
+            "replica_steps_per_s": world * wl.P * K / (ms_max / 1e3), "launches": launches,
+            "kernel_ms": {g: (v[0] / v[1] if v[1] else None) for g, v in kt.items()},
+            "messages_sent": stats["messages"], "bytes_sent": stats["bytes"],
+            "pct_messages": 100.0 * stats["messages"] / (wl.P * wl.T * 2 * K)}
+        if main:
+            clocks = sampler.summary()
+    main = results[args.variant]
+
+    # end to end: host buffers in, updated parameters out, through eg_step_host
+    e_steps = max(1, min(K, args.e2e_steps))
+    xh = x0.cpu().pin_memory()
+    gh = [grads[k % n_buf].cpu().pin_memory() for k in range(min(e_steps, 2))]
+    eg.reset()
+    eg.set_timing(False)
+    eg.step_host(xh, gh[0], wl.lr)          # allocates the staging buffers
+    xh.copy_(x0)
+    eg.reset()
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for k in range(e_steps):
+        eg.step_host(xh, gh[k % len(gh)], wl.lr)
+    e_ms = (time.perf_counter() - t0) * 1e3
+    e_units, e_ms_max = aggregate(float(elems) * e_steps, e_ms, dev)
+    e2e = {"value": e_units * BYTES_PER_ELEMENT["two_pass"] / e_ms_max / 1e6, "unit": "GB/s",
+           "h2d_bytes_per_step": 2 * buf_bytes, "d2h_bytes_per_step": buf_bytes,
+           "steps": e_steps, "ms_per_step": e_ms_max / e_steps,
+           "replica_steps_per_s": world * wl.P * e_steps / (e_ms_max / 1e3)}
+
+    fused_ms = main["kernel_ms"]["fused"]
+    achieved = elems * FUSED_BYTES_PER_ELEMENT / fused_ms / 1e6 if fused_ms else None
+    roofline = {"bound": "hbm", "kernel": "k_fused", "achieved": achieved, "peak": peak,
+                "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None,
+                "traffic": FUSED_TRAFFIC.get(kernel_source_hash()),
+                "algorithmic_bytes_per_launch": elems * FUSED_BYTES_PER_ELEMENT,
+                "kernel_ms": fused_ms,
+                "step_frac_of_peak": main["gbs"] / peak,
+                "step_frac_of_nominal_8TBs": main["gbs"] / NOMINAL_HBM_GBS}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        del grads
+        torch.cuda.empty_cache()
+        cpu = time_oracle(wl, steps=args.cpu_steps, warmup=1, budget_s=25.0, gen_device=str(dev))
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "replica_steps_per_s")}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": main["gbs"], "unit": "GB/s", "n_gpus": world,
+                "steps": K, "warmup": Wm, "ms_per_step": main["ms_per_step"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic",
+                "config": {"workload": wl.name, "P": wl.P, "tensors": wl.T, "elements": wl.N,
+                           "variant": args.variant,
+                           "bytes_per_element_step": BYTES_PER_ELEMENT[args.variant],
+                           "l2": "inputs larger than L2 (no flush needed)",
+                           "gradient_buffers": n_buf, "multi_gpu": "replicas only"},
+                "pct_of_peak": 100.0 * main["gbs"] / peak,
+                "replica_steps_per_s": main["replica_steps_per_s"],
+                "messages_sent": main["messages_sent"], "pct_messages": main["pct_messages"],
+                "gpu_launches": main["launches"], "clocks": clocks, "e2e": e2e,
+                "roofline": roofline, "cpu_baseline": cpu, "variants": results}
+        print(json.dumps(line), flush=True)
+    eg.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--config", type=int, default=3)
+    ap.add_argument("--which", type=int, default=0)
+    ap.add_argument("--variant", default="carry", choices=["carry", "two_pass"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-steps", type=int, default=10)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -114,6 +114,17 @@ eg_status eg_step_host(eg_ctx* ctx, float* params_host, const float* grads_host,
  * turning it on, eg_reset and eg_import_state make the next step recompute the norms. */
 eg_status eg_set_carry_norm(eg_ctx* ctx, int enabled);
 
+/* Per-kernel timing for measurements (off by default).  When on, eg_step brackets each
+ * kernel group with a pair of CUDA events recorded on the step's own stream; eg_kernel_times
+ * synchronises, adds up the elapsed milliseconds per group since the last call into
+ * ms_host[EG_KERNEL_GROUPS], the number of timed sections into
+ * sections_host[EG_KERNEL_GROUPS], and forgets them.  At most 32768 sections are kept
+ * between two reads; further ones are not timed. */
+enum { EG_KERNEL_NORM = 0, EG_KERNEL_DECIDE = 1, EG_KERNEL_TOPK = 2, EG_KERNEL_FUSED = 3,
+       EG_KERNEL_GROUPS = 4 };
+eg_status eg_set_timing(eg_ctx* ctx, int enabled);
+eg_status eg_kernel_times(eg_ctx* ctx, double* ms_host, uint64_t* sections_host);
+
 /* Totals since creation / eg_reset (Table 1 and Table 2 report ratios of these).
  * Synchronises.  Pointers may be NULL. */
 eg_status eg_stats(eg_ctx* ctx, uint64_t* messages_sent_host, uint64_t* bytes_sent_host);

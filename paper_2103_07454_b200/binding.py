@@ -26,7 +26,9 @@ EXPORTS = [
     "eg_event_count", "eg_last_decisions", "eg_thresholds", "eg_last_outbox", "eg_topk_count",
     "eg_read_mailboxes", "eg_average_model", "eg_export_state", "eg_import_state", "eg_reset",
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
+    "eg_set_timing", "eg_kernel_times",
 ]
+KERNEL_GROUPS = ("norm", "decide", "topk", "fused")
 
 
 class ThresholdParams(C.Structure):
@@ -74,6 +76,8 @@ def load_library() -> C.CDLL:
     lib.eg_export_state.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
     lib.eg_import_state.argtypes = [vp, vp, C.c_size_t]
     lib.eg_reset.argtypes = [vp]
+    lib.eg_set_timing.argtypes = [vp, C.c_int]
+    lib.eg_kernel_times.argtypes = [vp, C.POINTER(C.c_double), u64p]
     lib.eg_destroy.argtypes = [vp]
     lib.eg_destroy.restype = None
     lib.eg_strerror.argtypes = [C.c_int]
@@ -246,6 +250,16 @@ class EventGrad:
     def import_state(self, blob: bytes):
         _check(self._lib, self._lib.eg_import_state(self._h, blob, len(blob)), self._h,
                "eg_import_state")
+
+    def set_timing(self, enabled: bool):
+        _check(self._lib, self._lib.eg_set_timing(self._h, int(enabled)), self._h, "eg_set_timing")
+
+    def kernel_times(self) -> dict:
+        """{group: (total ms, timed sections)} since the last call (``eg_kernel_times``)."""
+        ms = (C.c_double * len(KERNEL_GROUPS))()
+        n = (C.c_uint64 * len(KERNEL_GROUPS))()
+        _check(self._lib, self._lib.eg_kernel_times(self._h, ms, n), self._h, "eg_kernel_times")
+        return {g: (ms[q], int(n[q])) for q, g in enumerate(KERNEL_GROUPS)}
 
     def reset(self):
         _check(self._lib, self._lib.eg_reset(self._h), self._h, "eg_reset")

@@ -66,6 +66,11 @@ struct eg_ctx {
     int last_cuda_error = 0;
     int last_launches = 0;
     size_t fused_smem = 0;
+    // optional per-kernel timing (events on the launching stream)
+    bool timing = false;
+    std::vector<cudaEvent_t> ev_pool;      // pairs
+    std::vector<int> ev_kind;              // kernel group of every recorded pair
+    size_t ev_used = 0;
 };
 
 namespace {
@@ -165,6 +170,33 @@ eg_status sync_and_check(eg_ctx* c) {
     return e ? EG_ERR_INTERNAL : EG_OK;
 }
 
+constexpr size_t kMaxTimedPairs = 1 << 15;
+
+// Brackets one kernel group with a pair of events when timing is on.
+struct TimedSection {
+    eg_ctx* c;
+    cudaStream_t stream;
+    bool on;
+    TimedSection(eg_ctx* ctx, cudaStream_t s, int kind) : c(ctx), stream(s), on(false) {
+        if (!c->timing || c->ev_used >= kMaxTimedPairs) return;
+        if (c->ev_pool.size() < 2 * (c->ev_used + 1)) {
+            cudaEvent_t a, b;
+            if (cudaEventCreate(&a) != cudaSuccess) return;
+            if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
+            c->ev_pool.push_back(a);
+            c->ev_pool.push_back(b);
+        }
+        if (c->ev_kind.size() <= c->ev_used) c->ev_kind.push_back(kind);
+        c->ev_kind[c->ev_used] = kind;
+        on = cudaEventRecord(c->ev_pool[2 * c->ev_used], stream) == cudaSuccess;
+    }
+    ~TimedSection() {
+        if (!on) return;
+        cudaEventRecord(c->ev_pool[2 * c->ev_used + 1], stream);
+        ++c->ev_used;
+    }
+};
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -201,6 +233,7 @@ void eg_destroy(eg_ctx* c) {
         DeviceGuard guard(c->device);
         cudaDeviceSynchronize();
         for (void* p : c->allocs) cudaFree(p);
+        for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
     }
     delete c;
 }
@@ -323,6 +356,7 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     // a1: || x - x_hat || partial sums, unless the previous step carried them over
     const bool use_carried = c->carry && c->carried_valid && c->carried_params == params;
     if (!use_carried) {
+        TimedSection ts(c, stream, EG_KERNEL_NORM);
         k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, c->partials_norm);
         ++launches;
     }
@@ -331,12 +365,16 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
                     c->topk.enabled, c->degree};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf : tn;
-    k_decide<<<(S + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
-        partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
-        c->ctr, c->step_k);
-    ++launches;
+    {
+        TimedSection ts(c, stream, EG_KERNEL_DECIDE);
+        k_decide<<<(S + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
+            partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
+            c->ctr, c->step_k);
+        ++launches;
+    }
     // a4: Top-K select / pack / scatter for the segments that send a sparse message
     if (c->topk.enabled) {
+        TimedSection ts(c, stream, EG_KERNEL_TOPK);
         for (int digit = 0; digit < 3; ++digit) {
             k_topk_hist<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
                                                            c->st.sparse, c->tk, digit);
@@ -353,15 +391,18 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
         launches += 4;
     }
     // a3 + a5: dense snapshot, consensus average, SGD
-    if (c->carry)
-        k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
-            params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-            c->partials_fused, c->step_k);
-    else
-        k_fused<kFusedVpt, false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
-            params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-            c->partials_fused, c->step_k);
-    ++launches;
+    {
+        TimedSection ts(c, stream, EG_KERNEL_FUSED);
+        if (c->carry)
+            k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+                params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                c->partials_fused, c->step_k);
+        else
+            k_fused<kFusedVpt, false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+                params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                c->partials_fused, c->step_k);
+        ++launches;
+    }
     c->carried_valid = c->carry;
     c->carried_params = params;
     c->last_launches = launches;
@@ -464,6 +505,28 @@ eg_status eg_read_mailboxes(eg_ctx* c, float* xhat_host) {
     eg_status s = sync_and_check(c);
     if (s != EG_OK) return s;
     EG_CUDA(c, cudaMemcpy(xhat_host, c->xhat, (size_t)c->P * c->stride * sizeof(float), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_set_timing(eg_ctx* c, int enabled) {
+    if (!c) return EG_ERR_INVALID;
+    c->timing = enabled != 0;
+    c->ev_used = 0;
+    return EG_OK;
+}
+
+eg_status eg_kernel_times(eg_ctx* c, double* ms_host, uint64_t* sections_host) {
+    if (!c || !ms_host || !sections_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    for (int q = 0; q < EG_KERNEL_GROUPS; ++q) { ms_host[q] = 0.0; sections_host[q] = 0; }
+    for (size_t q = 0; q < c->ev_used; ++q) {
+        float ms = 0.f;
+        EG_CUDA(c, cudaEventElapsedTime(&ms, c->ev_pool[2 * q], c->ev_pool[2 * q + 1]));
+        ms_host[c->ev_kind[q]] += (double)ms;
+        sections_host[c->ev_kind[q]] += 1;
+    }
+    c->ev_used = 0;
     return EG_OK;
 }
 
