@@ -165,7 +165,17 @@ def measured_peak():
 
 
 def pick_workload(args) -> W.Workload:
-    return W.config(args.config)[args.which]
+    wl = W.config(args.config)[args.which]
+    if args.max_elements:       # a smaller case of the same shapes (for profiler captures)
+        keep, total = [], 0
+        for t in wl.tensors:
+            if keep and total + t.numel > args.max_elements:
+                break
+            keep.append(t)
+            total += t.numel
+        wl.tensors = keep
+        wl.name += f"_first{len(keep)}tensors"
+    return wl
 
 
 def sample_tensors(wl: W.Workload, fraction: float):
@@ -385,6 +395,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--max-elements", type=int, default=0,
+                    help="keep only the leading tensors of the workload up to this many elements")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
