@@ -114,6 +114,13 @@ eg_status eg_step_host(eg_ctx* ctx, float* params_host, const float* grads_host,
  * turning it on, eg_reset and eg_import_state make the next step recompute the norms. */
 eg_status eg_set_carry_norm(eg_ctx* ctx, int enabled);
 
+/* Which implementation of the fused snapshot / average / SGD kernel eg_step launches.  Both
+ * compute bit-identical results.  EG_FUSED_PIPELINED (default) streams the operands through
+ * shared memory with bulk asynchronous copies; EG_FUSED_REGISTER keeps the ring walk in
+ * registers with plain vector loads. */
+enum { EG_FUSED_PIPELINED = 0, EG_FUSED_REGISTER = 1 };
+eg_status eg_set_fused_kernel(eg_ctx* ctx, int kind);
+
 /* Per-kernel timing for measurements (off by default).  When on, eg_step brackets each
  * kernel group with a pair of CUDA events recorded on the step's own stream; eg_kernel_times
  * synchronises, adds up the elapsed milliseconds per group since the last call into

@@ -26,8 +26,10 @@ EXPORTS = [
     "eg_event_count", "eg_last_decisions", "eg_thresholds", "eg_last_outbox", "eg_topk_count",
     "eg_read_mailboxes", "eg_average_model", "eg_export_state", "eg_import_state", "eg_reset",
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
-    "eg_set_timing", "eg_kernel_times",
+    "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel",
 ]
+FUSED_PIPELINED = 0
+FUSED_REGISTER = 1
 KERNEL_GROUPS = ("norm", "decide", "topk", "fused")
 
 
@@ -77,6 +79,7 @@ def load_library() -> C.CDLL:
     lib.eg_import_state.argtypes = [vp, vp, C.c_size_t]
     lib.eg_reset.argtypes = [vp]
     lib.eg_set_timing.argtypes = [vp, C.c_int]
+    lib.eg_set_fused_kernel.argtypes = [vp, C.c_int]
     lib.eg_kernel_times.argtypes = [vp, C.POINTER(C.c_double), u64p]
     lib.eg_destroy.argtypes = [vp]
     lib.eg_destroy.restype = None
@@ -250,6 +253,10 @@ class EventGrad:
     def import_state(self, blob: bytes):
         _check(self._lib, self._lib.eg_import_state(self._h, blob, len(blob)), self._h,
                "eg_import_state")
+
+    def set_fused_kernel(self, kind: int):
+        _check(self._lib, self._lib.eg_set_fused_kernel(self._h, int(kind)), self._h,
+               "eg_set_fused_kernel")
 
     def set_timing(self, enabled: bool):
         _check(self._lib, self._lib.eg_set_timing(self._h, int(enabled)), self._h, "eg_set_timing")

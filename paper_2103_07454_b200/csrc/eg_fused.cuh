@@ -52,7 +52,7 @@ k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ 
         const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
         int P, int T, long long stride, float lr, double* __restrict__ partials,
         long long* step_k) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     uint8_t* s_snap = smem;
     uint8_t* s_valid = smem + P;
     double* s_red = reinterpret_cast<double*>(smem + ((2 * P + 15) & ~15));

@@ -11,6 +11,7 @@
 
 #include "eg_common.cuh"
 #include "eg_fused.cuh"
+#include "eg_fused_pipe.cuh"
 #include "eg_norm.cuh"
 #include "eg_topk.cuh"
 
@@ -20,6 +21,7 @@ namespace {
 
 constexpr int kFusedVpt = EG_FUSED_VPT;               // float4 columns per thread
 constexpr int kFusedTile = kThreads * 4 * kFusedVpt;  // elements per CTA of the fused kernel
+static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
 constexpr uint64_t kStateMagic = 0x4547535441544531ull;  // "EGSTATE1"
 
 struct HostTiles {
@@ -66,6 +68,7 @@ struct eg_ctx {
     int last_cuda_error = 0;
     int last_launches = 0;
     size_t fused_smem = 0;
+    int fused_kind = EG_FUSED_PIPELINED;
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
     std::vector<cudaEvent_t> ev_pool;      // pairs
@@ -315,6 +318,15 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fused_smem);
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
+    {
+        const int pipe_smem = (int)PipeSmem::bytes(P, true);
+        cudaError_t e = cudaFuncSetAttribute(k_fused_pipe<true>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_fused_pipe<false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
+        if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
+    }
     if ((s = init_state(c)) != EG_OK) return fail(s);
     if (cudaDeviceSynchronize() != cudaSuccess) return fail(EG_ERR_CUDA);
     *out = c;
@@ -393,7 +405,16 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     // a3 + a5: dense snapshot, consensus average, SGD
     {
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
-        if (c->carry)
+        if (c->fused_kind == EG_FUSED_PIPELINED) {
+            if (c->carry)
+                k_fused_pipe<true><<<tf.n_tiles, kPipeThreads, PipeSmem::bytes(c->P, true), stream>>>(
+                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                    c->partials_fused, c->step_k, c->err);
+            else
+                k_fused_pipe<false><<<tf.n_tiles, kPipeThreads, PipeSmem::bytes(c->P, false), stream>>>(
+                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                    c->partials_fused, c->step_k, c->err);
+        } else if (c->carry)
             k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
                 params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
                 c->partials_fused, c->step_k);
@@ -505,6 +526,12 @@ eg_status eg_read_mailboxes(eg_ctx* c, float* xhat_host) {
     eg_status s = sync_and_check(c);
     if (s != EG_OK) return s;
     EG_CUDA(c, cudaMemcpy(xhat_host, c->xhat, (size_t)c->P * c->stride * sizeof(float), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_set_fused_kernel(eg_ctx* c, int kind) {
+    if (!c || (kind != EG_FUSED_PIPELINED && kind != EG_FUSED_REGISTER)) return EG_ERR_INVALID;
+    c->fused_kind = kind;
     return EG_OK;
 }
 

@@ -96,7 +96,8 @@ def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np
 def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "workload",
              gen_device: str = "cuda", tensors: Optional[Sequence[int]] = None,
              carry: bool = False, check_every: int = 1, oracle_kw: Optional[dict] = None,
-             eg_kw: Optional[dict] = None, outbox_samples: int = 8, grad_hook=None) -> Report:
+             eg_kw: Optional[dict] = None, outbox_samples: int = 8, grad_hook=None,
+             fused_kernel: int = B.FUSED_PIPELINED) -> Report:
     steps = wl.steps if steps is None else steps
     dev = torch.device("cuda")
     full = tensors is None
@@ -114,6 +115,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             ekw[key] = okw[key]
     eg = B.from_workload(wl, **ekw)
     eg.set_carry_norm(carry)
+    eg.set_fused_kernel(fused_kernel)
 
     x0 = W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)
     x_dev = eg.to_layout(x0)

@@ -16,12 +16,13 @@ RAGGED = [1, 3, 4, 5, 31, 32, 33, 1023, 1024, 1025, 4095, 4096, 4097, 10000, (1 
 INF = float("inf")
 
 
-@pytest.mark.parametrize("P", [1, 2, 3, 4, 64])
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 6, 7, 11, 64])
 @pytest.mark.parametrize("carry", [False, True])
-def test_ragged_dense(P, carry):
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
+def test_ragged_dense(P, carry, kernel):
     numel = RAGGED if P <= 4 else RAGGED[:-1]
     wl = W.synthetic(P, numel, steps=12, lr=0.1, grad_sigma=0.01)
-    rep = lockstep(wl, init="distinct", carry=carry)
+    rep = lockstep(wl, init="distinct", carry=carry, fused_kernel=kernel)
     assert rep.params_bit_exact and not rep.near_threshold
     assert 0 < rep.events < P * wl.T * wl.steps
 
@@ -60,9 +61,10 @@ def test_ragged_topk(P, frac):
     assert rep.params_bit_exact and rep.sparse_checked > 10
 
 
-def test_topk_carry_norm():
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
+def test_topk_carry_norm(kernel):
     wl = W.synthetic(4, RAGGED, steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
-    rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64)
+    rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64, fused_kernel=kernel)
     assert rep.params_bit_exact and rep.sparse_checked > 10
 
 
