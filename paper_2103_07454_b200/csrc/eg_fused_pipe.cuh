@@ -5,8 +5,8 @@
 // replicas, in ring order, into a ring of shared-memory stages with 1-D bulk asynchronous
 // copies (cp.async.bulk, completion on an mbarrier, no multicast), so the bytes in flight
 // are bounded by shared memory instead of registers; 8 consumer warps read their float4
-// column of three adjacent stages (replica j-1, j, j+1) and write the results straight to
-// global memory.  Every thread always owns the same column, so the two wrap-around operands
+// column of two adjacent stages (replica j and the contribution of replica j+1; that of
+// replica j-1 is carried in registers) and write the results straight to global memory.  Every thread always owns the same column, so the two wrap-around operands
 // (replica P-1 for replica 0, replica 0 for replica P-1) live in two extra shared buffers
 // that are private per column.
 //
@@ -18,9 +18,16 @@
 
 namespace eg {
 
-constexpr int kPipeTile = 1024;                 // elements per CTA (one float4 per consumer)
-constexpr int kPipeStages = 5;
-constexpr int kPipeThreads = kThreads + 32;     // 8 consumer warps + 1 producer warp
+#ifndef EG_PIPE_CONSUMERS
+#define EG_PIPE_CONSUMERS 256
+#endif
+#ifndef EG_PIPE_STAGES
+#define EG_PIPE_STAGES 5
+#endif
+constexpr int kPipeTile = 1024;                   // elements per CTA and stage
+constexpr int kPipeStages = EG_PIPE_STAGES;
+constexpr int kPipeConsumers = EG_PIPE_CONSUMERS; // consumer threads (+ one producer warp)
+constexpr int kPipeThreads = kPipeConsumers + 32;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
 constexpr unsigned kErrPipeTimeout = 8u;
 
@@ -71,38 +78,50 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     return true;
 }
 
-struct PipeSmem {   // offsets into dynamic shared memory, all multiples of 16
-    static constexpr int kTileBytes = kPipeTile * 4;
-    static constexpr int kStageBytes = 3 * kTileBytes;
-    static constexpr int kWrapL = kPipeStages * kStageBytes;
+struct PipeCfg {
+    int tile;        // elements per CTA and stage
+    int stages;
+    int consumers;   // consumer threads; each owns tile / (4 * consumers) float4 columns
+};
+
+// Shared-memory layout (dynamic), all offsets multiples of 16.
+template <int TILE, int STAGES>
+struct PipeSmem {
+    static constexpr int kTileBytes = TILE * 4;
+    static constexpr int kStageBytes = 3 * kTileBytes;            // x, g, x_hat
+    static constexpr int kWrapL = STAGES * kStageBytes;
     static constexpr int kWrapR = kWrapL + kTileBytes;
-    static constexpr int kBars = kWrapR + kTileBytes;              // full[S], empty[S], wrap
-    static constexpr int kFlags = kBars + 8 * (2 * kPipeStages + 1) + 8;
-    __host__ __device__ static size_t bytes(int P, bool carry) {
-        size_t b = kFlags + 16 + ((2 * (size_t)P + 15) & ~(size_t)15);
-        if (carry) b += (size_t)P * kWarps * sizeof(double);
+    static constexpr int kBars = kWrapR + kTileBytes;             // full[S], empty[S], wrap
+    static constexpr int kFlags = kBars + 8 * (2 * STAGES + 1) + 8;
+    __host__ __device__ static size_t bytes(int P, bool carry, int consumer_warps) {
+        size_t b = kFlags + 16 + (((size_t)P + 15) & ~(size_t)15);
+        if (carry) b += (size_t)P * consumer_warps * sizeof(double);
         return b;
     }
 };
 
-// grid n_tiles (tile table with kPipeTile elements per tile), kPipeThreads threads.
-template <bool CARRY>
-__global__ void __launch_bounds__(kPipeThreads)
+// grid n_tiles (tile table with TILE elements per tile), CONSUMERS + 32 threads.
+// COLS = TILE / (4 * CONSUMERS) float4 columns per consumer thread.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY>
+__global__ void __launch_bounds__(CONSUMERS + 32)
 k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
              long long* step_k, unsigned int* __restrict__ err) {
+    using L = PipeSmem<TILE, STAGES>;
+    constexpr int COLS = TILE / (4 * CONSUMERS);
+    constexpr int CWARPS = CONSUMERS / 32;
+    static_assert(COLS * 4 * CONSUMERS == TILE, "tile must be covered exactly");
     extern __shared__ __align__(128) unsigned char smem[];
     float* stages = reinterpret_cast<float*>(smem);
-    float* wrap_l = reinterpret_cast<float*>(smem + PipeSmem::kWrapL);   // contribution of replica P-1
-    float* wrap_r = reinterpret_cast<float*>(smem + PipeSmem::kWrapR);   // contribution of replica 0
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + PipeSmem::kBars);
-    uint64_t* empty = full + kPipeStages;
-    uint64_t* wrap_bar = empty + kPipeStages;
-    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + PipeSmem::kFlags);
-    uint8_t* s_snap = smem + PipeSmem::kFlags + 16;
-    uint8_t* s_valid = s_snap + P;
-    double* s_red = reinterpret_cast<double*>(s_snap + ((2 * P + 15) & ~15));
+    float* wrap_l = reinterpret_cast<float*>(smem + L::kWrapL);   // contribution of replica P-1
+    float* wrap_r = reinterpret_cast<float*>(smem + L::kWrapR);   // contribution of replica 0
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBars);
+    uint64_t* empty = full + STAGES;
+    uint64_t* wrap_bar = empty + STAGES;
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kFlags);
+    uint8_t* s_mode = smem + L::kFlags + 16;                      // bit 0: dense message, bit 1: valid
+    double* s_red = reinterpret_cast<double*>(s_mode + ((P + 15) & ~15));
 
     const int tile = blockIdx.x, tid = threadIdx.x;
     const int t = tt.tensor[tile];
@@ -110,14 +129,12 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
     const long long off = tt.offset[tile];
     const uint32_t copy_bytes = (uint32_t)(((len + 3) & ~3) * 4);
 
-    for (int j = tid; j < P; j += kPipeThreads) {
-        s_snap[j] = snap[(long long)j * T + t];
-        s_valid[j] = valid[(long long)j * T + t];
-    }
+    for (int j = tid; j < P; j += CONSUMERS + 32)
+        s_mode[j] = (uint8_t)((snap[(long long)j * T + t] ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0));
     if (tid == 0) {
-        for (int s = 0; s < kPipeStages; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], kWarps);
+            mbar_init(&empty[s], CWARPS);
         }
         mbar_init(wrap_bar, 1);
         *s_abort = 0;
@@ -126,98 +143,132 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
     }
     __syncthreads();
 
-    const bool snap_last = s_snap[P - 1] != 0;
+    const bool snap_last = (s_mode[P - 1] & 1) != 0;
     // Replica P-1 contributes wrap_l; its own stage then only needs what wrap_l does not hold.
     const bool last_opt = P >= 2;
 
-    if (tid >= kThreads) {
+    if (tid >= CONSUMERS) {
         // ------------------------------------------------------------------ producer
-        if (tid == kThreads) {
-            const long long lb = (long long)(P - 1) * stride + off;
+        if (tid == CONSUMERS) {
+            const float* xp = x + off;
+            const float* gp = g + off;
+            const float* hp = xhat + off;
             mbar_expect_tx(wrap_bar, copy_bytes);
-            bulk_g2s(wrap_l, (snap_last ? x : xhat) + lb, copy_bytes, wrap_bar);
+            bulk_g2s(wrap_l, (snap_last ? xp : hp) + (long long)(P - 1) * stride, copy_bytes, wrap_bar);
+            int s = 0;
+            uint32_t wait_parity = 1;     // parity of the phase before the one to wait for
             for (int j = 0; j < P; ++j) {
-                const int s = j % kPipeStages;
-                if (j >= kPipeStages &&
-                    !mbar_wait_bounded(&empty[s], (uint32_t)((j / kPipeStages - 1) & 1), s_abort, err))
-                    break;
-                float* st = stages + (size_t)s * 3 * kPipeTile;
-                const long long rb = (long long)j * stride + off;
-                const bool sn = s_snap[j] != 0;
+                if (j >= STAGES && !mbar_wait_bounded(&empty[s], wait_parity, s_abort, err)) break;
+                float* st = stages + s * (3 * TILE);
+                const bool sn = (s_mode[j] & 1) != 0;
                 const bool is_last = last_opt && (j == P - 1);
                 const bool need_x = !(is_last && sn);
                 const bool need_h = !sn && !is_last;
                 mbar_expect_tx(&full[s], copy_bytes * (1u + (need_x ? 1u : 0u) + (need_h ? 1u : 0u)));
-                bulk_g2s(st + kPipeTile, g + rb, copy_bytes, &full[s]);
-                if (need_x) bulk_g2s(st, x + rb, copy_bytes, &full[s]);
-                if (need_h) bulk_g2s(st + 2 * kPipeTile, xhat + rb, copy_bytes, &full[s]);
+                bulk_g2s(st + TILE, gp, copy_bytes, &full[s]);
+                if (need_x) bulk_g2s(st, xp, copy_bytes, &full[s]);
+                if (need_h) bulk_g2s(st + 2 * TILE, hp, copy_bytes, &full[s]);
+                xp += stride; gp += stride; hp += stride;
+                if (++s == STAGES) { s = 0; wait_parity ^= 1u; }
             }
         }
     } else {
         // ------------------------------------------------------------------ consumers
-        const int c = tid * 4;
-        const int nel = min(4, max(0, len - c));
         const int lane = tid & 31, warp = tid >> 5;
+        int nel[COLS];
+#pragma unroll
+        for (int v = 0; v < COLS; ++v) nel[v] = min(4, max(0, len - (v * CONSUMERS + tid) * 4));
+        const int c0 = tid * 4;                      // column v starts at c0 + v * 4 * CONSUMERS
         const double neg_lr = -(double)lr;
+        const double w_one = 1.0, w_half = 0.5, w_third = __ddiv_rn(1.0, 3.0);
         const bool has_left = P >= 2, has_right = P >= 3;
+        // contributions of replica j-1 and j to their neighbours, for this thread's columns,
+        // kept as doubles so that every value is converted once
+        double hp[COLS][4], hc[COLS][4];
         bool ok = mbar_wait_bounded(wrap_bar, 0, s_abort, err) &&
                   mbar_wait_bounded(&full[0], 0, s_abort, err);
+        unsigned mode_prev = s_mode[P - 1], mode_cur = s_mode[0];
+#pragma unroll
+        for (int v = 0; v < COLS; ++v) {
+            const int c = c0 + v * 4 * CONSUMERS;
+            const float4 a = ok ? *reinterpret_cast<const float4*>(wrap_l + c) : make_float4(0, 0, 0, 0);
+            const float4 b = ok ? *reinterpret_cast<const float4*>(((mode_cur & 1) ? stages : stages + 2 * TILE) + c)
+                                : make_float4(0, 0, 0, 0);
+            hp[v][0] = a.x; hp[v][1] = a.y; hp[v][2] = a.z; hp[v][3] = a.w;
+            hc[v][0] = b.x; hc[v][1] = b.y; hc[v][2] = b.z; hc[v][3] = b.w;
+        }
+        int s = 0, s1 = (STAGES > 1) ? 1 : 0;
+        uint32_t parity1 = (STAGES > 1) ? 0u : 1u;   // phase parity of the fill of stage s1 for j+1
+        float* xo = x + off + c0;                    // output pointers of replica j
+        float* ho = xhat + off + c0;
         for (int j = 0; ok && j < P; ++j) {
-            const int s = j % kPipeStages;
-            if (j + 1 < P) {
-                ok = mbar_wait_bounded(&full[(j + 1) % kPipeStages],
-                                       (uint32_t)(((j + 1) / kPipeStages) & 1), s_abort, err);
+            const bool more = j + 1 < P;
+            if (more) {
+                ok = mbar_wait_bounded(&full[s1], parity1, s_abort, err);
                 if (!ok) break;
             }
-            const float* st = stages + (size_t)s * 3 * kPipeTile;
-            const bool sn = s_snap[j] != 0;
-            const bool is_last = last_opt && (j == P - 1);
-            // where the operands of replica j sit
-            const float* xs = (is_last && sn) ? wrap_l : st;
-            const float* hs = is_last ? wrap_l : (sn ? st : st + 2 * kPipeTile);
-            const float* hl_s;
-            const float* hr_s;
-            if (j == 0) {
-                hl_s = wrap_l;
-            } else {
-                const float* sp = stages + (size_t)((j - 1) % kPipeStages) * 3 * kPipeTile;
-                hl_s = (s_snap[j - 1] != 0) ? sp : sp + 2 * kPipeTile;
-            }
-            if (j + 1 == P) {
-                hr_s = wrap_r;
-            } else if (last_opt && j + 1 == P - 1) {
-                hr_s = wrap_l;
-            } else {
-                const float* sq = stages + (size_t)((j + 1) % kPipeStages) * 3 * kPipeTile;
-                hr_s = (s_snap[j + 1] != 0) ? sq : sq + 2 * kPipeTile;
-            }
-            const int jl = (j == 0) ? P - 1 : j - 1, jr = (j + 1 == P) ? 0 : j + 1;
-            const bool ul = has_left && s_valid[jl] != 0;
-            const bool ur = has_right && s_valid[jr] != 0;
-            const double w = __ddiv_rn(1.0, (double)(1 + (ul ? 1 : 0) + (ur ? 1 : 0)));
+            const unsigned mode_next = s_mode[more ? j + 1 : 0];
+            const float* st = stages + s * (3 * TILE);
+            const bool sn = (mode_cur & 1) != 0;
+            const bool is_last = last_opt && !more;
+            // fp32 copy of this replica's contribution (its old x when it sends a dense message)
+            const float* hs = is_last ? wrap_l : (sn ? st : st + 2 * TILE);
+            // contribution of replica j+1
+            const float* sq = stages + s1 * (3 * TILE);
+            const float* hn_s = !more ? wrap_r
+                                      : ((last_opt && j + 2 == P) ? wrap_l
+                                                                  : ((mode_next & 1) ? sq : sq + 2 * TILE));
+            const bool ul = has_left && (mode_prev & 2) != 0;
+            const bool ur = has_right && (mode_next & 2) != 0;
+            const double w = (ul && ur) ? w_third : ((ul || ur) ? w_half : w_one);
             double acc = 0.0;
-            if (nel > 0) {
-                const float4 xc = *reinterpret_cast<const float4*>(xs + c);
-                const float4 gc = *reinterpret_cast<const float4*>(st + kPipeTile + c);
-                const float4 hc = *reinterpret_cast<const float4*>(hs + c);
-                const float4 hl = *reinterpret_cast<const float4*>(hl_s + c);
-                const float4 hr = *reinterpret_cast<const float4*>(hr_s + c);
-                if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hc;   // private to this thread
-                const long long rb = (long long)j * stride + off + c;
-                const float4 xn = upd4(xc, gc, hl, hr, ul, ur, w, neg_lr);
-                store_masked(x + rb, xn, nel);
-                if (sn) store_masked(xhat + rb, xc, nel);
-                if (CARRY) acc = sq_diff4(xn, hc, nel, acc);
+#pragma unroll
+            for (int v = 0; v < COLS; ++v) {
+                if (nel[v] > 0) {
+                    const int c = c0 + v * 4 * CONSUMERS;
+                    const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
+                    const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
+                    const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
+                    if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;   // private to this thread
+                    const double hn[4] = {(double)hnf.x, (double)hnf.y, (double)hnf.z, (double)hnf.w};
+                    const double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
+                    double xd[4];
+                    if (sn) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) xd[q] = hc[v][q];
+                    } else {
+                        const float4 xf = *reinterpret_cast<const float4*>(st + c);
+                        xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
+                    }
+                    float xn[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        double sum = xd[q];
+                        if (ul) sum = __dadd_rn(sum, hp[v][q]);
+                        if (ur) sum = __dadd_rn(sum, hn[q]);
+                        xn[q] = __double2float_rn(__fma_rn(neg_lr, gd[q], __dmul_rn(sum, w)));
+                    }
+                    const float4 xn4 = make_float4(xn[0], xn[1], xn[2], xn[3]);
+                    store_masked(xo + v * 4 * CONSUMERS, xn4, nel[v]);
+                    if (sn) store_masked(ho + v * 4 * CONSUMERS, hcf, nel[v]);
+                    if (CARRY) acc = sq_diff4(xn4, hcf, nel[v], acc);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) { hp[v][q] = hc[v][q]; hc[v][q] = hn[q]; }
+                }
             }
             if (CARRY) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1)
                     acc = __dadd_rn(acc, __shfl_down_sync(0xffffffffu, acc, o));
-                if (lane == 0) s_red[j * kWarps + warp] = acc;
+                if (lane == 0) s_red[j * CWARPS + warp] = acc;
             }
-            // replica j-1 is not needed any more
+            // everything later iterations need from this stage now sits in registers
             __syncwarp();
-            if (lane == 0 && j >= 1) mbar_arrive(&empty[(j - 1) % kPipeStages]);
+            if (lane == 0) mbar_arrive(&empty[s]);
+            xo += stride; ho += stride;
+            mode_prev = mode_cur; mode_cur = mode_next;
+            s = s1;
+            if (++s1 == STAGES) { s1 = 0; parity1 ^= 1u; }
         }
     }
     if (*s_abort) {
@@ -227,10 +278,10 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
     }
     if (CARRY) {
         __syncthreads();
-        for (int j = tid; j < P; j += kPipeThreads) {
+        for (int j = tid; j < P; j += CONSUMERS + 32) {
             double r = 0.0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) r = __dadd_rn(r, s_red[j * kWarps + w]);
+            for (int w = 0; w < CWARPS; ++w) r = __dadd_rn(r, s_red[j * CWARPS + w]);
             partials[(long long)j * tt.n_tiles + tile] = r;
         }
     }

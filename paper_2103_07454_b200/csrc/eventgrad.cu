@@ -21,6 +21,7 @@ namespace {
 
 constexpr int kFusedVpt = EG_FUSED_VPT;               // float4 columns per thread
 constexpr int kFusedTile = kThreads * 4 * kFusedVpt;  // elements per CTA of the fused kernel
+using PipeLayout = PipeSmem<kPipeTile, kPipeStages>;
 static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
 constexpr uint64_t kStateMagic = 0x4547535441544531ull;  // "EGSTATE1"
 
@@ -319,11 +320,11 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
     {
-        const int pipe_smem = (int)PipeSmem::bytes(P, true);
-        cudaError_t e = cudaFuncSetAttribute(k_fused_pipe<true>,
+        const int pipe_smem = (int)PipeLayout::bytes(P, true, kPipeConsumers / 32);
+        cudaError_t e = cudaFuncSetAttribute(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k_fused_pipe<false>,
+            e = cudaFuncSetAttribute(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
@@ -407,11 +408,13 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
         if (c->fused_kind == EG_FUSED_PIPELINED) {
             if (c->carry)
-                k_fused_pipe<true><<<tf.n_tiles, kPipeThreads, PipeSmem::bytes(c->P, true), stream>>>(
+                k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
+                    <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, true, kPipeConsumers / 32), stream>>>(
                     params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
                     c->partials_fused, c->step_k, c->err);
             else
-                k_fused_pipe<false><<<tf.n_tiles, kPipeThreads, PipeSmem::bytes(c->P, false), stream>>>(
+                k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>
+                    <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                     params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
                     c->partials_fused, c->step_k, c->err);
         } else if (c->carry)
