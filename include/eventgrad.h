@@ -173,6 +173,40 @@ eg_status eg_average_model(eg_ctx* ctx, const float* params, float* avg_dev,
 eg_status eg_export_state(eg_ctx* ctx, void* host_buf, size_t* bytes);
 eg_status eg_import_state(eg_ctx* ctx, const void* host_buf, size_t bytes);
 
+/* Change norms without any allocation.  (The paper has no counterpart: this is a service
+ * entry point of the library, not a step of the method.)
+ *
+ * Some callers may not allocate device memory at the moment they need the norms: code that
+ * runs while a stream is being captured, code inside a framework whose memory pool forbids
+ * raw cudaMalloc / cudaFree (both also synchronise the whole device), or a control loop with
+ * a hard latency budget.  For them this call computes
+ *     norms_dev[i*T + t] = || x[i][t] - x_hat[i][t] ||_2        (fp64, device array of P*T)
+ * exactly as the norm pass of eg_step does (same tiles, same summation order, hence the same
+ * bits), without a context and without allocating: the tensor table is passed by value to
+ * the kernels and the per-tile partial sums go to a fixed array of
+ * EG_STATIC_MAX_PARTIALS doubles (4 MiB) that is part of the library's device image -- every
+ * GPU that loads the library holds that array until the process exits.
+ *
+ * x_dev, xhat_dev: device, fp32, [P][replica_stride], 16-byte aligned; replica_stride and
+ * every tensor_offset_host[t] multiples of 4 elements (no padding between tensors needed).
+ * tensor_offset_host, layer_numel_host: host arrays of T entries.  Enqueues two kernels on
+ * `stream` and returns; it never synchronises.
+ *
+ * Limits, checked before anything is launched (EG_ERR_INVALID): T <= EG_STATIC_MAX_TENSORS,
+ * and P * sum_t ceil(n_t / 4096) <= EG_STATIC_MAX_PARTIALS.
+ *
+ * The first call on each device looks up the device address of the scratch array (a runtime
+ * query, no allocation); make that first call outside any stream capture.  All calls on one
+ * device share the scratch array: each call overwrites the part it uses (nothing has to be
+ * cleared beforehand), so two calls whose kernels may overlap on the GPU (different streams)
+ * race with each other -- keep them on one stream or order them with events. */
+#define EG_STATIC_MAX_TENSORS 192
+#define EG_STATIC_MAX_PARTIALS 524288
+eg_status eg_change_norms_static(const float* x_dev, const float* xhat_dev, int P,
+                                 int64_t replica_stride, const int64_t* tensor_offset_host,
+                                 const int64_t* layer_numel_host, int T, double* norms_dev,
+                                 void* stream);
+
 /* Back to iteration 0 with empty mailboxes, initial thresholds and zero counters. */
 eg_status eg_reset(eg_ctx* ctx);
 void eg_destroy(eg_ctx* ctx);

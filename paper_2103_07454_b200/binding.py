@@ -26,8 +26,10 @@ EXPORTS = [
     "eg_event_count", "eg_last_decisions", "eg_thresholds", "eg_last_outbox", "eg_topk_count",
     "eg_read_mailboxes", "eg_average_model", "eg_export_state", "eg_import_state", "eg_reset",
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
-    "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel",
+    "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static",
 ]
+STATIC_MAX_TENSORS = 192
+STATIC_MAX_PARTIALS = 524288
 FUSED_PIPELINED = 0
 FUSED_REGISTER = 1
 KERNEL_GROUPS = ("norm", "decide", "topk", "fused")
@@ -80,6 +82,7 @@ def load_library() -> C.CDLL:
     lib.eg_reset.argtypes = [vp]
     lib.eg_set_timing.argtypes = [vp, C.c_int]
     lib.eg_set_fused_kernel.argtypes = [vp, C.c_int]
+    lib.eg_change_norms_static.argtypes = [vp, vp, C.c_int, C.c_int64, i64p, i64p, C.c_int, vp, vp]
     lib.eg_kernel_times.argtypes = [vp, C.POINTER(C.c_double), u64p]
     lib.eg_destroy.argtypes = [vp]
     lib.eg_destroy.restype = None
@@ -274,6 +277,30 @@ class EventGrad:
     @property
     def last_launch_count(self) -> int:
         return int(self._lib.eg_last_launch_count(self._h))
+
+
+def change_norms_static(x: torch.Tensor, xhat: torch.Tensor, tensor_offset: Sequence[int],
+                        layer_numel: Sequence[int], out: torch.Tensor,
+                        stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """``eg_change_norms_static``: || x - x_hat || of every (replica, tensor) into ``out``
+    (float64 device tensor of ``P*T`` entries) without allocating anything.  ``x`` and ``xhat``
+    are ``[P, replica_stride]`` fp32 device tensors.  Raises EventGradError if the sizes exceed
+    the library's fixed scratch."""
+    lib = load_library()
+    assert x.is_cuda and xhat.is_cuda and out.is_cuda and out.dtype == torch.float64
+    assert x.dtype == xhat.dtype == torch.float32 and x.shape == xhat.shape and x.dim() == 2
+    assert x.is_contiguous() and xhat.is_contiguous() and out.is_contiguous()
+    T = len(layer_numel)
+    assert out.numel() == x.shape[0] * T
+    offs = (C.c_int64 * T)(*[int(o) for o in tensor_offset])
+    nums = (C.c_int64 * T)(*[int(n) for n in layer_numel])
+    s = stream if stream is not None else torch.cuda.current_stream(x.device)
+    with torch.cuda.device(x.device):
+        st = lib.eg_change_norms_static(x.data_ptr(), xhat.data_ptr(), int(x.shape[0]),
+                                        int(x.shape[1]), offs, nums, T, out.data_ptr(),
+                                        C.c_void_p(s.cuda_stream))
+    _check(lib, st, None, "eg_change_norms_static")
+    return out
 
 
 def from_workload(wl, **overrides) -> EventGrad:
