@@ -304,6 +304,11 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         EG_ALLOC(c->tk.hist, S * kMaxBins);
         EG_ALLOC(c->tk.prefix, S); EG_ALLOC(c->tk.remaining, S);
         EG_ALLOC(c->tk.tile_count, (size_t)P * c->tiles_norm.n_tiles);
+        EG_ALLOC(c->tk.tile_cand, (size_t)P * c->tiles_norm.n_tiles);
+        EG_ALLOC(c->tk.cand, (size_t)P * c->stride);
+        EG_ALLOC(c->tk.plan, 1);
+        EG_ALLOC(c->tk.sp_seg, S);
+        EG_ALLOC(c->tk.sp_begin, S + 1);
         EG_ALLOC(c->tk.outbox, (size_t)P * c->out_stride);
         c->tk.out_off = c->d_out_off;
         c->tk.count = c->d_kcount;
@@ -388,20 +393,19 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     // a4: Top-K select / pack / scatter for the segments that send a sparse message
     if (c->topk.enabled) {
         TimedSection ts(c, stream, EG_KERNEL_TOPK);
-        for (int digit = 0; digit < 3; ++digit) {
-            k_topk_hist<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
-                                                           c->st.sparse, c->tk, digit);
-            k_topk_pick<<<S, kThreads, 0, stream>>>(c->T, c->st.sparse, c->tk, digit);
-            launches += 2;
+        k_topk_plan<<<1, kPlanThreads, 0, stream>>>(S, c->T, c->st.sparse, tn.seg_begin, c->tk);
+        k_topk_hist<false><<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk, 0);
+        k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(c->T, c->tk, 0);
+        k_topk_collect<<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk);
+        for (int digit = 1; digit < 3; ++digit) {
+            k_topk_hist<true><<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk, digit);
+            k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(c->T, c->tk, digit);
         }
-        k_topk_count<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
-                                                        c->st.sparse, c->tk);
-        k_topk_scan<<<S, kThreads, 0, stream>>>(tn, c->T, c->st.sparse, c->tk);
-        k_topk_write<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride,
-                                                        c->st.sparse, c->tk, c->err);
-        k_topk_scatter<<<grid_norm, kThreads, 0, stream>>>(c->xhat, tn, c->T, c->stride,
-                                                          c->st.sparse, c->tk, c->d_numel, c->err);
-        launches += 4;
+        k_topk_count<<<kTopkGrid, kThreads, 0, stream>>>(tn, c->T, c->stride, c->tk);
+        k_topk_scan<<<kTopkSegGrid, kThreads, 0, stream>>>(tn, c->T, c->tk);
+        k_topk_write<<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk, c->err);
+        k_topk_scatter<<<kTopkGrid, kThreads, 0, stream>>>(c->xhat, tn, c->T, c->stride, c->tk, c->d_numel, c->err);
+        launches += 12;
     }
     // a3 + a5: dense snapshot, consensus average, SGD
     {
