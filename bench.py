@@ -348,7 +348,7 @@ def run_native(args):
 
     fused_ms = main["kernel_ms"]["fused"]
     achieved = elems * FUSED_BYTES_PER_ELEMENT / fused_ms / 1e6 if fused_ms else None
-    roofline = {"bound": "hbm", "kernel": "k_fused", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "k_fused_pipe", "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
                 "traffic": FUSED_TRAFFIC.get(kernel_source_hash()),

@@ -1,16 +1,16 @@
 // Top-K messages (Top-K paragraph of Section 7): for every segment whose event sends a
 // sparse message, find exactly the K_t entries with the largest |x - x_hat| (ties to the lower
 // index), pack them as (index, value) in ascending index order into the replica's outbox,
-// and scatter them into the mailbox x_hat "on receipt".
+// and deliver them into the mailbox x_hat.
 //
 // The rank key is the bit pattern of |x - x_hat| (fp32), which orders like the magnitude.
 // The K_t-th largest key tau is found by radix select over three digits (11 + 10 + 10 bits):
 //   pass A  (reads x, x_hat)  histogram of the top digit                     -> bin b0
 //   pass B  (reads x, x_hat)  keys whose top digit is b0 ("candidates") are copied, tile by
-//                             tile, into a candidate buffer; keys above b0 are counted per tile
-//   digits 1 and 2            histograms over the candidates only (a few percent of the data)
-//   per-tile counts           from the candidates only
-//   pass C  (reads x, x_hat)  ordered compaction into the outbox
+//                             tile, into a candidate buffer; keys above b0 are counted per tile;
+//                             digit 1 of the candidates is histogrammed on the way
+//   digit 2, per-tile counts  from the candidates only (a few percent of the data)
+//   pass C  (reads x, x_hat)  ordered compaction into the outbox and delivery into x_hat
 // so a sparse message costs three passes over its tensor.  The host knows nothing about the
 // decisions: a one-CTA planning kernel turns the device-side `sparse` flags into a compact list
 // of work tiles, and every other kernel runs a fixed-size grid over that list (an empty list
@@ -51,7 +51,6 @@ __device__ __forceinline__ unsigned int rank_key(float a, float b) {
 }
 
 // digit 0: bits 30..20, digit 1: bits 19..10, digit 2: bits 9..0
-__device__ __forceinline__ int digit_shift(int digit) { return digit == 0 ? 20 : (digit == 1 ? 10 : 0); }
 __device__ __forceinline__ int digit_bits(int digit) { return digit == 0 ? kDigitBits0 : kDigitBits1; }
 
 // One CTA: compact list of the sparse segments and of their tiles, in segment order.
@@ -111,53 +110,65 @@ __device__ __forceinline__ WorkRange work_range(const TopkState& tk) {
     return r;
 }
 
-// Pass A and the two candidate passes: histogram of one digit.
-// CANDIDATES == false: over the keys of the tile (digit 0).
-// CANDIDATES == true : over the candidate keys of the tile that match the resolved prefix.
-template <bool CANDIDATES>
+// Walks a CTA's share of the work list.  Segment-level values are re-read only when the
+// segment changes, so consecutive tiles of one tensor cost two dependent loads, not six.
+struct WorkCursor {
+    int q, end, s, i, t, first_tile, begin;
+    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int q0) {
+        q = q0 - 1;
+        end = -1;
+        (void)tk; (void)tt; (void)T;
+    }
+    // returns the tile id of work item w; `changed` tells whether a new segment started
+    __device__ __forceinline__ int advance(const TopkState& tk, const TileTable& tt, int T, int w,
+                                           bool& changed) {
+        changed = false;
+        while (w >= end) {
+            ++q;
+            begin = tk.sp_begin[q];
+            end = tk.sp_begin[q + 1];
+            changed = true;
+        }
+        if (changed) {
+            s = tk.sp_seg[q];
+            i = s / T;
+            t = s - i * T;
+            first_tile = tt.seg_begin[t];
+        }
+        return first_tile + (w - begin);
+    }
+};
+
+// Pass A: histogram of the top digit of every key of the work tiles.
 __global__ void __launch_bounds__(kThreads)
 k_topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
-            long long stride, TopkState tk, int digit) {
+            long long stride, TopkState tk) {
     __shared__ unsigned int s_hist[kMaxBins];
     WorkRange r = work_range(tk);
     if (r.w0 >= r.w1) return;
-    const int nbins = 1 << digit_bits(digit);
-    const int shift = digit_shift(digit);
-    const int hi_shift = shift + digit_bits(digit);
-    for (int b = threadIdx.x; b < nbins; b += kThreads) s_hist[b] = 0;
+    for (int b = threadIdx.x; b < kMaxBins; b += kThreads) s_hist[b] = 0;
     __syncthreads();
-    int q = r.q;
+    WorkCursor cur;
+    cur.init(tk, tt, T, r.q);
     for (int w = r.w0; w < r.w1; ++w) {
-        while (w >= tk.sp_begin[q + 1]) ++q;
-        const int s = tk.sp_seg[q];
-        const int i = s / T, t = s - i * T;
-        const int tile = tt.seg_begin[t] + (w - tk.sp_begin[q]);
-        if (!CANDIDATES) {
-            const int len = tt.length[tile];
-            const long long base = (long long)i * stride + tt.offset[tile];
-            for (int local = threadIdx.x * 4; local < len; local += kThreads * 4) {
-                const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
-                const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
-                                           rank_key(a.w, b.w)};
-                const int nel = min(4, len - local);
+        bool changed;
+        const int tile = cur.advance(tk, tt, T, w, changed);
+        const int len = tt.length[tile];
+        const long long base = (long long)cur.i * stride + tt.offset[tile];
+        for (int local = threadIdx.x * 4; local < len; local += kThreads * 4) {
+            const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
+            const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
+                                       rank_key(a.w, b.w)};
+            const int nel = min(4, len - local);
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (c < nel) atomicAdd(&s_hist[(k[c] >> shift) & (nbins - 1)], 1u);
-            }
-        } else {
-            const unsigned int want = tk.prefix[s];
-            const unsigned int* cd = tk.cand + (long long)i * stride + tt.offset[tile];
-            const int n = tk.tile_cand[(long long)i * tt.n_tiles + tile];
-            for (int e = threadIdx.x; e < n; e += kThreads) {
-                const unsigned int k = cd[e];
-                if ((k >> hi_shift) == want) atomicAdd(&s_hist[(k >> shift) & (nbins - 1)], 1u);
-            }
+            for (int c = 0; c < 4; ++c)
+                if (c < nel) atomicAdd(&s_hist[k[c] >> 20], 1u);
         }
         // flush when the next tile belongs to another segment (or this was the last one)
-        if (w + 1 == r.w1 || w + 1 >= tk.sp_begin[q + 1]) {
+        if (w + 1 == r.w1 || w + 1 >= cur.end) {
             __syncthreads();
-            unsigned int* gh = tk.hist + (long long)s * kMaxBins;
-            for (int b = threadIdx.x; b < nbins; b += kThreads) {
+            unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
+            for (int b = threadIdx.x; b < kMaxBins; b += kThreads) {
                 const unsigned int v = s_hist[b];
                 if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
             }
@@ -170,11 +181,11 @@ k_topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTab
 // largest key downwards; clear the histogram for the next digit.
 __global__ void __launch_bounds__(kThreads)
 k_topk_pick(int T, TopkState tk, int digit) {
-    __shared__ unsigned int s_sum[kThreads];
-    __shared__ unsigned int s_above[kThreads];
+    __shared__ unsigned int s_warp[kWarps];
     const int nq = tk.plan->n_sparse;
     const int nbins = 1 << digit_bits(digit);
     const int per = nbins / kThreads;                      // 8 or 4 bins per thread
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int q = blockIdx.x; q < nq; q += gridDim.x) {
         const int s = tk.sp_seg[q];
         const int t = s % T;
@@ -183,15 +194,20 @@ k_topk_pick(int T, TopkState tk, int digit) {
         unsigned int c[8];
         unsigned int mine = 0;
         for (int z = 0; z < per; ++z) { c[z] = gh[top - z]; mine += c[z]; gh[top - z] = 0; }
-        s_sum[threadIdx.x] = mine;
-        __syncthreads();
-        if (threadIdx.x == 0) {                            // exclusive scan from the top
-            unsigned int run = 0;
-            for (int z = 0; z < kThreads; ++z) { s_above[z] = run; run += s_sum[z]; }
+        // exclusive scan of `mine` over the CTA, from the highest bins down
+        unsigned int inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
         }
+        if (lane == 31) s_warp[warp] = inc;
         __syncthreads();
+        unsigned int above = inc - mine;
+#pragma unroll
+        for (int u = 0; u < kWarps; ++u)
+            if (u < warp) above += s_warp[u];
         const unsigned int rem = (digit == 0) ? (unsigned int)tk.count[t] : tk.remaining[s];
-        unsigned int above = s_above[threadIdx.x];
         if (above < rem && rem <= above + mine) {
             for (int z = 0; z < per; ++z) {
                 if (rem <= above + c[z]) {
@@ -208,20 +224,26 @@ k_topk_pick(int T, TopkState tk, int digit) {
 }
 
 // Pass B: per tile, copy the keys whose top digit equals the chosen bin into the tile's slice
-// of the candidate buffer (order inside the tile is irrelevant for selecting tau) and count the
-// keys whose top digit is larger.
-__global__ void __launch_bounds__(kThreads)
+// of the candidate buffer (order inside the tile is irrelevant for selecting tau), count the
+// keys whose top digit is larger, and histogram digit 1 of the candidates.
+__global__ void __launch_bounds__(kThreads, 4)
 k_topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
                long long stride, TopkState tk) {
+    constexpr int kBins1 = 1 << kDigitBits1;
+    __shared__ unsigned int s_hist[kBins1];
     __shared__ unsigned int s_n, s_gt;
     WorkRange r = work_range(tk);
-    int q = r.q;
+    if (r.w0 >= r.w1) return;
+    for (int b = threadIdx.x; b < kBins1; b += kThreads) s_hist[b] = 0;
+    __syncthreads();
+    WorkCursor cur;
+    cur.init(tk, tt, T, r.q);
+    unsigned int b0 = 0;
     for (int w = r.w0; w < r.w1; ++w) {
-        while (w >= tk.sp_begin[q + 1]) ++q;
-        const int s = tk.sp_seg[q];
-        const int i = s / T, t = s - i * T;
-        const int tile = tt.seg_begin[t] + (w - tk.sp_begin[q]);
-        const unsigned int b0 = tk.prefix[s];
+        bool changed;
+        const int tile = cur.advance(tk, tt, T, w, changed);
+        if (changed) b0 = tk.prefix[cur.s];
+        const int i = cur.i, s = cur.s;
         const int len = tt.length[tile];
         const long long base = (long long)i * stride + tt.offset[tile];
         unsigned int* cd = tk.cand + base;
@@ -238,7 +260,10 @@ k_topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, Tile
                 if (c < nel) {
                     const unsigned int d0 = k[c] >> 20;
                     gt += (d0 > b0);
-                    if (d0 == b0) cd[atomicAdd(&s_n, 1u)] = k[c];
+                    if (d0 == b0) {
+                        cd[atomicAdd(&s_n, 1u)] = k[c];
+                        atomicAdd(&s_hist[(k[c] >> 10) & (kBins1 - 1)], 1u);
+                    }
                 }
             }
         }
@@ -250,28 +275,68 @@ k_topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, Tile
             tk.tile_cand[(long long)i * tt.n_tiles + tile] = (int)s_n;
             tk.tile_count[(long long)i * tt.n_tiles + tile] = make_uint2(s_gt, 0u);
         }
+        if (w + 1 == r.w1 || w + 1 >= cur.end) {   // last tile of this segment here
+            unsigned int* gh = tk.hist + (long long)s * kMaxBins;
+            for (int b = threadIdx.x; b < kBins1; b += kThreads) {
+                const unsigned int v = s_hist[b];
+                if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
+            }
+        }
         __syncthreads();
     }
 }
 
-// Per tile, from its candidates only: keys greater than / equal to tau.
+// Work tile number w of this step (used by the one-warp-per-tile kernels).
+struct WarpTile {
+    int s, i, t, tile;
+};
+__device__ __forceinline__ WarpTile warp_tile(const TopkState& tk, const TileTable& tt, int T, int w) {
+    int lo = 0, hi = tk.plan->n_sparse - 1;      // last q with sp_begin[q] <= w
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (tk.sp_begin[mid] <= w) lo = mid; else hi = mid - 1;
+    }
+    WarpTile r;
+    r.s = tk.sp_seg[lo];
+    r.i = r.s / T;
+    r.t = r.s - r.i * T;
+    r.tile = tt.seg_begin[r.t] + (w - tk.sp_begin[lo]);
+    return r;
+}
+
+// Digit 2 over the candidates: one warp per tile, global histogram updated directly (only the
+// candidates that match the 21 resolved bits take part: about one in a thousand).
+__global__ void __launch_bounds__(kThreads)
+k_topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk) {
+    const int total = tk.plan->total_tiles;
+    const int lane = threadIdx.x & 31;
+    const int nwarps = gridDim.x * kWarps;
+    for (int w = blockIdx.x * kWarps + (threadIdx.x >> 5); w < total; w += nwarps) {
+        const WarpTile z = warp_tile(tk, tt, T, w);
+        const unsigned int want = tk.prefix[z.s];
+        const unsigned int* cd = tk.cand + (long long)z.i * stride + tt.offset[z.tile];
+        const int n = tk.tile_cand[(long long)z.i * tt.n_tiles + z.tile];
+        unsigned int* gh = tk.hist + (long long)z.s * kMaxBins;
+        for (int e = lane; e < n; e += 32) {
+            const unsigned int k = cd[e];
+            if ((k >> 10) == want) atomicAdd(&gh[k & ((1 << kDigitBits2) - 1)], 1u);
+        }
+    }
+}
+
+// Per tile, from its candidates only: keys greater than / equal to tau.  One warp per tile.
 __global__ void __launch_bounds__(kThreads)
 k_topk_count(TileTable tt, int T, long long stride, TopkState tk) {
-    __shared__ unsigned int s_gt, s_eq;
-    WorkRange r = work_range(tk);
-    int q = r.q;
-    for (int w = r.w0; w < r.w1; ++w) {
-        while (w >= tk.sp_begin[q + 1]) ++q;
-        const int s = tk.sp_seg[q];
-        const int i = s / T, t = s - i * T;
-        const int tile = tt.seg_begin[t] + (w - tk.sp_begin[q]);
-        const unsigned int tau = tk.prefix[s];
-        const unsigned int* cd = tk.cand + (long long)i * stride + tt.offset[tile];
-        const int n = tk.tile_cand[(long long)i * tt.n_tiles + tile];
-        if (threadIdx.x == 0) { s_gt = 0; s_eq = 0; }
-        __syncthreads();
+    const int total = tk.plan->total_tiles;
+    const int lane = threadIdx.x & 31;
+    const int nwarps = gridDim.x * kWarps;
+    for (int w = blockIdx.x * kWarps + (threadIdx.x >> 5); w < total; w += nwarps) {
+        const WarpTile z = warp_tile(tk, tt, T, w);
+        const unsigned int tau = tk.prefix[z.s];
+        const unsigned int* cd = tk.cand + (long long)z.i * stride + tt.offset[z.tile];
+        const int n = tk.tile_cand[(long long)z.i * tt.n_tiles + z.tile];
         unsigned int gt = 0, eq = 0;
-        for (int e = threadIdx.x; e < n; e += kThreads) {
+        for (int e = lane; e < n; e += 32) {
             const unsigned int k = cd[e];
             gt += (k > tau);
             eq += (k == tau);
@@ -281,25 +346,20 @@ k_topk_count(TileTable tt, int T, long long stride, TopkState tk) {
             gt += __shfl_down_sync(0xffffffffu, gt, o);
             eq += __shfl_down_sync(0xffffffffu, eq, o);
         }
-        if ((threadIdx.x & 31) == 0) {
-            if (gt) atomicAdd(&s_gt, gt);
-            if (eq) atomicAdd(&s_eq, eq);
+        if (lane == 0) {
+            uint2* tc = tk.tile_count + (long long)z.i * tt.n_tiles + z.tile;
+            *tc = make_uint2(tc->x + gt, eq);
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint2* tc = tk.tile_count + (long long)i * tt.n_tiles + tile;
-            *tc = make_uint2(tc->x + s_gt, s_eq);
-        }
-        __syncthreads();
     }
 }
 
 // One CTA per sparse segment: exclusive prefix of the tile counts, in tile order.
 __global__ void __launch_bounds__(kThreads)
 k_topk_scan(TileTable tt, int T, TopkState tk) {
-    __shared__ unsigned int s_gt[kThreads], s_eq[kThreads];
+    __shared__ unsigned int s_gt[kWarps], s_eq[kWarps];
     __shared__ unsigned int s_run[2];
     const int nq = tk.plan->n_sparse;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int q = blockIdx.x; q < nq; q += gridDim.x) {
         const int s = tk.sp_seg[q];
         const int i = s / T, t = s - i * T;
@@ -311,9 +371,7 @@ k_topk_scan(TileTable tt, int T, TopkState tk) {
             const int z = c0 + threadIdx.x;
             uint2 v = make_uint2(0, 0);
             if (z < q1) v = tc[z];
-            // inclusive scan over the chunk, in tile order
-            unsigned int a = v.x, b = v.y;
-            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            unsigned int a = v.x, b = v.y;     // inclusive scan over the chunk, in tile order
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const unsigned int pa = __shfl_up_sync(0xffffffffu, a, o);
@@ -336,105 +394,109 @@ k_topk_scan(TileTable tt, int T, TopkState tk) {
     }
 }
 
-// Pass C: ordered compaction of the selected entries of one tile into the outbox.
+// Pass C: ordered compaction of the selected entries of one tile into the outbox, and delivery:
+// the same (index, value) pairs are written into the mailbox x_hat, which is what the receivers
+// hold once the message has arrived.
 // An entry is selected if key > tau, or key == tau and fewer than `remaining` equal keys
 // precede it in the tensor.  Its slot is (#greater before it) + min(#equal before it, remaining).
-__global__ void __launch_bounds__(kThreads)
-k_topk_write(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
-             long long stride, TopkState tk, unsigned int* __restrict__ err) {
-    __shared__ unsigned int s_gt[kWarps], s_eq[kWarps];
+// A tile is read as four coalesced chunks of 1024 elements (thread t owns elements 4t..4t+3 of
+// every chunk); the four per-chunk counts of a thread travel through ONE scan, packed 16 bits
+// each into a 64-bit word (a chunk holds at most 1024 entries, so the fields cannot overflow).
+// A thread has read the x_hat entries it owns before it overwrites any of them, and no thread
+// touches another thread's entries.
+__global__ void __launch_bounds__(kThreads, 3)
+k_topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long long stride,
+             TopkState tk, unsigned int* __restrict__ err) {
+    constexpr int kChunks = kNormTile / (kThreads * 4);   // 4
+    static_assert(kChunks == 4, "the packed scan holds four 16-bit fields");
+    __shared__ unsigned long long s_pg[kWarps], s_pe[kWarps];
     WorkRange r = work_range(tk);
-    int q = r.q;
+    WorkCursor cur;
+    cur.init(tk, tt, T, r.q);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned int tau = 0, take = 0, K = 0;
+    int2* out = nullptr;
     for (int w = r.w0; w < r.w1; ++w) {
-        while (w >= tk.sp_begin[q + 1]) ++q;
-        const int s = tk.sp_seg[q];
-        const int i = s / T, t = s - i * T;
-        const int tile = tt.seg_begin[t] + (w - tk.sp_begin[q]);
-        const unsigned int tau = tk.prefix[s], take = tk.remaining[s];
+        bool changed;
+        const int tile = cur.advance(tk, tt, T, w, changed);
+        if (changed) {
+            tau = tk.prefix[cur.s];
+            take = tk.remaining[cur.s];
+            K = (unsigned int)tk.count[cur.t];
+            out = tk.outbox + (long long)cur.i * tk.out_stride + tk.out_off[cur.t];
+        }
+        const int i = cur.i;
         const int len = tt.length[tile];
         const long long base = (long long)i * stride + tt.offset[tile];
-        const int first = (int)(tt.offset[tile] - tt.offset[tt.seg_begin[t]]);  // index of the tile's first element
+        const int first = (tile - cur.first_tile) * kNormTile;   // index of the tile's first element
         const uint2 before = tk.tile_count[(long long)i * tt.n_tiles + tile];
-        const long long K = tk.count[t];
-        int2* out = tk.outbox + (long long)i * tk.out_stride + tk.out_off[t];
-        unsigned int run_gt = before.x, run_eq = before.y;       // entries before this chunk
-        for (int c0 = 0; c0 < len; c0 += kThreads * 4) {
-            const int local = c0 + threadIdx.x * 4;
-            unsigned int k[4] = {0, 0, 0, 0};
-            float xv[4] = {0.f, 0.f, 0.f, 0.f};
-            int nel = 0;
-            if (local < len) {
-                const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
-                k[0] = rank_key(a.x, b.x); k[1] = rank_key(a.y, b.y);
-                k[2] = rank_key(a.z, b.z); k[3] = rank_key(a.w, b.w);
-                xv[0] = a.x; xv[1] = a.y; xv[2] = a.z; xv[3] = a.w;
-                nel = min(4, len - local);
-            }
+        unsigned int k[kChunks][4];
+        float xv[kChunks][4];
+        unsigned long long pg = 0, pe = 0;
+#pragma unroll
+        for (int v = 0; v < kChunks; ++v) {
+            const int local = (v * kThreads + threadIdx.x) * 4;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            if (local < len) { a = ld_stream(x + base + local); b = ld_stream(xhat + base + local); }
+            xv[v][0] = a.x; xv[v][1] = a.y; xv[v][2] = a.z; xv[v][3] = a.w;
+            k[v][0] = rank_key(a.x, b.x); k[v][1] = rank_key(a.y, b.y);
+            k[v][2] = rank_key(a.z, b.z); k[v][3] = rank_key(a.w, b.w);
+        }
+#pragma unroll
+        for (int v = 0; v < kChunks; ++v) {
+            const int local = (v * kThreads + threadIdx.x) * 4;
             unsigned int gt = 0, eq = 0;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-                if (c < nel) { gt += (k[c] > tau); eq += (k[c] == tau); }
-            // exclusive scan over the CTA in thread order (= index order)
-            unsigned int sgt = gt, seq = eq;
+                if (local + c < len) { gt += (k[v][c] > tau); eq += (k[v][c] == tau); }
+            pg |= (unsigned long long)gt << (16 * v);
+            pe |= (unsigned long long)eq << (16 * v);
+        }
+        // inclusive scan over the CTA in thread order, all four chunks at once
+        unsigned long long sg = pg, se = pe;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned int a = __shfl_up_sync(0xffffffffu, sgt, o);
-                const unsigned int b = __shfl_up_sync(0xffffffffu, seq, o);
-                if (lane >= o) { sgt += a; seq += b; }
-            }
-            if (lane == 31) { s_gt[warp] = sgt; s_eq[warp] = seq; }
-            __syncthreads();
-            unsigned int wgt = 0, weq = 0, tot_gt = 0, tot_eq = 0;
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long a = __shfl_up_sync(0xffffffffu, sg, o);
+            const unsigned long long b = __shfl_up_sync(0xffffffffu, se, o);
+            if (lane >= o) { sg += a; se += b; }
+        }
+        if (lane == 31) { s_pg[warp] = sg; s_pe[warp] = se; }
+        __syncthreads();
+        unsigned long long wg = 0, we = 0, tg = 0, te = 0;
 #pragma unroll
-            for (int u = 0; u < kWarps; ++u) {
-                if (u < warp) { wgt += s_gt[u]; weq += s_eq[u]; }
-                tot_gt += s_gt[u]; tot_eq += s_eq[u];
-            }
-            unsigned int my_gt = run_gt + wgt + sgt - gt;         // greater keys before my first entry
-            unsigned int my_eq = run_eq + weq + seq - eq;         // equal keys before my first entry
+        for (int u = 0; u < kWarps; ++u) {
+            if (u < warp) { wg += s_pg[u]; we += s_pe[u]; }
+            tg += s_pg[u]; te += s_pe[u];
+        }
+        const unsigned long long xg = wg + sg - pg, xe = we + se - pe;   // exclusive, per chunk
+        unsigned int run_gt = before.x, run_eq = before.y;               // entries before chunk v
+        if (pg | pe) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (c < nel) {
-                    const bool is_gt = k[c] > tau, is_eq = k[c] == tau;
-                    if (is_gt || (is_eq && my_eq < take)) {
-                        const long long slot = (long long)my_gt + (long long)min(my_eq, take);
-                        if (slot < K) out[slot] = make_int2(first + local + c, __float_as_int(xv[c]));
-                        else atomicOr(err, 2u);
+            for (int v = 0; v < kChunks; ++v) {
+                const int local = (v * kThreads + threadIdx.x) * 4;
+                unsigned int my_gt = run_gt + (unsigned int)((xg >> (16 * v)) & 0xffffu);
+                unsigned int my_eq = run_eq + (unsigned int)((xe >> (16 * v)) & 0xffffu);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (local + c < len) {
+                        const bool is_gt = k[v][c] > tau, is_eq = k[v][c] == tau;
+                        if (is_gt || (is_eq && my_eq < take)) {
+                            const unsigned int slot = my_gt + min(my_eq, take);
+                            if (slot < K) {
+                                out[slot] = make_int2(first + local + c, __float_as_int(xv[v][c]));
+                                xhat[base + local + c] = xv[v][c];
+                            } else {
+                                atomicOr(err, 2u);
+                            }
+                        }
+                        my_gt += is_gt; my_eq += is_eq;
                     }
-                    my_gt += is_gt; my_eq += is_eq;
                 }
+                run_gt += (unsigned int)((tg >> (16 * v)) & 0xffffu);
+                run_eq += (unsigned int)((te >> (16 * v)) & 0xffffu);
             }
-            run_gt += tot_gt; run_eq += tot_eq;
-            __syncthreads();
         }
-    }
-}
-
-// The receiver's side: write the received values into the mailbox.  Work tile number r of a
-// tensor handles outbox entries [r*kNormTile, (r+1)*kNormTile) (K_t <= n_t, so the tensor's
-// tiles cover its outbox).
-__global__ void __launch_bounds__(kThreads)
-k_topk_scatter(float* __restrict__ xhat, TileTable tt, int T, long long stride, TopkState tk,
-               const long long* __restrict__ numel, unsigned int* __restrict__ err) {
-    WorkRange r = work_range(tk);
-    int q = r.q;
-    for (int w = r.w0; w < r.w1; ++w) {
-        while (w >= tk.sp_begin[q + 1]) ++q;
-        const int s = tk.sp_seg[q];
-        const int i = s / T, t = s - i * T;
-        const long long K = tk.count[t];
-        const long long lo = (long long)(w - tk.sp_begin[q]) * kNormTile;
-        if (lo >= K) continue;
-        const long long hi = min(K, lo + kNormTile);
-        const int2* in = tk.outbox + (long long)i * tk.out_stride + tk.out_off[t];
-        float* dst = xhat + (long long)i * stride + tt.offset[tt.seg_begin[t]];
-        const long long n = numel[t];
-        for (long long e = lo + threadIdx.x; e < hi; e += kThreads) {
-            const int2 m = in[e];
-            if (m.x >= 0 && m.x < n) dst[m.x] = __int_as_float(m.y);
-            else atomicOr(err, 4u);
-        }
+        __syncthreads();
     }
 }
 

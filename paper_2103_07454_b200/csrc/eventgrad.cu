@@ -390,22 +390,20 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
             c->ctr, c->step_k);
         ++launches;
     }
-    // a4: Top-K select / pack / scatter for the segments that send a sparse message
+    // a4: Top-K select / pack / deliver for the segments that send a sparse message
     if (c->topk.enabled) {
         TimedSection ts(c, stream, EG_KERNEL_TOPK);
         k_topk_plan<<<1, kPlanThreads, 0, stream>>>(S, c->T, c->st.sparse, tn.seg_begin, c->tk);
-        k_topk_hist<false><<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk, 0);
+        k_topk_hist<<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk);
         k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(c->T, c->tk, 0);
         k_topk_collect<<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk);
-        for (int digit = 1; digit < 3; ++digit) {
-            k_topk_hist<true><<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk, digit);
-            k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(c->T, c->tk, digit);
-        }
+        k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(c->T, c->tk, 1);
+        k_topk_hist_cand<<<kTopkGrid, kThreads, 0, stream>>>(tn, c->T, c->stride, c->tk);
+        k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(c->T, c->tk, 2);
         k_topk_count<<<kTopkGrid, kThreads, 0, stream>>>(tn, c->T, c->stride, c->tk);
         k_topk_scan<<<kTopkSegGrid, kThreads, 0, stream>>>(tn, c->T, c->tk);
         k_topk_write<<<kTopkGrid, kThreads, 0, stream>>>(params, c->xhat, tn, c->T, c->stride, c->tk, c->err);
-        k_topk_scatter<<<kTopkGrid, kThreads, 0, stream>>>(c->xhat, tn, c->T, c->stride, c->tk, c->d_numel, c->err);
-        launches += 12;
+        launches += 10;
     }
     // a3 + a5: dense snapshot, consensus average, SGD
     {
