@@ -114,6 +114,21 @@ eg_status eg_step_host(eg_ctx* ctx, float* params_host, const float* grads_host,
  * turning it on, eg_reset and eg_import_state make the next step recompute the norms. */
 eg_status eg_set_carry_norm(eg_ctx* ctx, int enabled);
 
+/* Two readings of the paper's text that differ from the defaults (both are what the text,
+ * rather than the displayed formulas or the defaults' rationale, literally says):
+ *  own_term       EG_OWN_CURRENT (default): a replica averages its CURRENT parameters with
+ *                 the neighbours' last received ones.  EG_OWN_LAST_SENT: its own term is
+ *                 x_hat_i as well, i.e. X_{k+1} = X_hat_k W - gamma G of Eq. (dist_sgd_event)
+ *                 taken literally.
+ *  trigger_metric EG_TRIGGER_NORM_OF_CHANGE (default): d = || x - x_hat || (the displayed
+ *                 trigger condition).  EG_TRIGGER_CHANGE_OF_NORM: d = | ||x|| - ||x at the
+ *                 last event|| | (Section 4 prose: "when the norm of a particular parameter
+ *                 has changed by some threshold"); the norm pass then reads x only.
+ * Allowed before the first step of a context or right after eg_reset (EG_ERR_STATE later). */
+enum { EG_OWN_CURRENT = 0, EG_OWN_LAST_SENT = 1 };
+enum { EG_TRIGGER_NORM_OF_CHANGE = 0, EG_TRIGGER_CHANGE_OF_NORM = 1 };
+eg_status eg_set_variant(eg_ctx* ctx, int own_term, int trigger_metric);
+
 /* Which implementation of the fused snapshot / average / SGD kernel eg_step launches.  Both
  * compute bit-identical results.  EG_FUSED_PIPELINED (default) streams the operands through
  * shared memory with bulk asynchronous copies; EG_FUSED_REGISTER keeps the ring walk in

@@ -40,6 +40,10 @@
  *  - a mailbox that never received anything is left out of the average and the weight is
  *    1/(1 + number of neighbours heard from); with the forced first event this never
  *    happens and the weight is 1/3 on a ring;
+ *  - two further readings of the text are available as variants (ego_set_variant), both off
+ *    by default: the own term taken literally from Eq. (dist_sgd_event) (x_hat_i instead of
+ *    x_i; with it a replica that never communicated averages with x_hat_i = X_0 = 0), and the
+ *    tested quantity taken as the change of the norm, | ||x|| - ||x at the last event|| |;
  *  - Top-K ranks by |x - x_hat| (fp32 difference), sends the parameter values x[e] with
  *    their indices, ties go to the lower index, the message is in ascending index order,
  *    K_t = max(1, ceil(n_t * k_num / k_den)); the first message of a tensor is dense.
@@ -95,6 +99,12 @@ typedef struct ego_ctx {
     uint64_t *seg_payload; /* scratch: payload bytes of this step's event, 0 if none */
     uint64_t messages, bytes, events;
     int threads;
+    /* variants the paper's text also admits (both off by default) */
+    int own_last_sent;    /* 1: the replica's own term of the average is x_hat_i, i.e.
+                             Eq. (dist_sgd_event) read literally (X_hat W) */
+    int change_of_norm;   /* 1: the tested quantity is | ||x|| - ||x|| at the last event |
+                             ("the norm of a parameter has changed by some threshold") */
+    double *sent_norm;    /* [P*T] ||x|| at the last event (0 before the first) */
 } ego_ctx;
 
 void ego_destroy(ego_ctx *c) {
@@ -102,7 +112,7 @@ void ego_destroy(ego_ctx *c) {
     free(c->numel); free(c->off); free(c->Kt); free(c->out_off); free(c->xhat);
     free(c->delta); free(c->khat); free(c->hist); free(c->hist_len); free(c->valid);
     free(c->flag); free(c->norm); free(c->thr_used); free(c->out_idx); free(c->out_val);
-    free(c->out_count); free(c->seg_events); free(c->seg_payload);
+    free(c->out_count); free(c->seg_events); free(c->seg_payload); free(c->sent_norm);
     free(c);
 }
 
@@ -121,6 +131,7 @@ void ego_reset(ego_ctx *c) {
         c->thr_used[s] = c->delta[s];
         c->out_count[s] = 0;
         c->seg_events[s] = 0;
+        c->sent_norm[s] = 0.0;
     }
     memset(c->hist, 0, sizeof(double) * (size_t)S * (size_t)c->H);
 }
@@ -175,8 +186,14 @@ ego_ctx *ego_create(int P, int T, const int64_t *numel, int mode, double horizon
     c->out_count = (int32_t *)malloc(sizeof(int32_t) * S);
     c->seg_events = (uint64_t *)malloc(sizeof(uint64_t) * S);
     c->seg_payload = (uint64_t *)malloc(sizeof(uint64_t) * S);
+    c->sent_norm = (double *)malloc(sizeof(double) * S);
     ego_reset(c);
     return c;
+}
+
+void ego_set_variant(ego_ctx *c, int own_last_sent, int change_of_norm) {
+    c->own_last_sent = own_last_sent != 0;
+    c->change_of_norm = change_of_norm != 0;
 }
 
 void ego_set_threads(ego_ctx *c, int threads) { c->threads = threads < 1 ? 1 : threads; }
@@ -228,14 +245,24 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
     const float *xs = x + (int64_t)i * c->N + c->off[t];
     float *hs = c->xhat + (int64_t)i * c->N + c->off[t];
 
-    /* 1-2: d = || x - x_hat ||_2 with fp32 differences, exact fp64 squares, fp64 sum */
+    /* 1-2: d = || x - x_hat ||_2 with fp32 differences, exact fp64 squares, fp64 sum;
+     * variant: d = | ||x||_2 - ||x at the last event||_2 | */
     double acc = 0.0;
-    for (int64_t e = 0; e < n; ++e) {
-        const float d32 = xs[e] - hs[e]; /* one fp32 subtraction (FLT_EVAL_METHOD 0) */
-        double dd = (double)d32;
-        acc = acc + dd * dd;
+    double d;
+    if (!c->change_of_norm) {
+        for (int64_t e = 0; e < n; ++e) {
+            const float d32 = xs[e] - hs[e]; /* one fp32 subtraction (FLT_EVAL_METHOD 0) */
+            double dd = (double)d32;
+            acc = acc + dd * dd;
+        }
+        d = sqrt(acc);
+    } else {
+        for (int64_t e = 0; e < n; ++e) {
+            double dd = (double)xs[e];
+            acc = acc + dd * dd;
+        }
+        d = fabs(sqrt(acc) - c->sent_norm[s]);
     }
-    const double d = sqrt(acc);
     const double thr = c->delta[s];
     c->norm[s] = d;
     c->thr_used[s] = thr;
@@ -290,6 +317,7 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
     c->seg_payload[s] = payload;
 
     /* 4c: bookkeeping */
+    if (c->change_of_norm) c->sent_norm[s] = sqrt(acc);
     c->khat[s] = c->k;
     c->valid[s] = 1;
     c->seg_events[s] += 1;
@@ -309,8 +337,9 @@ static void phase_b_segment(ego_ctx *c, float *x, const float *g, float lr, int 
     float *xs = x + (int64_t)i * c->N + c->off[t];
     const float *gs = g + (int64_t)i * c->N + c->off[t];
     const double neg_lr = -(double)lr;
+    const float *own = c->own_last_sent ? c->xhat + (int64_t)i * c->N + c->off[t] : xs;
     for (int64_t e = 0; e < c->numel[t]; ++e) {
-        double sum = (double)xs[e];
+        double sum = (double)own[e];
         for (int q = 0; q < cnt; ++q) sum = sum + (double)hn[q][e];
         const double avg = sum * w;
         const double r = fma(neg_lr, (double)gs[e], avg);
@@ -361,6 +390,7 @@ const double *ego_thresholds(const ego_ctx *c) { return c->delta; }
 const uint8_t *ego_valid(const ego_ctx *c) { return c->valid; }
 const int64_t *ego_last_event_iteration(const ego_ctx *c) { return c->khat; }
 const uint64_t *ego_segment_events(const ego_ctx *c) { return c->seg_events; }
+const double *ego_sent_norms(const ego_ctx *c) { return c->sent_norm; }
 const double *ego_history(const ego_ctx *c) { return c->hist; }
 const int *ego_history_len(const ego_ctx *c) { return c->hist_len; }
 float *ego_xhat(ego_ctx *c) { return c->xhat; }

@@ -44,6 +44,7 @@ def _load():
         lib.ego_destroy.argtypes = [C.c_void_p]
         lib.ego_reset.argtypes = [C.c_void_p]
         lib.ego_set_threads.argtypes = [C.c_void_p, C.c_int]
+        lib.ego_set_variant.argtypes = [C.c_void_p, C.c_int, C.c_int]
         lib.ego_threads_available.restype = C.c_int
         lib.ego_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
         lib.ego_stats.argtypes = [C.c_void_p] + [C.POINTER(C.c_uint64)] * 3
@@ -51,7 +52,7 @@ def _load():
         lib.ego_iteration.argtypes = [C.c_void_p]
         for name in ("ego_flags", "ego_norms", "ego_thresholds_used", "ego_thresholds",
                      "ego_valid", "ego_last_event_iteration", "ego_segment_events", "ego_xhat",
-                     "ego_history", "ego_history_len"):
+                     "ego_history", "ego_history_len", "ego_sent_norms"):
             getattr(lib, name).restype = C.c_void_p
             getattr(lib, name).argtypes = [C.c_void_p]
         lib.ego_topk_count.restype = C.c_int64
@@ -84,7 +85,8 @@ class Oracle:
     def __init__(self, P: int, numel: Sequence[int], *, mode: int = ADAPTIVE,
                  horizon: float = 1.0, history_len: int = 1, delta_init: float = 0.0,
                  delta_fixed: float = 0.0, force_first_event: bool = True,
-                 topk: Optional[tuple] = None, threads: int = 1):
+                 topk: Optional[tuple] = None, threads: int = 1,
+                 own_last_sent: bool = False, change_of_norm: bool = False):
         lib = _load()
         self._lib = lib
         self.P, self.T = int(P), len(numel)
@@ -98,6 +100,7 @@ class Oracle:
         if not self._h:
             raise ValueError("ego_create rejected the arguments")
         lib.ego_set_threads(self._h, int(threads))
+        lib.ego_set_variant(self._h, int(own_last_sent), int(change_of_norm))
         self.S = self.P * self.T
         self.history_len = int(history_len)
 
@@ -145,6 +148,10 @@ class Oracle:
     def thresholds(self):
         """Threshold in force after the last step."""
         return self._seg("ego_thresholds", np.float64)
+
+    def sent_norms(self):
+        """||x|| of every (replica, tensor) at its last event (change-of-norm variant)."""
+        return self._seg("ego_sent_norms", np.float64)
 
     def valid(self):
         return self._seg("ego_valid", np.uint8)

@@ -37,7 +37,12 @@ struct SegState {
     double* norm;                // d of this step
     double* thr_used;            // delta that d was compared with
     unsigned long long* events;  // events so far
+    double* sent_norm;           // ||x|| at the last event (change-of-norm variant)
 };
+
+// Variants of the method that the paper's text also admits (kernel argument `variant`).
+constexpr int kOwnLastSent = 1;    // own term of the average is x_hat_i (Eq. (dist_sgd_event) literally)
+constexpr int kChangeOfNorm = 2;   // tested quantity is | ||x|| - ||x at the last event|| |
 
 struct Counters {                // device-resident, 64-bit
     unsigned long long messages, bytes, events, pad;

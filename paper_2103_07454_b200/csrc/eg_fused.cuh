@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kThreads)
 k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
         const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
         int P, int T, long long stride, float lr, double* __restrict__ partials,
-        long long* step_k) {
+        long long* step_k, int variant) {
     extern __shared__ __align__(128) unsigned char smem[];
     uint8_t* s_snap = smem;
     uint8_t* s_valid = smem + P;
@@ -131,10 +131,11 @@ k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ 
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             if (nel[v] > 0) {
-                const float4 xn = upd4(x_cur[v], g_cur[v], h_prev[v], h_nxt[v], ul, ur, w, neg_lr);
+                const float4 own = (variant & kOwnLastSent) ? h_cur[v] : x_cur[v];
+                const float4 xn = upd4(own, g_cur[v], h_prev[v], h_nxt[v], ul, ur, w, neg_lr);
                 store_masked(x + rb + e[v], xn, nel[v]);
                 if (sn) store_masked(xhat + rb + e[v], x_cur[v], nel[v]);
-                if (CARRY) acc = sq_diff4(xn, h_cur[v], nel[v], acc);
+                if (CARRY) acc = sq_diff4(xn, (variant & kChangeOfNorm) ? zero4 : h_cur[v], nel[v], acc);
             }
         }
         if (CARRY) {

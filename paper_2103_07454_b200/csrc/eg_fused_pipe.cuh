@@ -44,8 +44,22 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+#ifndef EG_WAIT_HINT_NS
+#define EG_WAIT_HINT_NS 1000
+#endif
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
+#if EG_WAIT_HINT_NS > 0
+    // the hint lets the hardware keep the warp suspended (no issue slots used) until the phase
+    // completes or the time runs out
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"((uint32_t)EG_WAIT_HINT_NS)
+        : "memory");
+#else
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -53,6 +67,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
+#endif
     return ok != 0;
 }
 // 1-D bulk copy global -> this CTA's shared memory; src, dst 16-byte aligned, bytes % 16 == 0.
@@ -67,7 +82,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
                                                   unsigned int* err) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
+    unsigned int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) != 0) continue;       // look at the clock every 64 polls only
         if (*s_abort) return false;
         if (clock64() - t0 > kWaitLimitCycles) {
             *s_abort = 1;
@@ -107,7 +124,7 @@ __global__ void __launch_bounds__(CONSUMERS + 32)
 k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
-             long long* step_k, unsigned int* __restrict__ err) {
+             long long* step_k, unsigned int* __restrict__ err, int variant) {
     using L = PipeSmem<TILE, STAGES>;
     constexpr int COLS = TILE / (4 * CONSUMERS);
     constexpr int CWARPS = CONSUMERS / 32;
@@ -233,7 +250,7 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
                     const double hn[4] = {(double)hnf.x, (double)hnf.y, (double)hnf.z, (double)hnf.w};
                     const double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
                     double xd[4];
-                    if (sn) {
+                    if (sn || (variant & kOwnLastSent)) {   // own term = this replica's contribution
 #pragma unroll
                         for (int q = 0; q < 4; ++q) xd[q] = hc[v][q];
                     } else {
@@ -251,7 +268,9 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
                     const float4 xn4 = make_float4(xn[0], xn[1], xn[2], xn[3]);
                     store_masked(xo + v * 4 * CONSUMERS, xn4, nel[v]);
                     if (sn) store_masked(ho + v * 4 * CONSUMERS, hcf, nel[v]);
-                    if (CARRY) acc = sq_diff4(xn4, hcf, nel[v], acc);
+                    if (CARRY)
+                        acc = sq_diff4(xn4, (variant & kChangeOfNorm) ? make_float4(0.f, 0.f, 0.f, 0.f) : hcf,
+                                       nel[v], acc);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) { hp[v][q] = hc[v][q]; hc[v][q] = hn[q]; }
                 }

@@ -25,7 +25,7 @@ __device__ __forceinline__ double sq_diff4(float4 a, float4 b, int nel, double a
 // grid (n_tiles, P).  partials[i * n_tiles + tile].
 __global__ void __launch_bounds__(kThreads)
 k_norm_partial(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt,
-               long long stride, double* __restrict__ partials) {
+               long long stride, double* __restrict__ partials, int variant) {
     __shared__ double s_warp[kWarps];
     const int tile = blockIdx.x, i = blockIdx.y;
     const int len = tt.length[tile];
@@ -39,7 +39,9 @@ k_norm_partial(const float* __restrict__ x, const float* __restrict__ xhat, Tile
         nel[q] = min(4, max(0, len - local));
         if (nel[q] > 0) {
             a[q] = ld_stream(x + base + local);
-            b[q] = ld_stream(xhat + base + local);
+            // change-of-norm variant: sum of x^2 (x - 0 is exact), x_hat is not read
+            b[q] = (variant & kChangeOfNorm) ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                             : ld_stream(xhat + base + local);
         } else {
             a[q] = b[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
@@ -58,6 +60,7 @@ struct DecideParams {
     int force_first;
     int topk;                 // Top-K messages enabled
     int degree;               // distinct ring neighbours of every replica
+    int variant;              // kChangeOfNorm: d = | sqrt(sum) - sent_norm |
 };
 
 // One warp per (replica, tensor).  grid ceil(P*T / kWarps).
@@ -79,7 +82,8 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     if (lane != 0) return;
 
     const long long k = *step_k;
-    const double d = __dsqrt_rn(acc);
+    const double root = __dsqrt_rn(acc);
+    const double d = (dp.variant & kChangeOfNorm) ? fabs(__dsub_rn(root, st.sent_norm[s])) : root;
     const double thr = st.delta[s];
     st.norm[s] = d;
     st.thr_used[s] = thr;
@@ -112,6 +116,7 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
             out_count = (int)topk_count[t];
             payload = 8ull * (unsigned long long)topk_count[t];
         }
+        if (dp.variant & kChangeOfNorm) st.sent_norm[s] = root;
         st.khat[s] = k;
         st.valid[s] = 1;
         st.events[s] += 1ull;

@@ -23,7 +23,7 @@ constexpr int kFusedVpt = EG_FUSED_VPT;               // float4 columns per thre
 constexpr int kFusedTile = kThreads * 4 * kFusedVpt;  // elements per CTA of the fused kernel
 using PipeLayout = PipeSmem<kPipeTile, kPipeStages>;
 static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
-constexpr uint64_t kStateMagic = 0x4547535441544531ull;  // "EGSTATE1"
+constexpr uint64_t kStateMagic = 0x4547535441544532ull;  // "EGSTATE2"
 
 struct HostTiles {
     std::vector<int> tensor, length, seg_begin;
@@ -70,6 +70,8 @@ struct eg_ctx {
     int last_launches = 0;
     size_t fused_smem = 0;
     int fused_kind = EG_FUSED_PIPELINED;
+    int variant = 0;
+    bool stepped = false;   // a step has run since creation / reset / import
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
     std::vector<cudaEvent_t> ev_pool;      // pairs
@@ -153,6 +155,7 @@ eg_status init_state(eg_ctx* c) {
     EG_CUDA(c, cudaMemset(c->st.sparse, 0, S));
     EG_CUDA(c, cudaMemset(c->st.norm, 0, S * sizeof(double)));
     EG_CUDA(c, cudaMemset(c->st.events, 0, S * sizeof(unsigned long long)));
+    EG_CUDA(c, cudaMemset(c->st.sent_norm, 0, S * sizeof(double)));
     EG_CUDA(c, cudaMemset(c->ctr, 0, sizeof(Counters)));
     EG_CUDA(c, cudaMemset(c->step_k, 0, sizeof(long long)));
     EG_CUDA(c, cudaMemset(c->err, 0, sizeof(unsigned int)));
@@ -164,6 +167,7 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->tk.remaining, 0, S * sizeof(unsigned int)));
     }
     c->carried_valid = false;
+    c->stepped = false;
     return EG_OK;
 }
 
@@ -296,7 +300,7 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     EG_ALLOC(c->st.delta, S); EG_ALLOC(c->st.khat, S); EG_ALLOC(c->st.hist, S * c->H);
     EG_ALLOC(c->st.hist_len, S); EG_ALLOC(c->st.valid, S); EG_ALLOC(c->st.flag, S);
     EG_ALLOC(c->st.snap, S); EG_ALLOC(c->st.sparse, S); EG_ALLOC(c->st.norm, S);
-    EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S);
+    EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S); EG_ALLOC(c->st.sent_norm, S);
     EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 1);
     EG_ALLOC(c->outbox_count, S);
     EG_ALLOC(c->cons_partials, (size_t)c->tiles_fused.n_tiles + 1);
@@ -375,12 +379,13 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     const bool use_carried = c->carry && c->carried_valid && c->carried_params == params;
     if (!use_carried) {
         TimedSection ts(c, stream, EG_KERNEL_NORM);
-        k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, c->partials_norm);
+        k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, c->partials_norm,
+                                                          c->variant);
         ++launches;
     }
     // a2 + a6: decision, threshold update, counters
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
-                    c->topk.enabled, c->degree};
+                    c->topk.enabled, c->degree, c->variant};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf : tn;
     {
@@ -413,24 +418,25 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
                 k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
                     <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, true, kPipeConsumers / 32), stream>>>(
                     params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->err);
+                    c->partials_fused, c->step_k, c->err, c->variant);
             else
                 k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>
                     <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                     params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->err);
+                    c->partials_fused, c->step_k, c->err, c->variant);
         } else if (c->carry)
             k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
                 params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                c->partials_fused, c->step_k);
+                c->partials_fused, c->step_k, c->variant);
         else
             k_fused<kFusedVpt, false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
                 params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                c->partials_fused, c->step_k);
+                c->partials_fused, c->step_k, c->variant);
         ++launches;
     }
     c->carried_valid = c->carry;
     c->carried_params = params;
+    c->stepped = true;
     c->last_launches = launches;
     EG_CUDA(c, cudaGetLastError());
     return EG_OK;
@@ -531,6 +537,17 @@ eg_status eg_read_mailboxes(eg_ctx* c, float* xhat_host) {
     eg_status s = sync_and_check(c);
     if (s != EG_OK) return s;
     EG_CUDA(c, cudaMemcpy(xhat_host, c->xhat, (size_t)c->P * c->stride * sizeof(float), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_set_variant(eg_ctx* c, int own_term, int trigger_metric) {
+    if (!c || (own_term != EG_OWN_CURRENT && own_term != EG_OWN_LAST_SENT) ||
+        (trigger_metric != EG_TRIGGER_NORM_OF_CHANGE && trigger_metric != EG_TRIGGER_CHANGE_OF_NORM))
+        return EG_ERR_INVALID;
+    if (c->stepped) return EG_ERR_STATE;   // only before the first step (or after eg_reset)
+    c->variant = (own_term == EG_OWN_LAST_SENT ? kOwnLastSent : 0) |
+                 (trigger_metric == EG_TRIGGER_CHANGE_OF_NORM ? kChangeOfNorm : 0);
+    c->carried_valid = false;
     return EG_OK;
 }
 
@@ -643,14 +660,14 @@ eg_status eg_average_model(eg_ctx* c, const float* params, float* avg_dev, doubl
 // ---------------------------------------------------------------------------------------
 struct StateHeader {
     uint64_t magic;
-    int64_t P, T, H, stride, n_total, topk, k_num, k_den;
+    int64_t P, T, H, stride, n_total, topk, k_num, k_den, variant;
     int64_t step;
     uint64_t messages, bytes, events;
 };
 
 static size_t state_bytes(const eg_ctx* c) {
     const size_t S = (size_t)c->P * c->T;
-    return sizeof(StateHeader) + S * (sizeof(double) + sizeof(long long) + sizeof(int) + 1 +
+    return sizeof(StateHeader) + S * (2 * sizeof(double) + sizeof(long long) + sizeof(int) + 1 +
                                       sizeof(unsigned long long)) +
            S * c->H * sizeof(double) + (size_t)c->P * c->stride * sizeof(float);
 }
@@ -671,6 +688,7 @@ eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
     EG_CUDA(c, cudaMemcpy(&k, c->step_k, sizeof(k), cudaMemcpyDeviceToHost));
     h.magic = kStateMagic; h.P = c->P; h.T = c->T; h.H = c->H; h.stride = c->stride;
     h.n_total = c->n_total; h.topk = c->topk.enabled; h.k_num = c->topk.k_num; h.k_den = c->topk.k_den;
+    h.variant = c->variant;
     h.step = k; h.messages = ctr.messages; h.bytes = ctr.bytes; h.events = ctr.events;
     char* p = static_cast<char*>(host_buf);
     memcpy(p, &h, sizeof(h)); p += sizeof(h);
@@ -682,6 +700,7 @@ eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
     EG_PULL(c->st.valid, S);
     EG_PULL(c->st.events, S * sizeof(unsigned long long));
     EG_PULL(c->st.hist, S * c->H * sizeof(double));
+    EG_PULL(c->st.sent_norm, S * sizeof(double));
     EG_PULL(c->xhat, (size_t)c->P * c->stride * sizeof(float));
 #undef EG_PULL
     *bytes = need;
@@ -693,7 +712,7 @@ eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
     StateHeader h;
     memcpy(&h, host_buf, sizeof(h));
     if (h.magic != kStateMagic || h.P != c->P || h.T != c->T || h.H != c->H || h.stride != c->stride ||
-        h.n_total != c->n_total || h.topk != c->topk.enabled ||
+        h.n_total != c->n_total || h.topk != c->topk.enabled || h.variant != c->variant ||
         (h.topk && (h.k_num != c->topk.k_num || h.k_den != c->topk.k_den)))
         return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
@@ -714,10 +733,12 @@ eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
     EG_PUSH(c->st.valid, S);
     EG_PUSH(c->st.events, S * sizeof(unsigned long long));
     EG_PUSH(c->st.hist, S * c->H * sizeof(double));
+    EG_PUSH(c->st.sent_norm, S * sizeof(double));
     EG_PUSH(c->xhat, (size_t)c->P * c->stride * sizeof(float));
 #undef EG_PUSH
     EG_CUDA(c, cudaDeviceSynchronize());
     c->carried_valid = false;
+    c->stepped = h.step > 0;
     return EG_OK;
 }
 

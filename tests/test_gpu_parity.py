@@ -16,7 +16,7 @@ RAGGED = [1, 3, 4, 5, 31, 32, 33, 1023, 1024, 1025, 4095, 4096, 4097, 10000, (1 
 INF = float("inf")
 
 
-@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 6, 7, 11, 64])
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 6, 7, 11, 64, 130])
 @pytest.mark.parametrize("carry", [False, True])
 @pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
 def test_ragged_dense(P, carry, kernel):
@@ -25,6 +25,60 @@ def test_ragged_dense(P, carry, kernel):
     rep = lockstep(wl, init="distinct", carry=carry, fused_kernel=kernel)
     assert rep.params_bit_exact and not rep.near_threshold
     assert 0 < rep.events < P * wl.T * wl.steps
+
+
+@pytest.mark.parametrize("own,con", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("carry", [False, True])
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
+def test_variants_own_term_and_change_of_norm(own, con, carry, kernel):
+    wl = W.synthetic(5, RAGGED[:-1], steps=16, lr=0.1, grad_sigma=0.01, history_len=2)
+    rep = lockstep(wl, init="distinct", carry=carry, fused_kernel=kernel,
+                   oracle_kw=dict(own_last_sent=own, change_of_norm=con))
+    assert rep.params_bit_exact and not rep.near_threshold
+    assert 0 < rep.events < 5 * wl.T * wl.steps
+
+
+def test_variant_with_topk():
+    wl = W.synthetic(4, RAGGED[:-1], steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
+    rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64,
+                   oracle_kw=dict(own_last_sent=True, change_of_norm=True))
+    assert rep.params_bit_exact
+
+
+def test_variant_only_before_the_first_step():
+    wl = W.synthetic(2, [8, 100])
+    eg = B.from_workload(wl)
+    eg.set_variant(True, True)
+    x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+    eg.step(x, eg.to_layout(wl.grads(0, "cuda")), 0.1)
+    with pytest.raises(B.EventGradError):
+        eg.set_variant(False, False)
+    eg.reset()
+    eg.set_variant(False, False)
+    eg.close()
+
+
+def test_resynchronise_through_the_checkpoint_interface():
+    """The harness's recovery path (used after a reported near-threshold disagreement): the
+    CUDA context takes over the oracle's whole state and the comparison goes on."""
+    import numpy as np
+    from oracle import eg_oracle as eo
+    from parity_harness import resynchronise
+    wl = W.synthetic(3, [5, 1000, 4097], steps=10, lr=0.1, grad_sigma=0.01, history_len=3)
+    o, eg = eo.from_workload(wl), B.from_workload(wl)
+    xh = W.distinct_init_params(wl).numpy().copy()
+    xd = eg.to_layout(torch.from_numpy(xh))
+    for k in range(4):                      # only the oracle advances
+        o.step(xh, wl.grads(k).numpy(), wl.lr)
+    resynchronise(eg, o, xd, xh)
+    for k in range(4, 10):
+        g = wl.grads(k)
+        o.step(xh, g.numpy(), wl.lr)
+        eg.step(xd, eg.to_layout(g), wl.lr)
+        f, _, _ = eg.last_decisions()
+        assert np.array_equal(f, o.flags())
+    assert eg.stats() == o.stats()
+    assert np.array_equal(eg.from_layout(xd).cpu().numpy(), xh)
 
 
 @pytest.mark.parametrize("hist,horizon", [(1, 1.0), (4, 1.0), (2, 0.5)])

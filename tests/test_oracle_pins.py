@@ -217,8 +217,9 @@ def load_threshold_cases():
             if not line or line.startswith("#"):
                 continue
             if line.startswith("case"):
-                _, name, H, h = line.split()
-                cur = {"name": name, "H": int(H[2:]), "h": float(h[2:]), "rows": []}
+                _, name, H, h, *rest = line.split()
+                cur = {"name": name, "H": int(H[2:]), "h": float(h[2:]), "rows": [],
+                       "change_of_norm": "metric=change_of_norm" in rest}
                 cases.append(cur)
             else:
                 cur["rows"].append([float(v) for v in line.split()])
@@ -228,7 +229,8 @@ def load_threshold_cases():
 @pytest.mark.parametrize("case", load_threshold_cases(), ids=lambda c: c["name"])
 def test_hand_worked_threshold_sequence(case):
     rows = case["rows"]
-    o = eo.Oracle(1, [2], horizon=case["h"], history_len=case["H"], delta_init=0.0)
+    o = eo.Oracle(1, [2], horizon=case["h"], history_len=case["H"], delta_init=0.0,
+                  change_of_norm=case["change_of_norm"])
     x = np.array([[rows[0][1], rows[0][2]]], dtype=np.float32)
     for r, row in enumerate(rows):
         k, x0, x1, flag, d, thr_tested, thr_after = row
@@ -253,6 +255,65 @@ def test_fixed_threshold_never_adapts():
         assert o.thresholds()[0, 0] == 2.0
     # x_k = k*(0.6,0.8): k=0,1 below 2; k=2 fires (d~2, x_hat<-x_2); k=3 d~1; k=4 fires; ...
     assert fired[:2] == [0, 0] and sum(fired) >= 1
+
+
+# ---------------------------------------------------------------------------------------
+# variants: own term read literally from Eq. (dist_sgd_event); change-of-norm trigger
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("own,con", [(True, False), (False, True), (True, True)])
+def test_variants_reduce_to_dpsgd_at_zero_threshold(own, con):
+    P = 5
+    wl = small(P=P, steps=5, lr=0.1, grad_sigma=0.01)
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=0.0, own_last_sent=own, change_of_norm=con)
+    x = W.distinct_init_params(wl).numpy().copy()
+    Wm = ring_matrix(P)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        ref = Wm @ x.astype(np.float64) - np.float64(np.float32(wl.lr)) * g.astype(np.float64)
+        o.step(x, g, wl.lr)
+        assert o.flags().all()
+        assert np.all(np.abs(x.astype(np.float64) - ref) <= 0.5000001 * ulp32(ref) + 1e-300)
+
+
+def test_literal_own_term_uses_the_last_sent_value():
+    """X_{k+1} = X_hat_k W - gamma G read literally: with mailboxes frozen at x_0 (forced first
+    event, infinite threshold afterwards) nothing accumulates, x_{k+1} = W x_0 - gamma g_k;
+    and a replica that never sent anything averages with X_0 = 0."""
+    P = 5
+    wl = small(P=P, steps=4, lr=0.1, grad_sigma=0.05)
+    lr64 = np.float64(np.float32(wl.lr))
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=INF, force_first_event=True, own_last_sent=True)
+    x0 = W.distinct_init_params(wl).numpy().copy()
+    x = x0.copy()
+    base = ring_matrix(P) @ x0.astype(np.float64)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        o.step(x, g, wl.lr)
+        ref = base - lr64 * g.astype(np.float64)
+        assert np.all(np.abs(x - ref) <= ulp32(ref))
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=INF, force_first_event=False, own_last_sent=True)
+    x = x0.copy()
+    g = wl.grads(0).numpy()
+    o.step(x, g, wl.lr)
+    assert np.all(np.abs(x - (-lr64 * g.astype(np.float64))) <= ulp32(lr64 * g))
+
+
+def test_change_of_norm_ignores_rotations():
+    """A vector that turns without changing its length triggers the norm-of-change test but
+    not the change-of-norm test."""
+    fired = {}
+    for con in (False, True):
+        o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=0.5, force_first_event=True, change_of_norm=con)
+        x = np.array([[3.0, 4.0]], np.float32)
+        o.step(x, np.array([[-5.0, 2.0]], np.float32), 1.0)      # x becomes (8, 2)... any value
+        x[:] = [[4.0, 3.0]]                                         # same length as (3, 4), turned
+        o.step(x, np.zeros((1, 2), np.float32), 1.0)
+        fired[con] = int(o.flags()[0, 0])
+        if con:
+            assert o.norms()[0, 0] == 0.0 and o.sent_norms()[0, 0] == 5.0
+        else:
+            assert o.norms()[0, 0] == pytest.approx(math.sqrt(2.0), rel=1e-15)
+    assert fired == {False: 1, True: 0}
 
 
 # ---------------------------------------------------------------------------------------
