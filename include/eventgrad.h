@@ -38,7 +38,7 @@
  *    problem (an index outside its table) sets an error word that the next synchronising
  *    call returns as EG_ERR_INTERNAL.
  *  - Counters: an event of tensor t at replica i adds deg(i) to messages_sent (deg = number
- *    of distinct ring neighbours: 2, or 1 for P = 2, or 0 for P = 1) and deg(i)*payload to
+ *    of distinct ring neighbours: min(2*hops, P-1), i.e. 2 on the paper's ring) and deg(i)*payload to
  *    bytes_sent; payload = 4*n_t for a dense message, 8*K_t for a Top-K message
  *    ("2K percent", Section 7).  The paper's "percentage of messages" (Table 1) is
  *    messages_sent / (P * T * 2 * steps).
@@ -65,7 +65,11 @@ typedef enum {
     EG_ERR_INTERNAL = 6  /* device-side consistency check failed */
 } eg_status;
 
-enum { EG_TOPO_RING = 0 }; /* the topology the paper fixes (Section 3) */
+enum { EG_TOPO_RING = 0 }; /* the topology the paper fixes (Section 3): nearest neighbours */
+/* Ring in which every replica averages with the m nearest replicas on each side, 1 <= m <= 8
+ * (Section 7: more neighbours per PE let information flow sooner); W_ij = 1/(N_i + 1) over the
+ * distinct neighbours.  EG_TOPO_RING_HOPS(1) == EG_TOPO_RING. */
+#define EG_TOPO_RING_HOPS(m) ((m) - 1)
 enum { EG_THRESH_ADAPTIVE = 0, /* Eq. (thres) with a history of H slopes */
        EG_THRESH_FIXED = 1 };  /* one static threshold for all tensors (Section 4 calls it
                                   the simplest option); 0 gives regular D-PSGD, +inf none */

@@ -61,6 +61,7 @@
 #error "the oracle needs float expressions evaluated in float (FLT_EVAL_METHOD == 0)"
 #endif
 
+#define EGO_MAX_HOPS 8
 #define EGO_ADAPTIVE 0
 #define EGO_FIXED 1
 
@@ -105,6 +106,7 @@ typedef struct ego_ctx {
     int change_of_norm;   /* 1: the tested quantity is | ||x|| - ||x|| at the last event |
                              ("the norm of a parameter has changed by some threshold") */
     double *sent_norm;    /* [P*T] ||x|| at the last event (0 before the first) */
+    int hops;             /* ring neighbours on each side (1 = the paper's ring) */
 } ego_ctx;
 
 void ego_destroy(ego_ctx *c) {
@@ -154,7 +156,7 @@ ego_ctx *ego_create(int P, int T, const int64_t *numel, int mode, double horizon
     if (!c) return NULL;
     c->P = P; c->T = T; c->mode = mode; c->horizon = horizon; c->H = H;
     c->delta_init = delta_init; c->delta_fixed = delta_fixed; c->force_first = force_first;
-    c->topk = topk; c->k_num = k_num; c->k_den = k_den; c->threads = 1;
+    c->topk = topk; c->k_num = k_num; c->k_den = k_den; c->threads = 1; c->hops = 1;
     c->numel = (int64_t *)malloc(sizeof(int64_t) * T);
     c->off = (int64_t *)malloc(sizeof(int64_t) * T);
     c->Kt = (int64_t *)malloc(sizeof(int64_t) * T);
@@ -196,6 +198,12 @@ void ego_set_variant(ego_ctx *c, int own_last_sent, int change_of_norm) {
     c->change_of_norm = change_of_norm != 0;
 }
 
+int ego_set_hops(ego_ctx *c, int hops) {
+    if (hops < 1 || hops > EGO_MAX_HOPS) return 1;
+    c->hops = hops;
+    return 0;
+}
+
 void ego_set_threads(ego_ctx *c, int threads) { c->threads = threads < 1 ? 1 : threads; }
 
 int ego_threads_available(void) {
@@ -225,14 +233,22 @@ static int cmp_idx(const void *a, const void *b) {
     return (p->idx < q->idx) ? -1 : (p->idx > q->idx);
 }
 
-/* Number of distinct ring neighbours of replica i and their ids (left first). */
-static int ring_neighbours(int P, int i, int nbr[2]) {
-    if (P <= 1) return 0;
-    int left = (i - 1 + P) % P, right = (i + 1) % P;
-    nbr[0] = left;
-    if (right == left) return 1;
-    nbr[1] = right;
-    return 2;
+/* Distinct neighbours of replica i on a ring where every PE talks to the `hops` nearest PEs on
+ * each side (hops = 1: the paper's ring; more: "if the number of neighbors of each PE is
+ * increased, information can flow sooner", Section 7).  Order: distance 1 left, distance 1
+ * right, distance 2 left, ...; a PE reached twice on a small ring is listed once and the PE
+ * itself never. Returns their number. */
+static int ring_neighbours(int P, int hops, int i, int nbr[2 * EGO_MAX_HOPS]) {
+    int n = 0;
+    for (int d = 1; d <= hops; ++d) {
+        const int cand[2] = {((i - d) % P + P) % P, (i + d) % P};
+        for (int side = 0; side < 2; ++side) {
+            int seen = cand[side] == i;
+            for (int q = 0; q < n && !seen; ++q) seen = nbr[q] == cand[side];
+            if (!seen) nbr[n++] = cand[side];
+        }
+    }
+    return n;
 }
 
 /* Phase A for one (replica i, tensor t): norm of the change, trigger test, threshold
@@ -326,9 +342,9 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
 /* Phase B for one (replica i, tensor t): average with the neighbours' last received
  * values and apply the gradient (Eq. (dist_sgd_event) with W_ij = 1/(N_i + 1)). */
 static void phase_b_segment(ego_ctx *c, float *x, const float *g, float lr, int i, int t) {
-    int nbr[2];
-    const int deg = ring_neighbours(c->P, i, nbr);
-    const float *hn[2];
+    int nbr[2 * EGO_MAX_HOPS];
+    const int deg = ring_neighbours(c->P, c->hops, i, nbr);
+    const float *hn[2 * EGO_MAX_HOPS];
     int cnt = 0;
     for (int q = 0; q < deg; ++q)
         if (c->valid[(int64_t)nbr[q] * c->T + t])
@@ -358,8 +374,8 @@ void ego_step(ego_ctx *c, float *x, const float *g, float lr) {
     /* message accounting: one message per (event, neighbour) */
     for (int64_t s = 0; s < S; ++s) {
         if (!c->flag[s]) continue;
-        int nbr[2];
-        const uint64_t deg = (uint64_t)ring_neighbours(c->P, (int)(s / c->T), nbr);
+        int nbr[2 * EGO_MAX_HOPS];
+        const uint64_t deg = (uint64_t)ring_neighbours(c->P, c->hops, (int)(s / c->T), nbr);
         c->events += 1;
         c->messages += deg;
         c->bytes += deg * c->seg_payload[s];

@@ -45,6 +45,7 @@ def _load():
         lib.ego_reset.argtypes = [C.c_void_p]
         lib.ego_set_threads.argtypes = [C.c_void_p, C.c_int]
         lib.ego_set_variant.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        lib.ego_set_hops.argtypes = [C.c_void_p, C.c_int]
         lib.ego_threads_available.restype = C.c_int
         lib.ego_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
         lib.ego_stats.argtypes = [C.c_void_p] + [C.POINTER(C.c_uint64)] * 3
@@ -86,7 +87,7 @@ class Oracle:
                  horizon: float = 1.0, history_len: int = 1, delta_init: float = 0.0,
                  delta_fixed: float = 0.0, force_first_event: bool = True,
                  topk: Optional[tuple] = None, threads: int = 1,
-                 own_last_sent: bool = False, change_of_norm: bool = False):
+                 own_last_sent: bool = False, change_of_norm: bool = False, hops: int = 1):
         lib = _load()
         self._lib = lib
         self.P, self.T = int(P), len(numel)
@@ -101,6 +102,8 @@ class Oracle:
             raise ValueError("ego_create rejected the arguments")
         lib.ego_set_threads(self._h, int(threads))
         lib.ego_set_variant(self._h, int(own_last_sent), int(change_of_norm))
+        if lib.ego_set_hops(self._h, int(hops)):
+            raise ValueError("hops out of range")
         self.S = self.P * self.T
         self.history_len = int(history_len)
 

@@ -108,7 +108,7 @@ class EventGrad:
     def __init__(self, P: int, layer_numel: Sequence[int], *, mode: int = THRESH_ADAPTIVE,
                  horizon: float = 1.0, history_len: int = 1, delta_init: float = 0.0,
                  delta_fixed: float = 0.0, force_first_event: bool = True,
-                 topk: Optional[tuple] = None, device: Optional[int] = None):
+                 topk: Optional[tuple] = None, device: Optional[int] = None, hops: int = 1):
         self._h = None
         lib = load_library()
         self._lib = lib
@@ -123,7 +123,7 @@ class EventGrad:
         arr = (C.c_int64 * self.T)(*self.numel)
         h = C.c_void_p()
         with torch.cuda.device(self.device):
-            st = lib.eg_create(C.byref(h), TOPO_RING, self.P, arr, self.T, C.byref(thr),
+            st = lib.eg_create(C.byref(h), TOPO_RING + int(hops) - 1, self.P, arr, self.T, C.byref(thr),
                                C.byref(tk) if tk else None)
         _check(lib, st, None, "eg_create")
         self._h = h

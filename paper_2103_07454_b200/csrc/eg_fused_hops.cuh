@@ -1,0 +1,116 @@
+// Fused dense snapshot / consensus average / SGD update for a ring in which every replica
+// averages with the `hops` nearest replicas on EACH side (Section 7: more neighbours per PE
+// let information flow sooner; W_ij = 1/(N_i + 1) as in Section 3).  hops == 1 is served by
+// the specialised kernels (eg_fused_pipe.cuh, eg_fused.cuh); this one is the general form.
+//
+// Same element-axis tiling: a thread owns one float4 column and walks the replicas in order.
+// No rolling state is needed: the value replica r contributes is x_hat_r once the thread has
+// processed r (a dense message has been written into x_hat_r by then), and x_r (dense message
+// this step) or x_hat_r before.  Neighbour values are re-read from L1/L2.
+#pragma once
+#include "eg_common.cuh"
+#include "eg_fused.cuh"
+
+namespace eg {
+
+constexpr int kMaxHops = 8;
+
+// grid n_tiles (1024-element tiles), kThreads threads; dynamic shared memory:
+//   P bytes of per-replica mode, rounded up to 16, then P*kWarps doubles when CARRY.
+template <bool CARRY>
+__global__ void __launch_bounds__(kThreads)
+k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
+             const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
+             int P, int T, long long stride, float lr, double* __restrict__ partials,
+             long long* step_k, int variant, int hops) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint8_t* s_mode = smem;                                       // bit 0: dense message, bit 1: valid
+    double* s_red = reinterpret_cast<double*>(smem + ((P + 15) & ~15));
+    __shared__ int s_off[2 * kMaxHops];                           // distinct neighbour offsets, in order
+    __shared__ int s_noff;
+    __shared__ double s_w[2 * kMaxHops + 1];                      // 1 / (1 + number heard from)
+
+    const int tile = blockIdx.x, tid = threadIdx.x;
+    const int t = tt.tensor[tile];
+    const int len = tt.length[tile];
+    const long long off = tt.offset[tile];
+    for (int j = tid; j < P; j += kThreads)
+        s_mode[j] = (uint8_t)((snap[(long long)j * T + t] ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0));
+    if (tid == 0) {
+        // offsets -1, +1, -2, +2, ... reduced mod P; one entry per distinct neighbour
+        int n = 0;
+        for (int d = 1; d <= hops; ++d) {
+            const int cand[2] = {((-d) % P + P) % P, d % P};
+            for (int side = 0; side < 2; ++side) {
+                bool seen = cand[side] == 0;
+                for (int q = 0; q < n && !seen; ++q) seen = s_off[q] == cand[side];
+                if (!seen) s_off[n++] = cand[side];
+            }
+        }
+        s_noff = n;
+        for (int q = 0; q <= 2 * kMaxHops; ++q) s_w[q] = __ddiv_rn(1.0, (double)(1 + q));
+        if (blockIdx.x == 0) *step_k += 1;   // nothing in this launch reads it
+    }
+    __syncthreads();
+
+    const int c = tid * 4;
+    const int nel = min(4, max(0, len - c));
+    const double neg_lr = -(double)lr;
+    const int noff = s_noff;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    float* xc = x + off + c;
+    const float* gc = g + off + c;
+    float* hc = xhat + off + c;
+
+    for (int j = 0; j < P; ++j) {
+        const bool sn = (s_mode[j] & 1) != 0;
+        double acc = 0.0;
+        if (nel > 0) {
+            const long long rb = (long long)j * stride;
+            const float4 xj = *reinterpret_cast<const float4*>(xc + rb);
+            const float4 gj = ld_stream(gc + rb);
+            const float4 hj = sn ? xj : *reinterpret_cast<const float4*>(hc + rb);   // own contribution
+            const float4 own = (variant & kOwnLastSent) ? hj : xj;
+            double s0 = (double)own.x, s1 = (double)own.y, s2 = (double)own.z, s3 = (double)own.w;
+            int cnt = 0;
+            for (int q = 0; q < noff; ++q) {
+                int r = j + s_off[q];
+                if (r >= P) r -= P;
+                const unsigned mode = s_mode[r];
+                if (!(mode & 2)) continue;                         // never heard from
+                // processed replicas (r < j) have their message, if any, in x_hat already
+                const float* src = (r > j && (mode & 1)) ? xc : hc;
+                const float4 v = *reinterpret_cast<const float4*>(src + (long long)r * stride);
+                s0 = __dadd_rn(s0, (double)v.x); s1 = __dadd_rn(s1, (double)v.y);
+                s2 = __dadd_rn(s2, (double)v.z); s3 = __dadd_rn(s3, (double)v.w);
+                ++cnt;
+            }
+            const double w = s_w[cnt];
+            float4 xn;
+            xn.x = __double2float_rn(__fma_rn(neg_lr, (double)gj.x, __dmul_rn(s0, w)));
+            xn.y = __double2float_rn(__fma_rn(neg_lr, (double)gj.y, __dmul_rn(s1, w)));
+            xn.z = __double2float_rn(__fma_rn(neg_lr, (double)gj.z, __dmul_rn(s2, w)));
+            xn.w = __double2float_rn(__fma_rn(neg_lr, (double)gj.w, __dmul_rn(s3, w)));
+            // the message first (later replicas read it), then the parameters
+            if (sn) store_masked(hc + rb, xj, nel);
+            store_masked(xc + rb, xn, nel);
+            if (CARRY) acc = sq_diff4(xn, (variant & kChangeOfNorm) ? zero4 : hj, nel, acc);
+        }
+        if (CARRY) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc = __dadd_rn(acc, __shfl_down_sync(0xffffffffu, acc, o));
+            if ((tid & 31) == 0) s_red[j * kWarps + (tid >> 5)] = acc;
+        }
+    }
+    if (CARRY) {
+        __syncthreads();
+        for (int j = tid; j < P; j += kThreads) {
+            double r = 0.0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) r = __dadd_rn(r, s_red[j * kWarps + w]);
+            partials[(long long)j * tt.n_tiles + tile] = r;
+        }
+    }
+}
+
+}  // namespace eg

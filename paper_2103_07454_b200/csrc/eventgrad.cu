@@ -11,6 +11,7 @@
 
 #include "eg_common.cuh"
 #include "eg_fused.cuh"
+#include "eg_fused_hops.cuh"
 #include "eg_fused_pipe.cuh"
 #include "eg_norm.cuh"
 #include "eg_topk.cuh"
@@ -47,6 +48,7 @@ struct eg_ctx {
     std::vector<int64_t> numel, offset, kcount, out_off;
     int64_t stride = 0, n_total = 0, out_stride = 0;
     int degree = 0;
+    int hops = 1;
     DeviceTiles tiles_norm, tiles_fused;
     // device state
     float* xhat = nullptr;
@@ -250,7 +252,8 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
                     const eg_threshold_params* thr, const eg_topk_params* topk) {
     if (!out) return EG_ERR_INVALID;
     *out = nullptr;
-    if (topology != EG_TOPO_RING || P < 1 || P > kMaxReplicas || T < 1 || !layer_numel || !thr)
+    if (topology < EG_TOPO_RING || topology >= kMaxHops || P < 1 || P > kMaxReplicas || T < 1 ||
+        !layer_numel || !thr)
         return EG_ERR_INVALID;
     if (thr->mode != EG_THRESH_ADAPTIVE && thr->mode != EG_THRESH_FIXED) return EG_ERR_INVALID;
     if (thr->history_len < 1 || thr->history_len > kMaxHistory) return EG_ERR_INVALID;
@@ -267,7 +270,8 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     if (cudaGetDevice(&c->device) != cudaSuccess) return fail(EG_ERR_CUDA);
     c->P = P; c->T = T; c->H = thr->history_len; c->thr = *thr;
     if (topk) c->topk = *topk;
-    c->degree = P == 1 ? 0 : (P == 2 ? 1 : 2);
+    c->hops = topology + 1;                       // EG_TOPO_RING_HOPS(m) == m - 1
+    c->degree = std::min(2 * c->hops, P - 1);     // distinct neighbours of every replica
     // layout: every tensor starts on a 128-byte boundary
     int64_t off = 0, koff = 0;
     for (int t = 0; t < T; ++t) {
@@ -326,6 +330,12 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(k_fused<kFusedVpt, false>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fused_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_fused_hops<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)c->fused_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_fused_hops<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)c->fused_smem);
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
     {
@@ -413,7 +423,16 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     // a3 + a5: dense snapshot, consensus average, SGD
     {
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
-        if (c->fused_kind == EG_FUSED_PIPELINED) {
+        if (c->hops > 1) {
+            if (c->carry)
+                k_fused_hops<true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                    c->partials_fused, c->step_k, c->variant, c->hops);
+            else
+                k_fused_hops<false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                    c->partials_fused, c->step_k, c->variant, c->hops);
+        } else if (c->fused_kind == EG_FUSED_PIPELINED) {
             if (c->carry)
                 k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
                     <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, true, kPipeConsumers / 32), stream>>>(

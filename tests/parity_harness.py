@@ -111,6 +111,8 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     okw.update(oracle_kw or {})
     o = eo.Oracle(wl.P, sub_numel, **okw)
     ekw = dict(eg_kw or {})
+    if "hops" in okw:
+        ekw.setdefault("hops", okw["hops"])
     ekw.pop("own_last_sent", None)
     ekw.pop("change_of_norm", None)
     for key in ("mode", "delta_fixed", "force_first_event", "horizon", "history_len", "delta_init"):

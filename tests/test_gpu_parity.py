@@ -38,6 +38,21 @@ def test_variants_own_term_and_change_of_norm(own, con, carry, kernel):
     assert 0 < rep.events < 5 * wl.T * wl.steps
 
 
+@pytest.mark.parametrize("P,hops", [(1, 2), (2, 2), (3, 2), (4, 2), (5, 2), (7, 3), (16, 2), (16, 8)])
+@pytest.mark.parametrize("carry", [False, True])
+def test_more_neighbours_per_side(P, hops, carry):
+    wl = W.synthetic(P, RAGGED[:-1], steps=10, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(hops=hops))
+    assert rep.params_bit_exact and not rep.near_threshold
+
+
+def test_more_neighbours_with_topk_and_variants():
+    wl = W.synthetic(6, RAGGED[:-1], steps=12, lr=0.1, grad_sigma=0.01, topk=(5, 100))
+    rep = lockstep(wl, init="distinct", carry=True, outbox_samples=32,
+                   oracle_kw=dict(hops=2, own_last_sent=True, change_of_norm=True))
+    assert rep.params_bit_exact
+
+
 def test_variant_with_topk():
     wl = W.synthetic(4, RAGGED[:-1], steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
     rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64,

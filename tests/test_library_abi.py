@@ -41,7 +41,8 @@ def test_create_rejects_bad_arguments_before_touching_the_device():
     numel = (ctypes.c_int64 * 2)(4, 0)
     assert lib.eg_create(ctypes.byref(h), 0, 4, numel, 2, ctypes.byref(thr), None) == 1   # empty tensor
     numel = (ctypes.c_int64 * 2)(4, 5)
-    assert lib.eg_create(ctypes.byref(h), 7, 4, numel, 2, ctypes.byref(thr), None) == 1   # topology
+    assert lib.eg_create(ctypes.byref(h), 8, 4, numel, 2, ctypes.byref(thr), None) == 1   # topology
+    assert lib.eg_create(ctypes.byref(h), -1, 4, numel, 2, ctypes.byref(thr), None) == 1
     assert lib.eg_create(ctypes.byref(h), 0, 0, numel, 2, ctypes.byref(thr), None) == 1   # P
     thr.history_len = 0
     assert lib.eg_create(ctypes.byref(h), 0, 4, numel, 2, ctypes.byref(thr), None) == 1   # H

@@ -17,12 +17,12 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 INF = float("inf")
 
 
-def ring_matrix(P):
+def ring_matrix(P, hops=1):
     """Mixing matrix of Section 3: W_ij = 1/(N_i + 1) over the PE itself and its distinct
-    ring neighbours."""
+    ring neighbours (the `hops` nearest on each side)."""
     Wm = np.zeros((P, P))
     for i in range(P):
-        nb = {i, (i - 1) % P, (i + 1) % P}
+        nb = {i} | {(i + d) % P for d in range(-hops, hops + 1)}
         for j in nb:
             Wm[i, j] = 1.0 / len(nb)
     return Wm
@@ -57,6 +57,42 @@ def test_zero_threshold_is_dpsgd(P):
         assert st["messages"] == P * wl.T * deg * (k + 1)
         assert st["bytes"] == 4 * wl.N * P * deg * (k + 1)
         assert st["events"] == P * wl.T * (k + 1)
+
+
+@pytest.mark.parametrize("P,hops", [(2, 2), (3, 2), (4, 2), (5, 2), (7, 3), (9, 2), (16, 4)])
+def test_more_neighbours_zero_threshold_is_xw(P, hops):
+    """More neighbours per PE (Section 7): W stays symmetric doubly stochastic with
+    W_ij = 1/(N_i + 1); threshold 0 still gives X W - gamma G, and the message count follows
+    the number of distinct neighbours."""
+    wl = small(P=P, steps=4, lr=0.1, grad_sigma=0.01)
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=0.0, hops=hops)
+    x = W.distinct_init_params(wl).numpy().copy()
+    Wm = ring_matrix(P, hops)
+    assert np.allclose(Wm.sum(0), 1) and np.allclose(Wm.sum(1), 1) and np.allclose(Wm, Wm.T)
+    deg = min(2 * hops, P - 1)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        ref = Wm @ x.astype(np.float64) - np.float64(np.float32(wl.lr)) * g.astype(np.float64)
+        o.step(x, g, wl.lr)
+        assert np.all(np.abs(x.astype(np.float64) - ref) <= 0.5000001 * ulp32(ref) + 1e-300)
+        assert o.stats()["messages"] == P * wl.T * deg * (k + 1)
+
+
+def test_more_neighbours_eigenmode_decay():
+    """Circulant W with 2 neighbours per side: eigenvalue (1 + 2cos(a) + 2cos(2a)) / 5, a = 2 pi m / P."""
+    P, m, hops = 12, 1, 2
+    o = eo.Oracle(P, [3], mode=eo.FIXED, delta_fixed=0.0, hops=hops)
+    mode = np.cos(2 * np.pi * m * np.arange(P) / P)
+    amp = np.array([1.0, -2.0, 0.5])
+    x = (mode[:, None] * amp[None, :]).astype(np.float32)
+    x_init = x.astype(np.float64)
+    a = 2 * math.pi * m / P
+    lam = (1 + 2 * math.cos(a) + 2 * math.cos(2 * a)) / 5
+    lam1 = (1 + 2 * math.cos(a)) / 3
+    assert lam < lam1                                   # information flows sooner
+    for s_ in range(1, 9):
+        o.step(x, np.zeros_like(x), 0.1)
+        assert np.all(np.abs(x - lam ** s_ * x_init) <= 3e-7 * np.abs(amp)[None, :] * s_ + 1e-12)
 
 
 # ---------------------------------------------------------------------------------------
