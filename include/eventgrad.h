@@ -133,6 +133,14 @@ enum { EG_OWN_CURRENT = 0, EG_OWN_LAST_SENT = 1 };
 enum { EG_TRIGGER_NORM_OF_CHANGE = 0, EG_TRIGGER_CHANGE_OF_NORM = 1 };
 eg_status eg_set_variant(eg_ctx* ctx, int own_term, int trigger_metric);
 
+/* Bound on the thresholds (Assumption 1 of Section 5, with the geometric sequence
+ * g(k) = alpha * beta^k of Corollary 2): the threshold a tensor is tested against in iteration
+ * k becomes min(delta, sqrt(alpha * beta^k)); the adaptive delta itself is left as computed.
+ * alpha <= 0 removes the bound (default).  The bound of a step is evaluated on the host when
+ * eg_step is called (from the host's copy of the iteration counter) and passed to the device
+ * as a kernel argument. */
+eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
+
 /* Which implementation of the fused snapshot / average / SGD kernel eg_step launches.  Both
  * compute bit-identical results.  EG_FUSED_PIPELINED (default) streams the operands through
  * shared memory with bulk asynchronous copies; EG_FUSED_REGISTER keeps the ring walk in

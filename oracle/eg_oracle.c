@@ -107,6 +107,8 @@ typedef struct ego_ctx {
                              ("the norm of a parameter has changed by some threshold") */
     double *sent_norm;    /* [P*T] ||x|| at the last event (0 before the first) */
     int hops;             /* ring neighbours on each side (1 = the paper's ring) */
+    double cap_alpha, cap_beta; /* bound g(k) = alpha * beta^k on the squared threshold
+                                   (Assumption 1, Corollary 2); alpha <= 0: no bound */
 } ego_ctx;
 
 void ego_destroy(ego_ctx *c) {
@@ -198,6 +200,11 @@ void ego_set_variant(ego_ctx *c, int own_last_sent, int change_of_norm) {
     c->change_of_norm = change_of_norm != 0;
 }
 
+void ego_set_threshold_cap(ego_ctx *c, double alpha, double beta) {
+    c->cap_alpha = alpha;
+    c->cap_beta = beta;
+}
+
 int ego_set_hops(ego_ctx *c, int hops) {
     if (hops < 1 || hops > EGO_MAX_HOPS) return 1;
     c->hops = hops;
@@ -279,7 +286,13 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
         }
         d = fabs(sqrt(acc) - c->sent_norm[s]);
     }
-    const double thr = c->delta[s];
+    /* the threshold in force, bounded by sqrt(g(k)) when a bound is set (Assumption 1 with
+     * g(k) = alpha * beta^k of Corollary 2) */
+    double thr = c->delta[s];
+    if (c->cap_alpha > 0.0) {
+        const double cap = sqrt(c->cap_alpha * pow(c->cap_beta, (double)c->k));
+        if (cap < thr) thr = cap;
+    }
     c->norm[s] = d;
     c->thr_used[s] = thr;
 

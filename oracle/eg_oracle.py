@@ -46,6 +46,7 @@ def _load():
         lib.ego_set_threads.argtypes = [C.c_void_p, C.c_int]
         lib.ego_set_variant.argtypes = [C.c_void_p, C.c_int, C.c_int]
         lib.ego_set_hops.argtypes = [C.c_void_p, C.c_int]
+        lib.ego_set_threshold_cap.argtypes = [C.c_void_p, C.c_double, C.c_double]
         lib.ego_threads_available.restype = C.c_int
         lib.ego_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
         lib.ego_stats.argtypes = [C.c_void_p] + [C.POINTER(C.c_uint64)] * 3
@@ -87,7 +88,8 @@ class Oracle:
                  horizon: float = 1.0, history_len: int = 1, delta_init: float = 0.0,
                  delta_fixed: float = 0.0, force_first_event: bool = True,
                  topk: Optional[tuple] = None, threads: int = 1,
-                 own_last_sent: bool = False, change_of_norm: bool = False, hops: int = 1):
+                 own_last_sent: bool = False, change_of_norm: bool = False, hops: int = 1,
+                 threshold_cap: Optional[tuple] = None):
         lib = _load()
         self._lib = lib
         self.P, self.T = int(P), len(numel)
@@ -104,6 +106,8 @@ class Oracle:
         lib.ego_set_variant(self._h, int(own_last_sent), int(change_of_norm))
         if lib.ego_set_hops(self._h, int(hops)):
             raise ValueError("hops out of range")
+        if threshold_cap:
+            lib.ego_set_threshold_cap(self._h, float(threshold_cap[0]), float(threshold_cap[1]))
         self.S = self.P * self.T
         self.history_len = int(history_len)
 

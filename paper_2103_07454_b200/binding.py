@@ -26,7 +26,7 @@ EXPORTS = [
     "eg_event_count", "eg_last_decisions", "eg_thresholds", "eg_last_outbox", "eg_topk_count",
     "eg_read_mailboxes", "eg_average_model", "eg_export_state", "eg_import_state", "eg_reset",
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
-    "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant",
+    "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant", "eg_set_threshold_cap",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -83,6 +83,7 @@ def load_library() -> C.CDLL:
     lib.eg_set_timing.argtypes = [vp, C.c_int]
     lib.eg_set_fused_kernel.argtypes = [vp, C.c_int]
     lib.eg_set_variant.argtypes = [vp, C.c_int, C.c_int]
+    lib.eg_set_threshold_cap.argtypes = [vp, C.c_double, C.c_double]
     lib.eg_change_norms_static.argtypes = [vp, vp, C.c_int, C.c_int64, i64p, i64p, C.c_int, vp, vp]
     lib.eg_kernel_times.argtypes = [vp, C.POINTER(C.c_double), u64p]
     lib.eg_destroy.argtypes = [vp]
@@ -262,6 +263,11 @@ class EventGrad:
         """``eg_set_variant``: alternative readings of the own term / the tested quantity."""
         _check(self._lib, self._lib.eg_set_variant(self._h, int(own_last_sent), int(change_of_norm)),
                self._h, "eg_set_variant")
+
+    def set_threshold_cap(self, alpha: float, beta: float):
+        """``eg_set_threshold_cap``: thresholds bounded by sqrt(alpha * beta**k)."""
+        _check(self._lib, self._lib.eg_set_threshold_cap(self._h, float(alpha), float(beta)),
+               self._h, "eg_set_threshold_cap")
 
     def set_fused_kernel(self, kind: int):
         _check(self._lib, self._lib.eg_set_fused_kernel(self._h, int(kind)), self._h,

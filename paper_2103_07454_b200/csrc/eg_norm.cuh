@@ -61,6 +61,7 @@ struct DecideParams {
     int topk;                 // Top-K messages enabled
     int degree;               // distinct ring neighbours of every replica
     int variant;              // kChangeOfNorm: d = | sqrt(sum) - sent_norm |
+    double cap;               // bound sqrt(g(k)) on the threshold of this step (+inf: none)
 };
 
 // One warp per (replica, tensor).  grid ceil(P*T / kWarps).
@@ -84,7 +85,7 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     const long long k = *step_k;
     const double root = __dsqrt_rn(acc);
     const double d = (dp.variant & kChangeOfNorm) ? fabs(__dsub_rn(root, st.sent_norm[s])) : root;
-    const double thr = st.delta[s];
+    const double thr = fmin(st.delta[s], dp.cap);
     st.norm[s] = d;
     st.thr_used[s] = thr;
     const bool fire = (dp.force_first && k == 0) || (d >= thr);

@@ -73,6 +73,8 @@ struct eg_ctx {
     size_t fused_smem = 0;
     int fused_kind = EG_FUSED_PIPELINED;
     int variant = 0;
+    double cap_alpha = 0.0, cap_beta = 1.0;   // bound alpha*beta^k on the squared threshold
+    long long host_k = 0;                     // host copy of the iteration counter
     bool stepped = false;   // a step has run since creation / reset / import
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
@@ -170,6 +172,7 @@ eg_status init_state(eg_ctx* c) {
     }
     c->carried_valid = false;
     c->stepped = false;
+    c->host_k = 0;
     return EG_OK;
 }
 
@@ -395,7 +398,9 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     }
     // a2 + a6: decision, threshold update, counters
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
-                    c->topk.enabled, c->degree, c->variant};
+                    c->topk.enabled, c->degree, c->variant,
+                    c->cap_alpha > 0.0 ? std::sqrt(c->cap_alpha * std::pow(c->cap_beta, (double)c->host_k))
+                                       : HUGE_VAL};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf : tn;
     {
@@ -456,6 +461,7 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     c->carried_valid = c->carry;
     c->carried_params = params;
     c->stepped = true;
+    c->host_k += 1;
     c->last_launches = launches;
     EG_CUDA(c, cudaGetLastError());
     return EG_OK;
@@ -567,6 +573,13 @@ eg_status eg_set_variant(eg_ctx* c, int own_term, int trigger_metric) {
     c->variant = (own_term == EG_OWN_LAST_SENT ? kOwnLastSent : 0) |
                  (trigger_metric == EG_TRIGGER_CHANGE_OF_NORM ? kChangeOfNorm : 0);
     c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status eg_set_threshold_cap(eg_ctx* c, double alpha, double beta) {
+    if (!c || std::isnan(alpha) || std::isnan(beta) || (alpha > 0.0 && !(beta > 0.0))) return EG_ERR_INVALID;
+    c->cap_alpha = alpha;
+    c->cap_beta = beta;
     return EG_OK;
 }
 
@@ -758,6 +771,7 @@ eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
     EG_CUDA(c, cudaDeviceSynchronize());
     c->carried_valid = false;
     c->stepped = h.step > 0;
+    c->host_k = h.step;
     return EG_OK;
 }
 

@@ -111,8 +111,10 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     okw.update(oracle_kw or {})
     o = eo.Oracle(wl.P, sub_numel, **okw)
     ekw = dict(eg_kw or {})
+    cap = okw.get("threshold_cap")
     if "hops" in okw:
         ekw.setdefault("hops", okw["hops"])
+    ekw.pop("threshold_cap", None)
     ekw.pop("own_last_sent", None)
     ekw.pop("change_of_norm", None)
     for key in ("mode", "delta_fixed", "force_first_event", "horizon", "history_len", "delta_init"):
@@ -122,6 +124,8 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     eg.set_carry_norm(carry)
     eg.set_fused_kernel(fused_kernel)
     eg.set_variant(bool(okw.get("own_last_sent")), bool(okw.get("change_of_norm")))
+    if cap:
+        eg.set_threshold_cap(*cap)
 
     x0 = W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)
     x_dev = eg.to_layout(x0)

@@ -53,6 +53,15 @@ def test_more_neighbours_with_topk_and_variants():
     assert rep.params_bit_exact
 
 
+@pytest.mark.parametrize("carry", [False, True])
+def test_geometric_threshold_cap(carry):
+    wl = W.synthetic(4, RAGGED[:-1], steps=20, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(threshold_cap=(1e-3, 0.7)))
+    free = lockstep(wl, init="distinct", carry=carry)
+    assert rep.params_bit_exact and not rep.near_threshold
+    assert rep.events > free.events          # a shrinking bound makes tensors communicate more
+
+
 def test_variant_with_topk():
     wl = W.synthetic(4, RAGGED[:-1], steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
     rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64,

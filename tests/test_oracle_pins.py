@@ -281,6 +281,35 @@ def test_hand_worked_threshold_sequence(case):
         assert o.thresholds()[0, 0] == pytest.approx(thr_after, rel=1e-15, abs=0)
 
 
+def test_geometric_bound_on_the_threshold():
+    """Assumption 1 with g(k) = alpha beta^k (Corollary 2): the threshold in force is
+    min(delta, sqrt(g(k))).  alpha = 16, beta = 1/4: sqrt(g) = 4, 2, 1, 1/2, 1/4 (exact).
+    x moves along u = (0.75, 1), |u| = 1.25, by 1, 1, 1, 1/2, 1/4 units; fixed delta = 2."""
+    o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=2.0, force_first_event=False,
+                  threshold_cap=(16.0, 0.25))
+    steps_u = [1.0, 1.0, 1.0, 0.5, 0.25]
+    x = np.zeros((1, 2), np.float32)
+    pos = 0.0
+    want = [(0, 1.25, 2.0), (1, 2.5, 2.0), (1, 1.25, 1.0), (1, 0.625, 0.5), (1, 0.3125, 0.25)]
+    for k, du in enumerate(steps_u):
+        pos += du
+        x[0] = [0.75 * pos, pos]
+        o.step(x, np.zeros_like(x), 1.0)
+        flag, d, thr = want[k]
+        assert int(o.flags()[0, 0]) == flag and o.norms()[0, 0] == d
+        assert o.thresholds_used()[0, 0] == thr and o.thresholds()[0, 0] == 2.0
+    # without the bound: k = 1 fires (d = 2.5), then d = 1.25, 1.875, 2.1875 -> k = 4 fires again
+    o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=2.0, force_first_event=False)
+    x[:] = 0
+    pos, fired = 0.0, []
+    for du in steps_u:
+        pos += du
+        x[0] = [0.75 * pos, pos]
+        o.step(x, np.zeros_like(x), 1.0)
+        fired.append(int(o.flags()[0, 0]))
+    assert fired == [0, 1, 0, 0, 1]
+
+
 def test_fixed_threshold_never_adapts():
     o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=2.0, force_first_event=False)
     x = np.zeros((1, 2), np.float32)
