@@ -107,6 +107,13 @@ typedef struct ego_ctx {
                              ("the norm of a parameter has changed by some threshold") */
     double *sent_norm;    /* [P*T] ||x|| at the last event (0 before the first) */
     int hops;             /* ring neighbours on each side (1 = the paper's ring) */
+    /* intermittent delivery (Section 7 remarks on the "stochastic nature of the MPI one-sided
+     * implementation"): x_hat is what a replica has SENT, mailbox what its neighbours have
+     * RECEIVED; they differ while a message is in flight.  NULL until a delivery mask is used. */
+    float *mailbox;       /* [P][N] */
+    uint8_t *pending;     /* [P*T] something sent has not arrived yet */
+    uint8_t *recv_valid;  /* [P*T] the neighbours have received this tensor at least once */
+    uint64_t arrivals;
     double cap_alpha, cap_beta; /* bound g(k) = alpha * beta^k on the squared threshold
                                    (Assumption 1, Corollary 2); alpha <= 0: no bound */
 } ego_ctx;
@@ -117,6 +124,7 @@ void ego_destroy(ego_ctx *c) {
     free(c->delta); free(c->khat); free(c->hist); free(c->hist_len); free(c->valid);
     free(c->flag); free(c->norm); free(c->thr_used); free(c->out_idx); free(c->out_val);
     free(c->out_count); free(c->seg_events); free(c->seg_payload); free(c->sent_norm);
+    free(c->mailbox); free(c->pending); free(c->recv_valid);
     free(c);
 }
 
@@ -124,6 +132,12 @@ void ego_reset(ego_ctx *c) {
     int64_t S = (int64_t)c->P * c->T;
     c->k = 0;
     c->messages = c->bytes = c->events = 0;
+    c->arrivals = 0;
+    if (c->mailbox) {
+        memset(c->mailbox, 0, sizeof(float) * (size_t)c->P * (size_t)c->N);
+        memset(c->pending, 0, (size_t)S);
+        memset(c->recv_valid, 0, (size_t)S);
+    }
     memset(c->xhat, 0, sizeof(float) * (size_t)c->P * (size_t)c->N); /* X_0 = 0, Assumption 2.4 */
     for (int64_t s = 0; s < S; ++s) {
         c->delta[s] = (c->mode == EGO_FIXED) ? c->delta_fixed : c->delta_init;
@@ -359,9 +373,11 @@ static void phase_b_segment(ego_ctx *c, float *x, const float *g, float lr, int 
     const int deg = ring_neighbours(c->P, c->hops, i, nbr);
     const float *hn[2 * EGO_MAX_HOPS];
     int cnt = 0;
+    const float *box = c->mailbox ? c->mailbox : c->xhat;          /* what neighbours hold */
+    const uint8_t *heard = c->mailbox ? c->recv_valid : c->valid;
     for (int q = 0; q < deg; ++q)
-        if (c->valid[(int64_t)nbr[q] * c->T + t])
-            hn[cnt++] = c->xhat + (int64_t)nbr[q] * c->N + c->off[t];
+        if (heard[(int64_t)nbr[q] * c->T + t])
+            hn[cnt++] = box + (int64_t)nbr[q] * c->N + c->off[t];
     const double w = 1.0 / (double)(1 + cnt);
     float *xs = x + (int64_t)i * c->N + c->off[t];
     const float *gs = g + (int64_t)i * c->N + c->off[t];
@@ -376,9 +392,29 @@ static void phase_b_segment(ego_ctx *c, float *x, const float *g, float lr, int 
     }
 }
 
-/* One iteration of Algorithm B for all replicas.  x is updated in place. */
-void ego_step(ego_ctx *c, float *x, const float *g, float lr) {
+/* Switches to the two-copy model (sent / received).  Everything sent so far has arrived. */
+int ego_enable_delivery_masks(ego_ctx *c) {
+    if (c->mailbox) return 0;
     const int64_t S = (int64_t)c->P * c->T;
+    const size_t bytes = sizeof(float) * (size_t)c->P * (size_t)c->N;
+    c->mailbox = (float *)malloc(bytes);
+    c->pending = (uint8_t *)calloc((size_t)S, 1);
+    c->recv_valid = (uint8_t *)malloc((size_t)S);
+    if (!c->mailbox || !c->pending || !c->recv_valid) return 1;
+    memcpy(c->mailbox, c->xhat, bytes);
+    memcpy(c->recv_valid, c->valid, (size_t)S);
+    return 0;
+}
+
+/* One iteration of Algorithm B for all replicas.  x is updated in place.
+ * deliver (may be NULL = everything arrives at once): deliver[i*T+t] != 0 means that whatever
+ * replica i has sent of tensor t and has not arrived yet -- this iteration's message
+ * included -- arrives at its neighbours now, before they average; 0 keeps it in flight.
+ * A later message overwrites an earlier one in flight, as a later put into the same window
+ * location does. */
+void ego_step_masked(ego_ctx *c, float *x, const float *g, float lr, const uint8_t *deliver) {
+    const int64_t S = (int64_t)c->P * c->T;
+    if (deliver && !c->mailbox) ego_enable_delivery_masks(c);
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1) num_threads(c->threads)
 #endif
@@ -394,6 +430,21 @@ void ego_step(ego_ctx *c, float *x, const float *g, float lr) {
         c->bytes += deg * c->seg_payload[s];
     }
 
+    /* arrivals */
+    if (c->mailbox) {
+        for (int64_t s = 0; s < S; ++s) {
+            if (c->flag[s]) c->pending[s] = 1;
+            if (c->pending[s] && (!deliver || deliver[s])) {
+                const int i = (int)(s / c->T), t = (int)(s % c->T);
+                const int64_t o = (int64_t)i * c->N + c->off[t];
+                memcpy(c->mailbox + o, c->xhat + o, sizeof(float) * (size_t)c->numel[t]);
+                c->pending[s] = 0;
+                c->recv_valid[s] = 1;
+                c->arrivals += 1;
+            }
+        }
+    }
+
     /* every mailbox is final before anybody averages */
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1) num_threads(c->threads)
@@ -403,6 +454,8 @@ void ego_step(ego_ctx *c, float *x, const float *g, float lr) {
 
     c->k += 1;
 }
+
+void ego_step(ego_ctx *c, float *x, const float *g, float lr) { ego_step_masked(c, x, g, lr, NULL); }
 
 /* ---- readers ---------------------------------------------------------------------- */
 void ego_stats(const ego_ctx *c, uint64_t *messages, uint64_t *bytes, uint64_t *events) {
@@ -423,6 +476,9 @@ const double *ego_sent_norms(const ego_ctx *c) { return c->sent_norm; }
 const double *ego_history(const ego_ctx *c) { return c->hist; }
 const int *ego_history_len(const ego_ctx *c) { return c->hist_len; }
 float *ego_xhat(ego_ctx *c) { return c->xhat; }
+float *ego_received(ego_ctx *c) { return c->mailbox ? c->mailbox : c->xhat; }
+const uint8_t *ego_pending(const ego_ctx *c) { return c->pending; }
+uint64_t ego_arrivals(const ego_ctx *c) { return c->arrivals; }
 int64_t ego_topk_count(const ego_ctx *c, int t) { return c->Kt[t]; }
 int32_t ego_outbox(const ego_ctx *c, int i, int t, const int32_t **idx, const float **val) {
     const int64_t o = (int64_t)i * c->out_off[c->T] + c->out_off[t];

@@ -49,6 +49,14 @@ def _load():
         lib.ego_set_threshold_cap.argtypes = [C.c_void_p, C.c_double, C.c_double]
         lib.ego_threads_available.restype = C.c_int
         lib.ego_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
+        lib.ego_step_masked.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
+        lib.ego_enable_delivery_masks.argtypes = [C.c_void_p]
+        lib.ego_received.restype = C.c_void_p
+        lib.ego_received.argtypes = [C.c_void_p]
+        lib.ego_pending.restype = C.c_void_p
+        lib.ego_pending.argtypes = [C.c_void_p]
+        lib.ego_arrivals.restype = C.c_uint64
+        lib.ego_arrivals.argtypes = [C.c_void_p]
         lib.ego_stats.argtypes = [C.c_void_p] + [C.POINTER(C.c_uint64)] * 3
         lib.ego_iteration.restype = C.c_int64
         lib.ego_iteration.argtypes = [C.c_void_p]
@@ -124,11 +132,36 @@ class Oracle:
     def set_threads(self, n: int):
         self._lib.ego_set_threads(self._h, int(n))
 
-    def step(self, x: np.ndarray, g: np.ndarray, lr: float):
+    def step(self, x: np.ndarray, g: np.ndarray, lr: float, deliver: Optional[np.ndarray] = None):
+        """One iteration; ``deliver`` ([P, T] uint8, optional) says whose outstanding messages
+        arrive in this iteration (default: all, i.e. synchronous delivery)."""
         assert x.dtype == np.float32 and g.dtype == np.float32
         assert x.flags.c_contiguous and g.flags.c_contiguous
         assert x.shape == (self.P, self.N) and g.shape == (self.P, self.N)
-        self._lib.ego_step(self._h, x.ctypes.data, g.ctypes.data, C.c_float(lr))
+        if deliver is None:
+            self._lib.ego_step(self._h, x.ctypes.data, g.ctypes.data, C.c_float(lr))
+        else:
+            d = np.ascontiguousarray(deliver, dtype=np.uint8)
+            assert d.size == self.S
+            self._lib.ego_step_masked(self._h, x.ctypes.data, g.ctypes.data, C.c_float(lr), d.ctypes.data)
+
+    def enable_delivery_masks(self):
+        self._lib.ego_enable_delivery_masks(self._h)
+
+    def received(self) -> np.ndarray:
+        """Copy of what the neighbours hold of every replica (== xhat() under synchronous delivery)."""
+        return _view(self._lib.ego_received(self._h), np.float32, self.P * self.N).reshape(
+            self.P, self.N).copy()
+
+    def pending(self):
+        p = self._lib.ego_pending(self._h)
+        if not p:
+            return np.zeros((self.P, self.T), np.uint8)
+        return _view(p, np.uint8, self.S).reshape(self.P, self.T).copy()
+
+    @property
+    def arrivals(self) -> int:
+        return int(self._lib.ego_arrivals(self._h))
 
     @property
     def iteration(self) -> int:

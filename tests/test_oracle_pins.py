@@ -382,6 +382,86 @@ def test_change_of_norm_ignores_rotations():
 
 
 # ---------------------------------------------------------------------------------------
+# intermittent delivery (messages that stay in flight)
+# ---------------------------------------------------------------------------------------
+def test_delivering_everything_is_synchronous_delivery():
+    wl = small(P=4, steps=12, lr=0.1, grad_sigma=0.01, topk=(1, 4))
+    a, b = eo.from_workload(wl), eo.from_workload(wl)
+    xa = W.distinct_init_params(wl).numpy().copy()
+    xb = xa.copy()
+    ones = np.ones((wl.P, wl.T), np.uint8)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        a.step(xa, g, wl.lr)
+        b.step(xb, g, wl.lr, deliver=ones)
+        assert np.array_equal(xa, xb) and np.array_equal(a.flags(), b.flags())
+        assert np.array_equal(b.received(), b.xhat()) and not b.pending().any()
+    assert a.stats() == b.stats() and b.arrivals == b.stats()["events"]
+
+
+def test_nothing_ever_delivered_is_independent_sgd_although_events_happen():
+    wl = small(P=4, steps=6, lr=0.25, grad_sigma=0.02)
+    o = eo.from_workload(wl)
+    x0 = W.distinct_init_params(wl).numpy().copy()
+    x = x0.copy()
+    ref = x0.astype(np.float64)
+    none = np.zeros((wl.P, wl.T), np.uint8)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        o.step(x, g, wl.lr, deliver=none)
+        ref = (ref - np.float64(np.float32(wl.lr)) * g.astype(np.float64)).astype(np.float32).astype(np.float64)
+        assert np.all(np.abs(x - ref) <= ulp32(ref))
+    assert o.stats()["events"] >= wl.P * wl.T and o.arrivals == 0
+    assert o.pending().all() and np.all(o.received() == 0)
+
+
+def test_links_that_are_up_every_other_step():
+    """Threshold 0 (everything is sent every step); links deliver on even steps only.  On an even
+    step neighbours average with x_k, on an odd step with the stale x_{k-1}."""
+    P = 5
+    wl = small(P=P, steps=6, lr=0.1, grad_sigma=0.02)
+    lr64 = np.float64(np.float32(wl.lr))
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=0.0)
+    x = W.distinct_init_params(wl).numpy().copy()
+    stale = None
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        up = k % 2 == 0
+        cur = x.astype(np.float64)
+        box = cur if up else stale
+        ref = (cur + np.roll(box, 1, axis=0) + np.roll(box, -1, axis=0)) / 3.0 - lr64 * g.astype(np.float64)
+        o.step(x, g, wl.lr, deliver=np.full((P, wl.T), int(up), np.uint8))
+        assert np.all(np.abs(x - ref) <= ulp32(ref))
+        if up:
+            stale = cur
+        assert o.pending().all() == (not up) and np.array_equal(o.received(), stale.astype(np.float32))
+    assert o.arrivals == P * wl.T * 3
+
+
+def test_outstanding_sparse_messages_arrive_together():
+    """A delivery hands over everything outstanding: afterwards the receivers' copy equals
+    the sender's record, before it is untouched."""
+    wl = small(P=3, numel=(40, 300), steps=10, lr=0.1, grad_sigma=0.02, topk=(1, 10))
+    o = eo.Oracle(3, wl.numel, mode=eo.FIXED, delta_fixed=0.0, topk=wl.topk)
+    x = W.distinct_init_params(wl).numpy().copy()
+    rng = np.random.default_rng(0)
+    for k in range(wl.steps):
+        mask = (rng.random((3, wl.T)) < 0.4).astype(np.uint8)
+        before = o.received() if k else np.zeros_like(x)
+        o.step(x, wl.grads(k).numpy(), wl.lr, deliver=mask)
+        sent, got = o.xhat(), o.received()
+        off = 0
+        for t, n in enumerate(wl.numel):
+            for i in range(3):
+                seg = slice(off, off + n)
+                if mask[i, t]:
+                    assert np.array_equal(got[i, seg], sent[i, seg])
+                else:
+                    assert np.array_equal(got[i, seg], before[i, seg])
+            off += n
+
+
+# ---------------------------------------------------------------------------------------
 # Top-K
 # ---------------------------------------------------------------------------------------
 def brute_force_topk(x_row, xhat_row, K):
