@@ -133,6 +133,28 @@ enum { EG_OWN_CURRENT = 0, EG_OWN_LAST_SENT = 1 };
 enum { EG_TRIGGER_NORM_OF_CHANGE = 0, EG_TRIGGER_CHANGE_OF_NORM = 1 };
 eg_status eg_set_variant(eg_ctx* ctx, int own_term, int trigger_metric);
 
+/* Intermittent delivery.  Section 7 remarks that the one-sided puts of the paper's
+ * implementation arrive at unpredictable times; this models it with links that are up or down
+ * per iteration.  After eg_enable_delivery_masks the context keeps two copies per replica: what
+ * it has SENT (x_hat, the reference of its trigger test) and what its neighbours have RECEIVED
+ * (the mailbox they average with).  eg_step_masked is eg_step with a device array
+ * deliver_dev[P*T] (uint8): a non-zero entry [i*T + t] lets everything replica i has sent of
+ * tensor t and that has not arrived yet -- this iteration's message included -- arrive now,
+ * before the neighbours average; zero keeps it in flight (a later message replaces an earlier
+ * one in flight, as a later put into the same window does).  deliver_dev == NULL (and plain
+ * eg_step) delivers everything outstanding.  eg_enable_delivery_masks allocates the second
+ * copy (P*replica_stride floats) and synchronises; everything sent until then counts as
+ * arrived.  Not available together with EG_OWN_LAST_SENT, the carried norm is not used while
+ * it is on, and a context with it enabled cannot be checkpointed (EG_ERR_STATE).
+ * eg_read_received copies the received copies to the host ([P][replica_stride] fp32; equal to
+ * eg_read_mailboxes under synchronous delivery); eg_delivery_status returns the per-(replica,
+ * tensor) "in flight" flags (host, P*T bytes) and the number of arrivals so far. */
+eg_status eg_enable_delivery_masks(eg_ctx* ctx);
+eg_status eg_step_masked(eg_ctx* ctx, float* params, const float* grads, float lr,
+                         const uint8_t* deliver_dev, void* stream);
+eg_status eg_read_received(eg_ctx* ctx, float* received_host);
+eg_status eg_delivery_status(eg_ctx* ctx, uint8_t* pending_host, uint64_t* arrivals_host);
+
 /* Bound on the thresholds (Assumption 1 of Section 5, with the geometric sequence
  * g(k) = alpha * beta^k of Corollary 2): the threshold a tensor is tested against in iteration
  * k becomes min(delta, sqrt(alpha * beta^k)); the adaptive delta itself is left as computed.

@@ -27,6 +27,7 @@ EXPORTS = [
     "eg_read_mailboxes", "eg_average_model", "eg_export_state", "eg_import_state", "eg_reset",
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
     "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant", "eg_set_threshold_cap",
+    "eg_enable_delivery_masks", "eg_step_masked", "eg_read_received", "eg_delivery_status",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -84,6 +85,10 @@ def load_library() -> C.CDLL:
     lib.eg_set_fused_kernel.argtypes = [vp, C.c_int]
     lib.eg_set_variant.argtypes = [vp, C.c_int, C.c_int]
     lib.eg_set_threshold_cap.argtypes = [vp, C.c_double, C.c_double]
+    lib.eg_enable_delivery_masks.argtypes = [vp]
+    lib.eg_step_masked.argtypes = [vp, vp, vp, C.c_float, vp, vp]
+    lib.eg_read_received.argtypes = [vp, vp]
+    lib.eg_delivery_status.argtypes = [vp, vp, u64p]
     lib.eg_change_norms_static.argtypes = [vp, vp, C.c_int, C.c_int64, i64p, i64p, C.c_int, vp, vp]
     lib.eg_kernel_times.argtypes = [vp, C.POINTER(C.c_double), u64p]
     lib.eg_destroy.argtypes = [vp]
@@ -179,6 +184,36 @@ class EventGrad:
         st = self._lib.eg_step(self._h, params.data_ptr(), grads.data_ptr(), C.c_float(lr),
                                C.c_void_p(s.cuda_stream))
         _check(self._lib, st, self._h, "eg_step")
+
+    def enable_delivery_masks(self):
+        _check(self._lib, self._lib.eg_enable_delivery_masks(self._h), self._h,
+               "eg_enable_delivery_masks")
+
+    def step_masked(self, params: torch.Tensor, grads: torch.Tensor, lr: float,
+                    deliver: Optional[torch.Tensor], stream: Optional[torch.cuda.Stream] = None):
+        """``eg_step_masked``: ``deliver`` is a uint8 device tensor of ``P*T`` entries or None."""
+        assert params.shape == grads.shape == (self.P, self.replica_stride)
+        if deliver is not None:
+            assert deliver.is_cuda and deliver.dtype == torch.uint8 and deliver.is_contiguous()
+            assert deliver.numel() == self.P * self.T
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        st = self._lib.eg_step_masked(self._h, params.data_ptr(), grads.data_ptr(), C.c_float(lr),
+                                      deliver.data_ptr() if deliver is not None else None,
+                                      C.c_void_p(s.cuda_stream))
+        _check(self._lib, st, self._h, "eg_step_masked")
+
+    def received(self) -> torch.Tensor:
+        out = torch.empty((self.P, self.replica_stride), dtype=torch.float32)
+        _check(self._lib, self._lib.eg_read_received(self._h, out.data_ptr()), self._h,
+               "eg_read_received")
+        return out
+
+    def delivery_status(self):
+        pend = np.empty(self.P * self.T, np.uint8)
+        arr = C.c_uint64()
+        _check(self._lib, self._lib.eg_delivery_status(self._h, pend.ctypes.data, C.byref(arr)),
+               self._h, "eg_delivery_status")
+        return pend.reshape(self.P, self.T), int(arr.value)
 
     def step_host(self, params_host: torch.Tensor, grads_host: torch.Tensor, lr: float):
         """``eg_step_host``: the same iteration with host-resident buffers."""

@@ -22,9 +22,12 @@ __global__ void __launch_bounds__(kThreads)
 k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
-             long long* step_k, int variant, int hops) {
+             long long* step_k, int variant, int hops, float* mailbox = nullptr,
+             const uint8_t* __restrict__ arrive = nullptr) {
+    // Intermittent delivery (arrive != nullptr): x_hat is the SENT copy, `mailbox` the RECEIVED
+    // one, `valid` means "received at least once"; otherwise both copies are x_hat.
     extern __shared__ __align__(128) unsigned char smem[];
-    uint8_t* s_mode = smem;                                       // bit 0: dense message, bit 1: valid
+    uint8_t* s_mode = smem;   // bit 0: dense message, bit 1: valid, bit 2: contributes own x, bit 3: arrives
     double* s_red = reinterpret_cast<double*>(smem + ((P + 15) & ~15));
     __shared__ int s_off[2 * kMaxHops];                           // distinct neighbour offsets, in order
     __shared__ int s_noff;
@@ -34,8 +37,13 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
     const int t = tt.tensor[tile];
     const int len = tt.length[tile];
     const long long off = tt.offset[tile];
-    for (int j = tid; j < P; j += kThreads)
-        s_mode[j] = (uint8_t)((snap[(long long)j * T + t] ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0));
+    const bool async = arrive != nullptr;
+    for (int j = tid; j < P; j += kThreads) {
+        const bool sn = snap[(long long)j * T + t] != 0;
+        const bool ar = async ? (arrive[(long long)j * T + t] != 0) : sn;
+        s_mode[j] = (uint8_t)((sn ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0) |
+                              ((sn && ar) ? 4 : 0) | (ar ? 8 : 0));
+    }
     if (tid == 0) {
         // offsets -1, +1, -2, +2, ... reduced mod P; one entry per distinct neighbour
         int n = 0;
@@ -60,7 +68,8 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     float* xc = x + off + c;
     const float* gc = g + off + c;
-    float* hc = xhat + off + c;
+    float* hc = xhat + off + c;                         // sent copies
+    float* mc = (async ? mailbox : xhat) + off + c;     // received copies
 
     for (int j = 0; j < P; ++j) {
         const bool sn = (s_mode[j] & 1) != 0;
@@ -69,7 +78,10 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
             const long long rb = (long long)j * stride;
             const float4 xj = *reinterpret_cast<const float4*>(xc + rb);
             const float4 gj = ld_stream(gc + rb);
-            const float4 hj = sn ? xj : *reinterpret_cast<const float4*>(hc + rb);   // own contribution
+            const unsigned mj = s_mode[j];
+            // what this replica contributes to its neighbours in this step
+            const float4 hj = (mj & 4) ? xj
+                                       : *reinterpret_cast<const float4*>(((mj & 8) ? hc : mc) + rb);
             const float4 own = (variant & kOwnLastSent) ? hj : xj;
             double s0 = (double)own.x, s1 = (double)own.y, s2 = (double)own.z, s3 = (double)own.w;
             int cnt = 0;
@@ -78,8 +90,8 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
                 if (r >= P) r -= P;
                 const unsigned mode = s_mode[r];
                 if (!(mode & 2)) continue;                         // never heard from
-                // processed replicas (r < j) have their message, if any, in x_hat already
-                const float* src = (r > j && (mode & 1)) ? xc : hc;
+                // processed replicas (r < j) have whatever arrived in their mailbox already
+                const float* src = (r > j) ? ((mode & 4) ? xc : ((mode & 8) ? hc : mc)) : mc;
                 const float4 v = *reinterpret_cast<const float4*>(src + (long long)r * stride);
                 s0 = __dadd_rn(s0, (double)v.x); s1 = __dadd_rn(s1, (double)v.y);
                 s2 = __dadd_rn(s2, (double)v.z); s3 = __dadd_rn(s3, (double)v.w);
@@ -93,6 +105,7 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
             xn.w = __double2float_rn(__fma_rn(neg_lr, (double)gj.w, __dmul_rn(s3, w)));
             // the message first (later replicas read it), then the parameters
             if (sn) store_masked(hc + rb, xj, nel);
+            if (async && (mj & 8)) store_masked(mc + rb, hj, nel);
             store_masked(xc + rb, xn, nel);
             if (CARRY) acc = sq_diff4(xn, (variant & kChangeOfNorm) ? zero4 : hj, nel, acc);
         }

@@ -117,14 +117,30 @@ struct PipeSmem {
     }
 };
 
-// grid n_tiles (tile table with TILE elements per tile), CONSUMERS + 32 threads.
+// Body of the kernels below.  grid n_tiles (tile table with TILE elements per tile),
+// CONSUMERS + 32 threads.
 // COLS = TILE / (4 * CONSUMERS) float4 columns per consumer thread.
-template <int TILE, int STAGES, int CONSUMERS, bool CARRY>
-__global__ void __launch_bounds__(CONSUMERS + 32)
-k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
-             const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
-             int P, int T, long long stride, float lr, double* __restrict__ partials,
-             long long* step_k, unsigned int* __restrict__ err, int variant) {
+//
+// ASYNC (intermittent delivery): x_hat is what a replica has SENT, `mailbox` what its
+// neighbours have RECEIVED, `arrive` says whose outstanding messages arrive in this step and
+// `valid` is then "received at least once".  A replica contributes its own x (dense message
+// that arrives now), its sent copy (older message arriving now; copied into the mailbox on
+// the way) or its mailbox (nothing arrives).  Without ASYNC the two copies are one buffer and
+// every message arrives at once, which is the code path of the synchronous method.
+// PLAIN: the default readings only (the `variant` argument is ignored), so that the common
+// path carries no variant tests.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC, bool PLAIN>
+__device__ __forceinline__ void
+fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
+                const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, const TileTable& tt,
+                int P, int T, long long stride, float lr, double* __restrict__ partials,
+                long long* step_k, unsigned int* __restrict__ err, int variant_arg,
+                float* mailbox, const uint8_t* __restrict__ arrive) {
+    static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
+    const int variant = PLAIN ? 0 : variant_arg;
+    // mode bit that says "contributes its own x": the dense-message bit itself unless ASYNC
+    constexpr unsigned kCx = ASYNC ? 4u : 1u;
+    static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
     using L = PipeSmem<TILE, STAGES>;
     constexpr int COLS = TILE / (4 * CONSUMERS);
     constexpr int CWARPS = CONSUMERS / 32;
@@ -137,7 +153,8 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
     uint64_t* empty = full + STAGES;
     uint64_t* wrap_bar = empty + STAGES;
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kFlags);
-    uint8_t* s_mode = smem + L::kFlags + 16;                      // bit 0: dense message, bit 1: valid
+    // bit 0: dense message, bit 1: valid, bit 2: contributes its own x, bit 3: arrives now
+    uint8_t* s_mode = smem + L::kFlags + 16;
     double* s_red = reinterpret_cast<double*>(s_mode + ((P + 15) & ~15));
 
     const int tile = blockIdx.x, tid = threadIdx.x;
@@ -146,8 +163,12 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
     const long long off = tt.offset[tile];
     const uint32_t copy_bytes = (uint32_t)(((len + 3) & ~3) * 4);
 
-    for (int j = tid; j < P; j += CONSUMERS + 32)
-        s_mode[j] = (uint8_t)((snap[(long long)j * T + t] ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0));
+    for (int j = tid; j < P; j += CONSUMERS + 32) {
+        const bool sn = snap[(long long)j * T + t] != 0;
+        const bool ar = ASYNC ? (arrive[(long long)j * T + t] != 0) : sn;
+        s_mode[j] = (uint8_t)((sn ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0) |
+                              ((sn && ar) ? 4 : 0) | (ar ? 8 : 0));
+    }
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full[s], 1);
@@ -160,7 +181,7 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
     }
     __syncthreads();
 
-    const bool snap_last = (s_mode[P - 1] & 1) != 0;
+    const bool cx_last = (s_mode[P - 1] & kCx) != 0;
     // Replica P-1 contributes wrap_l; its own stage then only needs what wrap_l does not hold.
     const bool last_opt = P >= 2;
 
@@ -170,22 +191,25 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
             const float* xp = x + off;
             const float* gp = g + off;
             const float* hp = xhat + off;
+            const float* mp = ASYNC ? mailbox + off : hp;
             mbar_expect_tx(wrap_bar, copy_bytes);
-            bulk_g2s(wrap_l, (snap_last ? xp : hp) + (long long)(P - 1) * stride, copy_bytes, wrap_bar);
+            bulk_g2s(wrap_l,
+                     (cx_last ? xp : ((s_mode[P - 1] & 8) ? hp : mp)) + (long long)(P - 1) * stride,
+                     copy_bytes, wrap_bar);
             int s = 0;
             uint32_t wait_parity = 1;     // parity of the phase before the one to wait for
             for (int j = 0; j < P; ++j) {
                 if (j >= STAGES && !mbar_wait_bounded(&empty[s], wait_parity, s_abort, err)) break;
                 float* st = stages + s * (3 * TILE);
-                const bool sn = (s_mode[j] & 1) != 0;
+                const bool cx = (s_mode[j] & kCx) != 0;
                 const bool is_last = last_opt && (j == P - 1);
-                const bool need_x = !(is_last && sn);
-                const bool need_h = !sn && !is_last;
+                const bool need_x = !(is_last && cx);
+                const bool need_h = !cx && !is_last;
                 mbar_expect_tx(&full[s], copy_bytes * (1u + (need_x ? 1u : 0u) + (need_h ? 1u : 0u)));
                 bulk_g2s(st + TILE, gp, copy_bytes, &full[s]);
                 if (need_x) bulk_g2s(st, xp, copy_bytes, &full[s]);
-                if (need_h) bulk_g2s(st + 2 * TILE, hp, copy_bytes, &full[s]);
-                xp += stride; gp += stride; hp += stride;
+                if (need_h) bulk_g2s(st + 2 * TILE, (s_mode[j] & 8) ? hp : mp, copy_bytes, &full[s]);
+                xp += stride; gp += stride; hp += stride; mp += stride;
                 if (++s == STAGES) { s = 0; wait_parity ^= 1u; }
             }
         }
@@ -209,7 +233,7 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
         for (int v = 0; v < COLS; ++v) {
             const int c = c0 + v * 4 * CONSUMERS;
             const float4 a = ok ? *reinterpret_cast<const float4*>(wrap_l + c) : make_float4(0, 0, 0, 0);
-            const float4 b = ok ? *reinterpret_cast<const float4*>(((mode_cur & 1) ? stages : stages + 2 * TILE) + c)
+            const float4 b = ok ? *reinterpret_cast<const float4*>(((mode_cur & kCx) ? stages : stages + 2 * TILE) + c)
                                 : make_float4(0, 0, 0, 0);
             hp[v][0] = a.x; hp[v][1] = a.y; hp[v][2] = a.z; hp[v][3] = a.w;
             hc[v][0] = b.x; hc[v][1] = b.y; hc[v][2] = b.z; hc[v][3] = b.w;
@@ -218,6 +242,7 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
         uint32_t parity1 = (STAGES > 1) ? 0u : 1u;   // phase parity of the fill of stage s1 for j+1
         float* xo = x + off + c0;                    // output pointers of replica j
         float* ho = xhat + off + c0;
+        float* mo = ASYNC ? mailbox + off + c0 : nullptr;
         for (int j = 0; ok && j < P; ++j) {
             const bool more = j + 1 < P;
             if (more) {
@@ -227,14 +252,15 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
             const unsigned mode_next = s_mode[more ? j + 1 : 0];
             const float* st = stages + s * (3 * TILE);
             const bool sn = (mode_cur & 1) != 0;
+            const bool cx = (mode_cur & kCx) != 0;     // == sn unless ASYNC
             const bool is_last = last_opt && !more;
-            // fp32 copy of this replica's contribution (its old x when it sends a dense message)
-            const float* hs = is_last ? wrap_l : (sn ? st : st + 2 * TILE);
+            // fp32 copy of this replica's contribution (its old x when a dense message arrives)
+            const float* hs = is_last ? wrap_l : (cx ? st : st + 2 * TILE);
             // contribution of replica j+1
             const float* sq = stages + s1 * (3 * TILE);
             const float* hn_s = !more ? wrap_r
                                       : ((last_opt && j + 2 == P) ? wrap_l
-                                                                  : ((mode_next & 1) ? sq : sq + 2 * TILE));
+                                                                  : ((mode_next & kCx) ? sq : sq + 2 * TILE));
             const bool ul = has_left && (mode_prev & 2) != 0;
             const bool ur = has_right && (mode_next & 2) != 0;
             const double w = (ul && ur) ? w_third : ((ul || ur) ? w_half : w_one);
@@ -250,12 +276,15 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
                     const double hn[4] = {(double)hnf.x, (double)hnf.y, (double)hnf.z, (double)hnf.w};
                     const double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
                     double xd[4];
-                    if (sn || (variant & kOwnLastSent)) {   // own term = this replica's contribution
+                    float4 x_old = make_float4(0.f, 0.f, 0.f, 0.f);   // only needed under ASYNC
+                    if (cx || (variant & kOwnLastSent)) {   // own term = this replica's contribution
 #pragma unroll
                         for (int q = 0; q < 4; ++q) xd[q] = hc[v][q];
+                        if (ASYNC) x_old = hcf;
                     } else {
                         const float4 xf = *reinterpret_cast<const float4*>(st + c);
                         xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
+                        if (ASYNC) x_old = xf;
                     }
                     float xn[4];
 #pragma unroll
@@ -267,7 +296,9 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
                     }
                     const float4 xn4 = make_float4(xn[0], xn[1], xn[2], xn[3]);
                     store_masked(xo + v * 4 * CONSUMERS, xn4, nel[v]);
-                    if (sn) store_masked(ho + v * 4 * CONSUMERS, hcf, nel[v]);
+                    // a dense message: the sender's record becomes its old x (== hcf unless ASYNC)
+                    if (sn) store_masked(ho + v * 4 * CONSUMERS, ASYNC ? x_old : hcf, nel[v]);
+                    if (ASYNC && (mode_cur & 8)) store_masked(mo + v * 4 * CONSUMERS, hcf, nel[v]);
                     if (CARRY)
                         acc = sq_diff4(xn4, (variant & kChangeOfNorm) ? make_float4(0.f, 0.f, 0.f, 0.f) : hcf,
                                        nel[v], acc);
@@ -285,6 +316,7 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[s]);
             xo += stride; ho += stride;
+            if (ASYNC) mo += stride;
             mode_prev = mode_cur; mode_cur = mode_next;
             s = s1;
             if (++s1 == STAGES) { s1 = 0; parity1 ^= 1u; }
@@ -304,6 +336,31 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
             partials[(long long)j * tt.n_tiles + tile] = r;
         }
     }
+}
+
+// The method as the paper's formulas state it (default readings, synchronous delivery).  No
+// register bound is requested: the body needs 72 registers, which lets 3 CTAs share an SM.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY>
+__global__ void __launch_bounds__(CONSUMERS + 32)
+k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
+             const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
+             int P, int T, long long stride, float lr, double* __restrict__ partials,
+             long long* step_k, unsigned int* __restrict__ err) {
+    fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true>(x, g, xhat, snap, valid, tt, P, T, stride, lr,
+                                                                partials, step_k, err, 0, nullptr, nullptr);
+}
+
+// Variants (eg_set_variant) and intermittent delivery; bounded to 72 registers for 3 CTAs per SM.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC>
+__global__ void __launch_bounds__(CONSUMERS + 32, 3)
+k_fused_pipe_general(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
+                     const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
+                     int P, int T, long long stride, float lr, double* __restrict__ partials,
+                     long long* step_k, unsigned int* __restrict__ err, int variant, float* mailbox,
+                     const uint8_t* __restrict__ arrive) {
+    fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, ASYNC, false>(x, g, xhat, snap, valid, tt, P, T, stride,
+                                                                 lr, partials, step_k, err, variant, mailbox,
+                                                                 arrive);
 }
 
 }  // namespace eg

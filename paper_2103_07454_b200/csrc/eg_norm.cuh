@@ -64,12 +64,22 @@ struct DecideParams {
     double cap;               // bound sqrt(g(k)) on the threshold of this step (+inf: none)
 };
 
+// Intermittent delivery: which outstanding messages arrive in this step.
+struct DeliveryState {
+    const uint8_t* deliver;   // [P*T] host-supplied mask for this step (nullptr: everything arrives)
+    uint8_t* pending;         // [P*T] something sent has not arrived yet
+    uint8_t* recv_valid;      // [P*T] neighbours have received this tensor at least once
+    uint8_t* arrive;          // [P*T] out: arrives in this step
+    unsigned long long* arrivals;
+    int enabled;
+};
+
 // One warp per (replica, tensor).  grid ceil(P*T / kWarps).
 __global__ void __launch_bounds__(kThreads)
 k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin, int n_tiles,
          DecideParams dp, SegState st, const long long* __restrict__ numel,
          const long long* __restrict__ topk_count, int* __restrict__ outbox_count,
-         Counters* ctr, const long long* __restrict__ step_k) {
+         Counters* ctr, const long long* __restrict__ step_k, DeliveryState dl) {
     const int lane = threadIdx.x & 31;
     const long long s = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (s >= (long long)dp.P * dp.T) return;
@@ -125,6 +135,16 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
         if (dp.degree > 0) {
             atomicAdd(&ctr->messages, (unsigned long long)dp.degree);
             atomicAdd(&ctr->bytes, (unsigned long long)dp.degree * payload);
+        }
+    }
+    if (dl.enabled) {
+        const bool pend = fire || dl.pending[s] != 0;
+        const bool arr = pend && (dl.deliver == nullptr || dl.deliver[s] != 0);
+        dl.pending[s] = (pend && !arr) ? 1 : 0;
+        dl.arrive[s] = arr ? 1 : 0;
+        if (arr) {
+            dl.recv_valid[s] = 1;
+            atomicAdd(dl.arrivals, 1ull);
         }
     }
     st.flag[s] = fire ? 1 : 0;

@@ -75,6 +75,11 @@ struct eg_ctx {
     int variant = 0;
     double cap_alpha = 0.0, cap_beta = 1.0;   // bound alpha*beta^k on the squared threshold
     long long host_k = 0;                     // host copy of the iteration counter
+    // intermittent delivery (two copies: sent = xhat, received = mailbox)
+    bool async = false;
+    float* mailbox = nullptr;
+    uint8_t *pending = nullptr, *recv_valid = nullptr, *arrive = nullptr;
+    unsigned long long* arrivals = nullptr;
     bool stepped = false;   // a step has run since creation / reset / import
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
@@ -169,6 +174,13 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->tk.hist, 0, S * kMaxBins * sizeof(unsigned int)));
         EG_CUDA(c, cudaMemset(c->tk.prefix, 0, S * sizeof(unsigned int)));
         EG_CUDA(c, cudaMemset(c->tk.remaining, 0, S * sizeof(unsigned int)));
+    }
+    if (c->async) {
+        EG_CUDA(c, cudaMemset(c->mailbox, 0, (size_t)c->P * c->stride * sizeof(float)));
+        EG_CUDA(c, cudaMemset(c->pending, 0, S));
+        EG_CUDA(c, cudaMemset(c->recv_valid, 0, S));
+        EG_CUDA(c, cudaMemset(c->arrive, 0, S));
+        EG_CUDA(c, cudaMemset(c->arrivals, 0, sizeof(unsigned long long)));
     }
     c->carried_valid = false;
     c->stepped = false;
@@ -343,11 +355,16 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     }
     {
         const int pipe_smem = (int)PipeLayout::bytes(P, true, kPipeConsumers / 32);
-        cudaError_t e = cudaFuncSetAttribute(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
+        cudaError_t e = cudaSuccess;
+        auto raise = [&](const void* fn) {
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe_smem);
+        };
+        raise((const void*)k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>);
+        raise((const void*)k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>);
+        raise((const void*)k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, true, false>);
+        raise((const void*)k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, false>);
+        raise((const void*)k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>);
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
     if ((s = init_state(c)) != EG_OK) return fail(s);
@@ -377,7 +394,14 @@ eg_status eg_set_carry_norm(eg_ctx* c, int enabled) {
 }
 
 eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* stream_v) {
+    return eg_step_masked(c, params, grads, lr, nullptr, stream_v);
+}
+
+eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
+                         const uint8_t* deliver_dev, void* stream_v) {
     if (!c || !params || !grads) return EG_ERR_INVALID;
+    if (deliver_dev && !c->async) return EG_ERR_STATE;     // eg_enable_delivery_masks first
+    if (c->async && (c->variant & kOwnLastSent)) return EG_ERR_STATE;
     if (((uintptr_t)params & 15u) || ((uintptr_t)grads & 15u)) return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
     if (!guard.ok) return EG_ERR_CUDA;
@@ -389,7 +413,8 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     const int S = c->P * c->T;
 
     // a1: || x - x_hat || partial sums, unless the previous step carried them over
-    const bool use_carried = c->carry && c->carried_valid && c->carried_params == params;
+    const bool carry = c->carry && !c->async;   // no carried norm under intermittent delivery
+    const bool use_carried = carry && c->carried_valid && c->carried_params == params;
     if (!use_carried) {
         TimedSection ts(c, stream, EG_KERNEL_NORM);
         k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, c->partials_norm,
@@ -407,7 +432,8 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
         TimedSection ts(c, stream, EG_KERNEL_DECIDE);
         k_decide<<<(S + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
             partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
-            c->ctr, c->step_k);
+            c->ctr, c->step_k,
+            DeliveryState{deliver_dev, c->pending, c->recv_valid, c->arrive, c->arrivals, c->async ? 1 : 0});
         ++launches;
     }
     // a4: Top-K select / pack / deliver for the segments that send a sparse message
@@ -428,37 +454,53 @@ eg_status eg_step(eg_ctx* c, float* params, const float* grads, float lr, void* 
     // a3 + a5: dense snapshot, consensus average, SGD
     {
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
+        const uint8_t* valid = c->async ? c->recv_valid : c->st.valid;   // whom the neighbours have heard from
         if (c->hops > 1) {
-            if (c->carry)
+            if (carry)
                 k_fused_hops<true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
-                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
                     c->partials_fused, c->step_k, c->variant, c->hops);
             else
                 k_fused_hops<false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
-                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->variant, c->hops);
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    c->partials_fused, c->step_k, c->variant, c->hops,
+                    c->async ? c->mailbox : nullptr, c->async ? c->arrive : nullptr);
+        } else if (c->async) {
+            k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>
+                <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
+                params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                c->partials_fused, c->step_k, c->err, c->variant, c->mailbox, c->arrive);
         } else if (c->fused_kind == EG_FUSED_PIPELINED) {
-            if (c->carry)
-                k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
-                    <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, true, kPipeConsumers / 32), stream>>>(
-                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->err, c->variant);
-            else
-                k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>
-                    <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
-                    params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->err, c->variant);
-        } else if (c->carry)
+            const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
+#define EG_PIPE_ARGS params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, \
+                     c->partials_fused, c->step_k, c->err
+            if (c->variant == 0) {
+                if (carry)
+                    k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
+                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
+                else
+                    k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>
+                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
+            } else {
+                if (carry)
+                    k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, true, false>
+                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                else
+                    k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, false>
+                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+            }
+#undef EG_PIPE_ARGS
+        } else if (carry)
             k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
-                params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
                 c->partials_fused, c->step_k, c->variant);
         else
             k_fused<kFusedVpt, false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
-                params, grads, c->xhat, c->st.snap, c->st.valid, tf, c->P, c->T, c->stride, lr,
+                params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
                 c->partials_fused, c->step_k, c->variant);
         ++launches;
     }
-    c->carried_valid = c->carry;
+    c->carried_valid = carry;
     c->carried_params = params;
     c->stepped = true;
     c->host_k += 1;
@@ -570,9 +612,64 @@ eg_status eg_set_variant(eg_ctx* c, int own_term, int trigger_metric) {
         (trigger_metric != EG_TRIGGER_NORM_OF_CHANGE && trigger_metric != EG_TRIGGER_CHANGE_OF_NORM))
         return EG_ERR_INVALID;
     if (c->stepped) return EG_ERR_STATE;   // only before the first step (or after eg_reset)
+    if (c->async && own_term == EG_OWN_LAST_SENT) return EG_ERR_STATE;
     c->variant = (own_term == EG_OWN_LAST_SENT ? kOwnLastSent : 0) |
                  (trigger_metric == EG_TRIGGER_CHANGE_OF_NORM ? kChangeOfNorm : 0);
     c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status eg_enable_delivery_masks(eg_ctx* c) {
+    if (!c) return EG_ERR_INVALID;
+    if (c->async) return EG_OK;
+    if (c->variant & kOwnLastSent) return EG_ERR_STATE;
+    DeviceGuard guard(c->device);
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    const size_t S = (size_t)c->P * c->T, n = (size_t)c->P * c->stride;
+    eg_status s;
+    if ((s = dev_alloc(c, &c->mailbox, n, false)) != EG_OK) return s;
+    if ((s = dev_alloc(c, &c->pending, S)) != EG_OK) return s;
+    if ((s = dev_alloc(c, &c->recv_valid, S, false)) != EG_OK) return s;
+    if ((s = dev_alloc(c, &c->arrive, S)) != EG_OK) return s;
+    if ((s = dev_alloc(c, &c->arrivals, 1)) != EG_OK) return s;
+    // everything sent so far has arrived
+    EG_CUDA(c, cudaMemcpy(c->mailbox, c->xhat, n * sizeof(float), cudaMemcpyDeviceToDevice));
+    EG_CUDA(c, cudaMemcpy(c->recv_valid, c->st.valid, S, cudaMemcpyDeviceToDevice));
+    c->async = true;
+    c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status eg_read_received(eg_ctx* c, float* received_host) {
+    if (!c || !received_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    EG_CUDA(c, cudaMemcpy(received_host, c->async ? c->mailbox : c->xhat,
+                          (size_t)c->P * c->stride * sizeof(float), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_delivery_status(eg_ctx* c, uint8_t* pending_host, uint64_t* arrivals_host) {
+    if (!c) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    const size_t S = (size_t)c->P * c->T;
+    if (pending_host) {
+        if (c->async) EG_CUDA(c, cudaMemcpy(pending_host, c->pending, S, cudaMemcpyDeviceToHost));
+        else memset(pending_host, 0, S);
+    }
+    if (arrivals_host) {
+        unsigned long long a = 0;
+        if (c->async) EG_CUDA(c, cudaMemcpy(&a, c->arrivals, sizeof(a), cudaMemcpyDeviceToHost));
+        else {
+            Counters h{};
+            EG_CUDA(c, cudaMemcpy(&h, c->ctr, sizeof(h), cudaMemcpyDeviceToHost));
+            a = h.events;   // synchronous delivery: every event arrived
+        }
+        *arrivals_host = a;
+    }
     return EG_OK;
 }
 
@@ -706,6 +803,7 @@ static size_t state_bytes(const eg_ctx* c) {
 
 eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
     if (!c || !bytes) return EG_ERR_INVALID;
+    if (c->async) return EG_ERR_STATE;   // messages in flight are not part of a checkpoint
     const size_t need = state_bytes(c);
     if (!host_buf) { *bytes = need; return EG_OK; }
     if (*bytes < need) { *bytes = need; return EG_ERR_INVALID; }
@@ -741,6 +839,7 @@ eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
 
 eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
     if (!c || !host_buf || bytes < state_bytes(c)) return EG_ERR_INVALID;
+    if (c->async) return EG_ERR_STATE;
     StateHeader h;
     memcpy(&h, host_buf, sizeof(h));
     if (h.magic != kStateMagic || h.P != c->P || h.T != c->T || h.H != c->H || h.stride != c->stride ||

@@ -98,7 +98,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
              gen_device: str = "cuda", tensors: Optional[Sequence[int]] = None,
              carry: bool = False, check_every: int = 1, oracle_kw: Optional[dict] = None,
              eg_kw: Optional[dict] = None, outbox_samples: int = 8, grad_hook=None,
-             fused_kernel: int = B.FUSED_PIPELINED) -> Report:
+             fused_kernel: int = B.FUSED_PIPELINED, deliver_fn=None) -> Report:
     steps = wl.steps if steps is None else steps
     dev = torch.device("cuda")
     full = tensors is None
@@ -123,6 +123,9 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     eg = B.from_workload(wl, **ekw)
     eg.set_carry_norm(carry)
     eg.set_fused_kernel(fused_kernel)
+    if deliver_fn is not None:
+        eg.enable_delivery_masks()
+        o.enable_delivery_masks()
     eg.set_variant(bool(okw.get("own_last_sent")), bool(okw.get("change_of_norm")))
     if cap:
         eg.set_threshold_cap(*cap)
@@ -148,8 +151,14 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
         g_host = (g if full else g[:, cols]).cpu().numpy()
         del g
         sent_pre = o.sent_norms() if okw.get("change_of_norm") else None
-        o.step(x_host, np.ascontiguousarray(g_host), wl.lr)
-        eg.step(x_dev, g_dev, wl.lr)
+        mask = None if deliver_fn is None else deliver_fn(k)          # [P, T] uint8 or None
+        o.step(x_host, np.ascontiguousarray(g_host), wl.lr,
+               deliver=None if mask is None else np.ascontiguousarray(mask[:, tensors]))
+        if deliver_fn is None:
+            eg.step(x_dev, g_dev, wl.lr)
+        else:
+            eg.step_masked(x_dev, g_dev, wl.lr,
+                           None if mask is None else torch.from_numpy(np.ascontiguousarray(mask)).to(dev))
         rep.launches += eg.last_launch_count
         rep.steps += 1
         if (k % check_every) and k != steps - 1 and k >= 8:
@@ -213,6 +222,13 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             assert rep.max_param_rel <= PARAM_RTOL, f"parameters, step {k}: rel err {rep.max_param_rel}"
         xh_g = gpu_sub(eg.mailboxes().to(dev))
         assert np.array_equal(xh_g.view(np.uint32), o.xhat().view(np.uint32)), f"mailboxes, step {k}"
+        if deliver_fn is not None:
+            rc_g = gpu_sub(eg.received().to(dev))
+            assert np.array_equal(rc_g.view(np.uint32), o.received().view(np.uint32)), f"received, step {k}"
+            pend, arrivals = eg.delivery_status()
+            assert np.array_equal(pend[:, tensors], o.pending()), f"in flight, step {k}"
+            if full:
+                assert arrivals == o.arrivals, f"arrivals, step {k}"
 
     eg.close()
     o.close()

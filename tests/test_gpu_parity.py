@@ -62,6 +62,61 @@ def test_geometric_threshold_cap(carry):
     assert rep.events > free.events          # a shrinking bound makes tensors communicate more
 
 
+def _random_links(P, T, p_up, seed):
+    rng = np.random.default_rng(seed)
+
+    def fn(k):
+        if k % 7 == 6:
+            return None                      # NULL mask: everything outstanding arrives
+        return (rng.random((P, T)) < p_up).astype(np.uint8)
+    return fn
+
+
+@pytest.mark.parametrize("P,hops", [(1, 1), (2, 1), (3, 1), (5, 1), (16, 1), (5, 2), (9, 3)])
+@pytest.mark.parametrize("p_up", [0.0, 0.5, 1.0])
+def test_intermittent_delivery_dense(P, hops, p_up):
+    wl = W.synthetic(P, RAGGED[:-1], steps=16, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", oracle_kw=dict(hops=hops),
+                   deliver_fn=_random_links(P, wl.T, p_up, seed=P * 10 + hops))
+    assert rep.params_bit_exact and not rep.near_threshold
+
+
+@pytest.mark.parametrize("con", [False, True])
+def test_intermittent_delivery_topk(con):
+    wl = W.synthetic(6, RAGGED[:-1], steps=16, lr=0.1, grad_sigma=0.01, topk=(5, 100))
+    rep = lockstep(wl, init="distinct", outbox_samples=32, carry=True,     # carry is ignored here
+                   oracle_kw=dict(change_of_norm=con), deliver_fn=_random_links(6, wl.T, 0.4, seed=3))
+    assert rep.params_bit_exact
+
+
+def test_delivery_masks_enabled_mid_run_and_refusals():
+    from oracle import eg_oracle as eo
+    wl = W.synthetic(4, [5, 1000, 4097], steps=12, lr=0.1, grad_sigma=0.01)
+    o, eg = eo.from_workload(wl), B.from_workload(wl)
+    xh = W.distinct_init_params(wl).numpy().copy()
+    xd = eg.to_layout(torch.from_numpy(xh))
+    rng = np.random.default_rng(1)
+    with pytest.raises(B.EventGradError):          # a mask before the second copy exists
+        eg.step_masked(xd, xd, 0.1, torch.ones(4 * wl.T, dtype=torch.uint8, device="cuda"))
+    for k in range(wl.steps):
+        g = wl.grads(k)
+        if k == 4:
+            eg.enable_delivery_masks()
+            o.enable_delivery_masks()
+        mask = (rng.random((4, wl.T)) < 0.5).astype(np.uint8) if k >= 4 else None
+        o.step(xh, g.numpy(), wl.lr, deliver=mask)
+        if mask is None:
+            eg.step(xd, eg.to_layout(g), wl.lr)
+        else:
+            eg.step_masked(xd, eg.to_layout(g), wl.lr, torch.from_numpy(mask).cuda())
+        assert np.array_equal(eg.last_decisions()[0], o.flags())
+    assert np.array_equal(eg.from_layout(xd).cpu().numpy(), xh)
+    assert np.array_equal(eg.from_layout(eg.received()).numpy(), o.received())
+    with pytest.raises(B.EventGradError):
+        eg.export_state()                          # messages in flight are not checkpointed
+    eg.close()
+
+
 def test_variant_with_topk():
     wl = W.synthetic(4, RAGGED[:-1], steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
     rep = lockstep(wl, init="distinct", carry=True, outbox_samples=64,
