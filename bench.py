@@ -278,28 +278,19 @@ def time_steps(eg, x, grads, lr, steps, sampler=None):
     return e0.elapsed_time(e1), launches
 
 
-def run_native(args):
-    from paper_2103_07454_b200 import binding as B
-    rank, world, local = dist_setup("nccl")
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    wl = pick_workload(args)
-    K, Wm = args.steps, max(args.warmup, 3)
+def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_variant):
+    """Times K steps of `wl` for every variant; returns ({variant: figures}, context)."""
     eg = B.from_workload(wl)
     buf_bytes = wl.P * eg.replica_stride * 4
     free, _ = torch.cuda.mem_get_info()
-    n_buf = int(max(1, min(max(K, Wm), (free - (24 << 30)) // buf_bytes)))
+    reserve = (24 << 30) + 4 * buf_bytes + (2 * buf_bytes if wl.topk else 0)
+    n_buf = int(max(1, min(max(K, Wm), (free - reserve) // buf_bytes)))
     grads = [eg.to_layout(wl.grads(k, dev)) for k in range(n_buf)]
     x0 = eg.to_layout(wl.init_params(dev))
     x = x0.clone()
-    peak, peak_kind = measured_peak()
     elems = wl.P * wl.N
     results = {}
-    sampler = ClockSampler(local)
-    clocks = None
-    for variant in ([args.variant] + [v for v in ("carry", "two_pass") if v != args.variant]):
+    for variant in variants:
         eg.set_carry_norm(variant == "carry")
         x.copy_(x0)
         eg.reset()
@@ -310,8 +301,8 @@ def run_native(args):
         eg.reset()
         eg.set_carry_norm(variant == "carry")
         eg.set_timing(True)
-        main = variant == args.variant
-        ms, launches = time_steps(eg, x, grads, wl.lr, K, sampler if main else None)
+        ms, launches = time_steps(eg, x, grads, wl.lr, K,
+                                  sampler if (sampler and variant == sampled_variant) else None)
         kt = eg.kernel_times()
         stats = eg.stats()
         units, ms_max = aggregate(float(elems) * K, ms, dev)
@@ -320,9 +311,51 @@ def run_native(args):
             "replica_steps_per_s": world * wl.P * K / (ms_max / 1e3), "launches": launches,
             "kernel_ms": {g: (v[0] / v[1] if v[1] else None) for g, v in kt.items()},
             "messages_sent": stats["messages"], "bytes_sent": stats["bytes"],
-            "pct_messages": 100.0 * stats["messages"] / (wl.P * wl.T * 2 * K)}
-        if main:
-            clocks = sampler.summary()
+            "pct_messages": 100.0 * stats["messages"] / (wl.P * wl.T * 2 * K),
+            "gradient_buffers": n_buf}
+    del x
+    return results, (eg, x0, grads, n_buf, buf_bytes)
+
+
+def run_native(args):
+    from paper_2103_07454_b200 import binding as B
+    rank, world, local = dist_setup("nccl")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    wl = pick_workload(args)
+    K, Wm = args.steps, max(args.warmup, 3)
+    peak, peak_kind = measured_peak()
+    sampler = ClockSampler(local)
+    if args.all_configs:
+        rows = []
+        for idx in (1, 2, 3, 4, 5):
+            for w in W.config(idx):
+                r, ctx = measure_workload(B, w, w.steps, Wm, dev, world, ("carry", "two_pass"), None, None)
+                ctx[0].close()
+                del ctx
+                rows.append({"config": idx, "workload": w.name, "P": w.P, "tensors": w.T, "elements": w.N,
+                             "steps": w.steps, "topk": w.topk,
+                             **{v: {"ms_per_step": r[v]["ms_per_step"], "GB/s": r[v]["gbs"],
+                                    "pct_of_peak": 100.0 * r[v]["gbs"] / peak,
+                                    "replica_steps_per_s": r[v]["replica_steps_per_s"],
+                                    "kernel_ms": r[v]["kernel_ms"], "gradient_buffers": r[v]["gradient_buffers"]}
+                                for v in r},
+                             "messages_sent": r["carry"]["messages_sent"],
+                             "pct_messages": r["carry"]["pct_messages"],
+                             "bytes_sent": r["carry"]["bytes_sent"]})
+                torch.cuda.empty_cache()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "unit": "GB/s", "n_gpus": world, "peak": peak,
+                              "peak_kind": f"of {peak_kind}", "all_configs": rows}), flush=True)
+        return
+    results, ctx = measure_workload(B, wl, K, Wm, dev, world,
+                                    [args.variant] + [v for v in ("carry", "two_pass") if v != args.variant],
+                                    sampler, args.variant)
+    eg, x0, grads, n_buf, buf_bytes = ctx
+    clocks = sampler.summary()
+    elems = wl.P * wl.N
     main = results[args.variant]
 
     # end to end: host buffers in, updated parameters out, through eg_step_host
@@ -395,6 +428,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="time all five configurations (their own step counts) instead of the default one")
     ap.add_argument("--max-elements", type=int, default=0,
                     help="keep only the leading tensors of the workload up to this many elements")
     args = ap.parse_args()
