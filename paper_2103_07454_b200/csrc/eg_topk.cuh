@@ -38,7 +38,8 @@ struct TopkState {
     unsigned int* remaining;   // [P*T] rank still to resolve (after the last digit: number of
                                //       entries equal to tau that are part of the message)
     unsigned int* cand;        // [P][stride] candidate keys of a tile, at the tile's own offset
-    int* tile_cand;            // [P][n_tiles] candidates stored for the tile
+    int* tile_cand;            // [P][n_tiles][8] candidates stored by each warp for the tile
+    unsigned int* tile_gt;     // [P][n_tiles][8] keys above the chosen bin seen by each warp
     uint2* tile_count;         // [P][n_tiles] (greater, equal) per tile, then their prefixes
     int2* outbox;              // [P][sum K_t] (index, value bits)
     const long long* out_off;  // [T] start of tensor t inside one replica's outbox
@@ -223,19 +224,37 @@ k_topk_pick(int T, TopkState tk, int digit) {
     }
 }
 
-// Pass B: per tile, copy the keys whose top digit equals the chosen bin into the tile's slice
-// of the candidate buffer (order inside the tile is irrelevant for selecting tau), count the
-// keys whose top digit is larger, and histogram digit 1 of the candidates.
+constexpr int kSubSlices = kWarps;                       // candidate sub-slices per tile: one per warp
+
+// Warp w of a CTA owns, in every 1024-element chunk of a tile, the 128 elements starting at
+// 128*w.  Its candidate sub-slice starts after the elements owned by the warps before it, so
+// the eight sub-slices exactly fill the tile's own slice whatever the tile's length.
+__device__ __forceinline__ int sub_offset(int len, int w) {
+    int o = 0;
+#pragma unroll
+    for (int v = 0; v < kNormTile / (kThreads * 4); ++v)
+        o += min(max(len - v * kThreads * 4, 0), w * 128);
+    return o;
+}
+
+// Pass B: per tile, copy the keys whose top digit equals the chosen bin into the candidate
+// buffer (order is irrelevant for selecting tau), count the keys whose top digit is larger, and
+// histogram digit 1 of the candidates.  Every warp owns 512 elements of the tile and a private
+// sub-slice of the tile's candidate slice, so no counter is shared: a thread marks its
+// candidates in a 16-bit mask, a warp scan of the counts gives its first slot, and the keys
+// are fetched back from shared memory (written and read by the same thread).
 __global__ void __launch_bounds__(kThreads, 4)
 k_topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
                long long stride, TopkState tk) {
     constexpr int kBins1 = 1 << kDigitBits1;
+    constexpr int kChunks = kNormTile / (kThreads * 4);
     __shared__ unsigned int s_hist[kBins1];
-    __shared__ unsigned int s_n, s_gt;
+    __shared__ uint4 s_key[kNormTile / 4];
     WorkRange r = work_range(tk);
     if (r.w0 >= r.w1) return;
     for (int b = threadIdx.x; b < kBins1; b += kThreads) s_hist[b] = 0;
     __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     WorkCursor cur;
     cur.init(tk, tt, T, r.q);
     unsigned int b0 = 0;
@@ -243,46 +262,60 @@ k_topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, Tile
         bool changed;
         const int tile = cur.advance(tk, tt, T, w, changed);
         if (changed) b0 = tk.prefix[cur.s];
-        const int i = cur.i, s = cur.s;
+        const int i = cur.i;
         const int len = tt.length[tile];
         const long long base = (long long)i * stride + tt.offset[tile];
-        unsigned int* cd = tk.cand + base;
-        if (threadIdx.x == 0) { s_n = 0; s_gt = 0; }
-        __syncthreads();
-        unsigned int gt = 0;
-        for (int local = threadIdx.x * 4; local < len; local += kThreads * 4) {
-            const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
-            const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
-                                       rank_key(a.w, b.w)};
-            const int nel = min(4, len - local);
+        unsigned int mask = 0, gt = 0;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (c < nel) {
-                    const unsigned int d0 = k[c] >> 20;
-                    gt += (d0 > b0);
-                    if (d0 == b0) {
-                        cd[atomicAdd(&s_n, 1u)] = k[c];
-                        atomicAdd(&s_hist[(k[c] >> 10) & (kBins1 - 1)], 1u);
-                    }
+        for (int v = 0; v < kChunks; ++v) {
+            const int local = (v * kThreads + threadIdx.x) * 4;
+            if (local < len) {
+                const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
+                const uint4 k = make_uint4(rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
+                                           rank_key(a.w, b.w));
+                s_key[v * kThreads + threadIdx.x] = k;
+                const int nel = len - local;      // >= 1; 4 or more for all but the ragged end
+                const unsigned int d[4] = {k.x >> 20, k.y >> 20, k.z >> 20, k.w >> 20};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const bool live = c < nel;
+                    gt += (live && d[c] > b0);
+                    mask |= (live && d[c] == b0) ? (1u << (4 * v + c)) : 0u;
                 }
             }
         }
+        // first slot of this thread inside its warp's sub-slice
+        const unsigned int cnt = __popc(mask);
+        unsigned int inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int u = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += u;
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) gt += __shfl_down_sync(0xffffffffu, gt, o);
-        if ((threadIdx.x & 31) == 0 && gt) atomicAdd(&s_gt, gt);
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            tk.tile_cand[(long long)i * tt.n_tiles + tile] = (int)s_n;
-            tk.tile_count[(long long)i * tt.n_tiles + tile] = make_uint2(s_gt, 0u);
+        unsigned int* cd = tk.cand + base + sub_offset(len, warp);
+        unsigned int pos = inc - cnt;
+        const unsigned int* my_keys = reinterpret_cast<const unsigned int*>(s_key);
+        while (mask) {
+            const int bit = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const unsigned int key = my_keys[((bit >> 2) * kThreads + threadIdx.x) * 4 + (bit & 3)];
+            cd[pos++] = key;
+            atomicAdd(&s_hist[(key >> 10) & (kBins1 - 1)], 1u);
         }
+        const long long slot = ((long long)i * tt.n_tiles + tile) * kSubSlices + warp;
+        if (lane == 31) tk.tile_cand[slot] = (int)inc;          // candidates of this warp
+        if (lane == 0) tk.tile_gt[slot] = gt;                   // keys above the bin, this warp
         if (w + 1 == r.w1 || w + 1 >= cur.end) {   // last tile of this segment here
-            unsigned int* gh = tk.hist + (long long)s * kMaxBins;
+            __syncthreads();
+            unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
             for (int b = threadIdx.x; b < kBins1; b += kThreads) {
                 const unsigned int v = s_hist[b];
                 if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
             }
+            __syncthreads();
         }
-        __syncthreads();
     }
 }
 
@@ -315,16 +348,22 @@ k_topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk) {
         const WarpTile z = warp_tile(tk, tt, T, w);
         const unsigned int want = tk.prefix[z.s];
         const unsigned int* cd = tk.cand + (long long)z.i * stride + tt.offset[z.tile];
-        const int n = tk.tile_cand[(long long)z.i * tt.n_tiles + z.tile];
+        const int* n_sub = tk.tile_cand + ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices;
+        const int len = tt.length[z.tile];
         unsigned int* gh = tk.hist + (long long)z.s * kMaxBins;
-        for (int e = lane; e < n; e += 32) {
-            const unsigned int k = cd[e];
-            if ((k >> 10) == want) atomicAdd(&gh[k & ((1 << kDigitBits2) - 1)], 1u);
+        for (int sub = 0; sub < kSubSlices; ++sub) {
+            const int n = n_sub[sub];
+            const unsigned int* cs = cd + sub_offset(len, sub);
+            for (int e = lane; e < n; e += 32) {
+                const unsigned int k = cs[e];
+                if ((k >> 10) == want) atomicAdd(&gh[k & ((1 << kDigitBits2) - 1)], 1u);
+            }
         }
     }
 }
 
-// Per tile, from its candidates only: keys greater than / equal to tau.  One warp per tile.
+// Per tile: keys greater than / equal to tau, from the per-warp counts of pass B and the
+// tile's candidates.  One warp per tile.
 __global__ void __launch_bounds__(kThreads)
 k_topk_count(TileTable tt, int T, long long stride, TopkState tk) {
     const int total = tk.plan->total_tiles;
@@ -334,22 +373,24 @@ k_topk_count(TileTable tt, int T, long long stride, TopkState tk) {
         const WarpTile z = warp_tile(tk, tt, T, w);
         const unsigned int tau = tk.prefix[z.s];
         const unsigned int* cd = tk.cand + (long long)z.i * stride + tt.offset[z.tile];
-        const int n = tk.tile_cand[(long long)z.i * tt.n_tiles + z.tile];
-        unsigned int gt = 0, eq = 0;
-        for (int e = lane; e < n; e += 32) {
-            const unsigned int k = cd[e];
-            gt += (k > tau);
-            eq += (k == tau);
+        const long long slot = ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices;
+        const int len = tt.length[z.tile];
+        unsigned int gt = (lane < kSubSlices) ? tk.tile_gt[slot + lane] : 0u, eq = 0;
+        for (int sub = 0; sub < kSubSlices; ++sub) {
+            const int n = tk.tile_cand[slot + sub];
+            const unsigned int* cs = cd + sub_offset(len, sub);
+            for (int e = lane; e < n; e += 32) {
+                const unsigned int k = cs[e];
+                gt += (k > tau);
+                eq += (k == tau);
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             gt += __shfl_down_sync(0xffffffffu, gt, o);
             eq += __shfl_down_sync(0xffffffffu, eq, o);
         }
-        if (lane == 0) {
-            uint2* tc = tk.tile_count + (long long)z.i * tt.n_tiles + z.tile;
-            *tc = make_uint2(tc->x + gt, eq);
-        }
+        if (lane == 0) tk.tile_count[(long long)z.i * tt.n_tiles + z.tile] = make_uint2(gt, eq);
     }
 }
 
@@ -400,16 +441,19 @@ k_topk_scan(TileTable tt, int T, TopkState tk) {
 // An entry is selected if key > tau, or key == tau and fewer than `remaining` equal keys
 // precede it in the tensor.  Its slot is (#greater before it) + min(#equal before it, remaining).
 // A tile is read as four coalesced chunks of 1024 elements (thread t owns elements 4t..4t+3 of
-// every chunk); the four per-chunk counts of a thread travel through ONE scan, packed 16 bits
-// each into a 64-bit word (a chunk holds at most 1024 entries, so the fields cannot overflow).
-// A thread has read the x_hat entries it owns before it overwrites any of them, and no thread
-// touches another thread's entries.
-__global__ void __launch_bounds__(kThreads, 3)
+// every chunk).  A thread records which of its 16 elements are greater / equal in two 16-bit
+// masks and parks the x values in shared memory (read back by the same thread); the four
+// per-chunk counts travel through ONE scan, packed 16 bits each into a 64-bit word (a chunk
+// holds at most 1024 entries, so the fields cannot overflow); then only the marked elements
+// are visited.  A thread has read the x_hat entries it owns before it overwrites any of them,
+// and no thread touches another thread's entries.
+__global__ void __launch_bounds__(kThreads, 4)
 k_topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long long stride,
              TopkState tk, unsigned int* __restrict__ err) {
     constexpr int kChunks = kNormTile / (kThreads * 4);   // 4
     static_assert(kChunks == 4, "the packed scan holds four 16-bit fields");
     __shared__ unsigned long long s_pg[kWarps], s_pe[kWarps];
+    __shared__ float4 s_val[kNormTile / 4];
     WorkRange r = work_range(tk);
     WorkCursor cur;
     cur.init(tk, tt, T, r.q);
@@ -430,27 +474,29 @@ k_topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long
         const long long base = (long long)i * stride + tt.offset[tile];
         const int first = (tile - cur.first_tile) * kNormTile;   // index of the tile's first element
         const uint2 before = tk.tile_count[(long long)i * tt.n_tiles + tile];
-        unsigned int k[kChunks][4];
-        float xv[kChunks][4];
+        unsigned int gmask = 0, emask = 0;
         unsigned long long pg = 0, pe = 0;
 #pragma unroll
         for (int v = 0; v < kChunks; ++v) {
             const int local = (v * kThreads + threadIdx.x) * 4;
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-            if (local < len) { a = ld_stream(x + base + local); b = ld_stream(xhat + base + local); }
-            xv[v][0] = a.x; xv[v][1] = a.y; xv[v][2] = a.z; xv[v][3] = a.w;
-            k[v][0] = rank_key(a.x, b.x); k[v][1] = rank_key(a.y, b.y);
-            k[v][2] = rank_key(a.z, b.z); k[v][3] = rank_key(a.w, b.w);
-        }
+            if (local < len) {
+                const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
+                s_val[v * kThreads + threadIdx.x] = a;
+                const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
+                                           rank_key(a.w, b.w)};
+                const int nel = len - local;
+                unsigned int g = 0, e = 0;
 #pragma unroll
-        for (int v = 0; v < kChunks; ++v) {
-            const int local = (v * kThreads + threadIdx.x) * 4;
-            unsigned int gt = 0, eq = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (local + c < len) { gt += (k[v][c] > tau); eq += (k[v][c] == tau); }
-            pg |= (unsigned long long)gt << (16 * v);
-            pe |= (unsigned long long)eq << (16 * v);
+                for (int c = 0; c < 4; ++c) {
+                    const bool live = c < nel;
+                    g |= (live && k[c] > tau) ? (1u << c) : 0u;
+                    e |= (live && k[c] == tau) ? (1u << c) : 0u;
+                }
+                gmask |= g << (4 * v);
+                emask |= e << (4 * v);
+                pg |= (unsigned long long)__popc(g) << (16 * v);
+                pe |= (unsigned long long)__popc(e) << (16 * v);
+            }
         }
         // inclusive scan over the CTA in thread order, all four chunks at once
         unsigned long long sg = pg, se = pe;
@@ -470,31 +516,35 @@ k_topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long
         }
         const unsigned long long xg = wg + sg - pg, xe = we + se - pe;   // exclusive, per chunk
         unsigned int run_gt = before.x, run_eq = before.y;               // entries before chunk v
-        if (pg | pe) {
+        const float* my_val = reinterpret_cast<const float*>(s_val);
 #pragma unroll
-            for (int v = 0; v < kChunks; ++v) {
+        for (int v = 0; v < kChunks; ++v) {
+            unsigned int m = ((gmask | emask) >> (4 * v)) & 0xfu;
+            if (m) {
                 const int local = (v * kThreads + threadIdx.x) * 4;
                 unsigned int my_gt = run_gt + (unsigned int)((xg >> (16 * v)) & 0xffffu);
                 unsigned int my_eq = run_eq + (unsigned int)((xe >> (16 * v)) & 0xffffu);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (local + c < len) {
-                        const bool is_gt = k[v][c] > tau, is_eq = k[v][c] == tau;
-                        if (is_gt || (is_eq && my_eq < take)) {
-                            const unsigned int slot = my_gt + min(my_eq, take);
-                            if (slot < K) {
-                                out[slot] = make_int2(first + local + c, __float_as_int(xv[v][c]));
-                                xhat[base + local + c] = xv[v][c];
-                            } else {
-                                atomicOr(err, 2u);
-                            }
+                const unsigned int en = (emask >> (4 * v)) & 0xfu;
+                while (m) {
+                    const int c = __ffs(m) - 1;
+                    m &= m - 1;
+                    const bool is_eq = (en >> c) & 1u;
+                    if (!is_eq || my_eq < take) {
+                        const unsigned int slot = my_gt + min(my_eq, take);
+                        const float val = my_val[local + c];
+                        if (slot < K) {
+                            out[slot] = make_int2(first + local + c, __float_as_int(val));
+                            xhat[base + local + c] = val;
+                        } else {
+                            atomicOr(err, 2u);
                         }
-                        my_gt += is_gt; my_eq += is_eq;
                     }
+                    my_gt += is_eq ? 0u : 1u;
+                    my_eq += is_eq ? 1u : 0u;
                 }
-                run_gt += (unsigned int)((tg >> (16 * v)) & 0xffffu);
-                run_eq += (unsigned int)((te >> (16 * v)) & 0xffffu);
             }
+            run_gt += (unsigned int)((tg >> (16 * v)) & 0xffffu);
+            run_eq += (unsigned int)((te >> (16 * v)) & 0xffffu);
         }
         __syncthreads();
     }

@@ -327,7 +327,8 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         EG_ALLOC(c->tk.hist, S * kMaxBins);
         EG_ALLOC(c->tk.prefix, S); EG_ALLOC(c->tk.remaining, S);
         EG_ALLOC(c->tk.tile_count, (size_t)P * c->tiles_norm.n_tiles);
-        EG_ALLOC(c->tk.tile_cand, (size_t)P * c->tiles_norm.n_tiles);
+        EG_ALLOC(c->tk.tile_cand, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
+        EG_ALLOC(c->tk.tile_gt, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
         EG_ALLOC(c->tk.cand, (size_t)P * c->stride);
         EG_ALLOC(c->tk.plan, 1);
         EG_ALLOC(c->tk.sp_seg, S);
