@@ -278,7 +278,7 @@ def time_steps(eg, x, grads, lr, steps, sampler=None):
     return e0.elapsed_time(e1), launches
 
 
-def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_variant):
+def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_variant, graph_steps=0):
     """Times K steps of `wl` for every variant; returns ({variant: figures}, context)."""
     eg = B.from_workload(wl)
     buf_bytes = wl.P * eg.replica_stride * 4
@@ -313,6 +313,34 @@ def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_varian
             "messages_sent": stats["messages"], "bytes_sent": stats["bytes"],
             "pct_messages": 100.0 * stats["messages"] / (wl.P * wl.T * 2 * K),
             "gradient_buffers": n_buf}
+    if graph_steps:
+        # launch-bound cases: the same steady-state step replayed from a CUDA graph (gradients of
+        # one step, carried norm); shows what remains when the launch overhead is taken away
+        eg.set_timing(False)
+        eg.set_carry_norm(True)
+        x.copy_(x0)
+        eg.reset()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for k in range(3):
+                eg.step(x, grads[0], wl.lr)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            eg.step(x, grads[0], wl.lr)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(5):
+            g.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(graph_steps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        results["graph_replay_ms_per_step"] = e0.elapsed_time(e1) / graph_steps
+        del g
     del x
     return results, (eg, x0, grads, n_buf, buf_bytes)
 
@@ -332,7 +360,8 @@ def run_native(args):
         rows = []
         for idx in (1, 2, 3, 4, 5):
             for w in W.config(idx):
-                r, ctx = measure_workload(B, w, w.steps, Wm, dev, world, ("carry", "two_pass"), None, None)
+                r, ctx = measure_workload(B, w, w.steps, Wm, dev, world, ("carry", "two_pass"), None, None,
+                                          graph_steps=200 if w.N < 1_000_000 else 0)
                 ctx[0].close()
                 del ctx
                 rows.append({"config": idx, "workload": w.name, "P": w.P, "tensors": w.T, "elements": w.N,
@@ -341,7 +370,8 @@ def run_native(args):
                                     "pct_of_peak": 100.0 * r[v]["gbs"] / peak,
                                     "replica_steps_per_s": r[v]["replica_steps_per_s"],
                                     "kernel_ms": r[v]["kernel_ms"], "gradient_buffers": r[v]["gradient_buffers"]}
-                                for v in r},
+                                for v in ("carry", "two_pass")},
+                             "graph_replay_ms_per_step": r.get("graph_replay_ms_per_step"),
                              "messages_sent": r["carry"]["messages_sent"],
                              "pct_messages": r["carry"]["pct_messages"],
                              "bytes_sent": r["carry"]["bytes_sent"]})

@@ -299,6 +299,40 @@ def test_run_twice_is_deterministic():
     assert all(np.array_equal(a, b) for a, b in zip(outs[0][1], outs[1][1]))
 
 
+def test_steps_replayed_from_a_cuda_graph_match_direct_calls():
+    """eg_step only enqueues work and takes no decision on the host, so a captured step can be
+    replayed: the trigger state lives on the device and advances with every replay."""
+    wl = W.synthetic(4, [5, 1000, 4097, 70000], steps=8, lr=0.1, grad_sigma=0.01)
+    g = None
+    outs = []
+    for use_graph in (False, True):
+        eg = B.from_workload(wl)
+        eg.set_carry_norm(True)
+        x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+        grad = eg.to_layout(wl.grads(0, "cuda"))
+        eg.step(x, grad, wl.lr)                       # first step (computes the norms itself)
+        if use_graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                eg.step(x, grad, wl.lr)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):                 # recorded, not executed
+                eg.step(x, grad, wl.lr)
+            for _ in range(6):
+                g.replay()
+        else:
+            for _ in range(7):
+                eg.step(x, grad, wl.lr)
+        torch.cuda.synchronize()
+        outs.append((x.clone(), eg.stats(), eg.last_decisions()))
+        eg.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    assert all(np.array_equal(a, b) for a, b in zip(outs[0][2], outs[1][2]))
+
+
 def test_average_model_and_consensus():
     from oracle import eg_oracle as eo
     wl = W.synthetic(5, [3, 1000, 4097])
