@@ -108,7 +108,10 @@ eg_status eg_step(eg_ctx* ctx, float* params, const float* grads, float lr, void
 /* Same iteration for callers whose data lives in HOST memory: copies params_host and
  * grads_host ([P][replica_stride] fp32, ideally pinned) to device staging buffers owned by
  * the context (allocated on first use), runs eg_step, copies the updated parameters back
- * and synchronises. */
+ * and synchronises.  Tensors do not interact within an iteration, so for dense contexts on the
+ * nearest-neighbour ring the work is pipelined in groups of tensors: while one group is being
+ * computed the next is being copied in and the previous one copied out (pinned host buffers
+ * are needed for the copies to overlap).  The result is the same as that of eg_step. */
 eg_status eg_step_host(eg_ctx* ctx, float* params_host, const float* grads_host, float lr);
 
 /* Carried-norm mode (off by default).  When on, the fused average/update kernel of step k

@@ -177,7 +177,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         mbar_init(wrap_bar, 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (blockIdx.x == 0) *step_k += 1;   // nothing in this launch reads it
+        if (blockIdx.x == 0 && step_k) *step_k += 1;   // nothing in this launch reads it
     }
     __syncthreads();
 

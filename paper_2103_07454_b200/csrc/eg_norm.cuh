@@ -62,6 +62,7 @@ struct DecideParams {
     int degree;               // distinct ring neighbours of every replica
     int variant;              // kChangeOfNorm: d = | sqrt(sum) - sent_norm |
     double cap;               // bound sqrt(g(k)) on the threshold of this step (+inf: none)
+    int t0, tn;               // tensors [t0, t0 + tn) are decided by this launch
 };
 
 // Intermittent delivery: which outstanding messages arrive in this step.
@@ -81,9 +82,11 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
          const long long* __restrict__ topk_count, int* __restrict__ outbox_count,
          Counters* ctr, const long long* __restrict__ step_k, DeliveryState dl) {
     const int lane = threadIdx.x & 31;
-    const long long s = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (s >= (long long)dp.P * dp.T) return;
-    const int i = (int)(s / dp.T), t = (int)(s % dp.T);
+    // work item: (replica, tensor of the launch's range)
+    const long long w = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (w >= (long long)dp.P * dp.tn) return;
+    const int i = (int)(w / dp.tn), t = dp.t0 + (int)(w % dp.tn);
+    const long long s = (long long)i * dp.T + t;
     const int q0 = seg_begin[t], q1 = seg_begin[t + 1];
     const double* p = partials + (long long)i * n_tiles;
     double acc = 0.0;

@@ -75,6 +75,13 @@ struct eg_ctx {
     int variant = 0;
     double cap_alpha = 0.0, cap_beta = 1.0;   // bound alpha*beta^k on the squared threshold
     long long host_k = 0;                     // host copy of the iteration counter
+    // sub-range of the step that eg_step_masked launches (eg_step_host pipelines groups of
+    // tensors); the default is everything
+    std::vector<int> seg_begin_norm, seg_begin_fused;   // host copies, [T+1]
+    int range_t0 = 0, range_tn = 0;                      // tn == 0: all tensors
+    bool range_last = true;                              // the launch that ends the iteration
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    std::vector<cudaEvent_t> group_events;
     // intermittent delivery (two copies: sent = xhat, received = mailbox)
     bool async = false;
     float* mailbox = nullptr;
@@ -259,6 +266,9 @@ void eg_destroy(eg_ctx* c) {
         cudaDeviceSynchronize();
         for (void* p : c->allocs) cudaFree(p);
         for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+        for (cudaEvent_t e : c->group_events) cudaEventDestroy(e);
+        if (c->copy_in) cudaStreamDestroy(c->copy_in);
+        if (c->copy_out) cudaStreamDestroy(c->copy_out);
     }
     delete c;
 }
@@ -303,8 +313,14 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     c->out_stride = koff;
 
     const size_t S = (size_t)P * T;
-    if ((s = upload_tiles(c, build_tiles(c->numel, c->offset, kNormTile), &c->tiles_norm)) != EG_OK) return fail(s);
-    if ((s = upload_tiles(c, build_tiles(c->numel, c->offset, kFusedTile), &c->tiles_fused)) != EG_OK) return fail(s);
+    {
+        const HostTiles hn = build_tiles(c->numel, c->offset, kNormTile);
+        const HostTiles hf = build_tiles(c->numel, c->offset, kFusedTile);
+        c->seg_begin_norm = hn.seg_begin;
+        c->seg_begin_fused = hf.seg_begin;
+        if ((s = upload_tiles(c, hn, &c->tiles_norm)) != EG_OK) return fail(s);
+        if ((s = upload_tiles(c, hf, &c->tiles_fused)) != EG_OK) return fail(s);
+    }
     std::vector<long long> numel_ll(c->numel.begin(), c->numel.end());
     std::vector<long long> kcount_ll(c->kcount.begin(), c->kcount.end());
     std::vector<long long> out_off_ll(c->out_off.begin(), c->out_off.end());
@@ -409,16 +425,32 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     c->last_stream = stream;
     int launches = 0;
-    const TileTable tn = c->tiles_norm.view(), tf = c->tiles_fused.view();
-    const dim3 grid_norm(tn.n_tiles, c->P);
+    const TileTable tn_all = c->tiles_norm.view(), tf_all = c->tiles_fused.view();
     const int S = c->P * c->T;
+    // tensors [t0, t0 + tcount) of this launch and their tiles in both tile tables
+    const int t0 = c->range_tn ? c->range_t0 : 0, tcount = c->range_tn ? c->range_tn : c->T;
+    const int nb = c->seg_begin_norm[t0], ne = c->seg_begin_norm[t0 + tcount];
+    const int fb = c->seg_begin_fused[t0], fe = c->seg_begin_fused[t0 + tcount];
+    const bool whole = (tcount == c->T);
+    // views of the tile tables that start at the first tile of the range (per-tile arrays and
+    // the partial-sum arrays are shifted together, so the kernels index them as usual)
+    TileTable tn = tn_all, tf = tf_all;
+    tn.tensor += nb; tn.offset += nb; tn.length += nb;
+    tf.tensor += fb; tf.offset += fb; tf.length += fb;
+    const dim3 grid_norm(ne - nb, c->P);
+    const int grid_fused = fe - fb;
+    double* partials_norm = c->partials_norm + nb;
+    double* partials_fused = c->partials_fused + fb;
+    long long* step_k = c->range_last ? c->step_k : nullptr;
+    if (!whole && (c->topk.enabled || c->async || c->hops > 1 || c->fused_kind != EG_FUSED_PIPELINED))
+        return EG_ERR_STATE;
 
     // a1: || x - x_hat || partial sums, unless the previous step carried them over
     const bool carry = c->carry && !c->async;   // no carried norm under intermittent delivery
     const bool use_carried = carry && c->carried_valid && c->carried_params == params;
     if (!use_carried) {
         TimedSection ts(c, stream, EG_KERNEL_NORM);
-        k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, c->partials_norm,
+        k_norm_partial<<<grid_norm, kThreads, 0, stream>>>(params, c->xhat, tn, c->stride, partials_norm,
                                                           c->variant);
         ++launches;
     }
@@ -426,12 +458,13 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
                     c->topk.enabled, c->degree, c->variant,
                     c->cap_alpha > 0.0 ? std::sqrt(c->cap_alpha * std::pow(c->cap_beta, (double)c->host_k))
-                                       : HUGE_VAL};
+                                       : HUGE_VAL,
+                    t0, tcount};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
-    const TileTable& tp = use_carried ? tf : tn;
+    const TileTable& tp = use_carried ? tf_all : tn_all;
     {
         TimedSection ts(c, stream, EG_KERNEL_DECIDE);
-        k_decide<<<(S + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
+        k_decide<<<(c->P * tcount + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
             partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
             c->ctr, c->step_k,
             DeliveryState{deliver_dev, c->pending, c->recv_valid, c->arrive, c->arrivals, c->async ? 1 : 0});
@@ -458,53 +491,53 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         const uint8_t* valid = c->async ? c->recv_valid : c->st.valid;   // whom the neighbours have heard from
         if (c->hops > 1) {
             if (carry)
-                k_fused_hops<true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+                k_fused_hops<true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->variant, c->hops);
+                    partials_fused, step_k, c->variant, c->hops);
             else
-                k_fused_hops<false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+                k_fused_hops<false><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    c->partials_fused, c->step_k, c->variant, c->hops,
+                    partials_fused, step_k, c->variant, c->hops,
                     c->async ? c->mailbox : nullptr, c->async ? c->arrive : nullptr);
         } else if (c->async) {
             k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>
-                <<<tf.n_tiles, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
+                <<<grid_fused, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                 params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                c->partials_fused, c->step_k, c->err, c->variant, c->mailbox, c->arrive);
+                partials_fused, step_k, c->err, c->variant, c->mailbox, c->arrive);
         } else if (c->fused_kind == EG_FUSED_PIPELINED) {
             const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
 #define EG_PIPE_ARGS params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, \
-                     c->partials_fused, c->step_k, c->err
+                     partials_fused, step_k, c->err
             if (c->variant == 0) {
                 if (carry)
                     k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
-                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
                 else
                     k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>
-                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
             } else {
                 if (carry)
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, true, false>
-                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
                 else
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, false>
-                        <<<tf.n_tiles, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
             }
 #undef EG_PIPE_ARGS
         } else if (carry)
-            k_fused<kFusedVpt, true><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+            k_fused<kFusedVpt, true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                 params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                c->partials_fused, c->step_k, c->variant);
+                partials_fused, step_k, c->variant);
         else
-            k_fused<kFusedVpt, false><<<tf.n_tiles, kThreads, c->fused_smem, stream>>>(
+            k_fused<kFusedVpt, false><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                 params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                c->partials_fused, c->step_k, c->variant);
+                partials_fused, step_k, c->variant);
         ++launches;
     }
-    c->carried_valid = carry;
+    c->carried_valid = carry && whole;
     c->carried_params = params;
     c->stepped = true;
-    c->host_k += 1;
+    if (c->range_last) c->host_k += 1;
     c->last_launches = launches;
     EG_CUDA(c, cudaGetLastError());
     return EG_OK;
@@ -521,15 +554,81 @@ eg_status eg_step_host(eg_ctx* c, float* params_host, const float* grads_host, f
         if ((s = dev_alloc(c, &c->stage_g, (size_t)c->P * c->stride, false)) != EG_OK) return s;
     }
     cudaStream_t stream = c->last_stream;
-    EG_CUDA(c, cudaMemcpyAsync(c->stage_x, params_host, bytes, cudaMemcpyHostToDevice, stream));
-    EG_CUDA(c, cudaMemcpyAsync(c->stage_g, grads_host, bytes, cudaMemcpyHostToDevice, stream));
-    c->carried_valid = false;  // the parameters came from outside
-    eg_status s = eg_step(c, c->stage_x, c->stage_g, lr, stream);
-    if (s != EG_OK) return s;
-    EG_CUDA(c, cudaMemcpyAsync(params_host, c->stage_x, bytes, cudaMemcpyDeviceToHost, stream));
+    c->carried_valid = false;  // the parameters come from outside
+    const bool pipelined = !c->topk.enabled && !c->async && c->hops == 1 &&
+                           c->fused_kind == EG_FUSED_PIPELINED && c->T >= 2;
+    if (!pipelined) {
+        EG_CUDA(c, cudaMemcpyAsync(c->stage_x, params_host, bytes, cudaMemcpyHostToDevice, stream));
+        EG_CUDA(c, cudaMemcpyAsync(c->stage_g, grads_host, bytes, cudaMemcpyHostToDevice, stream));
+        eg_status s = eg_step(c, c->stage_x, c->stage_g, lr, stream);
+        if (s != EG_OK) return s;
+        EG_CUDA(c, cudaMemcpyAsync(params_host, c->stage_x, bytes, cudaMemcpyDeviceToHost, stream));
+        EG_CUDA(c, cudaStreamSynchronize(stream));
+        c->carried_valid = false;
+        return EG_OK;
+    }
+    // Tensors do not interact within a step, so the step is run group by group: while one group
+    // of tensors is being computed, the next one is on its way in and the previous one on its
+    // way out (the two directions of the host link work at the same time).
+    constexpr int kGroups = 8;
+    struct RangeReset {   // whatever happens below, later steps cover all tensors again
+        eg_ctx* c;
+        ~RangeReset() { c->range_t0 = 0; c->range_tn = 0; c->range_last = true; }
+    } range_reset{c};
+    if (!c->copy_in) {
+        EG_CUDA(c, cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking));
+        EG_CUDA(c, cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking));
+        for (int q = 0; q < 2 * kGroups + 1; ++q) {
+            cudaEvent_t e;
+            EG_CUDA(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            c->group_events.push_back(e);
+        }
+    }
+    // group boundaries at tensor starts, about equal numbers of elements
+    int bounds[kGroups + 1];
+    bounds[0] = 0;
+    {
+        int t = 0;
+        for (int gidx = 1; gidx < kGroups; ++gidx) {
+            const int64_t target = c->stride * gidx / kGroups;
+            while (t < c->T && c->offset[t] < target) ++t;
+            bounds[gidx] = std::max(bounds[gidx - 1], std::min(t, c->T));
+        }
+        bounds[kGroups] = c->T;
+    }
+    // the copies must not start before earlier work on the staging buffers has finished
+    EG_CUDA(c, cudaEventRecord(c->group_events[2 * kGroups], stream));
+    EG_CUDA(c, cudaStreamWaitEvent(c->copy_in, c->group_events[2 * kGroups], 0));
+    eg_status status = EG_OK;
+    int last_group = -1;
+    for (int gidx = 0; gidx < kGroups; ++gidx)
+        if (bounds[gidx + 1] > bounds[gidx]) last_group = gidx;
+    const size_t pitch = (size_t)c->stride * sizeof(float);
+    for (int gidx = 0; gidx < kGroups && status == EG_OK; ++gidx) {
+        const int t0 = bounds[gidx], t1 = bounds[gidx + 1];
+        if (t1 <= t0) continue;
+        const int64_t e0 = c->offset[t0], e1 = (t1 < c->T) ? c->offset[t1] : c->stride;
+        const size_t width = (size_t)(e1 - e0) * sizeof(float);
+        EG_CUDA(c, cudaMemcpy2DAsync(c->stage_x + e0, pitch, params_host + e0, pitch, width, c->P,
+                                     cudaMemcpyHostToDevice, c->copy_in));
+        EG_CUDA(c, cudaMemcpy2DAsync(c->stage_g + e0, pitch, grads_host + e0, pitch, width, c->P,
+                                     cudaMemcpyHostToDevice, c->copy_in));
+        EG_CUDA(c, cudaEventRecord(c->group_events[2 * gidx], c->copy_in));
+        EG_CUDA(c, cudaStreamWaitEvent(stream, c->group_events[2 * gidx], 0));
+        c->range_t0 = t0;
+        c->range_tn = t1 - t0;
+        c->range_last = (gidx == last_group);
+        status = eg_step(c, c->stage_x, c->stage_g, lr, stream);
+        if (status != EG_OK) break;
+        EG_CUDA(c, cudaEventRecord(c->group_events[2 * gidx + 1], stream));
+        EG_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->group_events[2 * gidx + 1], 0));
+        EG_CUDA(c, cudaMemcpy2DAsync(params_host + e0, pitch, c->stage_x + e0, pitch, width, c->P,
+                                     cudaMemcpyDeviceToHost, c->copy_out));
+    }
     EG_CUDA(c, cudaStreamSynchronize(stream));
+    EG_CUDA(c, cudaStreamSynchronize(c->copy_out));
     c->carried_valid = false;
-    return EG_OK;
+    return status;
 }
 
 eg_status eg_stats(eg_ctx* c, uint64_t* messages_sent_host, uint64_t* bytes_sent_host) {

@@ -272,8 +272,12 @@ def test_checkpoint_roundtrip_and_reset():
     eg.close()
 
 
-def test_host_buffer_entry_point():
-    wl = W.synthetic(3, [7, 3000], steps=3, lr=0.1, grad_sigma=0.01)
+@pytest.mark.parametrize("numel", [[7, 3000], RAGGED[:-1], [5000]])
+@pytest.mark.parametrize("hist", [1, 3])
+def test_host_buffer_entry_point(numel, hist):
+    """eg_step_host (host buffers; tensors pipelined in groups through the device when the
+    context allows it) gives the same iteration as eg_step on device buffers."""
+    wl = W.synthetic(3, numel, steps=6, lr=0.1, grad_sigma=0.01, history_len=hist)
     a, b = B.from_workload(wl), B.from_workload(wl)
     x0 = a.to_layout(W.distinct_init_params(wl, "cuda"))
     xa, xb = x0.clone(), x0.cpu().pin_memory()
@@ -281,7 +285,13 @@ def test_host_buffer_entry_point():
         g = a.to_layout(wl.grads(k, "cuda"))
         a.step(xa, g, wl.lr)
         b.step_host(xb, g.cpu().pin_memory(), wl.lr)
+        for u, v in zip(a.last_decisions(), b.last_decisions()):
+            assert np.array_equal(u, v)
     assert torch.equal(xa.cpu(), xb) and a.stats() == b.stats()
+    assert torch.equal(a.mailboxes(), b.mailboxes())
+    b.step(xa, g, wl.lr)        # a plain step afterwards covers all tensors again
+    a.step(xa.clone(), g, wl.lr)
+    assert a.stats() == b.stats()
 
 
 def test_run_twice_is_deterministic():
