@@ -12,17 +12,18 @@
 //   digit 2, per-tile counts  from the candidates only (a few percent of the data)
 //   pass C  (reads x, x_hat)  ordered compaction into the outbox and delivery into x_hat
 // so a sparse message costs three passes over its tensor.  The host knows nothing about the
-// decisions: a one-CTA planning kernel turns the device-side `sparse` flags into a compact list
-// of work tiles, and every other kernel runs a fixed-size grid over that list (an empty list
-// costs a few microseconds per launch).
+// decisions: a planning phase turns the device-side `sparse` flags into a compact list of work
+// tiles and every other phase runs a fixed-size grid over that list.  All phases run in one
+// cooperative launch (k_topk_all, bottom of this file).
 #pragma once
+#include <cooperative_groups.h>
+
 #include "eg_common.cuh"
 
 namespace eg {
 
 constexpr int kTopkGrid = 148 * 8;      // CTAs of the tile kernels (they loop over the work list)
 constexpr int kTopkSegGrid = 148 * 4;   // CTAs of the per-segment kernels
-constexpr int kPlanThreads = 1024;
 
 struct TopkPlan {
     int n_sparse;       // segments that send a sparse message in this step
@@ -54,12 +55,12 @@ __device__ __forceinline__ unsigned int rank_key(float a, float b) {
 // digit 0: bits 30..20, digit 1: bits 19..10, digit 2: bits 9..0
 __device__ __forceinline__ int digit_bits(int digit) { return digit == 0 ? kDigitBits0 : kDigitBits1; }
 
-// One CTA: compact list of the sparse segments and of their tiles, in segment order.
-__global__ void __launch_bounds__(kPlanThreads)
-k_topk_plan(int S, int T, const uint8_t* __restrict__ sparse, const int* __restrict__ seg_begin,
-            TopkState tk) {
-    __shared__ int s_cnt[kPlanThreads], s_tiles[kPlanThreads];
-    const int per = (S + kPlanThreads - 1) / kPlanThreads;
+// One CTA (of kThreads threads): compact list of the sparse segments and of their tiles, in
+// segment order.
+__device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restrict__ sparse,
+                                          const int* __restrict__ seg_begin, const TopkState& tk) {
+    __shared__ int s_cnt[kThreads], s_tiles[kThreads];
+    const int per = (S + kThreads - 1) / kThreads;
     const int lo = threadIdx.x * per, hi = min(S, lo + per);
     int cnt = 0, tiles = 0;
     for (int s = lo; s < hi; ++s)
@@ -67,8 +68,8 @@ k_topk_plan(int S, int T, const uint8_t* __restrict__ sparse, const int* __restr
     s_cnt[threadIdx.x] = cnt;
     s_tiles[threadIdx.x] = tiles;
     __syncthreads();
-    // inclusive scan (Hillis-Steele) over the 1024 per-thread totals
-    for (int o = 1; o < kPlanThreads; o <<= 1) {
+    // inclusive scan (Hillis-Steele) over the per-thread totals
+    for (int o = 1; o < kThreads; o <<= 1) {
         int a = 0, b = 0;
         if (threadIdx.x >= o) { a = s_cnt[threadIdx.x - o]; b = s_tiles[threadIdx.x - o]; }
         __syncthreads();
@@ -85,7 +86,7 @@ k_topk_plan(int S, int T, const uint8_t* __restrict__ sparse, const int* __restr
             ++q;
             w += seg_begin[t + 1] - seg_begin[t];
         }
-    if (threadIdx.x == kPlanThreads - 1) {
+    if (threadIdx.x == kThreads - 1) {
         tk.plan->n_sparse = s_cnt[threadIdx.x];
         tk.plan->total_tiles = s_tiles[threadIdx.x];
         tk.sp_begin[s_cnt[threadIdx.x]] = s_tiles[threadIdx.x];
@@ -141,8 +142,8 @@ struct WorkCursor {
 };
 
 // Pass A: histogram of the top digit of every key of the work tiles.
-__global__ void __launch_bounds__(kThreads)
-k_topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
+__device__ __forceinline__ void
+topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
             long long stride, TopkState tk) {
     __shared__ unsigned int s_hist[kMaxBins];
     WorkRange r = work_range(tk);
@@ -180,8 +181,8 @@ k_topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTab
 
 // One CTA per sparse segment: pick the bin that holds the wanted rank, counting from the
 // largest key downwards; clear the histogram for the next digit.
-__global__ void __launch_bounds__(kThreads)
-k_topk_pick(int T, TopkState tk, int digit) {
+__device__ __forceinline__ void
+topk_pick(int T, TopkState tk, int digit) {
     __shared__ unsigned int s_warp[kWarps];
     const int nq = tk.plan->n_sparse;
     const int nbins = 1 << digit_bits(digit);
@@ -243,8 +244,8 @@ __device__ __forceinline__ int sub_offset(int len, int w) {
 // sub-slice of the tile's candidate slice, so no counter is shared: a thread marks its
 // candidates in a 16-bit mask, a warp scan of the counts gives its first slot, and the keys
 // are fetched back from shared memory (written and read by the same thread).
-__global__ void __launch_bounds__(kThreads, 4)
-k_topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
+__device__ __forceinline__ void
+topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
                long long stride, TopkState tk) {
     constexpr int kBins1 = 1 << kDigitBits1;
     constexpr int kChunks = kNormTile / (kThreads * 4);
@@ -339,8 +340,8 @@ __device__ __forceinline__ WarpTile warp_tile(const TopkState& tk, const TileTab
 
 // Digit 2 over the candidates: one warp per tile, global histogram updated directly (only the
 // candidates that match the 21 resolved bits take part: about one in a thousand).
-__global__ void __launch_bounds__(kThreads)
-k_topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk) {
+__device__ __forceinline__ void
+topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk) {
     const int total = tk.plan->total_tiles;
     const int lane = threadIdx.x & 31;
     const int nwarps = gridDim.x * kWarps;
@@ -364,8 +365,8 @@ k_topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk) {
 
 // Per tile: keys greater than / equal to tau, from the per-warp counts of pass B and the
 // tile's candidates.  One warp per tile.
-__global__ void __launch_bounds__(kThreads)
-k_topk_count(TileTable tt, int T, long long stride, TopkState tk) {
+__device__ __forceinline__ void
+topk_count(TileTable tt, int T, long long stride, TopkState tk) {
     const int total = tk.plan->total_tiles;
     const int lane = threadIdx.x & 31;
     const int nwarps = gridDim.x * kWarps;
@@ -395,8 +396,8 @@ k_topk_count(TileTable tt, int T, long long stride, TopkState tk) {
 }
 
 // One CTA per sparse segment: exclusive prefix of the tile counts, in tile order.
-__global__ void __launch_bounds__(kThreads)
-k_topk_scan(TileTable tt, int T, TopkState tk) {
+__device__ __forceinline__ void
+topk_scan(TileTable tt, int T, TopkState tk) {
     __shared__ unsigned int s_gt[kWarps], s_eq[kWarps];
     __shared__ unsigned int s_run[2];
     const int nq = tk.plan->n_sparse;
@@ -447,8 +448,8 @@ k_topk_scan(TileTable tt, int T, TopkState tk) {
 // holds at most 1024 entries, so the fields cannot overflow); then only the marked elements
 // are visited.  A thread has read the x_hat entries it owns before it overwrites any of them,
 // and no thread touches another thread's entries.
-__global__ void __launch_bounds__(kThreads, 4)
-k_topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long long stride,
+__device__ __forceinline__ void
+topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long long stride,
              TopkState tk, unsigned int* __restrict__ err) {
     constexpr int kChunks = kNormTile / (kThreads * 4);   // 4
     static_assert(kChunks == 4, "the packed scan holds four 16-bit fields");
@@ -548,6 +549,66 @@ k_topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long
         }
         __syncthreads();
     }
+}
+
+// ---------------------------------------------------------------------------------------
+// Launch forms.  k_topk_all runs the whole sequence in ONE cooperative launch with grid-wide
+// barriers between the phases, and every CTA leaves after the first barrier when no segment
+// sends a sparse message in this step -- a quiet step then costs one launch instead of ten.
+// The single-phase kernels below are the fallback where a cooperative launch is not available.
+// ---------------------------------------------------------------------------------------
+struct TopkArgs {
+    const float* x;
+    float* xhat;
+    TileTable tt;
+    int S, T;
+    long long stride;
+    const uint8_t* sparse;
+    TopkState tk;
+    unsigned int* err;
+};
+
+__global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
+    cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+    if (blockIdx.x == 0) topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk);
+    grid.sync();
+    if (a.tk.plan->n_sparse == 0) return;          // the same for every CTA
+    topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+    grid.sync();
+    topk_pick(a.T, a.tk, 0);
+    grid.sync();
+    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+    grid.sync();
+    topk_pick(a.T, a.tk, 1);
+    grid.sync();
+    topk_hist_cand(a.tt, a.T, a.stride, a.tk);
+    grid.sync();
+    topk_pick(a.T, a.tk, 2);
+    grid.sync();
+    topk_count(a.tt, a.T, a.stride, a.tk);
+    grid.sync();
+    topk_scan(a.tt, a.T, a.tk);
+    grid.sync();
+    topk_write(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
+}
+
+__global__ void __launch_bounds__(kThreads) k_topk_plan(TopkArgs a) {
+    topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_hist(TopkArgs a) {
+    topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int digit) { topk_pick(a.T, a.tk, digit); }
+__global__ void __launch_bounds__(kThreads, 4) k_topk_collect(TopkArgs a) {
+    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_hist_cand(TopkArgs a) {
+    topk_hist_cand(a.tt, a.T, a.stride, a.tk);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_count(TopkArgs a) { topk_count(a.tt, a.T, a.stride, a.tk); }
+__global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) { topk_scan(a.tt, a.T, a.tk); }
+__global__ void __launch_bounds__(kThreads, 4) k_topk_write(TopkArgs a) {
+    topk_write(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
 }
 
 }  // namespace eg

@@ -194,6 +194,15 @@ def test_ragged_topk(P, frac):
     assert rep.params_bit_exact and rep.sparse_checked > 10
 
 
+def test_topk_with_separate_launches(monkeypatch):
+    """The ten single-phase Top-K launches (fallback where a cooperative launch is unavailable)."""
+    monkeypatch.setenv("EG_TOPK_SEPARATE_LAUNCHES", "1")
+    wl = W.synthetic(3, RAGGED, steps=10, lr=0.1, grad_sigma=0.01, topk=(10, 100))
+    rep = lockstep(wl, init="distinct", outbox_samples=64)
+    assert rep.params_bit_exact and rep.sparse_checked > 5
+    assert rep.launches == 10 * 13
+
+
 @pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
 def test_topk_carry_norm(kernel):
     wl = W.synthetic(4, RAGGED, steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100))
