@@ -194,6 +194,23 @@ def test_ragged_topk(P, frac):
     assert rep.params_bit_exact and rep.sparse_checked > 10
 
 
+@pytest.mark.parametrize("separate", [False, True])
+def test_topk_degenerate_all_keys_equal(separate, monkeypatch):
+    """Threshold 0 with zero gradients and identical replicas: every |x - x_hat| is exactly 0
+    from the third step on, so all keys tie, every element is a candidate and the message is
+    the first K_t indices."""
+    if separate:
+        monkeypatch.setenv("EG_TOPK_SEPARATE_LAUNCHES", "1")
+    wl = W.synthetic(3, [1, 5, 33, 4095, 4096, 4097, 20000], steps=6, lr=0.1, grad_sigma=0.01, topk=(7, 100))
+
+    def zero_after_first(k, g):
+        return g if k == 0 else torch.zeros_like(g)
+
+    rep = lockstep(wl, oracle_kw=dict(mode=1, delta_fixed=0.0), outbox_samples=10 ** 6,
+                   grad_hook=zero_after_first)
+    assert rep.params_bit_exact and rep.events == 3 * wl.T * wl.steps and rep.sparse_checked >= 3 * wl.T * 4
+
+
 def test_topk_with_separate_launches(monkeypatch):
     """The ten single-phase Top-K launches (fallback where a cooperative launch is unavailable)."""
     monkeypatch.setenv("EG_TOPK_SEPARATE_LAUNCHES", "1")
