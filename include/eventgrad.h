@@ -35,8 +35,8 @@
  *  - One context belongs to one device (the one current at eg_create) and is used from one
  *    stream at a time.
  *  - Every function returns an eg_status; nothing throws, aborts or traps.  A device-side
- *    problem (an index outside its table) sets an error word that the next synchronising
- *    call returns as EG_ERR_INTERNAL.
+ *    problem (an index outside its table, a bounded wait that ran out) sets an error word that
+ *    the next synchronising call returns as EG_ERR_INTERNAL or EG_ERR_TIMEOUT.
  *  - Counters: an event of tensor t at replica i adds deg(i) to messages_sent (deg = number
  *    of distinct ring neighbours: min(2*hops, P-1), i.e. 2 on the paper's ring) and deg(i)*payload to
  *    bytes_sent; payload = 4*n_t for a dense message, 8*K_t for a Top-K message
@@ -61,7 +61,7 @@ typedef enum {
     EG_ERR_OOM = 2,      /* host or device allocation failed */
     EG_ERR_CUDA = 3,     /* a CUDA runtime call failed; see eg_last_cuda_error */
     EG_ERR_STATE = 4,    /* call not allowed in the context's current state */
-    EG_ERR_TIMEOUT = 5,  /* reserved */
+    EG_ERR_TIMEOUT = 5,  /* a bounded device-side wait gave up (see eg_selftest_wait_timeout) */
     EG_ERR_INTERNAL = 6  /* device-side consistency check failed */
 } eg_status;
 
@@ -258,6 +258,14 @@ eg_status eg_change_norms_static(const float* x_dev, const float* xhat_dev, int 
                                  int64_t replica_stride, const int64_t* tensor_offset_host,
                                  const int64_t* layer_numel_host, int T, double* norms_dev,
                                  void* stream);
+
+/* Self-test of the failure path of the pipelined kernels.  Their waits on shared-memory
+ * barriers are bounded: a wait that runs out sets a bit in the context's error word and the
+ * kernel returns instead of hanging.  This call launches one warp that waits (for about a
+ * millisecond) on a barrier that nothing completes.  It returns EG_OK when the wait gave up as
+ * designed; from then on the calls that synchronise (eg_stats, eg_last_*, ...) return
+ * EG_ERR_TIMEOUT until eg_reset clears the error word.  The context stays usable. */
+eg_status eg_selftest_wait_timeout(eg_ctx* ctx, void* stream);
 
 /* Back to iteration 0 with empty mailboxes, initial thresholds and zero counters. */
 eg_status eg_reset(eg_ctx* ctx);

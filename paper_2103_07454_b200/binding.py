@@ -28,6 +28,7 @@ EXPORTS = [
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
     "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant", "eg_set_threshold_cap",
     "eg_enable_delivery_masks", "eg_step_masked", "eg_read_received", "eg_delivery_status",
+    "eg_selftest_wait_timeout",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -86,6 +87,7 @@ def load_library() -> C.CDLL:
     lib.eg_set_variant.argtypes = [vp, C.c_int, C.c_int]
     lib.eg_set_threshold_cap.argtypes = [vp, C.c_double, C.c_double]
     lib.eg_enable_delivery_masks.argtypes = [vp]
+    lib.eg_selftest_wait_timeout.argtypes = [vp, vp]
     lib.eg_step_masked.argtypes = [vp, vp, vp, C.c_float, vp, vp]
     lib.eg_read_received.argtypes = [vp, vp]
     lib.eg_delivery_status.argtypes = [vp, vp, u64p]
@@ -317,6 +319,11 @@ class EventGrad:
         n = (C.c_uint64 * len(KERNEL_GROUPS))()
         _check(self._lib, self._lib.eg_kernel_times(self._h, ms, n), self._h, "eg_kernel_times")
         return {g: (ms[q], int(n[q])) for q, g in enumerate(KERNEL_GROUPS)}
+
+    def selftest_wait_timeout(self) -> int:
+        """``eg_selftest_wait_timeout``; returns the raw status (0 = the wait gave up as designed)."""
+        s = torch.cuda.current_stream(self.device)
+        return int(self._lib.eg_selftest_wait_timeout(self._h, C.c_void_p(s.cuda_stream)))
 
     def reset(self):
         _check(self._lib, self._lib.eg_reset(self._h), self._h, "eg_reset")

@@ -79,14 +79,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 }
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* s_abort,
-                                                  unsigned int* err) {
+                                                  unsigned int* err,
+                                                  long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     unsigned int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) != 0) continue;       // look at the clock every 64 polls only
         if (*s_abort) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit_cycles) {
             *s_abort = 1;
             atomicOr(err, kErrPipeTimeout);
             return false;
@@ -361,6 +362,23 @@ k_fused_pipe_general(float* __restrict__ x, const float* __restrict__ g, float* 
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, ASYNC, false>(x, g, xhat, snap, valid, tt, P, T, stride,
                                                                  lr, partials, step_k, err, variant, mailbox,
                                                                  arrive);
+}
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes.  The
+// wait gives up after `limit_cycles`, sets the time-out bit in the error word and the kernel
+// returns normally, so the context stays usable.
+__global__ void __launch_bounds__(32) k_selftest_wait(unsigned int* err, long long limit_cycles,
+                                                      int* gave_up) {
+    __shared__ uint64_t bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = mbar_wait_bounded(&bar, 0, &s_abort, err, limit_cycles);
+    if (threadIdx.x == 0) *gave_up = ok ? 0 : 1;
 }
 
 }  // namespace eg

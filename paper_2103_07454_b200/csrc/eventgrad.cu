@@ -200,6 +200,7 @@ eg_status sync_and_check(eg_ctx* c) {
     EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
     unsigned int e = 0;
     EG_CUDA(c, cudaMemcpy(&e, c->err, sizeof(e), cudaMemcpyDeviceToHost));
+    if (e & kErrPipeTimeout) return EG_ERR_TIMEOUT;   // a bounded device-side wait gave up
     return e ? EG_ERR_INTERNAL : EG_OK;
 }
 
@@ -337,7 +338,7 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     EG_ALLOC(c->st.hist_len, S); EG_ALLOC(c->st.valid, S); EG_ALLOC(c->st.flag, S);
     EG_ALLOC(c->st.snap, S); EG_ALLOC(c->st.sparse, S); EG_ALLOC(c->st.norm, S);
     EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S); EG_ALLOC(c->st.sent_norm, S);
-    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 1);
+    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 2);
     EG_ALLOC(c->outbox_count, S);
     EG_ALLOC(c->cons_partials, (size_t)c->tiles_fused.n_tiles + 1);
     if (c->topk.enabled) {
@@ -795,6 +796,21 @@ eg_status eg_delivery_status(eg_ctx* c, uint8_t* pending_host, uint64_t* arrival
         *arrivals_host = a;
     }
     return EG_OK;
+}
+
+eg_status eg_selftest_wait_timeout(eg_ctx* c, void* stream_v) {
+    if (!c) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    c->last_stream = stream;
+    // reuse the plan-sized scratch word of the Top-K state? no: a dedicated int next to the error word
+    int* gave_up = reinterpret_cast<int*>(c->err) + 1;
+    k_selftest_wait<<<1, 32, 0, stream>>>(c->err, 2000000ll /* about a millisecond */, gave_up);
+    EG_CUDA(c, cudaGetLastError());
+    EG_CUDA(c, cudaStreamSynchronize(stream));
+    int h = 0;
+    EG_CUDA(c, cudaMemcpy(&h, gave_up, sizeof(h), cudaMemcpyDeviceToHost));
+    return h ? EG_OK : EG_ERR_INTERNAL;
 }
 
 eg_status eg_set_threshold_cap(eg_ctx* c, double alpha, double beta) {

@@ -392,6 +392,25 @@ def test_generator_is_device_independent():
     assert torch.equal(wl.init_params("cpu"), wl.init_params("cuda").cpu())
 
 
+def test_bounded_wait_gives_up_and_the_context_survives():
+    """Failure detection without a fault: a wait that nothing satisfies runs out after about a
+    millisecond, the kernel returns, the error surfaces as a status, and after eg_reset the
+    context works as before."""
+    wl = W.synthetic(3, [7, 3000], steps=3, lr=0.1, grad_sigma=0.01)
+    eg, ref = B.from_workload(wl), B.from_workload(wl)
+    assert eg.selftest_wait_timeout() == 0
+    with pytest.raises(B.EventGradError, match="timeout"):
+        eg.stats()
+    eg.reset()
+    x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+    y = x.clone()
+    for k in range(wl.steps):
+        g = eg.to_layout(wl.grads(k, "cuda"))
+        eg.step(x, g, wl.lr)
+        ref.step(y, g, wl.lr)
+    assert torch.equal(x, y) and eg.stats() == ref.stats()
+
+
 def test_invalid_arguments_are_reported():
     wl = W.synthetic(2, [8])
     eg = B.from_workload(wl)
