@@ -189,7 +189,8 @@ def sample_tensors(wl: W.Workload, fraction: float):
     return picked
 
 
-def time_oracle(wl: W.Workload, steps: int, warmup: int, budget_s: float, gen_device: str):
+def time_oracle(wl: W.Workload, steps: int, warmup: int, budget_s: float, gen_device: str,
+                single_thread_s: float = 0.0):
     """Times the CPU oracle, as it stands, on all host cores.  If ``steps`` full-size steps do
     not fit ``budget_s`` the run uses a subset of the tensors (they do not interact)."""
     import numpy as np
@@ -229,13 +230,32 @@ def time_oracle(wl: W.Workload, steps: int, warmup: int, budget_s: float, gen_de
     sec = time.perf_counter() - t0
     stats = o.stats()
     o.close()
+    # one thread, for context: a few seconds on the leading tensors
+    one = None
+    if single_thread_s > 0:
+        frac1 = min(1.0, single_thread_s / max(1e-9, 2 * full_step_s * threads))
+        t1 = sample_tensors(wl, frac1) if frac1 < 1.0 else list(range(wl.T))
+        numel1 = [wl.numel[t] for t in t1]
+        cols1 = torch.from_numpy(np.concatenate([np.arange(off[t], off[t] + wl.numel[t]) for t in t1])).to(gen_device)
+        g1 = np.ascontiguousarray(wl.grads(0, gen_device)[:, cols1].cpu().numpy())
+        x1 = np.ascontiguousarray(wl.init_params(gen_device)[:, cols1].cpu().numpy())
+        o1 = eo.Oracle(wl.P, numel1, horizon=wl.horizon, history_len=wl.history_len,
+                       delta_init=wl.delta_init, topk=wl.topk, threads=1)
+        o1.step(x1, g1, wl.lr)
+        t0 = time.perf_counter()
+        o1.step(x1, g1, wl.lr)
+        s1 = time.perf_counter() - t0
+        o1.close()
+        one = {"value": wl.P * sum(numel1) * BYTES_PER_ELEMENT["two_pass"] / s1 / 1e9, "unit": "GB/s",
+               "replica_steps_per_s": wl.P * (sum(numel1) / wl.N) / s1,
+               "sample": f"1 step of {len(t1)}/{wl.T} tensors ({sum(numel1)} elements per replica)"}
     elems = wl.P * n_sub * steps
     gbs = elems * BYTES_PER_ELEMENT["two_pass"] / sec / 1e9
     sample = (f"{steps} steps of all {wl.P} replicas x {len(tensors)}/{wl.T} tensors "
               f"({n_sub}/{wl.N} elements per replica)")
     return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample,
             "replica_steps_per_s": wl.P * steps * (n_sub / wl.N) / sec, "seconds": sec,
-            "messages_sent": stats["messages"]}
+            "messages_sent": stats["messages"], "single_thread": one}
 
 
 def run_reference(args):
@@ -306,13 +326,29 @@ def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_varian
         kt = eg.kernel_times()
         stats = eg.stats()
         units, ms_max = aggregate(float(elems) * K, ms, dev)
+        # the same K steps once more with an event between steps: spread of the single steps
+        # (the figures above come from the two outer events only)
+        x.copy_(x0)
+        eg.reset()
+        eg.set_carry_norm(variant == "carry")
+        eg.set_timing(False)
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+        torch.cuda.synchronize()
+        marks[0].record()
+        for k in range(K):
+            eg.step(x, grads[k % n_buf], wl.lr)
+            marks[k + 1].record()
+        torch.cuda.synchronize()
+        per_step = sorted(marks[k].elapsed_time(marks[k + 1]) for k in range(K))
         results[variant] = {
             "ms_per_step": ms_max / K, "gbs": units * BYTES_PER_ELEMENT[variant] / ms_max / 1e6,
             "replica_steps_per_s": world * wl.P * K / (ms_max / 1e3), "launches": launches,
             "kernel_ms": {g: (v[0] / v[1] if v[1] else None) for g, v in kt.items()},
             "messages_sent": stats["messages"], "bytes_sent": stats["bytes"],
             "pct_messages": 100.0 * stats["messages"] / (wl.P * wl.T * 2 * K),
-            "gradient_buffers": n_buf}
+            "gradient_buffers": n_buf, "cuda_graph": False,
+            "step_ms": {"median": statistics.median(per_step), "best": per_step[0],
+                        "worst": per_step[-1]}}
     if graph_steps:
         # launch-bound cases: the same steady-state step replayed from a CUDA graph (gradients of
         # one step, carried norm); shows what remains when the launch overhead is taken away
@@ -424,8 +460,10 @@ def run_native(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         del grads
         torch.cuda.empty_cache()
-        cpu = time_oracle(wl, steps=args.cpu_steps, warmup=1, budget_s=25.0, gen_device=str(dev))
-        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "replica_steps_per_s")}
+        cpu = time_oracle(wl, steps=args.cpu_steps, warmup=1, budget_s=25.0, gen_device=str(dev),
+                          single_thread_s=4.0)
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "replica_steps_per_s",
+                                   "single_thread")}
 
     if rank == 0:
         line = {"metric": METRIC, "value": main["gbs"], "unit": "GB/s", "n_gpus": world,
@@ -440,6 +478,7 @@ def run_native(args):
                 "pct_of_peak": 100.0 * main["gbs"] / peak,
                 "replica_steps_per_s": main["replica_steps_per_s"],
                 "messages_sent": main["messages_sent"], "pct_messages": main["pct_messages"],
+                "step_ms": main["step_ms"], "cuda_graph": False,
                 "gpu_launches": main["launches"], "clocks": clocks, "e2e": e2e,
                 "roofline": roofline, "cpu_baseline": cpu, "variants": results}
         print(json.dumps(line), flush=True)

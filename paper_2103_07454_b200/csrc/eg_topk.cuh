@@ -6,14 +6,16 @@
 // The rank key is the bit pattern of |x - x_hat| (fp32), which orders like the magnitude.
 // The K_t-th largest key tau is found by radix select over three digits (11 + 10 + 10 bits):
 //   pass A  (reads x, x_hat)  histogram of the top digit                     -> bin b0
-//   pass B  (reads x, x_hat)  keys whose top digit is b0 ("candidates") are copied, tile by
-//                             tile, into a candidate buffer; keys above b0 are counted per tile;
-//                             digit 1 of the candidates is histogrammed on the way
-//   digit 2, per-tile counts  from the candidates only (a few percent of the data)
-//   pass C  (reads x, x_hat)  ordered compaction into the outbox and delivery into x_hat
-// so a sparse message costs three passes over its tensor.  The host knows nothing about the
+//   pass B  (reads x, x_hat)  every element whose top digit is >= b0 is copied, tile by tile and
+//                             in index order, into an entry buffer as (20 low key bits, position,
+//                             value of x); digit 1 of the undecided ones (top digit == b0) is
+//                             histogrammed on the way
+//   digit 2, per-tile counts, ordered compaction into the outbox and delivery into x_hat:
+//                             from the entries only (K_t plus the population of one bin: a few
+//                             percent of the tensor)
+// so a sparse message costs two passes over its tensor.  The host knows nothing about the
 // decisions: a planning phase turns the device-side `sparse` flags into a compact list of work
-// tiles and every other phase runs a fixed-size grid over that list.  All phases run in one
+// tiles and every other phase runs a fixed-size grid over that list.  All phases can run in one
 // cooperative launch (k_topk_all, bottom of this file).
 #pragma once
 #include <cooperative_groups.h>
@@ -28,19 +30,21 @@ constexpr int kTopkSegGrid = 148 * 4;   // CTAs of the per-segment kernels
 struct TopkPlan {
     int n_sparse;       // segments that send a sparse message in this step
     int total_tiles;    // their tiles
+    int chunk;          // work tiles per planned share (kTopkGrid shares, or one per CTA of the single launch)
 };
 
 struct TopkState {
     TopkPlan* plan;
     int* sp_seg;               // [P*T] segment id of the q-th sparse segment
     int* sp_begin;             // [P*T+1] first work tile of the q-th sparse segment
+    int* cta_q;                // [kTopkGrid] sparse slot that holds the first work tile of CTA c's share
     unsigned int* hist;        // [P*T][kMaxBins]
     unsigned int* prefix;      // [P*T] key bits resolved so far (after the last digit: tau)
     unsigned int* remaining;   // [P*T] rank still to resolve (after the last digit: number of
                                //       entries equal to tau that are part of the message)
-    unsigned int* cand;        // [P][stride] candidate keys of a tile, at the tile's own offset
-    int* tile_cand;            // [P][n_tiles][8] candidates stored by each warp for the tile
-    unsigned int* tile_gt;     // [P][n_tiles][8] keys above the chosen bin seen by each warp
+    uint2* ent;                // [P][stride] entries (meta, value bits) of a tile, at the tile's own offset
+    int* tile_cand;            // [P][n_tiles][8] entries stored by each warp for the tile
+    unsigned int* tile_sub;    // [P][n_tiles][8] of those, (greater than tau) | (equal to tau) << 16
     uint2* tile_count;         // [P][n_tiles] (greater, equal) per tile, then their prefixes
     int2* outbox;              // [P][sum K_t] (index, value bits)
     const long long* out_off;  // [T] start of tensor t inside one replica's outbox
@@ -58,7 +62,8 @@ __device__ __forceinline__ int digit_bits(int digit) { return digit == 0 ? kDigi
 // One CTA (of kThreads threads): compact list of the sparse segments and of their tiles, in
 // segment order.
 __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restrict__ sparse,
-                                          const int* __restrict__ seg_begin, const TopkState& tk) {
+                                          const int* __restrict__ seg_begin, const TopkState& tk,
+                                          int n_cta) {
     __shared__ int s_cnt[kThreads], s_tiles[kThreads];
     const int per = (S + kThreads - 1) / kThreads;
     const int lo = threadIdx.x * per, hi = min(S, lo + per);
@@ -77,14 +82,20 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
         s_tiles[threadIdx.x] += b;
         __syncthreads();
     }
+    // the tile phases give CTA c the work tiles [c * chunk, (c + 1) * chunk): note for every c
+    // the sparse slot its first tile falls into, so that no phase has to search for it
+    const int chunk = (s_tiles[kThreads - 1] + n_cta - 1) / n_cta;
+    if (threadIdx.x == 0) tk.plan->chunk = chunk;
     int q = s_cnt[threadIdx.x] - cnt, w = s_tiles[threadIdx.x] - tiles;
     for (int s = lo; s < hi; ++s)
         if (sparse[s]) {
             const int t = s % T;
+            const int w_end = w + seg_begin[t + 1] - seg_begin[t];
             tk.sp_seg[q] = s;
             tk.sp_begin[q] = w;
+            for (int c = (w + chunk - 1) / chunk; c < n_cta && c * chunk < w_end; ++c) tk.cta_q[c] = q;
             ++q;
-            w += seg_begin[t + 1] - seg_begin[t];
+            w = w_end;
         }
     if (threadIdx.x == kThreads - 1) {
         tk.plan->n_sparse = s_cnt[threadIdx.x];
@@ -97,18 +108,14 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
 struct WorkRange {
     int w0, w1, q;
 };
-__device__ __forceinline__ WorkRange work_range(const TopkState& tk) {
-    const int total = tk.plan->total_tiles, nq = tk.plan->n_sparse;
-    const int chunk = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+// `shares`: planned shares per CTA (a phase may run with a grid `shares` times smaller than planned).
+__device__ __forceinline__ WorkRange work_range(const TopkState& tk, int shares = 1) {
+    const int total = tk.plan->total_tiles;
+    const int chunk = tk.plan->chunk;
     WorkRange r;
-    r.w0 = min(total, (int)blockIdx.x * chunk);
-    r.w1 = min(total, r.w0 + chunk);
-    int lo = 0, hi = max(nq - 1, 0);            // last q with sp_begin[q] <= w0
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (tk.sp_begin[mid] <= r.w0) lo = mid; else hi = mid - 1;
-    }
-    r.q = lo;
+    r.w0 = min(total, (int)blockIdx.x * shares * chunk);
+    r.w1 = min(total, r.w0 + shares * chunk);
+    r.q = (r.w0 < r.w1) ? tk.cta_q[blockIdx.x * shares] : 0;
     return r;
 }
 
@@ -179,78 +186,100 @@ topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable
     }
 }
 
-// One CTA per sparse segment: pick the bin that holds the wanted rank, counting from the
-// largest key downwards; clear the histogram for the next digit.
+// One warp per sparse segment: pick the bin that holds the wanted rank, counting from the
+// largest key downwards; clear the histogram for the next digit.  The histogram is walked in
+// blocks of 1024 bins from the top; a lane owns 32 consecutive bins of a block (eight 16-byte
+// loads, all in flight together), one warp scan places the rank in a lane, which then walks
+// its own bins.
 __device__ __forceinline__ void
 topk_pick(int T, TopkState tk, int digit) {
-    __shared__ unsigned int s_warp[kWarps];
+    constexpr int kBlock = 1024, kPer = kBlock / 32;
     const int nq = tk.plan->n_sparse;
     const int nbins = 1 << digit_bits(digit);
-    const int per = nbins / kThreads;                      // 8 or 4 bins per thread
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int q = blockIdx.x; q < nq; q += gridDim.x) {
+    const int lane = threadIdx.x & 31;
+    const int nwarps = gridDim.x * kWarps;
+    for (int q = blockIdx.x * kWarps + (threadIdx.x >> 5); q < nq; q += nwarps) {
         const int s = tk.sp_seg[q];
         const int t = s % T;
         unsigned int* gh = tk.hist + (long long)s * kMaxBins;
-        const int top = nbins - 1 - threadIdx.x * per;     // thread 0 owns the highest bins
-        unsigned int c[8];
-        unsigned int mine = 0;
-        for (int z = 0; z < per; ++z) { c[z] = gh[top - z]; mine += c[z]; gh[top - z] = 0; }
-        // exclusive scan of `mine` over the CTA, from the highest bins down
-        unsigned int inc = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned int v = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += v;
-        }
-        if (lane == 31) s_warp[warp] = inc;
-        __syncthreads();
-        unsigned int above = inc - mine;
-#pragma unroll
-        for (int u = 0; u < kWarps; ++u)
-            if (u < warp) above += s_warp[u];
         const unsigned int rem = (digit == 0) ? (unsigned int)tk.count[t] : tk.remaining[s];
-        if (above < rem && rem <= above + mine) {
-            for (int z = 0; z < per; ++z) {
-                if (rem <= above + c[z]) {
-                    const unsigned int old = (digit == 0) ? 0u : tk.prefix[s];
-                    tk.prefix[s] = (old << digit_bits(digit)) | (unsigned int)(top - z);
-                    tk.remaining[s] = rem - above;
-                    break;
-                }
-                above += c[z];
+        unsigned int above_blocks = 0;      // keys in the blocks already walked
+        bool found = false;                 // the same in every lane
+        for (int blk = nbins / kBlock - 1; blk >= 0; --blk) {
+            uint4* g4 = reinterpret_cast<uint4*>(gh + blk * kBlock + lane * kPer);
+            if (found) {                    // only the clearing is left
+#pragma unroll
+                for (int j = 0; j < kPer / 4; ++j) g4[j] = make_uint4(0u, 0u, 0u, 0u);
+                continue;
             }
+            unsigned int c[kPer];
+#pragma unroll
+            for (int j = 0; j < kPer / 4; ++j) {
+                const uint4 v = g4[j];
+                c[4 * j] = v.x; c[4 * j + 1] = v.y; c[4 * j + 2] = v.z; c[4 * j + 3] = v.w;
+            }
+#pragma unroll
+            for (int j = 0; j < kPer / 4; ++j) g4[j] = make_uint4(0u, 0u, 0u, 0u);
+            unsigned int mine = 0;
+#pragma unroll
+            for (int z = 0; z < kPer; ++z) mine += c[z];
+            unsigned int inc = mine;        // inclusive sum over this and the higher lanes
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int v = __shfl_down_sync(0xffffffffu, inc, o);
+                if (lane + o < 32) inc += v;
+            }
+            unsigned int above = above_blocks + inc - mine;
+            const bool here = above < rem && rem <= above + mine;
+            if (here) {
+                bool done = false;
+#pragma unroll
+                for (int z = kPer - 1; z >= 0; --z) {
+                    if (!done && rem <= above + c[z]) {
+                        const unsigned int old = (digit == 0) ? 0u : tk.prefix[s];
+                        tk.prefix[s] = (old << digit_bits(digit)) | (unsigned int)(blk * kBlock + lane * kPer + z);
+                        tk.remaining[s] = rem - above;
+                        done = true;
+                    }
+                    above += c[z];
+                }
+            }
+            found = __any_sync(0xffffffffu, here);
+            above_blocks += __shfl_sync(0xffffffffu, inc, 0);
         }
-        __syncthreads();
     }
 }
 
-constexpr int kSubSlices = kWarps;                       // candidate sub-slices per tile: one per warp
+constexpr int kSubSlices = kWarps;                       // entry sub-slices per tile: one per warp
+constexpr int kWarpSpan = kNormTile / kWarps;            // 512 consecutive elements of a tile per warp
+constexpr int kSubChunks = kWarpSpan / 128;              // read as 4 chunks of 128 (one float4 per lane)
+static_assert(kWarpSpan == 512 && kSubChunks == 4, "entry words hold a 9-bit position and four 8-bit counts");
 
-// Warp w of a CTA owns, in every 1024-element chunk of a tile, the 128 elements starting at
-// 128*w.  Its candidate sub-slice starts after the elements owned by the warps before it, so
-// the eight sub-slices exactly fill the tile's own slice whatever the tile's length.
-__device__ __forceinline__ int sub_offset(int len, int w) {
-    int o = 0;
-#pragma unroll
-    for (int v = 0; v < kNormTile / (kThreads * 4); ++v)
-        o += min(max(len - v * kThreads * 4, 0), w * 128);
-    return o;
-}
+// An entry describes one element whose top digit is at least the chosen bin b0:
+//   meta = sure << 29 | (key & 0xfffff) << 9 | position inside the warp's 512 elements
+//   val  = bits of x at that element
+// `sure` marks a top digit above b0 (the element is part of the message whatever the lower
+// digits say); otherwise the top digit equals b0 and the 20 low key bits decide.
+constexpr unsigned int kEntSure = 1u << 29;
+__device__ __forceinline__ unsigned int ent_low20(unsigned int meta) { return (meta >> 9) & 0xfffffu; }
+__device__ __forceinline__ bool ent_sure(unsigned int meta) { return (meta & kEntSure) != 0u; }
 
-// Pass B: per tile, copy the keys whose top digit equals the chosen bin into the candidate
-// buffer (order is irrelevant for selecting tau), count the keys whose top digit is larger, and
-// histogram digit 1 of the candidates.  Every warp owns 512 elements of the tile and a private
-// sub-slice of the tile's candidate slice, so no counter is shared: a thread marks its
-// candidates in a 16-bit mask, a warp scan of the counts gives its first slot, and the keys
-// are fetched back from shared memory (written and read by the same thread).
+// Warp w of a CTA owns elements [512 w, 512 w + 512) of a tile; its entries start at the same
+// place in the tile's slice of the entry buffer, so the slices can never overlap.
+__device__ __forceinline__ int sub_offset(int len, int w) { return min(len, w * kWarpSpan); }
+
+// Pass B: per tile, every element whose top digit is at least b0 is copied as an entry into the
+// tile's slice of the entry buffer, IN ASCENDING INDEX ORDER inside each warp's sub-slice (the
+// later phases rely on that order: concatenating the sub-slices of a tensor's tiles lists its
+// entries by index).  Digit 1 of the undecided entries is histogrammed on the way.  Nothing is
+// shared between warps except that histogram: a lane marks its elements in four 4-bit masks,
+// one warp scan of the four packed 8-bit counts (a chunk holds 128 elements, so a field cannot
+// overflow) gives every lane its first slot in each chunk.
 __device__ __forceinline__ void
 topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
                long long stride, TopkState tk) {
     constexpr int kBins1 = 1 << kDigitBits1;
-    constexpr int kChunks = kNormTile / (kThreads * 4);
     __shared__ unsigned int s_hist[kBins1];
-    __shared__ uint4 s_key[kNormTile / 4];
     WorkRange r = work_range(tk);
     if (r.w0 >= r.w1) return;
     for (int b = threadIdx.x; b < kBins1; b += kThreads) s_hist[b] = 0;
@@ -266,48 +295,51 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
         const int i = cur.i;
         const int len = tt.length[tile];
         const long long base = (long long)i * stride + tt.offset[tile];
-        unsigned int mask = 0, gt = 0;
+        unsigned int key[4 * kSubChunks];
+        float val[4 * kSubChunks];
+        unsigned int mask = 0, packed = 0;      // bit 4j+c: element c of chunk j is an entry
 #pragma unroll
-        for (int v = 0; v < kChunks; ++v) {
-            const int local = (v * kThreads + threadIdx.x) * 4;
-            if (local < len) {
-                const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
-                const uint4 k = make_uint4(rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
-                                           rank_key(a.w, b.w));
-                s_key[v * kThreads + threadIdx.x] = k;
-                const int nel = len - local;      // >= 1; 4 or more for all but the ragged end
-                const unsigned int d[4] = {k.x >> 20, k.y >> 20, k.z >> 20, k.w >> 20};
+        for (int j = 0; j < kSubChunks; ++j) {
+            const int local = warp * kWarpSpan + j * 128 + lane * 4;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+            if (local < len) { a = ld_stream(x + base + local); b = ld_stream(xhat + base + local); }
+            key[4 * j + 0] = rank_key(a.x, b.x); key[4 * j + 1] = rank_key(a.y, b.y);
+            key[4 * j + 2] = rank_key(a.z, b.z); key[4 * j + 3] = rank_key(a.w, b.w);
+            val[4 * j + 0] = a.x; val[4 * j + 1] = a.y; val[4 * j + 2] = a.z; val[4 * j + 3] = a.w;
+            const int nel = len - local;          // live elements of this float4 (<= 0: none)
+            unsigned int m = 0;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const bool live = c < nel;
-                    gt += (live && d[c] > b0);
-                    mask |= (live && d[c] == b0) ? (1u << (4 * v + c)) : 0u;
-                }
-            }
+            for (int c = 0; c < 4; ++c) m |= (c < nel && (key[4 * j + c] >> 20) >= b0) ? (1u << c) : 0u;
+            mask |= m << (4 * j);
+            packed |= (unsigned int)__popc(m) << (8 * j);
         }
-        // first slot of this thread inside its warp's sub-slice
-        const unsigned int cnt = __popc(mask);
-        unsigned int inc = cnt;
+        unsigned int inc = packed;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const unsigned int u = __shfl_up_sync(0xffffffffu, inc, o);
             if (lane >= o) inc += u;
         }
+        const unsigned int tot = __shfl_sync(0xffffffffu, inc, 31);
+        const unsigned int excl = inc - packed;
+        uint2* ent = tk.ent + base + sub_offset(len, warp);
+        unsigned int chunk_first = 0;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) gt += __shfl_down_sync(0xffffffffu, gt, o);
-        unsigned int* cd = tk.cand + base + sub_offset(len, warp);
-        unsigned int pos = inc - cnt;
-        const unsigned int* my_keys = reinterpret_cast<const unsigned int*>(s_key);
-        while (mask) {
-            const int bit = __ffs(mask) - 1;
-            mask &= mask - 1;
-            const unsigned int key = my_keys[((bit >> 2) * kThreads + threadIdx.x) * 4 + (bit & 3)];
-            cd[pos++] = key;
-            atomicAdd(&s_hist[(key >> 10) & (kBins1 - 1)], 1u);
+        for (int j = 0; j < kSubChunks; ++j) {
+            unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (mask & (1u << (4 * j + c))) {
+                    const unsigned int k = key[4 * j + c];
+                    const bool sure = (k >> 20) > b0;
+                    ent[pos++] = make_uint2((sure ? kEntSure : 0u) | ((k & 0xfffffu) << 9) |
+                                                (unsigned int)(j * 128 + lane * 4 + c),
+                                            __float_as_uint(val[4 * j + c]));
+                    if (!sure) atomicAdd(&s_hist[(k >> 10) & (kBins1 - 1)], 1u);
+                }
+            }
+            chunk_first += (tot >> (8 * j)) & 0xffu;
         }
-        const long long slot = ((long long)i * tt.n_tiles + tile) * kSubSlices + warp;
-        if (lane == 31) tk.tile_cand[slot] = (int)inc;          // candidates of this warp
-        if (lane == 0) tk.tile_gt[slot] = gt;                   // keys above the bin, this warp
+        if (lane == 0) tk.tile_cand[((long long)i * tt.n_tiles + tile) * kSubSlices + warp] = (int)chunk_first;
         if (w + 1 == r.w1 || w + 1 >= cur.end) {   // last tile of this segment here
             __syncthreads();
             unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
@@ -320,78 +352,164 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
     }
 }
 
-// Work tile number w of this step (used by the one-warp-per-tile kernels).
+// The one-warp-per-tile phases: a CTA takes a contiguous share of the work list (one search
+// per CTA), its warps take the tiles of that share in turn, each walking forward with its own
+// cursor.
 struct WarpTile {
     int s, i, t, tile;
 };
-__device__ __forceinline__ WarpTile warp_tile(const TopkState& tk, const TileTable& tt, int T, int w) {
-    int lo = 0, hi = tk.plan->n_sparse - 1;      // last q with sp_begin[q] <= w
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (tk.sp_begin[mid] <= w) lo = mid; else hi = mid - 1;
+struct WarpWalk {
+    WorkRange r;
+    WorkCursor cur;
+    int w;
+    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int shares = 1) {
+        r = work_range(tk, shares);
+        cur.init(tk, tt, T, r.q);
+        w = r.w0 + (int)(threadIdx.x >> 5);
     }
-    WarpTile r;
-    r.s = tk.sp_seg[lo];
-    r.i = r.s / T;
-    r.t = r.s - r.i * T;
-    r.tile = tt.seg_begin[r.t] + (w - tk.sp_begin[lo]);
-    return r;
-}
-
-// Digit 2 over the candidates: one warp per tile, global histogram updated directly (only the
-// candidates that match the 21 resolved bits take part: about one in a thousand).
-__device__ __forceinline__ void
-topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk) {
-    const int total = tk.plan->total_tiles;
-    const int lane = threadIdx.x & 31;
-    const int nwarps = gridDim.x * kWarps;
-    for (int w = blockIdx.x * kWarps + (threadIdx.x >> 5); w < total; w += nwarps) {
-        const WarpTile z = warp_tile(tk, tt, T, w);
-        const unsigned int want = tk.prefix[z.s];
-        const unsigned int* cd = tk.cand + (long long)z.i * stride + tt.offset[z.tile];
-        const int* n_sub = tk.tile_cand + ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices;
-        const int len = tt.length[z.tile];
-        unsigned int* gh = tk.hist + (long long)z.s * kMaxBins;
-        for (int sub = 0; sub < kSubSlices; ++sub) {
-            const int n = n_sub[sub];
-            const unsigned int* cs = cd + sub_offset(len, sub);
-            for (int e = lane; e < n; e += 32) {
-                const unsigned int k = cs[e];
-                if ((k >> 10) == want) atomicAdd(&gh[k & ((1 << kDigitBits2) - 1)], 1u);
-            }
-        }
+    __device__ __forceinline__ bool next(const TopkState& tk, const TileTable& tt, int T, WarpTile& z) {
+        if (w >= r.w1) return false;
+        bool changed;
+        z.tile = cur.advance(tk, tt, T, w, changed);
+        z.s = cur.s; z.i = cur.i; z.t = cur.t;
+        w += kWarps;
+        return true;
     }
-}
+};
 
-// Per tile: keys greater than / equal to tau, from the per-warp counts of pass B and the
-// tile's candidates.  One warp per tile.
-__device__ __forceinline__ void
-topk_count(TileTable tt, int T, long long stride, TopkState tk) {
-    const int total = tk.plan->total_tiles;
-    const int lane = threadIdx.x & 31;
-    const int nwarps = gridDim.x * kWarps;
-    for (int w = blockIdx.x * kWarps + (threadIdx.x >> 5); w < total; w += nwarps) {
-        const WarpTile z = warp_tile(tk, tt, T, w);
-        const unsigned int tau = tk.prefix[z.s];
-        const unsigned int* cd = tk.cand + (long long)z.i * stride + tt.offset[z.tile];
-        const long long slot = ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices;
-        const int len = tt.length[z.tile];
-        unsigned int gt = (lane < kSubSlices) ? tk.tile_gt[slot + lane] : 0u, eq = 0;
-        for (int sub = 0; sub < kSubSlices; ++sub) {
-            const int n = tk.tile_cand[slot + sub];
-            const unsigned int* cs = cd + sub_offset(len, sub);
-            for (int e = lane; e < n; e += 32) {
-                const unsigned int k = cs[e];
-                gt += (k > tau);
-                eq += (k == tau);
-            }
-        }
+// The entries of one tile: sub-slice u (the elements [512 u, 512 u + 512) of the tile, in index
+// order) holds n[u] entries starting at place min(len, 512 u) of the tile's slice.  The phases
+// below walk four sub-slices side by side -- round r touches entries 32 r + lane of each of
+// them, four independent loads per lane -- because a tile rarely holds more than a few
+// dozen entries per sub-slice and a walk one after the other would wait for memory eight times
+// instead of twice.
+constexpr int kSubGroup = 4;        // sub-slices walked side by side
+struct TileEntries {
+    int n[kSubSlices];
+    const uint2* slice;
+    int len;
+    long long slot;                 // first of the tile's eight per-sub-slice records
+    // `mine`: lane u < 8 brings the entry count of sub-slice u (see TileFeed)
+    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, long long stride,
+                                         const WarpTile& z, int mine) {
+        slot = ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            gt += __shfl_down_sync(0xffffffffu, gt, o);
-            eq += __shfl_down_sync(0xffffffffu, eq, o);
+        for (int u = 0; u < kSubSlices; ++u) n[u] = __shfl_sync(0xffffffffu, mine, u);
+        slice = tk.ent + (long long)z.i * stride + tt.offset[z.tile];
+        len = tt.length[z.tile];
+    }
+    __device__ __forceinline__ const uint2* sub(int u) const { return slice + min(len, u * kWarpSpan); }
+    // largest entry count among the sub-slices u0 .. u0 + kSubGroup - 1
+    __device__ __forceinline__ int most_of(int u0) const {
+        int m = 0;
+#pragma unroll
+        for (int v = 0; v < kSubGroup; ++v) m = max(m, n[u0 + v]);
+        return m;
+    }
+};
+
+// A warp's tiles, one ahead: while a tile is worked on, the entry counts of the warp's next
+// tile are already on their way, so a tile costs one wait less.
+struct TileFeed {
+    WarpWalk walk;
+    WarpTile ahead;
+    int ahead_mine;
+    bool have;
+    __device__ __forceinline__ int fetch(const TopkState& tk, const TileTable& tt) const {
+        const int lane = threadIdx.x & 31;
+        return (lane < kSubSlices)
+                   ? tk.tile_cand[((long long)ahead.i * tt.n_tiles + ahead.tile) * kSubSlices + lane] : 0;
+    }
+    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int shares) {
+        walk.init(tk, tt, T, shares);
+        have = walk.next(tk, tt, T, ahead);
+        ahead_mine = have ? fetch(tk, tt) : 0;
+    }
+    __device__ __forceinline__ bool next(const TopkState& tk, const TileTable& tt, int T, WarpTile& z, int& mine) {
+        if (!have) return false;
+        z = ahead;
+        mine = ahead_mine;
+        have = walk.next(tk, tt, T, ahead);
+        ahead_mine = have ? fetch(tk, tt) : 0;
+        return true;
+    }
+};
+
+// Digit 2 over the entries: one warp per tile, global histogram updated directly (only the
+// undecided entries that match the 21 resolved bits take part: about one in a thousand).
+__device__ __forceinline__ void
+topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk, int shares = 1) {
+    const int lane = threadIdx.x & 31;
+    TileFeed feed;
+    feed.init(tk, tt, T, shares);
+    WarpTile z;
+    int mine_n;
+    int s_now = -1;
+    unsigned int want = 0;
+    while (feed.next(tk, tt, T, z, mine_n)) {
+        if (z.s != s_now) { s_now = z.s; want = tk.prefix[z.s] & ((1u << kDigitBits1) - 1); }   // digit 1 of tau
+        unsigned int* gh = tk.hist + (long long)z.s * kMaxBins;
+        TileEntries te;
+        te.init(tk, tt, stride, z, mine_n);
+#pragma unroll
+        for (int u0 = 0; u0 < kSubSlices; u0 += kSubGroup) {
+            for (int f = lane; f - lane < te.most_of(u0); f += 32) {
+                unsigned int meta[kSubGroup];
+#pragma unroll
+                for (int v = 0; v < kSubGroup; ++v) meta[v] = (f < te.n[u0 + v]) ? te.sub(u0 + v)[f].x : kEntSure;
+#pragma unroll
+                for (int v = 0; v < kSubGroup; ++v) {
+                    const unsigned int low = ent_low20(meta[v]);
+                    if (!ent_sure(meta[v]) && (low >> kDigitBits2) == want)
+                        atomicAdd(&gh[low & ((1u << kDigitBits2) - 1)], 1u);
+                }
+            }
         }
-        if (lane == 0) tk.tile_count[(long long)z.i * tt.n_tiles + z.tile] = make_uint2(gt, eq);
+    }
+}
+
+// Per tile and per sub-slice: keys greater than / equal to tau, from the entries.  One warp per
+// tile.  tile_sub gets the eight (greater | equal << 16) pairs, tile_count the tile's totals.
+__device__ __forceinline__ void
+topk_count(TileTable tt, int T, long long stride, TopkState tk, int shares = 1) {
+    const int lane = threadIdx.x & 31;
+    TileFeed feed;
+    feed.init(tk, tt, T, shares);
+    WarpTile z;
+    int mine_n;
+    int s_now = -1;
+    unsigned int tau20 = 0;
+    while (feed.next(tk, tt, T, z, mine_n)) {
+        if (z.s != s_now) { s_now = z.s; tau20 = tk.prefix[z.s] & 0xfffffu; }
+        TileEntries te;
+        te.init(tk, tt, stride, z, mine_n);
+        unsigned int mine = 0, all_gt = 0, all_eq = 0;
+#pragma unroll
+        for (int u0 = 0; u0 < kSubSlices; u0 += kSubGroup) {
+            unsigned int gt[kSubGroup], eq[kSubGroup];        // the same in every lane
+#pragma unroll
+            for (int v = 0; v < kSubGroup; ++v) gt[v] = eq[v] = 0;
+            for (int f = lane; f - lane < te.most_of(u0); f += 32) {
+                unsigned int meta[kSubGroup];
+#pragma unroll
+                for (int v = 0; v < kSubGroup; ++v) meta[v] = (f < te.n[u0 + v]) ? te.sub(u0 + v)[f].x : 0u;
+#pragma unroll
+                for (int v = 0; v < kSubGroup; ++v) {
+                    const bool live = f < te.n[u0 + v];
+                    const unsigned int low = ent_low20(meta[v]);
+                    gt[v] += __popc(__ballot_sync(0xffffffffu, live && (ent_sure(meta[v]) || low > tau20)));
+                    eq[v] += __popc(__ballot_sync(0xffffffffu, live && !ent_sure(meta[v]) && low == tau20));
+                }
+            }
+#pragma unroll
+            for (int v = 0; v < kSubGroup; ++v) {
+                if (lane == u0 + v) mine = gt[v] | (eq[v] << 16);
+                all_gt += gt[v];
+                all_eq += eq[v];
+            }
+        }
+        if (lane < kSubSlices) tk.tile_sub[te.slot + lane] = mine;
+        if (lane == 0) tk.tile_count[(long long)z.i * tt.n_tiles + z.tile] = make_uint2(all_gt, all_eq);
     }
 }
 
@@ -436,118 +554,80 @@ topk_scan(TileTable tt, int T, TopkState tk) {
     }
 }
 
-// Pass C: ordered compaction of the selected entries of one tile into the outbox, and delivery:
-// the same (index, value) pairs are written into the mailbox x_hat, which is what the receivers
-// hold once the message has arrived.
+// Pass C: ordered compaction of the selected entries into the outbox, and delivery: the same
+// (index, value) pairs are written into the mailbox x_hat, which is what the receivers hold
+// once the message has arrived.  Works from the entries alone (a few percent of the tensor);
+// x and x_hat are not read again.
 // An entry is selected if key > tau, or key == tau and fewer than `remaining` equal keys
 // precede it in the tensor.  Its slot is (#greater before it) + min(#equal before it, remaining).
-// A tile is read as four coalesced chunks of 1024 elements (thread t owns elements 4t..4t+3 of
-// every chunk).  A thread records which of its 16 elements are greater / equal in two 16-bit
-// masks and parks the x values in shared memory (read back by the same thread); the four
-// per-chunk counts travel through ONE scan, packed 16 bits each into a 64-bit word (a chunk
-// holds at most 1024 entries, so the fields cannot overflow); then only the marked elements
-// are visited.  A thread has read the x_hat entries it owns before it overwrites any of them,
-// and no thread touches another thread's entries.
+// One warp per tile walks the tile's entries in index order, 32 at a time; ballots give every
+// lane the number of greater / equal entries before its own.
 __device__ __forceinline__ void
-topk_write(const float* __restrict__ x, float* xhat, TileTable tt, int T, long long stride,
-             TopkState tk, unsigned int* __restrict__ err) {
-    constexpr int kChunks = kNormTile / (kThreads * 4);   // 4
-    static_assert(kChunks == 4, "the packed scan holds four 16-bit fields");
-    __shared__ unsigned long long s_pg[kWarps], s_pe[kWarps];
-    __shared__ float4 s_val[kNormTile / 4];
-    WorkRange r = work_range(tk);
-    WorkCursor cur;
-    cur.init(tk, tt, T, r.q);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    unsigned int tau = 0, take = 0, K = 0;
+topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, unsigned int* __restrict__ err,
+           int shares = 1) {
+    const int lane = threadIdx.x & 31;
+    const unsigned int below = (1u << lane) - 1u;
+    TileFeed feed;
+    feed.init(tk, tt, T, shares);
+    WarpTile z;
+    int mine_n;
+    int s_now = -1;
+    unsigned int tau20 = 0, take = 0, K = 0;
     int2* out = nullptr;
-    for (int w = r.w0; w < r.w1; ++w) {
-        bool changed;
-        const int tile = cur.advance(tk, tt, T, w, changed);
-        if (changed) {
-            tau = tk.prefix[cur.s];
-            take = tk.remaining[cur.s];
-            K = (unsigned int)tk.count[cur.t];
-            out = tk.outbox + (long long)cur.i * tk.out_stride + tk.out_off[cur.t];
+    while (feed.next(tk, tt, T, z, mine_n)) {
+        if (z.s != s_now) {
+            s_now = z.s;
+            tau20 = tk.prefix[z.s] & 0xfffffu;
+            take = tk.remaining[z.s];
+            K = (unsigned int)tk.count[z.t];
+            out = tk.outbox + (long long)z.i * tk.out_stride + tk.out_off[z.t];
         }
-        const int i = cur.i;
-        const int len = tt.length[tile];
-        const long long base = (long long)i * stride + tt.offset[tile];
-        const int first = (tile - cur.first_tile) * kNormTile;   // index of the tile's first element
-        const uint2 before = tk.tile_count[(long long)i * tt.n_tiles + tile];
-        unsigned int gmask = 0, emask = 0;
-        unsigned long long pg = 0, pe = 0;
+        TileEntries te;
+        te.init(tk, tt, stride, z, mine_n);
+        const uint2 before = tk.tile_count[(long long)z.i * tt.n_tiles + z.tile];
+        const unsigned int sub_mine = (lane < kSubSlices) ? tk.tile_sub[te.slot + lane] : 0u;
+        const long long base = (long long)z.i * stride + tt.offset[z.tile];
+        const int first = (z.tile - tt.seg_begin[z.t]) * kNormTile;   // index of the tile's first element
+        unsigned int gt_before = before.x, eq_before = before.y;   // entries before sub-slice u0, whole tensor
 #pragma unroll
-        for (int v = 0; v < kChunks; ++v) {
-            const int local = (v * kThreads + threadIdx.x) * 4;
-            if (local < len) {
-                const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
-                s_val[v * kThreads + threadIdx.x] = a;
-                const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
-                                           rank_key(a.w, b.w)};
-                const int nel = len - local;
-                unsigned int g = 0, e = 0;
+        for (int u0 = 0; u0 < kSubSlices; u0 += kSubGroup) {
+            unsigned int run_gt[kSubGroup], run_eq[kSubGroup];     // the same in every lane
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const bool live = c < nel;
-                    g |= (live && k[c] > tau) ? (1u << c) : 0u;
-                    e |= (live && k[c] == tau) ? (1u << c) : 0u;
-                }
-                gmask |= g << (4 * v);
-                emask |= e << (4 * v);
-                pg |= (unsigned long long)__popc(g) << (16 * v);
-                pe |= (unsigned long long)__popc(e) << (16 * v);
+            for (int v = 0; v < kSubGroup; ++v) {
+                const unsigned int packed = __shfl_sync(0xffffffffu, sub_mine, u0 + v);
+                run_gt[v] = gt_before;
+                run_eq[v] = eq_before;
+                gt_before += packed & 0xffffu;
+                eq_before += packed >> 16;
             }
-        }
-        // inclusive scan over the CTA in thread order, all four chunks at once
-        unsigned long long sg = pg, se = pe;
+            for (int f = lane; f - lane < te.most_of(u0); f += 32) {
+                uint2 e[kSubGroup];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned long long a = __shfl_up_sync(0xffffffffu, sg, o);
-            const unsigned long long b = __shfl_up_sync(0xffffffffu, se, o);
-            if (lane >= o) { sg += a; se += b; }
-        }
-        if (lane == 31) { s_pg[warp] = sg; s_pe[warp] = se; }
-        __syncthreads();
-        unsigned long long wg = 0, we = 0, tg = 0, te = 0;
+                for (int v = 0; v < kSubGroup; ++v)
+                    e[v] = (f < te.n[u0 + v]) ? te.sub(u0 + v)[f] : make_uint2(0u, 0u);
 #pragma unroll
-        for (int u = 0; u < kWarps; ++u) {
-            if (u < warp) { wg += s_pg[u]; we += s_pe[u]; }
-            tg += s_pg[u]; te += s_pe[u];
-        }
-        const unsigned long long xg = wg + sg - pg, xe = we + se - pe;   // exclusive, per chunk
-        unsigned int run_gt = before.x, run_eq = before.y;               // entries before chunk v
-        const float* my_val = reinterpret_cast<const float*>(s_val);
-#pragma unroll
-        for (int v = 0; v < kChunks; ++v) {
-            unsigned int m = ((gmask | emask) >> (4 * v)) & 0xfu;
-            if (m) {
-                const int local = (v * kThreads + threadIdx.x) * 4;
-                unsigned int my_gt = run_gt + (unsigned int)((xg >> (16 * v)) & 0xffffu);
-                unsigned int my_eq = run_eq + (unsigned int)((xe >> (16 * v)) & 0xffffu);
-                const unsigned int en = (emask >> (4 * v)) & 0xfu;
-                while (m) {
-                    const int c = __ffs(m) - 1;
-                    m &= m - 1;
-                    const bool is_eq = (en >> c) & 1u;
-                    if (!is_eq || my_eq < take) {
+                for (int v = 0; v < kSubGroup; ++v) {
+                    const bool live = f < te.n[u0 + v];
+                    const unsigned int low = ent_low20(e[v].x);
+                    const bool g = live && (ent_sure(e[v].x) || low > tau20);
+                    const bool q = live && !ent_sure(e[v].x) && low == tau20;
+                    const unsigned int bg = __ballot_sync(0xffffffffu, g), bq = __ballot_sync(0xffffffffu, q);
+                    const unsigned int my_gt = run_gt[v] + __popc(bg & below), my_eq = run_eq[v] + __popc(bq & below);
+                    if (g || (q && my_eq < take)) {
                         const unsigned int slot = my_gt + min(my_eq, take);
-                        const float val = my_val[local + c];
-                        if (slot < K) {
-                            out[slot] = make_int2(first + local + c, __float_as_int(val));
-                            xhat[base + local + c] = val;
+                        const int local = (u0 + v) * kWarpSpan + (int)(e[v].x & 0x1ffu);
+                        if (slot < K && local < te.len) {
+                            out[slot] = make_int2(first + local, (int)e[v].y);
+                            xhat[base + local] = __uint_as_float(e[v].y);
                         } else {
                             atomicOr(err, 2u);
                         }
                     }
-                    my_gt += is_eq ? 0u : 1u;
-                    my_eq += is_eq ? 1u : 0u;
+                    run_gt[v] += __popc(bg);
+                    run_eq[v] += __popc(bq);
                 }
             }
-            run_gt += (unsigned int)((tg >> (16 * v)) & 0xffffu);
-            run_eq += (unsigned int)((te >> (16 * v)) & 0xffffu);
         }
-        __syncthreads();
     }
 }
 
@@ -570,7 +650,7 @@ struct TopkArgs {
 
 __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     cooperative_groups::grid_group grid = cooperative_groups::this_grid();
-    if (blockIdx.x == 0) topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk);
+    if (blockIdx.x == 0) topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, (int)gridDim.x);
     grid.sync();
     if (a.tk.plan->n_sparse == 0) return;          // the same for every CTA
     topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
@@ -589,26 +669,34 @@ __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     grid.sync();
     topk_scan(a.tt, a.T, a.tk);
     grid.sync();
-    topk_write(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
+    topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
 }
 
 __global__ void __launch_bounds__(kThreads) k_topk_plan(TopkArgs a) {
-    topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk);
+    topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, kTopkGrid);   // every tile phase runs kTopkGrid CTAs
 }
 __global__ void __launch_bounds__(kThreads) k_topk_hist(TopkArgs a) {
     topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
 }
 __global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int digit) { topk_pick(a.T, a.tk, digit); }
-__global__ void __launch_bounds__(kThreads, 4) k_topk_collect(TopkArgs a) {
+#ifndef EG_COLLECT_MINB
+#define EG_COLLECT_MINB 4
+#endif
+__global__ void __launch_bounds__(kThreads, EG_COLLECT_MINB) k_topk_collect(TopkArgs a) {
     topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
 }
-__global__ void __launch_bounds__(kThreads) k_topk_hist_cand(TopkArgs a) {
-    topk_hist_cand(a.tt, a.T, a.stride, a.tk);
+// The phases that work from the entries keep more registers than the streaming passes: they
+// run half the planned CTAs, each taking two planned shares.
+constexpr int kEntryShares = 2;
+__global__ void __launch_bounds__(kThreads, 4) k_topk_hist_cand(TopkArgs a) {
+    topk_hist_cand(a.tt, a.T, a.stride, a.tk, kEntryShares);
 }
-__global__ void __launch_bounds__(kThreads) k_topk_count(TopkArgs a) { topk_count(a.tt, a.T, a.stride, a.tk); }
+__global__ void __launch_bounds__(kThreads, 4) k_topk_count(TopkArgs a) {
+    topk_count(a.tt, a.T, a.stride, a.tk, kEntryShares);
+}
 __global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) { topk_scan(a.tt, a.T, a.tk); }
 __global__ void __launch_bounds__(kThreads, 4) k_topk_write(TopkArgs a) {
-    topk_write(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
+    topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.err, kEntryShares);
 }
 
 }  // namespace eg

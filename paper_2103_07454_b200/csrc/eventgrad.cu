@@ -346,11 +346,12 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         EG_ALLOC(c->tk.prefix, S); EG_ALLOC(c->tk.remaining, S);
         EG_ALLOC(c->tk.tile_count, (size_t)P * c->tiles_norm.n_tiles);
         EG_ALLOC(c->tk.tile_cand, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
-        EG_ALLOC(c->tk.tile_gt, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
-        EG_ALLOC(c->tk.cand, (size_t)P * c->stride);
+        EG_ALLOC(c->tk.tile_sub, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
+        EG_ALLOC(c->tk.ent, (size_t)P * c->stride);
         EG_ALLOC(c->tk.plan, 1);
         EG_ALLOC(c->tk.sp_seg, S);
         EG_ALLOC(c->tk.sp_begin, S + 1);
+        EG_ALLOC(c->tk.cta_q, kTopkGrid);
         EG_ALLOC(c->tk.outbox, (size_t)P * c->out_stride);
         {
             // one cooperative launch needs all its CTAs resident at the same time
@@ -502,11 +503,11 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
             k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(ta, 0);
             k_topk_collect<<<kTopkGrid, kThreads, 0, stream>>>(ta);
             k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(ta, 1);
-            k_topk_hist_cand<<<kTopkGrid, kThreads, 0, stream>>>(ta);
+            k_topk_hist_cand<<<kTopkGrid / kEntryShares, kThreads, 0, stream>>>(ta);
             k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(ta, 2);
-            k_topk_count<<<kTopkGrid, kThreads, 0, stream>>>(ta);
+            k_topk_count<<<kTopkGrid / kEntryShares, kThreads, 0, stream>>>(ta);
             k_topk_scan<<<kTopkSegGrid, kThreads, 0, stream>>>(ta);
-            k_topk_write<<<kTopkGrid, kThreads, 0, stream>>>(ta);
+            k_topk_write<<<kTopkGrid / kEntryShares, kThreads, 0, stream>>>(ta);
             launches += 10;
         }
     }
@@ -803,7 +804,7 @@ eg_status eg_selftest_wait_timeout(eg_ctx* c, void* stream_v) {
     DeviceGuard guard(c->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     c->last_stream = stream;
-    // reuse the plan-sized scratch word of the Top-K state? no: a dedicated int next to the error word
+    // the result word sits next to the error word
     int* gave_up = reinterpret_cast<int*>(c->err) + 1;
     k_selftest_wait<<<1, 32, 0, stream>>>(c->err, 2000000ll /* about a millisecond */, gave_up);
     EG_CUDA(c, cudaGetLastError());
