@@ -42,6 +42,7 @@ FUSED_BYTES_PER_ELEMENT = 16       # fused kernel: reads x, g, touches x_hat onc
 # DRAM traffic of the fused kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum per launch on the default workload), keyed by the hash of the kernel
 # sources it was taken with; reported as null once the sources change.
+FUSED_TRAFFIC_ELEMENTS = 16 * 11173962     # element-replicas of one launch on the default workload
 FUSED_TRAFFIC = {"9248f56a16a9": 2.630e9}   # profiles/k_fused_pipe_resnet18_first45tensors.md
 
 
@@ -447,10 +448,15 @@ def run_native(args):
 
     fused_ms = main["kernel_ms"]["fused"]
     achieved = elems * FUSED_BYTES_PER_ELEMENT / fused_ms / 1e6 if fused_ms else None
+    # the capture was taken on a prefix of the default workload; a streaming kernel's traffic
+    # grows with the elements, so it is scaled to the elements of one launch of this run
+    traffic = FUSED_TRAFFIC.get(kernel_source_hash())
+    if traffic is not None:
+        traffic *= elems / FUSED_TRAFFIC_ELEMENTS
     roofline = {"bound": "hbm", "kernel": "k_fused_pipe", "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
-                "traffic": FUSED_TRAFFIC.get(kernel_source_hash()),
+                "traffic": traffic,
                 "algorithmic_bytes_per_launch": elems * FUSED_BYTES_PER_ELEMENT,
                 "kernel_ms": fused_ms,
                 "step_frac_of_peak": main["gbs"] / peak,
