@@ -866,31 +866,69 @@ eg_status eg_reset(eg_ctx* c) {
 // ---------------------------------------------------------------------------------------
 namespace eg {
 
-// grid n_tiles (fused tile table).  avg[e] = (1/P) sum_i x_i[e]; cons[tile] = sum over the
-// tile and all replicas of (x_i[e] - mean)^2 with the mean kept in fp64.
+// CTAs loop over the fused tile table (1024 elements: one float4 per thread).
+// avg[e] = (1/P) sum_i x_i[e] with the sum and the mean in fp64; cons[cta] = sum over the CTA's
+// tiles and all replicas of (x_i[e] - mean)^2.  The first kAvgCache replicas stay in registers
+// for the second sweep; further ones are read again.
+constexpr int kAvgCache = 16;
 __global__ void __launch_bounds__(kThreads)
 k_average_model(const float* __restrict__ x, float* __restrict__ avg, TileTable tt, int P,
                 long long stride, double* __restrict__ cons) {
+    static_assert(kFusedTile == kThreads * 4, "one float4 per thread and tile");
     __shared__ double s_warp[kWarps];
-    const int tile = blockIdx.x;
-    const int len = tt.length[tile];
-    const long long off = tt.offset[tile];
     double acc = 0.0;
-    for (int local = threadIdx.x; local < len; local += kThreads) {
-        double s = 0.0;
-        for (int i = 0; i < P; ++i) s = __dadd_rn(s, (double)x[(long long)i * stride + off + local]);
-        const double m = __ddiv_rn(s, (double)P);
-        avg[off + local] = __double2float_rn(m);
-        if (cons) {
-            for (int i = 0; i < P; ++i) {
-                const double d = __dsub_rn((double)x[(long long)i * stride + off + local], m);
-                acc = __fma_rn(d, d, acc);
+    const double dP = (double)P;
+    for (int tile = blockIdx.x; tile < tt.n_tiles; tile += gridDim.x) {
+        const int local = threadIdx.x * 4;
+        const int nel = min(4, tt.length[tile] - local);      // live elements of this thread's float4
+        if (nel <= 0) continue;
+        const float* col = x + tt.offset[tile] + local;        // padding inside a tensor's slot may be read
+        float4 v[kAvgCache];
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+        // all loads first and without a branch on P (a row index past the last replica is
+        // clamped and its value not used), so that they are in flight together
+#pragma unroll
+        for (int i = 0; i < kAvgCache; ++i) v[i] = ld_stream(col + (long long)min(i, P - 1) * stride);
+#pragma unroll
+        for (int i = 0; i < kAvgCache; ++i) {
+            if (i < P) {
+                s0 = __dadd_rn(s0, (double)v[i].x); s1 = __dadd_rn(s1, (double)v[i].y);
+                s2 = __dadd_rn(s2, (double)v[i].z); s3 = __dadd_rn(s3, (double)v[i].w);
             }
+        }
+        for (int i = kAvgCache; i < P; ++i) {
+            const float4 a = ld_stream(col + (long long)i * stride);
+            s0 = __dadd_rn(s0, (double)a.x); s1 = __dadd_rn(s1, (double)a.y);
+            s2 = __dadd_rn(s2, (double)a.z); s3 = __dadd_rn(s3, (double)a.w);
+        }
+        const double m0 = __ddiv_rn(s0, dP), m1 = __ddiv_rn(s1, dP), m2 = __ddiv_rn(s2, dP), m3 = __ddiv_rn(s3, dP);
+        float* out = avg + tt.offset[tile] + local;
+        if (nel == 4) {
+            *reinterpret_cast<float4*>(out) = make_float4(__double2float_rn(m0), __double2float_rn(m1),
+                                                          __double2float_rn(m2), __double2float_rn(m3));
+        } else {                                               // padding is never written
+            out[0] = __double2float_rn(m0);
+            if (nel > 1) out[1] = __double2float_rn(m1);
+            if (nel > 2) out[2] = __double2float_rn(m2);
+        }
+        if (cons) {
+            auto add = [&](float4 a) {
+                const double d0 = __dsub_rn((double)a.x, m0), d1 = __dsub_rn((double)a.y, m1);
+                const double d2 = __dsub_rn((double)a.z, m2), d3 = __dsub_rn((double)a.w, m3);
+                acc = __fma_rn(d0, d0, acc);
+                if (nel > 1) acc = __fma_rn(d1, d1, acc);
+                if (nel > 2) acc = __fma_rn(d2, d2, acc);
+                if (nel > 3) acc = __fma_rn(d3, d3, acc);
+            };
+#pragma unroll
+            for (int i = 0; i < kAvgCache; ++i)
+                if (i < P) add(v[i]);
+            for (int i = kAvgCache; i < P; ++i) add(ld_stream(col + (long long)i * stride));
         }
     }
     if (cons) {
         const double total = block_sum(acc, s_warp);
-        if (threadIdx.x == 0) cons[tile] = total;
+        if (threadIdx.x == 0) cons[blockIdx.x] = total;
     }
 }
 
@@ -913,11 +951,12 @@ eg_status eg_average_model(eg_ctx* c, const float* params, float* avg_dev, doubl
     DeviceGuard guard(c->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const TileTable tf = c->tiles_fused.view();
-    k_average_model<<<tf.n_tiles, kThreads, 0, stream>>>(params, avg_dev, tf, c->P, c->stride,
-                                                        consensus_host ? c->cons_partials : nullptr);
+    const int grid = std::min(tf.n_tiles, 148 * 8);
+    k_average_model<<<grid, kThreads, 0, stream>>>(params, avg_dev, tf, c->P, c->stride,
+                                                   consensus_host ? c->cons_partials : nullptr);
     if (consensus_host) {
-        k_sum_partials<<<1, kThreads, 0, stream>>>(c->cons_partials, tf.n_tiles, c->cons_partials + tf.n_tiles);
-        EG_CUDA(c, cudaMemcpyAsync(consensus_host, c->cons_partials + tf.n_tiles, sizeof(double),
+        k_sum_partials<<<1, kThreads, 0, stream>>>(c->cons_partials, grid, c->cons_partials + grid);
+        EG_CUDA(c, cudaMemcpyAsync(consensus_host, c->cons_partials + grid, sizeof(double),
                                    cudaMemcpyDeviceToHost, stream));
         EG_CUDA(c, cudaStreamSynchronize(stream));
     }
