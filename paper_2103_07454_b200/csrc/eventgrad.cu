@@ -243,6 +243,52 @@ struct DeviceGuard {
 
 }  // namespace
 
+// The staged general-neighbourhood kernel: prefetch distance chosen so that two CTAs fit an SM.
+constexpr int kMaxStagedHops = 4;
+template <int M> struct StagedDepth;
+template <> struct StagedDepth<2> { static constexpr int D = 4; };
+template <> struct StagedDepth<3> { static constexpr int D = 3; };
+template <> struct StagedDepth<4> { static constexpr int D = 2; };
+
+template <int M>
+static cudaError_t raise_hops_staged(int P) {
+    constexpr int D = StagedDepth<M>::D;
+    cudaError_t e = cudaFuncSetAttribute(k_fused_hops_staged<true, M, D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)HopsStaged<M, D>::bytes(P, true));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_fused_hops_staged<false, M, D>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)HopsStaged<M, D>::bytes(P, false));
+    return e;
+}
+
+template <int M>
+static void launch_hops_staged_m(eg_ctx* c, bool carry, int grid, cudaStream_t stream, float* params,
+                                 const float* grads, const uint8_t* valid, const TileTable& tf, float lr,
+                                 double* partials, long long* step_k) {
+    constexpr int D = StagedDepth<M>::D;
+    const size_t smem = HopsStaged<M, D>::bytes(c->P, carry);
+    if (carry)
+        k_fused_hops_staged<true, M, D><<<grid, kThreads, smem, stream>>>(
+            params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, partials, step_k,
+            c->variant);
+    else
+        k_fused_hops_staged<false, M, D><<<grid, kThreads, smem, stream>>>(
+            params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, partials, step_k,
+            c->variant, c->async ? c->mailbox : nullptr, c->async ? c->arrive : nullptr);
+}
+
+static void launch_hops_staged(eg_ctx* c, bool carry, int grid, cudaStream_t stream, float* params,
+                               const float* grads, const uint8_t* valid, const TileTable& tf, float lr,
+                               double* partials, long long* step_k) {
+    switch (c->hops) {
+        case 2: launch_hops_staged_m<2>(c, carry, grid, stream, params, grads, valid, tf, lr, partials, step_k); break;
+        case 3: launch_hops_staged_m<3>(c, carry, grid, stream, params, grads, valid, tf, lr, partials, step_k); break;
+        default: launch_hops_staged_m<4>(c, carry, grid, stream, params, grads, valid, tf, lr, partials, step_k); break;
+    }
+}
+
 extern "C" {
 
 const char* eg_strerror(eg_status s) {
@@ -388,6 +434,11 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
                                      (int)c->fused_smem);
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
+    if (c->hops >= 2 && c->hops <= kMaxStagedHops && P >= 2 * c->hops + 1) {
+        const cudaError_t e = c->hops == 2 ? raise_hops_staged<2>(P)
+                              : c->hops == 3 ? raise_hops_staged<3>(P) : raise_hops_staged<4>(P);
+        if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
+    }
     {
         const int pipe_smem = (int)PipeLayout::bytes(P, true, kPipeConsumers / 32);
         cudaError_t e = cudaSuccess;
@@ -515,7 +566,11 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     {
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
         const uint8_t* valid = c->async ? c->recv_valid : c->st.valid;   // whom the neighbours have heard from
-        if (c->hops > 1) {
+        if (c->hops > 1 && c->hops <= kMaxStagedHops && c->P >= 2 * c->hops + 1 &&
+            c->fused_kind == EG_FUSED_PIPELINED) {
+            // rows staged through shared memory; the register kernel choice keeps the plain form
+            launch_hops_staged(c, carry, grid_fused, stream, params, grads, valid, tf, lr, partials_fused, step_k);
+        } else if (c->hops > 1) {
             if (carry)
                 k_fused_hops<true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,

@@ -38,11 +38,15 @@ def test_variants_own_term_and_change_of_norm(own, con, carry, kernel):
     assert 0 < rep.events < 5 * wl.T * wl.steps
 
 
-@pytest.mark.parametrize("P,hops", [(1, 2), (2, 2), (3, 2), (4, 2), (5, 2), (7, 3), (16, 2), (16, 8)])
+@pytest.mark.parametrize("P,hops", [(1, 2), (2, 2), (3, 2), (4, 2), (5, 2), (6, 2), (7, 3), (8, 3), (9, 4),
+                                    (13, 4), (16, 2), (16, 3), (16, 8), (64, 2)])
 @pytest.mark.parametrize("carry", [False, True])
-def test_more_neighbours_per_side(P, hops, carry):
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
+def test_more_neighbours_per_side(P, hops, carry, kernel):
+    """Rings of at least 2 hops + 1 replicas with up to 4 hops take the staged kernel under the
+    default kernel choice and the plain one under the other; the rest always take the plain one."""
     wl = W.synthetic(P, RAGGED[:-1], steps=10, lr=0.1, grad_sigma=0.01)
-    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(hops=hops))
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(hops=hops), fused_kernel=kernel)
     assert rep.params_bit_exact and not rep.near_threshold
 
 
@@ -72,7 +76,7 @@ def _random_links(P, T, p_up, seed):
     return fn
 
 
-@pytest.mark.parametrize("P,hops", [(1, 1), (2, 1), (3, 1), (5, 1), (16, 1), (5, 2), (9, 3)])
+@pytest.mark.parametrize("P,hops", [(1, 1), (2, 1), (3, 1), (5, 1), (16, 1), (5, 2), (9, 3), (4, 2), (12, 4)])
 @pytest.mark.parametrize("p_up", [0.0, 0.5, 1.0])
 def test_intermittent_delivery_dense(P, hops, p_up):
     wl = W.synthetic(P, RAGGED[:-1], steps=16, lr=0.1, grad_sigma=0.01)
