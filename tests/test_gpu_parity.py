@@ -93,6 +93,37 @@ def test_intermittent_delivery_topk(con):
     assert rep.params_bit_exact
 
 
+def _random_case(seed):
+    """One seeded draw over the options of a context; combinations the library documents as
+    unavailable (delivery masks with the own-term variant) are not drawn."""
+    rng = np.random.default_rng(1000 + seed)
+    P = int(rng.integers(1, 12))
+    sizes = [int(v) for v in rng.choice(RAGGED[:-1], size=int(rng.integers(1, 6)), replace=False)]
+    topk = [None, (1, 100), (7, 100), (1, 2)][int(rng.integers(0, 4))]
+    hops = int(rng.integers(1, 5))
+    deliver = bool(rng.integers(0, 3) == 0)
+    okw = dict(hops=hops, history_len=int(rng.integers(1, 5)), horizon=float(rng.choice([0.5, 1.0, 2.0])),
+               own_last_sent=bool(rng.integers(0, 2)) and not deliver,
+               change_of_norm=bool(rng.integers(0, 2)))
+    if rng.integers(0, 4) == 0:
+        okw["threshold_cap"] = (1e-3, 0.8)
+    if rng.integers(0, 5) == 0:
+        okw.update(mode=1, delta_fixed=float(rng.choice([0.0, 0.01])), force_first_event=bool(rng.integers(0, 2)))
+    return dict(P=P, sizes=sizes, topk=topk, okw=okw, carry=bool(rng.integers(0, 2)),
+                kernel=[B.FUSED_PIPELINED, B.FUSED_REGISTER][int(rng.integers(0, 2))],
+                deliver=_random_links(P, len(sizes), float(rng.choice([0.3, 0.8])), seed) if deliver else None)
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_option_combinations(seed):
+    case = _random_case(seed)
+    wl = W.synthetic(case["P"], case["sizes"], steps=14, lr=0.1, grad_sigma=0.01, topk=case["topk"],
+                     seed=77 + seed)
+    rep = lockstep(wl, init="distinct", carry=case["carry"], fused_kernel=case["kernel"],
+                   oracle_kw=case["okw"], deliver_fn=case["deliver"], outbox_samples=16)
+    assert rep.params_bit_exact, case
+
+
 def test_delivery_masks_enabled_mid_run_and_refusals():
     from oracle import eg_oracle as eo
     wl = W.synthetic(4, [5, 1000, 4097], steps=12, lr=0.1, grad_sigma=0.01)
