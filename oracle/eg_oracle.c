@@ -46,7 +46,12 @@
  *    tested quantity taken as the change of the norm, | ||x|| - ||x at the last event|| |;
  *  - Top-K ranks by |x - x_hat| (fp32 difference), sends the parameter values x[e] with
  *    their indices, ties go to the lower index, the message is in ascending index order,
- *    K_t = max(1, ceil(n_t * k_num / k_den)); the first message of a tensor is dense.
+ *    K_t = max(1, ceil(n_t * k_num / k_den)); the first message of a tensor is dense;
+ *  - another training algorithm (the Introduction names extensions to other optimizers without
+ *    giving one): heavy-ball momentum (ego_set_momentum), off by default.  Every replica keeps
+ *    a velocity v of its own, never communicated, v <- mu * v + g, and the gradient term of
+ *    Eq. (dist_sgd_event) becomes gamma * v.  Pinned against torch.optim.SGD(momentum=mu), a
+ *    closed-form geometric series, mu = 0 == the plain update, and the dense X W - gamma V.
  */
 #include <float.h>
 #include <math.h>
@@ -116,6 +121,9 @@ typedef struct ego_ctx {
     uint64_t arrivals;
     double cap_alpha, cap_beta; /* bound g(k) = alpha * beta^k on the squared threshold
                                    (Assumption 1, Corollary 2); alpha <= 0: no bound */
+    /* heavy-ball momentum (an extension to another training algorithm, Introduction) */
+    float *vel;           /* [P][N] velocity of every replica, fp32 like the parameters; NULL: off */
+    double mu;            /* momentum coefficient */
 } ego_ctx;
 
 void ego_destroy(ego_ctx *c) {
@@ -124,7 +132,7 @@ void ego_destroy(ego_ctx *c) {
     free(c->delta); free(c->khat); free(c->hist); free(c->hist_len); free(c->valid);
     free(c->flag); free(c->norm); free(c->thr_used); free(c->out_idx); free(c->out_val);
     free(c->out_count); free(c->seg_events); free(c->seg_payload); free(c->sent_norm);
-    free(c->mailbox); free(c->pending); free(c->recv_valid);
+    free(c->mailbox); free(c->pending); free(c->recv_valid); free(c->vel);
     free(c);
 }
 
@@ -139,6 +147,7 @@ void ego_reset(ego_ctx *c) {
         memset(c->recv_valid, 0, (size_t)S);
     }
     memset(c->xhat, 0, sizeof(float) * (size_t)c->P * (size_t)c->N); /* X_0 = 0, Assumption 2.4 */
+    if (c->vel) memset(c->vel, 0, sizeof(float) * (size_t)c->P * (size_t)c->N);
     for (int64_t s = 0; s < S; ++s) {
         c->delta[s] = (c->mode == EGO_FIXED) ? c->delta_fixed : c->delta_init;
         c->khat[s] = 0;
@@ -224,6 +233,19 @@ int ego_set_hops(ego_ctx *c, int hops) {
     c->hops = hops;
     return 0;
 }
+
+/* Heavy-ball momentum with coefficient mu (0 <= mu < 1); the velocities start at zero.
+ * Returns non-zero when mu is out of range or memory is short. */
+int ego_set_momentum(ego_ctx *c, double mu) {
+    if (!(mu >= 0.0 && mu < 1.0)) return 1;
+    if (!c->vel) {
+        c->vel = (float *)calloc((size_t)c->P * (size_t)c->N, sizeof(float));
+        if (!c->vel) return 1;
+    }
+    c->mu = mu;
+    return 0;
+}
+float *ego_velocity(ego_ctx *c) { return c->vel; }
 
 void ego_set_threads(ego_ctx *c, int threads) { c->threads = threads < 1 ? 1 : threads; }
 
@@ -383,11 +405,19 @@ static void phase_b_segment(ego_ctx *c, float *x, const float *g, float lr, int 
     const float *gs = g + (int64_t)i * c->N + c->off[t];
     const double neg_lr = -(double)lr;
     const float *own = c->own_last_sent ? c->xhat + (int64_t)i * c->N + c->off[t] : xs;
+    float *vs = c->vel ? c->vel + (int64_t)i * c->N + c->off[t] : NULL;
     for (int64_t e = 0; e < c->numel[t]; ++e) {
         double sum = (double)own[e];
         for (int q = 0; q < cnt; ++q) sum = sum + (double)hn[q][e];
         const double avg = sum * w;
-        const double r = fma(neg_lr, (double)gs[e], avg);
+        double step = (double)gs[e];
+        if (vs) {
+            /* v <- mu * v + g, stored in fp32 like every other state; the update uses the
+             * stored value */
+            vs[e] = (float)fma(c->mu, (double)vs[e], (double)gs[e]);
+            step = (double)vs[e];
+        }
+        const double r = fma(neg_lr, step, avg);
         xs[e] = (float)r;
     }
 }

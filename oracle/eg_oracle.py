@@ -47,6 +47,10 @@ def _load():
         lib.ego_set_variant.argtypes = [C.c_void_p, C.c_int, C.c_int]
         lib.ego_set_hops.argtypes = [C.c_void_p, C.c_int]
         lib.ego_set_threshold_cap.argtypes = [C.c_void_p, C.c_double, C.c_double]
+        lib.ego_set_momentum.restype = C.c_int
+        lib.ego_set_momentum.argtypes = [C.c_void_p, C.c_double]
+        lib.ego_velocity.restype = C.c_void_p
+        lib.ego_velocity.argtypes = [C.c_void_p]
         lib.ego_threads_available.restype = C.c_int
         lib.ego_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
         lib.ego_step_masked.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
@@ -97,7 +101,7 @@ class Oracle:
                  delta_fixed: float = 0.0, force_first_event: bool = True,
                  topk: Optional[tuple] = None, threads: int = 1,
                  own_last_sent: bool = False, change_of_norm: bool = False, hops: int = 1,
-                 threshold_cap: Optional[tuple] = None):
+                 threshold_cap: Optional[tuple] = None, momentum: Optional[float] = None):
         lib = _load()
         self._lib = lib
         self.P, self.T = int(P), len(numel)
@@ -116,6 +120,8 @@ class Oracle:
             raise ValueError("hops out of range")
         if threshold_cap:
             lib.ego_set_threshold_cap(self._h, float(threshold_cap[0]), float(threshold_cap[1]))
+        if momentum is not None and lib.ego_set_momentum(self._h, float(momentum)):
+            raise ValueError("momentum must be in [0, 1)")
         self.S = self.P * self.T
         self.history_len = int(history_len)
 
@@ -213,6 +219,13 @@ class Oracle:
         """Copy of the mailboxes (last communicated values), packed ``[P, N]``."""
         return _view(self._lib.ego_xhat(self._h), np.float32, self.P * self.N).reshape(
             self.P, self.N).copy()
+
+    def velocity(self) -> Optional[np.ndarray]:
+        """Copy of the momentum buffers, packed ``[P, N]`` (None when momentum is off)."""
+        p = self._lib.ego_velocity(self._h)
+        if not p:
+            return None
+        return _view(p, np.float32, self.P * self.N).reshape(self.P, self.N).copy()
 
     def topk_count(self, t: int) -> int:
         return int(self._lib.ego_topk_count(self._h, t))

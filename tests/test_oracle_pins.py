@@ -562,6 +562,99 @@ def test_topk_counts_of_the_resnet18_tensors():
 
 
 # ---------------------------------------------------------------------------------------
+# Heavy-ball momentum (the Introduction names other training algorithms as extensions and
+# gives none; the oracle takes v <- mu v + g, x <- average - gamma v, velocities local)
+# ---------------------------------------------------------------------------------------
+def test_momentum_zero_is_the_plain_update():
+    wl = small(P=5, steps=7, lr=0.1, grad_sigma=0.01)
+    a = eo.from_workload(wl)
+    b = eo.from_workload(wl, momentum=0.0)
+    xa = W.distinct_init_params(wl).numpy().copy()
+    xb = xa.copy()
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        a.step(xa, g, wl.lr)
+        b.step(xb, g, wl.lr)
+        assert np.array_equal(xa, xb) and np.array_equal(a.flags(), b.flags())
+        assert np.array_equal(b.velocity(), g)          # mu = 0: the velocity is the gradient
+    assert a.stats() == b.stats()
+    assert a.velocity() is None
+
+
+def test_momentum_matches_torch_sgd_on_independent_replicas():
+    """No messages (infinite threshold): every replica is torch.optim.SGD(momentum=mu) on its
+    own parameters.  torch runs in fp64 with an fp64 velocity; the oracle stores both in fp32,
+    so the two drift apart by roundings only."""
+    import torch
+    mu, lr, steps = 0.9, 0.05, 12
+    wl = small(P=3, steps=steps, lr=lr, grad_sigma=0.02)
+    o = eo.Oracle(3, wl.numel, mode=eo.FIXED, delta_fixed=INF, force_first_event=False, momentum=mu)
+    x = W.distinct_init_params(wl).numpy().copy()
+    p = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([p], lr=float(np.float32(lr)), momentum=mu)
+    vmax = 0.0
+    for k in range(steps):
+        g = wl.grads(k).numpy()
+        o.step(x, g, lr)
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        ref = p.detach().numpy()
+        buf = opt.state[p]["momentum_buffer"].numpy()
+        vmax = max(vmax, float(np.abs(buf).max()))
+        assert np.max(np.abs(o.velocity() - buf)) <= (k + 1) * 2.0 ** -23 * vmax
+        assert np.max(np.abs(x - ref)) <= (k + 1) * 2.0 ** -23 * (float(np.abs(ref).max()) + vmax)
+    assert o.stats()["messages"] == 0
+    # a wrong sign or a velocity that is not accumulated is far outside those bounds
+    plain = W.distinct_init_params(wl).numpy().astype(np.float64)
+    for k in range(steps):
+        plain -= float(np.float32(lr)) * wl.grads(k).numpy()
+    assert np.max(np.abs(plain - p.detach().numpy())) > 1e-3
+
+
+def test_momentum_closed_form_with_a_constant_gradient():
+    """mu = 1/2, g = 1, gamma = 1/4, one replica: v_k = 2 - 2^(1-k) and
+    x_k = x_0 - gamma * sum_{j<=k} v_j = x_0 - (2k - 2 + 2^(1-k)) / 4, all exact in fp32."""
+    o = eo.Oracle(1, [4], mode=eo.FIXED, delta_fixed=INF, force_first_event=False, momentum=0.5)
+    x = np.full((1, 4), 3.0, np.float32)
+    g = np.ones((1, 4), np.float32)
+    for k in range(1, 11):
+        o.step(x, g, 0.25)
+        assert np.all(o.velocity() == np.float32(2.0 - 2.0 ** (1 - k)))
+        assert np.all(x == np.float32(3.0 - (2 * k - 2 + 2.0 ** (1 - k)) / 4))
+
+
+@pytest.mark.parametrize("P", [2, 3, 6])
+def test_momentum_zero_threshold_is_xw_minus_gamma_v(P):
+    mu = 0.75
+    wl = small(P=P, steps=6, lr=0.1, grad_sigma=0.01)
+    o = eo.Oracle(P, wl.numel, mode=eo.FIXED, delta_fixed=0.0, force_first_event=False, momentum=mu)
+    x = W.distinct_init_params(wl).numpy().copy()
+    Wm = ring_matrix(P)
+    v = np.zeros_like(x)
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        v = (mu * v.astype(np.float64) + g.astype(np.float64)).astype(np.float32)
+        ref = Wm @ x.astype(np.float64) - np.float64(np.float32(wl.lr)) * v.astype(np.float64)
+        o.step(x, g, wl.lr)
+        assert np.array_equal(o.velocity(), v)
+        assert np.all(np.abs(x.astype(np.float64) - ref) <= 0.5000001 * ulp32(ref) + 1e-300)
+
+
+def test_momentum_reset_clears_the_velocity_and_range_is_checked():
+    wl = small(P=2, steps=2)
+    o = eo.from_workload(wl, momentum=0.9)
+    x = W.distinct_init_params(wl).numpy().copy()
+    o.step(x, wl.grads(0).numpy(), wl.lr)
+    assert np.any(o.velocity() != 0)
+    o.reset()
+    assert np.all(o.velocity() == 0)
+    for bad in (-0.1, 1.0, float("nan")):
+        with pytest.raises(ValueError):
+            eo.from_workload(wl, momentum=bad)
+
+
+
+# ---------------------------------------------------------------------------------------
 # after training: averaged model (last line of Algorithms A and B)
 # ---------------------------------------------------------------------------------------
 def test_average_model_and_consensus_distance():
