@@ -38,6 +38,7 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used if n
 NOMINAL_HBM_GBS = 8000.0
 BYTES_PER_ELEMENT = {"carry": 16, "two_pass": 24}   # algorithmic bytes per element-replica-step
 FUSED_BYTES_PER_ELEMENT = 16       # fused kernel: reads x, g, touches x_hat once, writes x
+MOMENTUM_BYTES_PER_ELEMENT = 8     # --momentum: the velocity is read and written once more
 
 # DRAM traffic of the fused kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum per launch on the default workload), keyed by the hash of the kernel
@@ -299,9 +300,13 @@ def time_steps(eg, x, grads, lr, steps, sampler=None):
     return e0.elapsed_time(e1), launches
 
 
-def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_variant, graph_steps=0):
+def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_variant, graph_steps=0,
+                     momentum=None):
     """Times K steps of `wl` for every variant; returns ({variant: figures}, context)."""
     eg = B.from_workload(wl)
+    if momentum is not None:      # heavy-ball update: the velocity is read and written as well
+        eg.set_momentum(momentum)
+    extra = MOMENTUM_BYTES_PER_ELEMENT if momentum is not None else 0
     buf_bytes = wl.P * eg.replica_stride * 4
     free, _ = torch.cuda.mem_get_info()
     reserve = (24 << 30) + 4 * buf_bytes + (2 * buf_bytes if wl.topk else 0)
@@ -342,7 +347,7 @@ def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_varian
         torch.cuda.synchronize()
         per_step = sorted(marks[k].elapsed_time(marks[k + 1]) for k in range(K))
         results[variant] = {
-            "ms_per_step": ms_max / K, "gbs": units * BYTES_PER_ELEMENT[variant] / ms_max / 1e6,
+            "ms_per_step": ms_max / K, "gbs": units * (BYTES_PER_ELEMENT[variant] + extra) / ms_max / 1e6,
             "replica_steps_per_s": world * wl.P * K / (ms_max / 1e3), "launches": launches,
             "kernel_ms": {g: (v[0] / v[1] if v[1] else None) for g, v in kt.items()},
             "messages_sent": stats["messages"], "bytes_sent": stats["bytes"],
@@ -419,8 +424,9 @@ def run_native(args):
         return
     results, ctx = measure_workload(B, wl, K, Wm, dev, world,
                                     [args.variant] + [v for v in ("carry", "two_pass") if v != args.variant],
-                                    sampler, args.variant)
+                                    sampler, args.variant, momentum=args.momentum)
     eg, x0, grads, n_buf, buf_bytes = ctx
+    extra = MOMENTUM_BYTES_PER_ELEMENT if args.momentum is not None else 0
     clocks = sampler.summary()
     elems = wl.P * wl.N
     main = results[args.variant]
@@ -441,23 +447,24 @@ def run_native(args):
         eg.step_host(xh, gh[k % len(gh)], wl.lr)
     e_ms = (time.perf_counter() - t0) * 1e3
     e_units, e_ms_max = aggregate(float(elems) * e_steps, e_ms, dev)
-    e2e = {"value": e_units * BYTES_PER_ELEMENT["two_pass"] / e_ms_max / 1e6, "unit": "GB/s",
+    e2e = {"value": e_units * (BYTES_PER_ELEMENT["two_pass"] + extra) / e_ms_max / 1e6, "unit": "GB/s",
            "h2d_bytes_per_step": 2 * buf_bytes, "d2h_bytes_per_step": buf_bytes,
            "steps": e_steps, "ms_per_step": e_ms_max / e_steps,
            "replica_steps_per_s": world * wl.P * e_steps / (e_ms_max / 1e3)}
 
     fused_ms = main["kernel_ms"]["fused"]
-    achieved = elems * FUSED_BYTES_PER_ELEMENT / fused_ms / 1e6 if fused_ms else None
+    achieved = elems * (FUSED_BYTES_PER_ELEMENT + extra) / fused_ms / 1e6 if fused_ms else None
     # the capture was taken on a prefix of the default workload; a streaming kernel's traffic
     # grows with the elements, so it is scaled to the elements of one launch of this run
-    traffic = FUSED_TRAFFIC.get(kernel_source_hash())
+    traffic = FUSED_TRAFFIC.get(kernel_source_hash()) if args.momentum is None else None
     if traffic is not None:
         traffic *= elems / FUSED_TRAFFIC_ELEMENTS
-    roofline = {"bound": "hbm", "kernel": "k_fused_pipe", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "k_fused_pipe" if args.momentum is None else "k_fused_pipe_momentum",
+                "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
                 "traffic": traffic,
-                "algorithmic_bytes_per_launch": elems * FUSED_BYTES_PER_ELEMENT,
+                "algorithmic_bytes_per_launch": elems * (FUSED_BYTES_PER_ELEMENT + extra),
                 "kernel_ms": fused_ms,
                 "step_frac_of_peak": main["gbs"] / peak,
                 "step_frac_of_nominal_8TBs": main["gbs"] / NOMINAL_HBM_GBS}
@@ -478,7 +485,8 @@ def run_native(args):
                 "data": "synthetic",
                 "config": {"workload": wl.name, "P": wl.P, "tensors": wl.T, "elements": wl.N,
                            "variant": args.variant,
-                           "bytes_per_element_step": BYTES_PER_ELEMENT[args.variant],
+                           "bytes_per_element_step": BYTES_PER_ELEMENT[args.variant] + extra,
+                           "momentum": args.momentum,
                            "l2": "inputs larger than L2 (no flush needed)",
                            "gradient_buffers": n_buf, "multi_gpu": "replicas only"},
                 "pct_of_peak": 100.0 * main["gbs"] / peak,
@@ -505,6 +513,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--all-configs", action="store_true",
                     help="time all five configurations (their own step counts) instead of the default one")
+    ap.add_argument("--momentum", type=float, default=None,
+                    help="heavy-ball momentum coefficient (default: plain SGD update, the paper's)")
     ap.add_argument("--max-elements", type=int, default=0,
                     help="keep only the leading tensors of the workload up to this many elements")
     args = ap.parse_args()

@@ -166,6 +166,25 @@ eg_status eg_delivery_status(eg_ctx* ctx, uint8_t* pending_host, uint64_t* arriv
  * as a kernel argument. */
 eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
 
+/* Heavy-ball momentum.  The Introduction says that event-triggered communication extends to
+ * other training algorithms and gives none; this is the plain momentum method with a velocity
+ * per replica that is never communicated:
+ *     v_i <- mu * v_i + g_i,     x_i <- w * (x_i + sum of the neighbours' x_hat_j) - lr * v_i,
+ * i.e. Eq. (dist_sgd_event) with the gradient replaced by the velocity.  v is fp32, laid out
+ * like params, owned by the context (allocated and zeroed by the first enabling call, zeroed
+ * again by eg_reset); mu * v + g is one fp64 fused multiply-add rounded to fp32, and the update
+ * uses that rounded value.  mu = 0 reproduces the plain update bit for bit.  0 <= mu < 1
+ * (EG_ERR_INVALID otherwise).  Available with the default readings on the nearest-neighbour ring
+ * and the pipelined kernel, dense or Top-K (EG_ERR_STATE with eg_set_variant choices,
+ * EG_TOPO_RING_HOPS(m > 1), intermittent delivery or EG_FUSED_REGISTER).  enabled = 0 returns to
+ * the plain update and keeps the buffer.  The velocity is optimizer state like the parameters
+ * themselves and not part of eg_export_state: eg_read_velocity / eg_write_velocity copy it to /
+ * from a host buffer of P*replica_stride floats (both synchronise; EG_ERR_STATE before the
+ * first enabling call). */
+eg_status eg_set_momentum(eg_ctx* ctx, int enabled, double mu);
+eg_status eg_read_velocity(eg_ctx* ctx, float* velocity_host);
+eg_status eg_write_velocity(eg_ctx* ctx, const float* velocity_host);
+
 /* Which implementation of the fused snapshot / average / SGD kernel eg_step launches.  Both
  * compute bit-identical results.  EG_FUSED_PIPELINED (default) streams the operands through
  * shared memory with bulk asynchronous copies; EG_FUSED_REGISTER keeps the ring walk in

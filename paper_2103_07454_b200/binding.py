@@ -28,7 +28,7 @@ EXPORTS = [
     "eg_destroy", "eg_strerror", "eg_last_cuda_error", "eg_last_launch_count",
     "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant", "eg_set_threshold_cap",
     "eg_enable_delivery_masks", "eg_step_masked", "eg_read_received", "eg_delivery_status",
-    "eg_selftest_wait_timeout",
+    "eg_selftest_wait_timeout", "eg_set_momentum", "eg_read_velocity", "eg_write_velocity",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -86,6 +86,9 @@ def load_library() -> C.CDLL:
     lib.eg_set_fused_kernel.argtypes = [vp, C.c_int]
     lib.eg_set_variant.argtypes = [vp, C.c_int, C.c_int]
     lib.eg_set_threshold_cap.argtypes = [vp, C.c_double, C.c_double]
+    lib.eg_set_momentum.argtypes = [vp, C.c_int, C.c_double]
+    lib.eg_read_velocity.argtypes = [vp, vp]
+    lib.eg_write_velocity.argtypes = [vp, vp]
     lib.eg_enable_delivery_masks.argtypes = [vp]
     lib.eg_selftest_wait_timeout.argtypes = [vp, vp]
     lib.eg_step_masked.argtypes = [vp, vp, vp, C.c_float, vp, vp]
@@ -305,6 +308,25 @@ class EventGrad:
         """``eg_set_threshold_cap``: thresholds bounded by sqrt(alpha * beta**k)."""
         _check(self._lib, self._lib.eg_set_threshold_cap(self._h, float(alpha), float(beta)),
                self._h, "eg_set_threshold_cap")
+
+    def set_momentum(self, mu: Optional[float]):
+        """``eg_set_momentum``: heavy-ball momentum with coefficient ``mu``; ``None`` turns it off."""
+        with torch.cuda.device(self.device):
+            st = self._lib.eg_set_momentum(self._h, int(mu is not None), float(mu or 0.0))
+        _check(self._lib, st, self._h, "eg_set_momentum")
+
+    def velocity(self) -> torch.Tensor:
+        """Host copy of the velocities in the library's layout ``[P, replica_stride]``."""
+        out = torch.empty((self.P, self.replica_stride), dtype=torch.float32)
+        _check(self._lib, self._lib.eg_read_velocity(self._h, out.data_ptr()), self._h,
+               "eg_read_velocity")
+        return out
+
+    def write_velocity(self, v: torch.Tensor):
+        assert v.dtype == torch.float32 and v.is_contiguous() and not v.is_cuda
+        assert tuple(v.shape) == (self.P, self.replica_stride)
+        _check(self._lib, self._lib.eg_write_velocity(self._h, v.data_ptr()), self._h,
+               "eg_write_velocity")
 
     def set_fused_kernel(self, kind: int):
         _check(self._lib, self._lib.eg_set_fused_kernel(self._h, int(kind)), self._h,

@@ -103,10 +103,10 @@ struct PipeCfg {
 };
 
 // Shared-memory layout (dynamic), all offsets multiples of 16.
-template <int TILE, int STAGES>
+template <int TILE, int STAGES, int ARRAYS = 3>
 struct PipeSmem {
     static constexpr int kTileBytes = TILE * 4;
-    static constexpr int kStageBytes = 3 * kTileBytes;            // x, g, x_hat
+    static constexpr int kStageBytes = ARRAYS * kTileBytes;       // x, g, x_hat (, velocity)
     static constexpr int kWrapL = STAGES * kStageBytes;
     static constexpr int kWrapR = kWrapL + kTileBytes;
     static constexpr int kBars = kWrapR + kTileBytes;             // full[S], empty[S], wrap
@@ -130,19 +130,25 @@ struct PipeSmem {
 // every message arrives at once, which is the code path of the synchronous method.
 // PLAIN: the default readings only (the `variant` argument is ignored), so that the common
 // path carries no variant tests.
-template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC, bool PLAIN>
+// MOM (heavy-ball momentum, an extension to another training algorithm): every replica owns a
+// velocity `vel` laid out like x; a stage carries a fourth tile (v), the consumers form
+// v <- fp32(mu * v + g) in fp64, write it back and use it in place of the gradient.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC, bool PLAIN, bool MOM = false>
 __device__ __forceinline__ void
 fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
                 const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, const TileTable& tt,
                 int P, int T, long long stride, float lr, double* __restrict__ partials,
                 long long* step_k, unsigned int* __restrict__ err, int variant_arg,
-                float* mailbox, const uint8_t* __restrict__ arrive) {
+                float* mailbox, const uint8_t* __restrict__ arrive, float* __restrict__ vel = nullptr,
+                double mu = 0.0) {
+    static_assert(!(MOM && ASYNC), "momentum is not combined with intermittent delivery");
+    constexpr int kArr = MOM ? 4 : 3;              // tiles per stage
     static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
     const int variant = PLAIN ? 0 : variant_arg;
     // mode bit that says "contributes its own x": the dense-message bit itself unless ASYNC
     constexpr unsigned kCx = ASYNC ? 4u : 1u;
     static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
-    using L = PipeSmem<TILE, STAGES>;
+    using L = PipeSmem<TILE, STAGES, kArr>;
     constexpr int COLS = TILE / (4 * CONSUMERS);
     constexpr int CWARPS = CONSUMERS / 32;
     static_assert(COLS * 4 * CONSUMERS == TILE, "tile must be covered exactly");
@@ -193,6 +199,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             const float* gp = g + off;
             const float* hp = xhat + off;
             const float* mp = ASYNC ? mailbox + off : hp;
+            const float* vp = MOM ? vel + off : nullptr;
             mbar_expect_tx(wrap_bar, copy_bytes);
             bulk_g2s(wrap_l,
                      (cx_last ? xp : ((s_mode[P - 1] & 8) ? hp : mp)) + (long long)(P - 1) * stride,
@@ -201,13 +208,14 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             uint32_t wait_parity = 1;     // parity of the phase before the one to wait for
             for (int j = 0; j < P; ++j) {
                 if (j >= STAGES && !mbar_wait_bounded(&empty[s], wait_parity, s_abort, err)) break;
-                float* st = stages + s * (3 * TILE);
+                float* st = stages + s * (kArr * TILE);
                 const bool cx = (s_mode[j] & kCx) != 0;
                 const bool is_last = last_opt && (j == P - 1);
                 const bool need_x = !(is_last && cx);
                 const bool need_h = !cx && !is_last;
-                mbar_expect_tx(&full[s], copy_bytes * (1u + (need_x ? 1u : 0u) + (need_h ? 1u : 0u)));
+                mbar_expect_tx(&full[s], copy_bytes * ((MOM ? 2u : 1u) + (need_x ? 1u : 0u) + (need_h ? 1u : 0u)));
                 bulk_g2s(st + TILE, gp, copy_bytes, &full[s]);
+                if (MOM) { bulk_g2s(st + 3 * TILE, vp, copy_bytes, &full[s]); vp += stride; }
                 if (need_x) bulk_g2s(st, xp, copy_bytes, &full[s]);
                 if (need_h) bulk_g2s(st + 2 * TILE, (s_mode[j] & 8) ? hp : mp, copy_bytes, &full[s]);
                 xp += stride; gp += stride; hp += stride; mp += stride;
@@ -244,6 +252,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         float* xo = x + off + c0;                    // output pointers of replica j
         float* ho = xhat + off + c0;
         float* mo = ASYNC ? mailbox + off + c0 : nullptr;
+        float* vo = MOM ? vel + off + c0 : nullptr;
         for (int j = 0; ok && j < P; ++j) {
             const bool more = j + 1 < P;
             if (more) {
@@ -251,14 +260,14 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                 if (!ok) break;
             }
             const unsigned mode_next = s_mode[more ? j + 1 : 0];
-            const float* st = stages + s * (3 * TILE);
+            const float* st = stages + s * (kArr * TILE);
             const bool sn = (mode_cur & 1) != 0;
             const bool cx = (mode_cur & kCx) != 0;     // == sn unless ASYNC
             const bool is_last = last_opt && !more;
             // fp32 copy of this replica's contribution (its old x when a dense message arrives)
             const float* hs = is_last ? wrap_l : (cx ? st : st + 2 * TILE);
             // contribution of replica j+1
-            const float* sq = stages + s1 * (3 * TILE);
+            const float* sq = stages + s1 * (kArr * TILE);
             const float* hn_s = !more ? wrap_r
                                       : ((last_opt && j + 2 == P) ? wrap_l
                                                                   : ((mode_next & kCx) ? sq : sq + 2 * TILE));
@@ -275,7 +284,17 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
                     if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;   // private to this thread
                     const double hn[4] = {(double)hnf.x, (double)hnf.y, (double)hnf.z, (double)hnf.w};
-                    const double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
+                    double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
+                    if (MOM) {      // v <- mu * v + g, kept in fp32; the update then uses gamma * v
+                        const float4 vf = *reinterpret_cast<const float4*>(st + 3 * TILE + c);
+                        const float vn[4] = {__double2float_rn(__fma_rn(mu, (double)vf.x, gd[0])),
+                                             __double2float_rn(__fma_rn(mu, (double)vf.y, gd[1])),
+                                             __double2float_rn(__fma_rn(mu, (double)vf.z, gd[2])),
+                                             __double2float_rn(__fma_rn(mu, (double)vf.w, gd[3]))};
+                        store_masked(vo + v * 4 * CONSUMERS, make_float4(vn[0], vn[1], vn[2], vn[3]), nel[v]);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) gd[q] = (double)vn[q];
+                    }
                     double xd[4];
                     float4 x_old = make_float4(0.f, 0.f, 0.f, 0.f);   // only needed under ASYNC
                     if (cx || (variant & kOwnLastSent)) {   // own term = this replica's contribution
@@ -318,6 +337,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             if (lane == 0) mbar_arrive(&empty[s]);
             xo += stride; ho += stride;
             if (ASYNC) mo += stride;
+            if (MOM) vo += stride;
             mode_prev = mode_cur; mode_cur = mode_next;
             s = s1;
             if (++s1 == STAGES) { s1 = 0; parity1 ^= 1u; }
@@ -349,6 +369,18 @@ k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restri
              long long* step_k, unsigned int* __restrict__ err) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true>(x, g, xhat, snap, valid, tt, P, T, stride, lr,
                                                                 partials, step_k, err, 0, nullptr, nullptr);
+}
+
+// Heavy-ball momentum on the default readings (eg_set_momentum): four tiles per stage.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY>
+__global__ void __launch_bounds__(CONSUMERS + 32)
+k_fused_pipe_momentum(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
+                      const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
+                      int P, int T, long long stride, float lr, double* __restrict__ partials,
+                      long long* step_k, unsigned int* __restrict__ err, float* __restrict__ vel, double mu) {
+    fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true, true>(x, g, xhat, snap, valid, tt, P, T, stride,
+                                                                      lr, partials, step_k, err, 0, nullptr,
+                                                                      nullptr, vel, mu);
 }
 
 // Variants (eg_set_variant) and intermittent delivery; bounded to 72 registers for 3 CTAs per SM.

@@ -23,6 +23,8 @@ namespace {
 constexpr int kFusedVpt = EG_FUSED_VPT;               // float4 columns per thread
 constexpr int kFusedTile = kThreads * 4 * kFusedVpt;  // elements per CTA of the fused kernel
 using PipeLayout = PipeSmem<kPipeTile, kPipeStages>;
+constexpr int kMomStages = 4;                         // four tiles per stage: same footprint as 5 x 3
+using MomLayout = PipeSmem<kPipeTile, kMomStages, 4>;
 static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
 constexpr uint64_t kStateMagic = 0x4547535441544532ull;  // "EGSTATE2"
 
@@ -89,6 +91,10 @@ struct eg_ctx {
     uint8_t *pending = nullptr, *recv_valid = nullptr, *arrive = nullptr;
     unsigned long long* arrivals = nullptr;
     bool stepped = false;   // a step has run since creation / reset / import
+    // heavy-ball momentum: velocity of every replica, laid out like the parameters
+    bool momentum = false;
+    double mu = 0.0;
+    float* vel = nullptr;
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
     std::vector<cudaEvent_t> ev_pool;      // pairs
@@ -190,6 +196,7 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->arrive, 0, S));
         EG_CUDA(c, cudaMemset(c->arrivals, 0, sizeof(unsigned long long)));
     }
+    if (c->vel) EG_CUDA(c, cudaMemset(c->vel, 0, (size_t)c->P * c->stride * sizeof(float)));
     c->carried_valid = false;
     c->stepped = false;
     c->host_k = 0;
@@ -488,6 +495,8 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     if (!c || !params || !grads) return EG_ERR_INVALID;
     if (deliver_dev && !c->async) return EG_ERR_STATE;     // eg_enable_delivery_masks first
     if (c->async && (c->variant & kOwnLastSent)) return EG_ERR_STATE;
+    if (c->momentum && (c->async || c->variant != 0 || c->hops > 1 || c->fused_kind != EG_FUSED_PIPELINED))
+        return EG_ERR_STATE;
     if (((uintptr_t)params & 15u) || ((uintptr_t)grads & 15u)) return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
     if (!guard.ok) return EG_ERR_CUDA;
@@ -585,6 +594,18 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                 <<<grid_fused, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                 params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
                 partials_fused, step_k, c->err, c->variant, c->mailbox, c->arrive);
+        } else if (c->momentum) {
+            const size_t smem = MomLayout::bytes(c->P, carry, kPipeConsumers / 32);
+            if (carry)
+                k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, true>
+                    <<<grid_fused, kPipeThreads, smem, stream>>>(
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    partials_fused, step_k, c->err, c->vel, c->mu);
+            else
+                k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, false>
+                    <<<grid_fused, kPipeThreads, smem, stream>>>(
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    partials_fused, step_k, c->err, c->vel, c->mu);
         } else if (c->fused_kind == EG_FUSED_PIPELINED) {
             const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
 #define EG_PIPE_ARGS params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, \
@@ -901,6 +922,51 @@ eg_status eg_kernel_times(eg_ctx* c, double* ms_host, uint64_t* sections_host) {
         sections_host[c->ev_kind[q]] += 1;
     }
     c->ev_used = 0;
+    return EG_OK;
+}
+
+eg_status eg_set_momentum(eg_ctx* c, int enabled, double mu) {
+    if (!c) return EG_ERR_INVALID;
+    if (!enabled) { c->momentum = false; return EG_OK; }
+    if (!(mu >= 0.0 && mu < 1.0)) return EG_ERR_INVALID;
+    if (c->async || c->variant != 0 || c->hops > 1) return EG_ERR_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return EG_ERR_CUDA;
+    if (!c->vel) {
+        float* v = nullptr;
+        const eg_status s = dev_alloc(c, &v, (size_t)c->P * c->stride);   // zeroed
+        if (s != EG_OK) return s;
+        const int smem = (int)MomLayout::bytes(c->P, true, kPipeConsumers / 32);
+        EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, true>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, false>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        EG_CUDA(c, cudaDeviceSynchronize());
+        c->vel = v;
+    }
+    c->momentum = true;
+    c->mu = mu;
+    return EG_OK;
+}
+
+eg_status eg_read_velocity(eg_ctx* c, float* velocity_host) {
+    if (!c || !velocity_host) return EG_ERR_INVALID;
+    if (!c->vel) return EG_ERR_STATE;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    EG_CUDA(c, cudaMemcpy(velocity_host, c->vel, (size_t)c->P * c->stride * sizeof(float),
+                          cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
+eg_status eg_write_velocity(eg_ctx* c, const float* velocity_host) {
+    if (!c || !velocity_host) return EG_ERR_INVALID;
+    if (!c->vel) return EG_ERR_STATE;
+    DeviceGuard guard(c->device);
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    EG_CUDA(c, cudaMemcpy(c->vel, velocity_host, (size_t)c->P * c->stride * sizeof(float),
+                          cudaMemcpyHostToDevice));
     return EG_OK;
 }
 

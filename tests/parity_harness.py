@@ -4,7 +4,8 @@ Both sides are fed the same seeded inputs, step by step.  Compared every step:
 trigger flags (bit-exact, except decisions whose norm lies within 1e-6 relative of the
 threshold, which are reported and followed by a re-synchronisation), change norms and
 thresholds (1e-12 relative: only the summation order differs), message / byte / event
-counters (exact), Top-K messages (exact index sets and values), mailboxes and parameters.
+counters (exact), Top-K messages (exact index sets and values), mailboxes, parameters and,
+with momentum, the velocities.
 
 Tensors never interact with each other in the method, so at sizes where the oracle would be
 too slow it is run on a subset of the tensors (``tensors=[...]``) while the CUDA library runs
@@ -92,6 +93,10 @@ def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np
     assert pos == len(blob)
     eg.import_state(bytes(blob))
     eg.pack_into(x_dev, torch.from_numpy(x_host).to(x_dev.device))
+    if o.velocity() is not None:
+        vel = torch.zeros((eg.P, eg.replica_stride), dtype=torch.float32)
+        eg.pack_into(vel, torch.from_numpy(o.velocity()))
+        eg.write_velocity(vel)
 
 
 def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "workload",
@@ -117,6 +122,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     ekw.pop("threshold_cap", None)
     ekw.pop("own_last_sent", None)
     ekw.pop("change_of_norm", None)
+    ekw.pop("momentum", None)
     for key in ("mode", "delta_fixed", "force_first_event", "horizon", "history_len", "delta_init"):
         if key in okw and key not in ekw:
             ekw[key] = okw[key]
@@ -129,6 +135,8 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     eg.set_variant(bool(okw.get("own_last_sent")), bool(okw.get("change_of_norm")))
     if cap:
         eg.set_threshold_cap(*cap)
+    if okw.get("momentum") is not None:
+        eg.set_momentum(okw["momentum"])
 
     x0 = W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)
     x_dev = eg.to_layout(x0)
@@ -222,6 +230,9 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             assert rep.max_param_rel <= PARAM_RTOL, f"parameters, step {k}: rel err {rep.max_param_rel}"
         xh_g = gpu_sub(eg.mailboxes().to(dev))
         assert np.array_equal(xh_g.view(np.uint32), o.xhat().view(np.uint32)), f"mailboxes, step {k}"
+        if okw.get("momentum") is not None:
+            v_g = gpu_sub(eg.velocity().to(dev))
+            assert np.array_equal(v_g.view(np.uint32), o.velocity().view(np.uint32)), f"velocity, step {k}"
         if deliver_fn is not None:
             rc_g = gpu_sub(eg.received().to(dev))
             assert np.array_equal(rc_g.view(np.uint32), o.received().view(np.uint32)), f"received, step {k}"

@@ -262,6 +262,78 @@ def test_topk_carry_norm(kernel):
     assert rep.params_bit_exact and rep.sparse_checked > 10
 
 
+@pytest.mark.parametrize("P", [1, 2, 3, 5, 16])
+@pytest.mark.parametrize("carry", [False, True])
+def test_momentum_ragged_dense(P, carry):
+    numel = RAGGED if P <= 3 else RAGGED[:-1]
+    wl = W.synthetic(P, numel, steps=12, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(momentum=0.9))
+    assert rep.params_bit_exact and not rep.near_threshold
+    assert 0 < rep.events < P * wl.T * wl.steps
+
+
+@pytest.mark.parametrize("carry", [False, True])
+def test_momentum_with_topk_and_history(carry):
+    wl = W.synthetic(4, RAGGED, steps=14, lr=0.1, grad_sigma=0.01, topk=(5, 100), history_len=3)
+    rep = lockstep(wl, init="distinct", carry=carry, outbox_samples=32, oracle_kw=dict(momentum=0.5))
+    assert rep.params_bit_exact and rep.sparse_checked > 10
+
+
+def test_momentum_zero_reset_roundtrip_and_refusals():
+    wl = W.synthetic(3, RAGGED[:-1], steps=6, lr=0.1, grad_sigma=0.01)
+    dev = torch.device("cuda")
+    plain, mom = B.from_workload(wl), B.from_workload(wl)
+    mom.set_momentum(0.0)
+    xa = plain.to_layout(W.distinct_init_params(wl, dev))
+    xb = xa.clone()
+    for k in range(wl.steps):
+        g = plain.to_layout(wl.grads(k, dev))
+        plain.step(xa, g, wl.lr)
+        mom.step(xb, g, wl.lr)
+    assert torch.equal(xa, xb) and plain.stats() == mom.stats()      # mu = 0: the plain update, bit for bit
+    v = mom.velocity()
+    assert torch.equal(mom.from_layout(v), wl.grads(wl.steps - 1))
+    # read / write round trip; reset clears; turning it off leaves the plain path
+    w = torch.randn_like(v)
+    mom.write_velocity(w)
+    assert torch.equal(mom.velocity(), w)
+    mom.reset()
+    assert not mom.velocity().any()
+    mom.set_momentum(None)
+    plain.reset()
+    xa = plain.to_layout(W.distinct_init_params(wl, dev))
+    xb = xa.clone()
+    g = plain.to_layout(wl.grads(0, dev))
+    plain.step(xa, g, wl.lr)
+    mom.step(xb, g, wl.lr)
+    assert torch.equal(xa, xb) and not mom.velocity().any()
+    with pytest.raises(B.EventGradError):
+        plain.velocity()                      # never enabled: no buffer
+    for bad in (-0.5, 1.0, float("nan")):
+        with pytest.raises(B.EventGradError):
+            mom.set_momentum(bad)
+    # combinations that have no momentum kernel are refused, not silently computed without it
+    mom.set_momentum(0.9)
+    mom.set_fused_kernel(B.FUSED_REGISTER)
+    with pytest.raises(B.EventGradError):
+        mom.step(xb, g, wl.lr)
+    mom.set_fused_kernel(B.FUSED_PIPELINED)
+    mom.step(xb, g, wl.lr)
+    wide = B.from_workload(wl, hops=2)
+    with pytest.raises(B.EventGradError):
+        wide.set_momentum(0.9)
+    for e in (plain, mom, wide):
+        e.close()
+
+
+def test_momentum_resnet18_shapes_p16():
+    """Many tiles, tensors of 10 ... 2.4 M elements, carried norm; the oracle follows a sample."""
+    (wl,) = W.config(3)
+    rep = lockstep(wl, steps=12, tensors=_sample_tensors(wl), carry=True, check_every=3,
+                   oracle_kw=dict(momentum=0.9))
+    assert rep.params_bit_exact
+
+
 def test_config1_mlp():
     (wl,) = W.config(1)
     rep = lockstep(wl)
