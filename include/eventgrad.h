@@ -175,7 +175,7 @@ eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
  * again by eg_reset); mu * v + g is one fp64 fused multiply-add rounded to fp32, and the update
  * uses that rounded value.  mu = 0 reproduces the plain update bit for bit.  0 <= mu < 1
  * (EG_ERR_INVALID otherwise).  Available with the default readings on the nearest-neighbour ring
- * and the pipelined kernel, dense or Top-K (EG_ERR_STATE with eg_set_variant choices,
+ * and the default kernel choice, dense or Top-K (EG_ERR_STATE with eg_set_variant choices,
  * EG_TOPO_RING_HOPS(m > 1), intermittent delivery or EG_FUSED_REGISTER).  enabled = 0 returns to
  * the plain update and keeps the buffer.  The velocity is optimizer state like the parameters
  * themselves and not part of eg_export_state: eg_read_velocity / eg_write_velocity copy it to /
@@ -185,11 +185,17 @@ eg_status eg_set_momentum(eg_ctx* ctx, int enabled, double mu);
 eg_status eg_read_velocity(eg_ctx* ctx, float* velocity_host);
 eg_status eg_write_velocity(eg_ctx* ctx, const float* velocity_host);
 
-/* Which implementation of the fused snapshot / average / SGD kernel eg_step launches.  Both
- * compute bit-identical results.  EG_FUSED_PIPELINED (default) streams the operands through
- * shared memory with bulk asynchronous copies; EG_FUSED_REGISTER keeps the ring walk in
- * registers with plain vector loads. */
-enum { EG_FUSED_PIPELINED = 0, EG_FUSED_REGISTER = 1 };
+/* Which implementation of the fused snapshot / average / SGD kernel eg_step launches.  All
+ * compute bit-identical parameters, mailboxes, flags and counters.
+ *  EG_FUSED_AUTO (default)  for small problems (dense messages on the nearest-neighbour ring,
+ *                      default readings, P <= 16, few enough tiles of 1024 elements for all
+ *                      their thread blocks to be resident at once) the whole iteration -- decisions, snapshot, average, update,
+ *                      next norms -- runs as ONE kernel launch, because such an iteration is
+ *                      bound by launch latency; everything else takes EG_FUSED_PIPELINED.
+ *  EG_FUSED_PIPELINED  streams the operands through shared memory with bulk asynchronous
+ *                      copies (a decision kernel runs before it).
+ *  EG_FUSED_REGISTER   keeps the ring walk in registers with plain vector loads. */
+enum { EG_FUSED_PIPELINED = 0, EG_FUSED_REGISTER = 1, EG_FUSED_AUTO = 2 };
 eg_status eg_set_fused_kernel(eg_ctx* ctx, int kind);
 
 /* Per-kernel timing for measurements (off by default).  When on, eg_step brackets each

@@ -34,6 +34,7 @@ STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
 FUSED_PIPELINED = 0
 FUSED_REGISTER = 1
+FUSED_AUTO = 2
 KERNEL_GROUPS = ("norm", "decide", "topk", "fused")
 
 

@@ -75,20 +75,9 @@ struct DeliveryState {
     int enabled;
 };
 
-// One warp per (replica, tensor).  grid ceil(P*T / kWarps).
-__global__ void __launch_bounds__(kThreads)
-k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin, int n_tiles,
-         DecideParams dp, SegState st, const long long* __restrict__ numel,
-         const long long* __restrict__ topk_count, int* __restrict__ outbox_count,
-         Counters* ctr, const long long* __restrict__ step_k, DeliveryState dl) {
-    const int lane = threadIdx.x & 31;
-    // work item: (replica, tensor of the launch's range)
-    const long long w = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (w >= (long long)dp.P * dp.tn) return;
-    const int i = (int)(w / dp.tn), t = dp.t0 + (int)(w % dp.tn);
-    const long long s = (long long)i * dp.T + t;
-    const int q0 = seg_begin[t], q1 = seg_begin[t + 1];
-    const double* p = partials + (long long)i * n_tiles;
+// Sum of the partials [q0, q1) of one segment by one warp, lane-strided and in a fixed order;
+// the total is valid in lane 0.
+__device__ __forceinline__ double segment_sum(const double* __restrict__ p, int q0, int q1, int lane) {
     double acc = 0.0;
     // same order of additions as a plain strided loop, but eight loads are in flight at a time
     int q = q0 + lane;
@@ -102,9 +91,15 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     for (; q < q1; q += 32) acc = __dadd_rn(acc, p[q]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc = __dadd_rn(acc, __shfl_down_sync(0xffffffffu, acc, o));
-    if (lane != 0) return;
+    return acc;
+}
 
-    const long long k = *step_k;
+// The decision of segment s = (replica, tensor t) in iteration k from `acc`, the sum of its
+// partials: test, threshold update, message accounting, flags (one thread).
+__device__ __forceinline__ void
+decide_segment(double acc, long long s, int t, long long k, const DecideParams& dp, const SegState& st,
+               const long long* __restrict__ numel, const long long* __restrict__ topk_count,
+               int* __restrict__ outbox_count, Counters* ctr, const DeliveryState& dl) {
     const double root = __dsqrt_rn(acc);
     const double d = (dp.variant & kChangeOfNorm) ? fabs(__dsub_rn(root, st.sent_norm[s])) : root;
     const double thr = fmin(st.delta[s], dp.cap);
@@ -163,6 +158,23 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     st.snap[s] = snap;
     st.sparse[s] = sparse;
     if (outbox_count) outbox_count[s] = out_count;
+}
+
+// One warp per (replica, tensor).  grid ceil(P*T / kWarps).
+__global__ void __launch_bounds__(kThreads)
+k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin, int n_tiles,
+         DecideParams dp, SegState st, const long long* __restrict__ numel,
+         const long long* __restrict__ topk_count, int* __restrict__ outbox_count,
+         Counters* ctr, const long long* __restrict__ step_k, DeliveryState dl) {
+    const int lane = threadIdx.x & 31;
+    // work item: (replica, tensor of the launch's range)
+    const long long w = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (w >= (long long)dp.P * dp.tn) return;
+    const int i = (int)(w / dp.tn), t = dp.t0 + (int)(w % dp.tn);
+    const long long s = (long long)i * dp.T + t;
+    const double acc = segment_sum(partials + (long long)i * n_tiles, seg_begin[t], seg_begin[t + 1], lane);
+    if (lane != 0) return;
+    decide_segment(acc, s, t, *step_k, dp, st, numel, topk_count, outbox_count, ctr, dl);
 }
 
 }  // namespace eg

@@ -14,6 +14,7 @@
 #include "eg_fused_hops.cuh"
 #include "eg_fused_pipe.cuh"
 #include "eg_norm.cuh"
+#include "eg_step_small.cuh"
 #include "eg_topk.cuh"
 
 using namespace eg;
@@ -73,7 +74,12 @@ struct eg_ctx {
     int last_cuda_error = 0;
     int last_launches = 0;
     size_t fused_smem = 0;
-    int fused_kind = EG_FUSED_PIPELINED;
+    int fused_kind = EG_FUSED_AUTO;
+    // single-launch iteration for small problems (k_step_small)
+    bool small_eligible = false;
+    double* partials_small = nullptr;   // second buffer of carried partials
+    int *small_arrived = nullptr, *small_done = nullptr;
+    int2 *small_range_fused = nullptr, *small_range_norm = nullptr;   // per fused tile: its tensor's tiles
     int topk_coop_grid = 0;   // CTAs of the one-launch Top-K kernel; 0: use the ten single-phase launches
     int variant = 0;
     double cap_alpha = 0.0, cap_beta = 1.0;   // bound alpha*beta^k on the squared threshold
@@ -164,6 +170,14 @@ int64_t topk_entries(int64_t n, uint32_t num, uint32_t den) {
     return (int64_t)q;
 }
 
+// The instantiation of the single-launch kernel for P replicas (nullptr: none).
+const void* small_kernel(int P) {
+    if (P <= 4) return (const void*)k_step_small<4>;
+    if (P <= 8) return (const void*)k_step_small<8>;
+    if (P <= kSmallMaxP) return (const void*)k_step_small<16>;
+    return nullptr;
+}
+
 eg_status init_state(eg_ctx* c) {
     const size_t S = (size_t)c->P * c->T;
     std::vector<double> delta(S, c->thr.mode == EG_THRESH_FIXED ? c->thr.delta_fixed : c->thr.delta_init);
@@ -195,6 +209,10 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->recv_valid, 0, S));
         EG_CUDA(c, cudaMemset(c->arrive, 0, S));
         EG_CUDA(c, cudaMemset(c->arrivals, 0, sizeof(unsigned long long)));
+    }
+    if (c->small_arrived) {
+        EG_CUDA(c, cudaMemset(c->small_arrived, 0, (size_t)c->T * sizeof(int)));
+        EG_CUDA(c, cudaMemset(c->small_done, 0, sizeof(int)));
     }
     if (c->vel) EG_CUDA(c, cudaMemset(c->vel, 0, (size_t)c->P * c->stride * sizeof(float)));
     c->carried_valid = false;
@@ -460,6 +478,34 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         raise((const void*)k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>);
         if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
     }
+    {
+        // one launch per iteration where a few hundred CTAs cover the whole parameter set
+        // ... and all of them are resident at the same time (a second wave would double the latency)
+        int sms = 0, max_smem = 0, per_sm = 0;
+        const void* fn = small_kernel(P);
+        if (fn && !c->topk.enabled && c->hops == 1 &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess &&
+            cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) == cudaSuccess &&
+            small_smem_bytes(P) <= (size_t)max_smem &&
+            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)small_smem_bytes(P)) ==
+                cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, small_smem_bytes(P)) ==
+                cudaSuccess &&
+            c->tiles_fused.n_tiles <= per_sm * sms) {
+            if ((s = dev_alloc(c, &c->partials_small, (size_t)P * c->tiles_fused.n_tiles)) != EG_OK) return fail(s);
+            if ((s = dev_alloc(c, &c->small_arrived, (size_t)T)) != EG_OK) return fail(s);
+            if ((s = dev_alloc(c, &c->small_done, 1)) != EG_OK) return fail(s);
+            std::vector<int2> rf, rn;
+            for (int t = 0; t < T; ++t)
+                for (int q = c->seg_begin_fused[t]; q < c->seg_begin_fused[t + 1]; ++q) {
+                    rf.push_back(make_int2(c->seg_begin_fused[t], c->seg_begin_fused[t + 1]));
+                    rn.push_back(make_int2(c->seg_begin_norm[t], c->seg_begin_norm[t + 1]));
+                }
+            if ((s = upload(c, &c->small_range_fused, rf)) != EG_OK) return fail(s);
+            if ((s = upload(c, &c->small_range_norm, rn)) != EG_OK) return fail(s);
+            c->small_eligible = true;
+        }
+    }
     if ((s = init_state(c)) != EG_OK) return fail(s);
     if (cudaDeviceSynchronize() != cudaSuccess) return fail(EG_ERR_CUDA);
     *out = c;
@@ -495,7 +541,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     if (!c || !params || !grads) return EG_ERR_INVALID;
     if (deliver_dev && !c->async) return EG_ERR_STATE;     // eg_enable_delivery_masks first
     if (c->async && (c->variant & kOwnLastSent)) return EG_ERR_STATE;
-    if (c->momentum && (c->async || c->variant != 0 || c->hops > 1 || c->fused_kind != EG_FUSED_PIPELINED))
+    if (c->momentum && (c->async || c->variant != 0 || c->hops > 1 || c->fused_kind == EG_FUSED_REGISTER))
         return EG_ERR_STATE;
     if (((uintptr_t)params & 15u) || ((uintptr_t)grads & 15u)) return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
@@ -520,7 +566,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     double* partials_norm = c->partials_norm + nb;
     double* partials_fused = c->partials_fused + fb;
     long long* step_k = c->range_last ? c->step_k : nullptr;
-    if (!whole && (c->topk.enabled || c->async || c->hops > 1 || c->fused_kind != EG_FUSED_PIPELINED))
+    if (!whole && (c->topk.enabled || c->async || c->hops > 1 || c->fused_kind == EG_FUSED_REGISTER))
         return EG_ERR_STATE;
 
     // a1: || x - x_hat || partial sums, unless the previous step carried them over
@@ -532,6 +578,8 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                                                           c->variant);
         ++launches;
     }
+    const bool small = c->fused_kind == EG_FUSED_AUTO && c->small_eligible && whole && !c->async &&
+                       c->variant == 0 && !c->momentum;
     // a2 + a6: decision, threshold update, counters
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
                     c->topk.enabled, c->degree, c->variant,
@@ -540,7 +588,23 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                     t0, tcount};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf_all : tn_all;
-    {
+    if (small) {
+        // decisions, snapshot, average, update and the next norms in one launch
+        TimedSection ts(c, stream, EG_KERNEL_FUSED);
+        SmallArgs sa{use_carried ? nullptr : c->partials_norm, tn_all.n_tiles,
+                     {c->partials_fused, c->partials_small}, carry ? 1 : 0, c->small_range_fused,
+                     c->small_range_norm, c->small_arrived, c->small_done};
+#define EG_SMALL_ARGS params, grads, c->xhat, tf, c->P, c->stride, lr, sa, dp, c->st, c->d_numel, c->ctr, \
+                      c->step_k, c->err
+        if (c->P <= 4)
+            k_step_small<4><<<grid_fused, kThreads, small_smem_bytes(c->P), stream>>>(EG_SMALL_ARGS);
+        else if (c->P <= 8)
+            k_step_small<8><<<grid_fused, kThreads, small_smem_bytes(c->P), stream>>>(EG_SMALL_ARGS);
+        else
+            k_step_small<16><<<grid_fused, kThreads, small_smem_bytes(c->P), stream>>>(EG_SMALL_ARGS);
+#undef EG_SMALL_ARGS
+        ++launches;
+    } else {
         TimedSection ts(c, stream, EG_KERNEL_DECIDE);
         k_decide<<<(c->P * tcount + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
             partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
@@ -549,7 +613,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         ++launches;
     }
     // a4: Top-K select / pack / deliver for the segments that send a sparse message
-    if (c->topk.enabled) {
+    if (c->topk.enabled && !small) {
         TimedSection ts(c, stream, EG_KERNEL_TOPK);
         TopkArgs ta{params, c->xhat, tn, S, c->T, c->stride, c->st.sparse, c->tk, c->err};
         if (c->topk_coop_grid > 0) {
@@ -572,11 +636,11 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         }
     }
     // a3 + a5: dense snapshot, consensus average, SGD
-    {
+    if (!small) {
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
         const uint8_t* valid = c->async ? c->recv_valid : c->st.valid;   // whom the neighbours have heard from
         if (c->hops > 1 && c->hops <= kMaxStagedHops && c->P >= 2 * c->hops + 1 &&
-            c->fused_kind == EG_FUSED_PIPELINED) {
+            c->fused_kind != EG_FUSED_REGISTER) {
             // rows staged through shared memory; the register kernel choice keeps the plain form
             launch_hops_staged(c, carry, grid_fused, stream, params, grads, valid, tf, lr, partials_fused, step_k);
         } else if (c->hops > 1) {
@@ -606,7 +670,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                     <<<grid_fused, kPipeThreads, smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
                     partials_fused, step_k, c->err, c->vel, c->mu);
-        } else if (c->fused_kind == EG_FUSED_PIPELINED) {
+        } else if (c->fused_kind != EG_FUSED_REGISTER) {
             const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
 #define EG_PIPE_ARGS params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, \
                      partials_fused, step_k, c->err
@@ -658,7 +722,7 @@ eg_status eg_step_host(eg_ctx* c, float* params_host, const float* grads_host, f
     cudaStream_t stream = c->last_stream;
     c->carried_valid = false;  // the parameters come from outside
     const bool pipelined = !c->topk.enabled && !c->async && c->hops == 1 &&
-                           c->fused_kind == EG_FUSED_PIPELINED && c->T >= 2;
+                           c->fused_kind != EG_FUSED_REGISTER && c->T >= 2;
     if (!pipelined) {
         EG_CUDA(c, cudaMemcpyAsync(c->stage_x, params_host, bytes, cudaMemcpyHostToDevice, stream));
         EG_CUDA(c, cudaMemcpyAsync(c->stage_g, grads_host, bytes, cudaMemcpyHostToDevice, stream));
@@ -898,7 +962,9 @@ eg_status eg_set_threshold_cap(eg_ctx* c, double alpha, double beta) {
 }
 
 eg_status eg_set_fused_kernel(eg_ctx* c, int kind) {
-    if (!c || (kind != EG_FUSED_PIPELINED && kind != EG_FUSED_REGISTER)) return EG_ERR_INVALID;
+    if (!c || (kind != EG_FUSED_PIPELINED && kind != EG_FUSED_REGISTER && kind != EG_FUSED_AUTO))
+        return EG_ERR_INVALID;
+    if (kind != c->fused_kind) c->carried_valid = false;   // the kernels keep their carried sums apart
     c->fused_kind = kind;
     return EG_OK;
 }
@@ -927,7 +993,7 @@ eg_status eg_kernel_times(eg_ctx* c, double* ms_host, uint64_t* sections_host) {
 
 eg_status eg_set_momentum(eg_ctx* c, int enabled, double mu) {
     if (!c) return EG_ERR_INVALID;
-    if (!enabled) { c->momentum = false; return EG_OK; }
+    if (!enabled) { c->momentum = false; c->carried_valid = false; return EG_OK; }
     if (!(mu >= 0.0 && mu < 1.0)) return EG_ERR_INVALID;
     if (c->async || c->variant != 0 || c->hops > 1) return EG_ERR_STATE;
     DeviceGuard guard(c->device);
@@ -946,6 +1012,7 @@ eg_status eg_set_momentum(eg_ctx* c, int enabled, double mu) {
     }
     c->momentum = true;
     c->mu = mu;
+    c->carried_valid = false;
     return EG_OK;
 }
 

@@ -18,8 +18,10 @@ INF = float("inf")
 
 @pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 6, 7, 11, 64, 130])
 @pytest.mark.parametrize("carry", [False, True])
-@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER, B.FUSED_AUTO])
 def test_ragged_dense(P, carry, kernel):
+    """Under the automatic choice the cases without the 2^20 + 1 element tensor and with at most
+    16 replicas run as one launch per iteration; the others take the pipelined kernel."""
     numel = RAGGED if P <= 4 else RAGGED[:-1]
     wl = W.synthetic(P, numel, steps=12, lr=0.1, grad_sigma=0.01)
     rep = lockstep(wl, init="distinct", carry=carry, fused_kernel=kernel)
@@ -58,10 +60,12 @@ def test_more_neighbours_with_topk_and_variants():
 
 
 @pytest.mark.parametrize("carry", [False, True])
-def test_geometric_threshold_cap(carry):
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_AUTO])
+def test_geometric_threshold_cap(carry, kernel):
     wl = W.synthetic(4, RAGGED[:-1], steps=20, lr=0.1, grad_sigma=0.01)
-    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(threshold_cap=(1e-3, 0.7)))
-    free = lockstep(wl, init="distinct", carry=carry)
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(threshold_cap=(1e-3, 0.7)),
+                   fused_kernel=kernel)
+    free = lockstep(wl, init="distinct", carry=carry, fused_kernel=kernel)
     assert rep.params_bit_exact and not rep.near_threshold
     assert rep.events > free.events          # a shrinking bound makes tensors communicate more
 
@@ -196,18 +200,20 @@ def test_resynchronise_through_the_checkpoint_interface():
 
 
 @pytest.mark.parametrize("hist,horizon", [(1, 1.0), (4, 1.0), (2, 0.5)])
-def test_history_and_horizon(hist, horizon):
+@pytest.mark.parametrize("kernel,carry", [(B.FUSED_PIPELINED, False), (B.FUSED_AUTO, False), (B.FUSED_AUTO, True)])
+def test_history_and_horizon(hist, horizon, kernel, carry):
     wl = W.synthetic(5, RAGGED[:-1], steps=25, lr=0.1, grad_sigma=0.01, history_len=hist,
                      horizon=horizon)
-    rep = lockstep(wl, init="distinct")
+    rep = lockstep(wl, init="distinct", fused_kernel=kernel, carry=carry)
     assert rep.params_bit_exact and not rep.near_threshold
 
 
 @pytest.mark.parametrize("delta,force", [(0.0, False), (INF, False), (INF, True), (0.02, True)])
-def test_fixed_threshold_modes(delta, force):
+@pytest.mark.parametrize("kernel,carry", [(B.FUSED_PIPELINED, False), (B.FUSED_AUTO, False), (B.FUSED_AUTO, True)])
+def test_fixed_threshold_modes(delta, force, kernel, carry):
     wl = W.synthetic(4, RAGGED[:-1], steps=6, lr=0.1, grad_sigma=0.01)
     kw = dict(mode=1, delta_fixed=delta, force_first_event=force)
-    rep = lockstep(wl, init="distinct", oracle_kw=kw)
+    rep = lockstep(wl, init="distinct", oracle_kw=kw, fused_kernel=kernel, carry=carry)
     assert rep.params_bit_exact
     if delta == 0.0:
         assert rep.events == 4 * wl.T * wl.steps
@@ -334,16 +340,24 @@ def test_momentum_resnet18_shapes_p16():
     assert rep.params_bit_exact
 
 
-def test_config1_mlp():
+@pytest.mark.parametrize("carry", [False, True])
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_AUTO])
+def test_config1_mlp(carry, kernel):
     (wl,) = W.config(1)
-    rep = lockstep(wl)
+    rep = lockstep(wl, carry=carry, fused_kernel=kernel)
     assert rep.params_bit_exact and not rep.near_threshold
+    if kernel == B.FUSED_AUTO:      # one launch per iteration (plus the norm pass when nothing is carried)
+        assert rep.launches == (wl.steps + 1 if carry else 2 * wl.steps)
 
 
-def test_config2_resnet20():
+@pytest.mark.parametrize("carry", [False, True])
+@pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_AUTO])
+def test_config2_resnet20(carry, kernel):
     (wl,) = W.config(2)
-    rep = lockstep(wl)
+    rep = lockstep(wl, carry=carry, fused_kernel=kernel)
     assert rep.params_bit_exact and not rep.near_threshold
+    if kernel == B.FUSED_AUTO:
+        assert rep.launches == (wl.steps + 1 if carry else 2 * wl.steps)
 
 
 @pytest.mark.parametrize("carry", [False, True])
