@@ -111,9 +111,11 @@ struct PipeSmem {
     static constexpr int kWrapR = kWrapL + kTileBytes;
     static constexpr int kBars = kWrapR + kTileBytes;             // full[S], empty[S], wrap
     static constexpr int kFlags = kBars + 8 * (2 * STAGES + 1) + 8;
+    // carried norm: per stage one slot of 8 doubles per consumer warp (see the consumers' end of
+    // a replica and the producer warp's reduce_slot)
     __host__ __device__ static size_t bytes(int P, bool carry, int consumer_warps) {
         size_t b = kFlags + 16 + (((size_t)P + 15) & ~(size_t)15);
-        if (carry) b += (size_t)P * consumer_warps * sizeof(double);
+        if (carry) b += (size_t)STAGES * consumer_warps * 8 * sizeof(double);
         return b;
     }
 };
@@ -162,7 +164,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kFlags);
     // bit 0: dense message, bit 1: valid, bit 2: contributes its own x, bit 3: arrives now
     uint8_t* s_mode = smem + L::kFlags + 16;
-    double* s_red = reinterpret_cast<double*>(s_mode + ((P + 15) & ~15));
+    double* s_part = reinterpret_cast<double*>(s_mode + ((P + 15) & ~15));   // [STAGES][CWARPS * 8]
 
     const int tile = blockIdx.x, tid = threadIdx.x;
     const int t = tt.tensor[tile];
@@ -194,32 +196,65 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
 
     if (tid >= CONSUMERS) {
         // ------------------------------------------------------------------ producer
-        if (tid == CONSUMERS) {
+        // CARRY: the whole warp walks the loop, because it also finishes the sums of squares that
+        // the consumers leave behind (8 values per consumer warp and replica, in the slot of the
+        // replica's stage): once a stage has been released, its slot is complete.
+        const int pl = tid - CONSUMERS;
+        auto reduce_slot = [&](int slot, int j) {
+            static_assert(CWARPS == 8, "a slot holds 64 values: two per lane");
+            const double* sp = s_part + slot * (CWARPS * 8);
+            double r = __dadd_rn(sp[pl], sp[32 + pl]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) r = __dadd_rn(r, __shfl_xor_sync(0xffffffffu, r, o));
+            if (pl == 0) partials[(long long)j * tt.n_tiles + tile] = r;
+        };
+        if (CARRY || tid == CONSUMERS) {
             const float* xp = x + off;
             const float* gp = g + off;
             const float* hp = xhat + off;
             const float* mp = ASYNC ? mailbox + off : hp;
             const float* vp = MOM ? vel + off : nullptr;
-            mbar_expect_tx(wrap_bar, copy_bytes);
-            bulk_g2s(wrap_l,
-                     (cx_last ? xp : ((s_mode[P - 1] & 8) ? hp : mp)) + (long long)(P - 1) * stride,
-                     copy_bytes, wrap_bar);
+            if (pl == 0) {
+                mbar_expect_tx(wrap_bar, copy_bytes);
+                bulk_g2s(wrap_l,
+                         (cx_last ? xp : ((s_mode[P - 1] & 8) ? hp : mp)) + (long long)(P - 1) * stride,
+                         copy_bytes, wrap_bar);
+            }
             int s = 0;
             uint32_t wait_parity = 1;     // parity of the phase before the one to wait for
+            bool alive = true;
             for (int j = 0; j < P; ++j) {
-                if (j >= STAGES && !mbar_wait_bounded(&empty[s], wait_parity, s_abort, err)) break;
-                float* st = stages + s * (kArr * TILE);
-                const bool cx = (s_mode[j] & kCx) != 0;
-                const bool is_last = last_opt && (j == P - 1);
-                const bool need_x = !(is_last && cx);
-                const bool need_h = !cx && !is_last;
-                mbar_expect_tx(&full[s], copy_bytes * ((MOM ? 2u : 1u) + (need_x ? 1u : 0u) + (need_h ? 1u : 0u)));
-                bulk_g2s(st + TILE, gp, copy_bytes, &full[s]);
-                if (MOM) { bulk_g2s(st + 3 * TILE, vp, copy_bytes, &full[s]); vp += stride; }
-                if (need_x) bulk_g2s(st, xp, copy_bytes, &full[s]);
-                if (need_h) bulk_g2s(st + 2 * TILE, (s_mode[j] & 8) ? hp : mp, copy_bytes, &full[s]);
-                xp += stride; gp += stride; hp += stride; mp += stride;
+                if (j >= STAGES) {
+                    alive = mbar_wait_bounded(&empty[s], wait_parity, s_abort, err);
+                    if (CARRY) alive = __all_sync(0xffffffffu, alive);
+                    if (!alive) break;
+                    if (CARRY) reduce_slot(s, j - STAGES);     // before the stage is filled again
+                }
+                if (pl == 0) {
+                    float* st = stages + s * (kArr * TILE);
+                    const bool cx = (s_mode[j] & kCx) != 0;
+                    const bool is_last = last_opt && (j == P - 1);
+                    const bool need_x = !(is_last && cx);
+                    const bool need_h = !cx && !is_last;
+                    mbar_expect_tx(&full[s],
+                                   copy_bytes * ((MOM ? 2u : 1u) + (need_x ? 1u : 0u) + (need_h ? 1u : 0u)));
+                    bulk_g2s(st + TILE, gp, copy_bytes, &full[s]);
+                    if (MOM) { bulk_g2s(st + 3 * TILE, vp, copy_bytes, &full[s]); vp += stride; }
+                    if (need_x) bulk_g2s(st, xp, copy_bytes, &full[s]);
+                    if (need_h) bulk_g2s(st + 2 * TILE, (s_mode[j] & 8) ? hp : mp, copy_bytes, &full[s]);
+                    xp += stride; gp += stride; hp += stride; mp += stride;
+                }
                 if (++s == STAGES) { s = 0; wait_parity ^= 1u; }
+            }
+            if (CARRY && alive) {
+                // the replicas whose stages are not filled again
+                for (int j = max(0, P - STAGES); j < P; ++j) {
+                    const int sj = j % STAGES;
+                    alive = __all_sync(0xffffffffu,
+                                       mbar_wait_bounded(&empty[sj], (uint32_t)((j / STAGES) & 1), s_abort, err));
+                    if (!alive) break;
+                    reduce_slot(sj, j);
+                }
             }
         }
     } else {
@@ -327,10 +362,11 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                 }
             }
             if (CARRY) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1)
-                    acc = __dadd_rn(acc, __shfl_down_sync(0xffffffffu, acc, o));
-                if (lane == 0) s_red[j * CWARPS + warp] = acc;
+                // two of the five rounds of the warp sum; the producer warp does the rest once
+                // this stage has been released by all consumer warps
+                acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, 16));
+                acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, 8));
+                if (lane < 8) s_part[s * (CWARPS * 8) + warp * 8 + lane] = acc;
             }
             // everything later iterations need from this stage now sits in registers
             __syncwarp();
@@ -347,15 +383,6 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         // failure path only: give copies in flight time to land before the CTA retires
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000ll) {}
-    }
-    if (CARRY) {
-        __syncthreads();
-        for (int j = tid; j < P; j += CONSUMERS + 32) {
-            double r = 0.0;
-#pragma unroll
-            for (int w = 0; w < CWARPS; ++w) r = __dadd_rn(r, s_red[j * CWARPS + w]);
-            partials[(long long)j * tt.n_tiles + tile] = r;
-        }
     }
 }
 
