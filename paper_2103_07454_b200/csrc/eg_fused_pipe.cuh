@@ -288,11 +288,15 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         float* ho = xhat + off + c0;
         float* mo = ASYNC ? mailbox + off + c0 : nullptr;
         float* vo = MOM ? vel + off + c0 : nullptr;
-        for (int j = 0; ok && j < P; ++j) {
+        // One replica.  A = contributions of replica j-1, B = of replica j, C receives those of
+        // replica j+1.  The three arrays swap roles from one replica to the next (see the loop
+        // below), so nothing is copied between them.
+        auto one_replica = [&](const int j, double (&hA)[COLS][4], double (&hB)[COLS][4],
+                               double (&hC)[COLS][4]) -> bool {
             const bool more = j + 1 < P;
             if (more) {
                 ok = mbar_wait_bounded(&full[s1], parity1, s_abort, err);
-                if (!ok) break;
+                if (!ok) return false;
             }
             const unsigned mode_next = s_mode[more ? j + 1 : 0];
             const float* st = stages + s * (kArr * TILE);
@@ -318,7 +322,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
                     const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
                     if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;   // private to this thread
-                    const double hn[4] = {(double)hnf.x, (double)hnf.y, (double)hnf.z, (double)hnf.w};
+                    hC[v][0] = (double)hnf.x; hC[v][1] = (double)hnf.y; hC[v][2] = (double)hnf.z; hC[v][3] = (double)hnf.w;
                     double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
                     if (MOM) {      // v <- mu * v + g, kept in fp32; the update then uses gamma * v
                         const float4 vf = *reinterpret_cast<const float4*>(st + 3 * TILE + c);
@@ -334,7 +338,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     float4 x_old = make_float4(0.f, 0.f, 0.f, 0.f);   // only needed under ASYNC
                     if (cx || (variant & kOwnLastSent)) {   // own term = this replica's contribution
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) xd[q] = hc[v][q];
+                        for (int q = 0; q < 4; ++q) xd[q] = hB[v][q];
                         if (ASYNC) x_old = hcf;
                     } else {
                         const float4 xf = *reinterpret_cast<const float4*>(st + c);
@@ -345,8 +349,8 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         double sum = xd[q];
-                        if (ul) sum = __dadd_rn(sum, hp[v][q]);
-                        if (ur) sum = __dadd_rn(sum, hn[q]);
+                        if (ul) sum = __dadd_rn(sum, hA[v][q]);
+                        if (ur) sum = __dadd_rn(sum, hC[v][q]);
                         xn[q] = __double2float_rn(__fma_rn(neg_lr, gd[q], __dmul_rn(sum, w)));
                     }
                     const float4 xn4 = make_float4(xn[0], xn[1], xn[2], xn[3]);
@@ -357,8 +361,6 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     if (CARRY)
                         acc = sq_diff4(xn4, (variant & kChangeOfNorm) ? make_float4(0.f, 0.f, 0.f, 0.f) : hcf,
                                        nel[v], acc);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) { hp[v][q] = hc[v][q]; hc[v][q] = hn[q]; }
                 }
             }
             if (CARRY) {
@@ -377,6 +379,13 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             mode_prev = mode_cur; mode_cur = mode_next;
             s = s1;
             if (++s1 == STAGES) { s1 = 0; parity1 ^= 1u; }
+            return true;
+        };
+        double hn[COLS][4];
+        for (int j = 0; ok && j < P; j += 3) {
+            if (!one_replica(j, hp, hc, hn)) break;
+            if (j + 1 < P && !one_replica(j + 1, hc, hn, hp)) break;
+            if (j + 2 < P && !one_replica(j + 2, hn, hp, hc)) break;
         }
     }
     if (*s_abort) {
@@ -389,7 +398,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
 // The method as the paper's formulas state it (default readings, synchronous delivery).  No
 // register bound is requested: the body needs 72 registers, which lets 3 CTAs share an SM.
 template <int TILE, int STAGES, int CONSUMERS, bool CARRY>
-__global__ void __launch_bounds__(CONSUMERS + 32)
+__global__ void __launch_bounds__(CONSUMERS + 32, 3)
 k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
