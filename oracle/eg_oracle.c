@@ -22,8 +22,10 @@
  * a hand-worked threshold sequence from Eq. (thres) with and without history
  * (tests/golden/threshold_sequence.txt); Top-K against a brute-force sort, K = n == dense,
  * payload = 2K percent (Section 7).
- * Parity unpinned: the paper prints no worked numeric trigger sequence, so the readings
- * listed below are pinned by consistency with its equations, not by printed values.
+ * Every function here has at least one such pin.  What the pins cannot settle is the choice
+ * between two readings of an ambiguous passage: the paper prints no worked numeric trigger
+ * sequence, so the pins fix the arithmetic of the readings listed below, not which reading
+ * the authors meant.
  *
  * Readings where the paper is silent (kept in one place so they can be checked by eye):
  *  - the tested quantity is the L2 norm of the element-wise difference x - x_hat
