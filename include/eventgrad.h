@@ -296,6 +296,16 @@ eg_status eg_selftest_wait_timeout(eg_ctx* ctx, void* stream);
 eg_status eg_reset(eg_ctx* ctx);
 void eg_destroy(eg_ctx* ctx);
 
+/* Test hook for the allocation-failure paths: the nth device allocation the library makes from
+ * now on (in any context of this process) fails as if the device were out of memory, without
+ * touching the device; 0 switches the hook off.  eg_create then frees what it had allocated,
+ * stores NULL in *out and returns EG_ERR_OOM. */
+void eg_debug_fail_allocation(int nth);
+
+/* Tracing: with EG_NVTX set (to anything but 0) in the environment when a context is created,
+ * eg_step wraps the launches of every kernel group in a named NVTX range ("eventgrad:norm",
+ * ":decide", ":topk", ":fused"); without a profiler attached the ranges cost nothing. */
+
 const char* eg_strerror(eg_status s);
 /* cudaError_t of the most recent failed CUDA call of this context (0 if none). */
 int eg_last_cuda_error(const eg_ctx* ctx);

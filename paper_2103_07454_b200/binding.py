@@ -29,6 +29,7 @@ EXPORTS = [
     "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant", "eg_set_threshold_cap",
     "eg_enable_delivery_masks", "eg_step_masked", "eg_read_received", "eg_delivery_status",
     "eg_selftest_wait_timeout", "eg_set_momentum", "eg_read_velocity", "eg_write_velocity",
+    "eg_debug_fail_allocation",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -97,6 +98,8 @@ def load_library() -> C.CDLL:
     lib.eg_delivery_status.argtypes = [vp, vp, u64p]
     lib.eg_change_norms_static.argtypes = [vp, vp, C.c_int, C.c_int64, i64p, i64p, C.c_int, vp, vp]
     lib.eg_kernel_times.argtypes = [vp, C.POINTER(C.c_double), u64p]
+    lib.eg_debug_fail_allocation.argtypes = [C.c_int]
+    lib.eg_debug_fail_allocation.restype = None
     lib.eg_destroy.argtypes = [vp]
     lib.eg_destroy.restype = None
     lib.eg_strerror.argtypes = [C.c_int]

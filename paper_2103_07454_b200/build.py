@@ -13,7 +13,7 @@ NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--fmad=false",            # every fused multiply-add of the path is written out
-    "-Xcompiler", "-fPIC", "-shared", "-DEG_FUSED_VPT=1",
+    "-Xcompiler", "-fPIC", "-shared", "-DEG_FUSED_VPT=1", "-ldl",
 ]
 
 

@@ -9,6 +9,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "eg_common.cuh"
 #include "eg_fused.cuh"
 #include "eg_fused_hops.cuh"
@@ -103,6 +105,7 @@ struct eg_ctx {
     float* vel = nullptr;
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
+    bool nvtx = false;      // EG_NVTX in the environment at eg_create: named ranges around the kernel groups
     std::vector<cudaEvent_t> ev_pool;      // pairs
     std::vector<int> ev_kind;              // kernel group of every recorded pair
     size_t ev_used = 0;
@@ -119,10 +122,18 @@ namespace {
         }                                                    \
     } while (0)
 
+// Test hook (eg_debug_fail_allocation): the n-th device allocation from now on reports
+// cudaErrorMemoryAllocation without calling the runtime; 0: off.
+int g_fail_alloc_in = 0;
+
 template <typename Tp>
 eg_status dev_alloc(eg_ctx* c, Tp** out, size_t count, bool zero = true) {
     void* p = nullptr;
     const size_t bytes = (count ? count : 1) * sizeof(Tp);
+    if (g_fail_alloc_in > 0 && --g_fail_alloc_in == 0) {
+        c->last_cuda_error = (int)cudaErrorMemoryAllocation;
+        return EG_ERR_OOM;
+    }
     EG_CUDA(c, cudaMalloc(&p, bytes));
     c->allocs.push_back(p);
     if (zero) EG_CUDA(c, cudaMemset(p, 0, bytes));
@@ -235,8 +246,11 @@ constexpr size_t kMaxTimedPairs = 1 << 15;
 struct TimedSection {
     eg_ctx* c;
     cudaStream_t stream;
-    bool on;
-    TimedSection(eg_ctx* ctx, cudaStream_t s, int kind) : c(ctx), stream(s), on(false) {
+    bool on, range;
+    TimedSection(eg_ctx* ctx, cudaStream_t s, int kind) : c(ctx), stream(s), on(false), range(ctx->nvtx) {
+        static const char* const kNames[EG_KERNEL_GROUPS] = {"eventgrad:norm", "eventgrad:decide",
+                                                             "eventgrad:topk", "eventgrad:fused"};
+        if (range) nvtxRangePushA(kNames[kind]);      // host-side range around the launches of the group
         if (!c->timing || c->ev_used >= kMaxTimedPairs) return;
         if (c->ev_pool.size() < 2 * (c->ev_used + 1)) {
             cudaEvent_t a, b;
@@ -250,9 +264,11 @@ struct TimedSection {
         on = cudaEventRecord(c->ev_pool[2 * c->ev_used], stream) == cudaSuccess;
     }
     ~TimedSection() {
-        if (!on) return;
-        cudaEventRecord(c->ev_pool[2 * c->ev_used + 1], stream);
-        ++c->ev_used;
+        if (on) {
+            cudaEventRecord(c->ev_pool[2 * c->ev_used + 1], stream);
+            ++c->ev_used;
+        }
+        if (range) nvtxRangePop();
     }
 };
 
@@ -316,6 +332,8 @@ static void launch_hops_staged(eg_ctx* c, bool carry, int grid, cudaStream_t str
 
 extern "C" {
 
+void eg_debug_fail_allocation(int nth) { g_fail_alloc_in = nth > 0 ? nth : 0; }
+
 const char* eg_strerror(eg_status s) {
     switch (s) {
         case EG_OK: return "ok";
@@ -366,6 +384,7 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     eg_status s = EG_OK;
     auto fail = [&](eg_status code) { eg_destroy(c); return code; };
     if (cudaGetDevice(&c->device) != cudaSuccess) return fail(EG_ERR_CUDA);
+    { const char* e = getenv("EG_NVTX"); c->nvtx = e && *e && *e != '0'; }
     c->P = P; c->T = T; c->H = thr->history_len; c->thr = *thr;
     if (topk) c->topk = *topk;
     c->hops = topology + 1;                       // EG_TOPO_RING_HOPS(m) == m - 1

@@ -532,6 +532,60 @@ def test_bounded_wait_gives_up_and_the_context_survives():
     assert torch.equal(x, y) and eg.stats() == ref.stats()
 
 
+def test_every_allocation_failure_is_reported_and_leaks_nothing():
+    """Host-made failure: the n-th device allocation of eg_create fails (test hook, the device
+    is not touched).  Every n must give EG_ERR_OOM and a NULL handle, release what was allocated
+    before it, and leave the library usable."""
+    import ctypes
+    lib = B.load_library()
+    wl = W.synthetic(4, [5, 1000, 70000], steps=2, topk=(5, 100))
+    thr = B.ThresholdParams(0, 1.0, 2, 0.0, 0.0, 1)
+    tk = B.TopkParams(1, 5, 100)
+    numel = (ctypes.c_int64 * wl.T)(*wl.numel)
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    free0, _ = torch.cuda.mem_get_info()
+    n = 1
+    while True:
+        lib.eg_debug_fail_allocation(n)
+        h = ctypes.c_void_p()
+        st = lib.eg_create(ctypes.byref(h), 0, wl.P, numel, wl.T, ctypes.byref(thr), ctypes.byref(tk))
+        if st == 0:
+            break
+        assert st == 2 and not h.value, f"allocation {n}: status {st}"
+        assert lib.eg_strerror(st) == b"out of memory"
+        n += 1
+        assert n < 200
+    lib.eg_debug_fail_allocation(0)
+    assert n > 20                       # a Top-K context makes dozens of allocations
+    lib.eg_destroy(h)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 >= free0 - (4 << 20), "memory of the failed creations was not released"
+    # the hook is off again: the library works as before
+    rep = lockstep(wl, init="distinct", outbox_samples=4)
+    assert rep.params_bit_exact
+    # later allocations fail the same way: the velocity buffer and the second copy of the mailboxes
+    eg = B.from_workload(W.synthetic(3, [100, 5000], steps=2))
+    lib.eg_debug_fail_allocation(1)
+    with pytest.raises(B.EventGradError):
+        eg.set_momentum(0.9)
+    lib.eg_debug_fail_allocation(1)
+    with pytest.raises(B.EventGradError):
+        eg.enable_delivery_masks()
+    lib.eg_debug_fail_allocation(0)
+    eg.set_momentum(0.9)
+    eg.close()
+
+
+def test_named_ranges_do_not_change_results(monkeypatch):
+    """EG_NVTX wraps the kernel groups in named ranges (no-ops without a profiler attached)."""
+    monkeypatch.setenv("EG_NVTX", "1")
+    wl = W.synthetic(4, RAGGED, steps=6, lr=0.1, grad_sigma=0.01, topk=(5, 100))
+    rep = lockstep(wl, init="distinct", carry=True, outbox_samples=8)
+    assert rep.params_bit_exact
+
+
 def test_invalid_arguments_are_reported():
     wl = W.synthetic(2, [8])
     eg = B.from_workload(wl)
