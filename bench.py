@@ -12,6 +12,11 @@ an independent copy of the workload on its own GPU ("replicas only": the method 
 one device's memory, nothing is exchanged); the value is the sum over ranks divided by the
 slowest rank's time.
 
+Every GB/s figure of one line (``value``, ``e2e``, ``cpu_baseline``, and the line of
+``--impl reference``) counts the same bytes per element-step, those of the timed variant
+(``config.bytes_per_element_step``: 16 with the carried norm, 24 with the separate norm pass), so
+their ratios are ratios of step rates; ``replica_steps_per_s`` beside each needs no convention.
+
 Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
@@ -192,7 +197,7 @@ def sample_tensors(wl: W.Workload, fraction: float):
 
 
 def time_oracle(wl: W.Workload, steps: int, warmup: int, budget_s: float, gen_device: str,
-                single_thread_s: float = 0.0):
+                single_thread_s: float = 0.0, bytes_per_element: int = 16):
     """Times the CPU oracle, as it stands, on all host cores.  If ``steps`` full-size steps do
     not fit ``budget_s`` the run uses a subset of the tensors (they do not interact)."""
     import numpy as np
@@ -248,11 +253,11 @@ def time_oracle(wl: W.Workload, steps: int, warmup: int, budget_s: float, gen_de
         o1.step(x1, g1, wl.lr)
         s1 = time.perf_counter() - t0
         o1.close()
-        one = {"value": wl.P * sum(numel1) * BYTES_PER_ELEMENT["two_pass"] / s1 / 1e9, "unit": "GB/s",
+        one = {"value": wl.P * sum(numel1) * bytes_per_element / s1 / 1e9, "unit": "GB/s",
                "replica_steps_per_s": wl.P * (sum(numel1) / wl.N) / s1,
                "sample": f"1 step of {len(t1)}/{wl.T} tensors ({sum(numel1)} elements per replica)"}
     elems = wl.P * n_sub * steps
-    gbs = elems * BYTES_PER_ELEMENT["two_pass"] / sec / 1e9
+    gbs = elems * bytes_per_element / sec / 1e9
     sample = (f"{steps} steps of all {wl.P} replicas x {len(tensors)}/{wl.T} tensors "
               f"({n_sub}/{wl.N} elements per replica)")
     return {"value": gbs, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample,
@@ -266,13 +271,14 @@ def run_reference(args):
         return
     wl = pick_workload(args)
     gen = "cuda" if torch.cuda.is_available() else "cpu"
-    r = time_oracle(wl, args.steps, args.warmup, budget_s=120.0, gen_device=gen)
+    r = time_oracle(wl, args.steps, args.warmup, budget_s=120.0, gen_device=gen,
+                    bytes_per_element=BYTES_PER_ELEMENT[args.variant])
     line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": "GB/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * r["seconds"] / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": wl.name, "P": wl.P, "tensors": wl.T, "elements": wl.N,
-                       "bytes_per_element_step": BYTES_PER_ELEMENT["two_pass"]},
+                       "variant": args.variant, "bytes_per_element_step": BYTES_PER_ELEMENT[args.variant]},
             "replica_steps_per_s": r["replica_steps_per_s"],
             "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
             "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0,
@@ -447,7 +453,7 @@ def run_native(args):
         eg.step_host(xh, gh[k % len(gh)], wl.lr)
     e_ms = (time.perf_counter() - t0) * 1e3
     e_units, e_ms_max = aggregate(float(elems) * e_steps, e_ms, dev)
-    e2e = {"value": e_units * (BYTES_PER_ELEMENT["two_pass"] + extra) / e_ms_max / 1e6, "unit": "GB/s",
+    e2e = {"value": e_units * (BYTES_PER_ELEMENT[args.variant] + extra) / e_ms_max / 1e6, "unit": "GB/s",
            "h2d_bytes_per_step": 2 * buf_bytes, "d2h_bytes_per_step": buf_bytes,
            "steps": e_steps, "ms_per_step": e_ms_max / e_steps,
            "replica_steps_per_s": world * wl.P * e_steps / (e_ms_max / 1e3)}
@@ -474,7 +480,7 @@ def run_native(args):
         del grads
         torch.cuda.empty_cache()
         cpu = time_oracle(wl, steps=args.cpu_steps, warmup=1, budget_s=25.0, gen_device=str(dev),
-                          single_thread_s=4.0)
+                          single_thread_s=4.0, bytes_per_element=BYTES_PER_ELEMENT[args.variant] + extra)
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample", "replica_steps_per_s",
                                    "single_thread")}
 
