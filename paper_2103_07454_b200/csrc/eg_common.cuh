@@ -38,6 +38,7 @@ struct SegState {
     double* thr_used;            // delta that d was compared with
     unsigned long long* events;  // events so far
     double* sent_norm;           // ||x|| at the last event (change-of-norm variant)
+    unsigned int* sparse_steps;  // [2] Top-K messages decided in the iteration of this parity (nullptr: dense)
 };
 
 // Variants of the method that the paper's text also admits (kernel argument `variant`).

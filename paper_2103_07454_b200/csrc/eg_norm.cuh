@@ -131,6 +131,7 @@ decide_segment(double acc, long long s, int t, long long k, const DecideParams& 
             payload = 4ull * (unsigned long long)numel[t];
         } else {
             sparse = 1;
+            if (st.sparse_steps) atomicAdd(&st.sparse_steps[k & 1], 1u);   // tells the Top-K launch there is work
             out_count = (int)topk_count[t];
             payload = 8ull * (unsigned long long)topk_count[t];
         }
@@ -174,7 +175,9 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     const long long s = (long long)i * dp.T + t;
     const double acc = segment_sum(partials + (long long)i * n_tiles, seg_begin[t], seg_begin[t + 1], lane);
     if (lane != 0) return;
-    decide_segment(acc, s, t, *step_k, dp, st, numel, topk_count, outbox_count, ctr, dl);
+    const long long k = *step_k;
+    if (w == 0 && st.sparse_steps) st.sparse_steps[(k + 1) & 1] = 0;   // the next iteration's count starts at zero
+    decide_segment(acc, s, t, k, dp, st, numel, topk_count, outbox_count, ctr, dl);
 }
 
 }  // namespace eg

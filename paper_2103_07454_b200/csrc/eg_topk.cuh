@@ -646,10 +646,15 @@ struct TopkArgs {
     const uint8_t* sparse;
     TopkState tk;
     unsigned int* err;
+    const unsigned int* sparse_steps;   // [2] sparse messages decided in the iteration of this parity
+    const long long* step_k;
 };
 
 __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+    // a quiet iteration (the decision kernel counted no sparse message) ends here, before any
+    // grid-wide barrier: the same answer in every CTA
+    if (a.sparse_steps[*a.step_k & 1] == 0) return;
     if (blockIdx.x == 0) topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, (int)gridDim.x);
     grid.sync();
     if (a.tk.plan->n_sparse == 0) return;          // the same for every CTA

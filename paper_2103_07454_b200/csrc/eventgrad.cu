@@ -208,6 +208,7 @@ eg_status init_state(eg_ctx* c) {
     EG_CUDA(c, cudaMemset(c->step_k, 0, sizeof(long long)));
     EG_CUDA(c, cudaMemset(c->err, 0, sizeof(unsigned int)));
     EG_CUDA(c, cudaMemset(c->outbox_count, 0, S * sizeof(int)));
+    if (c->st.sparse_steps) EG_CUDA(c, cudaMemset(c->st.sparse_steps, 0, 2 * sizeof(unsigned int)));
     EG_CUDA(c, cudaMemset(c->xhat, 0, (size_t)c->P * c->stride * sizeof(float)));
     if (c->topk.enabled) {
         EG_CUDA(c, cudaMemset(c->tk.hist, 0, S * kMaxBins * sizeof(unsigned int)));
@@ -430,6 +431,7 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S); EG_ALLOC(c->st.sent_norm, S);
     EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 2);
     EG_ALLOC(c->outbox_count, S);
+    if (c->topk.enabled) EG_ALLOC(c->st.sparse_steps, 2);
     EG_ALLOC(c->cons_partials, (size_t)c->tiles_fused.n_tiles + 1);
     if (c->topk.enabled) {
         EG_ALLOC(c->tk.hist, S * kMaxBins);
@@ -634,7 +636,8 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     // a4: Top-K select / pack / deliver for the segments that send a sparse message
     if (c->topk.enabled && !small) {
         TimedSection ts(c, stream, EG_KERNEL_TOPK);
-        TopkArgs ta{params, c->xhat, tn, S, c->T, c->stride, c->st.sparse, c->tk, c->err};
+        TopkArgs ta{params, c->xhat, tn, S, c->T, c->stride, c->st.sparse, c->tk, c->err, c->st.sparse_steps,
+                    c->step_k};
         if (c->topk_coop_grid > 0) {
             void* args[] = {&ta};
             EG_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_topk_all, dim3(c->topk_coop_grid),
