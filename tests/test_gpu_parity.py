@@ -420,12 +420,16 @@ def test_checkpoint_roundtrip_and_reset():
 
 
 @pytest.mark.parametrize("numel", [[7, 3000], RAGGED[:-1], [5000]])
-@pytest.mark.parametrize("hist", [1, 3])
-def test_host_buffer_entry_point(numel, hist):
+@pytest.mark.parametrize("hist,mu", [(1, None), (3, None), (1, 0.9)])
+def test_host_buffer_entry_point(numel, hist, mu):
     """eg_step_host (host buffers; tensors pipelined in groups through the device when the
-    context allows it) gives the same iteration as eg_step on device buffers."""
+    context allows it) gives the same iteration as eg_step on device buffers, with and without
+    momentum (the velocities stay on the device)."""
     wl = W.synthetic(3, numel, steps=6, lr=0.1, grad_sigma=0.01, history_len=hist)
     a, b = B.from_workload(wl), B.from_workload(wl)
+    if mu is not None:
+        a.set_momentum(mu)
+        b.set_momentum(mu)
     x0 = a.to_layout(W.distinct_init_params(wl, "cuda"))
     xa, xb = x0.clone(), x0.cpu().pin_memory()
     for k in range(wl.steps):
@@ -436,6 +440,8 @@ def test_host_buffer_entry_point(numel, hist):
             assert np.array_equal(u, v)
     assert torch.equal(xa.cpu(), xb) and a.stats() == b.stats()
     assert torch.equal(a.mailboxes(), b.mailboxes())
+    if mu is not None:
+        assert torch.equal(a.velocity(), b.velocity()) and a.velocity().any()
     b.step(xa, g, wl.lr)        # a plain step afterwards covers all tensors again
     a.step(xa.clone(), g, wl.lr)
     assert a.stats() == b.stats()
