@@ -128,6 +128,28 @@ def test_random_option_combinations(seed):
     assert rep.params_bit_exact, case
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_random_momentum_and_kernel_choice_combinations(seed):
+    """Seeded draws over what momentum and the automatic kernel choice combine with: ring size,
+    tensor sizes, dense / Top-K, history, horizon, threshold bound, fixed thresholds, carried norm."""
+    rng = np.random.default_rng(5000 + seed)
+    P = int(rng.integers(1, 20))
+    sizes = [int(v) for v in rng.choice(RAGGED[:-1], size=int(rng.integers(1, 7)), replace=False)]
+    topk = [None, None, (1, 100), (1, 3)][int(rng.integers(0, 4))]
+    okw = dict(history_len=int(rng.integers(1, 5)), horizon=float(rng.choice([0.5, 1.0, 2.0])))
+    if rng.integers(0, 2):
+        okw["momentum"] = float(rng.choice([0.0, 0.5, 0.9, 0.99]))
+    if rng.integers(0, 4) == 0:
+        okw["threshold_cap"] = (1e-3, 0.8)
+    if rng.integers(0, 5) == 0:
+        okw.update(mode=1, delta_fixed=float(rng.choice([0.0, 0.01])), force_first_event=bool(rng.integers(0, 2)))
+    kernel = [B.FUSED_PIPELINED, B.FUSED_AUTO][int(rng.integers(0, 2))]
+    wl = W.synthetic(P, sizes, steps=14, lr=0.1, grad_sigma=0.01, topk=topk, seed=177 + seed)
+    rep = lockstep(wl, init="distinct", carry=bool(rng.integers(0, 2)), fused_kernel=kernel, oracle_kw=okw,
+                   outbox_samples=16)
+    assert rep.params_bit_exact, (P, sizes, topk, okw, kernel)
+
+
 def test_delivery_masks_enabled_mid_run_and_refusals():
     from oracle import eg_oracle as eo
     wl = W.synthetic(4, [5, 1000, 4097], steps=12, lr=0.1, grad_sigma=0.01)
