@@ -316,7 +316,44 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             double acc = 0.0;
 #pragma unroll
             for (int v = 0; v < COLS; ++v) {
-                if (nel[v] > 0) {
+                if (PLAIN && !ASYNC && !MOM && nel[v] == 4 && ul && ur) {
+                    // The common case -- a full float4, both neighbours heard from, default
+                    // readings -- as straight-line code: the same operations in the same order
+                    // as the general form below, without its per-element conditions.
+                    const int c = c0 + v * 4 * CONSUMERS;
+                    const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
+                    const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
+                    const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
+                    if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;
+                    hC[v][0] = (double)hnf.x; hC[v][1] = (double)hnf.y; hC[v][2] = (double)hnf.z; hC[v][3] = (double)hnf.w;
+                    double xd[4];
+                    if (cx) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) xd[q] = hB[v][q];
+                    } else {
+                        const float4 xf = *reinterpret_cast<const float4*>(st + c);
+                        xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
+                    }
+                    float4 xn4;
+                    xn4.x = __double2float_rn(__fma_rn(neg_lr, (double)gf.x,
+                                __dmul_rn(__dadd_rn(__dadd_rn(xd[0], hA[v][0]), hC[v][0]), w_third)));
+                    xn4.y = __double2float_rn(__fma_rn(neg_lr, (double)gf.y,
+                                __dmul_rn(__dadd_rn(__dadd_rn(xd[1], hA[v][1]), hC[v][1]), w_third)));
+                    xn4.z = __double2float_rn(__fma_rn(neg_lr, (double)gf.z,
+                                __dmul_rn(__dadd_rn(__dadd_rn(xd[2], hA[v][2]), hC[v][2]), w_third)));
+                    xn4.w = __double2float_rn(__fma_rn(neg_lr, (double)gf.w,
+                                __dmul_rn(__dadd_rn(__dadd_rn(xd[3], hA[v][3]), hC[v][3]), w_third)));
+                    st_stream(xo + v * 4 * CONSUMERS, xn4);
+                    if (sn) st_stream(ho + v * 4 * CONSUMERS, hcf);
+                    if (CARRY) {
+                        const float d0 = __fsub_rn(xn4.x, hcf.x), d1 = __fsub_rn(xn4.y, hcf.y);
+                        const float d2 = __fsub_rn(xn4.z, hcf.z), d3 = __fsub_rn(xn4.w, hcf.w);
+                        acc = __fma_rn((double)d0, (double)d0, acc);
+                        acc = __fma_rn((double)d1, (double)d1, acc);
+                        acc = __fma_rn((double)d2, (double)d2, acc);
+                        acc = __fma_rn((double)d3, (double)d3, acc);
+                    }
+                } else if (nel[v] > 0) {
                     const int c = c0 + v * 4 * CONSUMERS;
                     const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
                     const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
