@@ -4,8 +4,8 @@
 // how the operands reach the SM.  One producer thread streams the (x, g, x_hat) tiles of the
 // replicas, in ring order, into a ring of shared-memory stages with 1-D bulk asynchronous
 // copies (cp.async.bulk, completion on an mbarrier, no multicast), so the bytes in flight
-// are bounded by shared memory instead of registers; 8 consumer warps read their float4
-// column of two adjacent stages (replica j and the contribution of replica j+1; that of
+// are bounded by shared memory instead of registers; 4 consumer warps read their float4
+// columns (two per thread) of two adjacent stages (replica j and the contribution of replica j+1; that of
 // replica j-1 is carried in registers) and write the results straight to global memory.  Every thread always owns the same column, so the two wrap-around operands
 // (replica P-1 for replica 0, replica 0 for replica P-1) live in two extra shared buffers
 // that are private per column.
@@ -19,7 +19,8 @@
 namespace eg {
 
 #ifndef EG_PIPE_CONSUMERS
-#define EG_PIPE_CONSUMERS 256
+#define EG_PIPE_CONSUMERS 128   // two float4 columns per consumer thread: the per-replica control
+                                // flow is paid once per eight elements (256 measured 0-3 % slower)
 #endif
 #ifndef EG_PIPE_STAGES
 #define EG_PIPE_STAGES 5
@@ -201,9 +202,11 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         // replica's stage): once a stage has been released, its slot is complete.
         const int pl = tid - CONSUMERS;
         auto reduce_slot = [&](int slot, int j) {
-            static_assert(CWARPS == 8, "a slot holds 64 values: two per lane");
+            static_assert(CWARPS == 8 || CWARPS == 4 || CWARPS == 2, "a slot holds 64, 32 or 16 values");
             const double* sp = s_part + slot * (CWARPS * 8);
-            double r = __dadd_rn(sp[pl], sp[32 + pl]);
+            double r = (CWARPS == 8) ? __dadd_rn(sp[pl], sp[32 + pl])
+                                     : ((CWARPS == 4 || pl < 16) ? sp[pl & (CWARPS * 8 - 1)] : 0.0);
+            if (CWARPS == 2 && pl >= 16) r = 0.0;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) r = __dadd_rn(r, __shfl_xor_sync(0xffffffffu, r, o));
             if (pl == 0) partials[(long long)j * tt.n_tiles + tile] = r;
