@@ -329,15 +329,24 @@ def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_varian
         eg.set_timing(False)
         for k in range(Wm):
             eg.step(x, grads[k % n_buf], wl.lr)
+        # pass 1, the timed region of `value`: K steps between two events, nothing in between
+        x.copy_(x0)
+        eg.reset()
+        eg.set_carry_norm(variant == "carry")
+        eg.set_timing(False)
+        ms, launches = time_steps(eg, x, grads, wl.lr, K,
+                                  sampler if (sampler and variant == sampled_variant) else None)
+        stats = eg.stats()
+        units, ms_max = aggregate(float(elems) * K, ms, dev)
+        # pass 2, the same K steps with a pair of events around every kernel group (the events
+        # keep a kernel from starting under the tail of the one before it, so this pass is a
+        # little slower than pass 1): per-kernel durations for the roofline
         x.copy_(x0)
         eg.reset()
         eg.set_carry_norm(variant == "carry")
         eg.set_timing(True)
-        ms, launches = time_steps(eg, x, grads, wl.lr, K,
-                                  sampler if (sampler and variant == sampled_variant) else None)
+        ms_instr, _ = time_steps(eg, x, grads, wl.lr, K, None)
         kt = eg.kernel_times()
-        stats = eg.stats()
-        units, ms_max = aggregate(float(elems) * K, ms, dev)
         # the same K steps once more with an event between steps: spread of the single steps
         # (the figures above come from the two outer events only)
         x.copy_(x0)
@@ -356,6 +365,7 @@ def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_varian
             "ms_per_step": ms_max / K, "gbs": units * (BYTES_PER_ELEMENT[variant] + extra) / ms_max / 1e6,
             "replica_steps_per_s": world * wl.P * K / (ms_max / 1e3), "launches": launches,
             "kernel_ms": {g: (v[0] / v[1] if v[1] else None) for g, v in kt.items()},
+            "ms_per_step_with_kernel_events": ms_instr / K,
             "messages_sent": stats["messages"], "bytes_sent": stats["bytes"],
             "pct_messages": 100.0 * stats["messages"] / (wl.P * wl.T * 2 * K),
             "gradient_buffers": n_buf, "cuda_graph": False,
@@ -472,6 +482,10 @@ def run_native(args):
                 "traffic": traffic,
                 "algorithmic_bytes_per_launch": elems * (FUSED_BYTES_PER_ELEMENT + extra),
                 "kernel_ms": fused_ms,
+                "kernel_timed_in": "a second pass over the same K steps with CUDA events around every kernel "
+                                   "group on the step's stream; the pass that gives `value` carries no events "
+                                   "between its kernels",
+                "ms_per_step_with_kernel_events": main["ms_per_step_with_kernel_events"],
                 "step_frac_of_peak": main["gbs"] / peak,
                 "step_frac_of_nominal_8TBs": main["gbs"] / NOMINAL_HBM_GBS}
 

@@ -49,6 +49,14 @@ struct Counters {                // device-resident, 64-bit
     unsigned long long messages, bytes, events, pad;
 };
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization
+// attribute may start while its predecessor in the stream is still running; pdl_wait() returns
+// once that predecessor has completed and its writes are visible (a no-op for an ordinary
+// launch), so everything before it must touch only data that no earlier kernel writes.
+// pdl_release() lets the next kernel of the stream start its own preamble early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float4 ld_stream(const float* p) {
     return __ldcs(reinterpret_cast<const float4*>(p));
 }

@@ -173,6 +173,9 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
     const long long off = tt.offset[tile];
     const uint32_t copy_bytes = (uint32_t)(((len + 3) & ~3) * 4);
 
+    // up to here only the tile table, which no kernel writes, has been read
+    pdl_release();
+    pdl_wait();
     for (int j = tid; j < P; j += CONSUMERS + 32) {
         const bool sn = snap[(long long)j * T + t] != 0;
         const bool ar = ASYNC ? (arrive[(long long)j * T + t] != 0) : sn;

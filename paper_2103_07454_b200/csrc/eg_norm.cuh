@@ -167,6 +167,8 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
          DecideParams dp, SegState st, const long long* __restrict__ numel,
          const long long* __restrict__ topk_count, int* __restrict__ outbox_count,
          Counters* ctr, const long long* __restrict__ step_k, DeliveryState dl) {
+    pdl_release();      // the kernel after this one may set itself up meanwhile
+    pdl_wait();         // the partial sums come from the kernel before this one
     const int lane = threadIdx.x & 31;
     // work item: (replica, tensor of the launch's range)
     const long long w = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);

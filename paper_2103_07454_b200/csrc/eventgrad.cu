@@ -243,6 +243,24 @@ eg_status sync_and_check(eg_ctx* c) {
 
 constexpr size_t kMaxTimedPairs = 1 << 15;
 
+// Launch with the programmatic-serialization attribute: the kernel may begin while its
+// predecessor in the stream finishes; it calls pdl_wait() before it depends on that kernel.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                       Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Brackets one kernel group with a pair of events when timing is on.
 struct TimedSection {
     eg_ctx* c;
@@ -627,10 +645,12 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         ++launches;
     } else {
         TimedSection ts(c, stream, EG_KERNEL_DECIDE);
-        k_decide<<<(c->P * tcount + kWarps - 1) / kWarps, kThreads, 0, stream>>>(
-            partials, tp.seg_begin, tp.n_tiles, dp, c->st, c->d_numel, c->d_kcount, c->outbox_count,
-            c->ctr, c->step_k,
-            DeliveryState{deliver_dev, c->pending, c->recv_valid, c->arrive, c->arrivals, c->async ? 1 : 0});
+        EG_CUDA(c, launch_pdl(k_decide, dim3((c->P * tcount + kWarps - 1) / kWarps), dim3(kThreads), 0, stream,
+                              partials, (const int*)tp.seg_begin, tp.n_tiles, dp, c->st,
+                              (const long long*)c->d_numel, (const long long*)c->d_kcount, c->outbox_count,
+                              c->ctr, (const long long*)c->step_k,
+                              DeliveryState{deliver_dev, c->pending, c->recv_valid, c->arrive, c->arrivals,
+                                            c->async ? 1 : 0}));
         ++launches;
     }
     // a4: Top-K select / pack / deliver for the segments that send a sparse message
@@ -694,15 +714,17 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                     partials_fused, step_k, c->err, c->vel, c->mu);
         } else if (c->fused_kind != EG_FUSED_REGISTER) {
             const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
-#define EG_PIPE_ARGS params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr, \
-                     partials_fused, step_k, c->err
+#define EG_PIPE_ARGS params, grads, c->xhat, (const uint8_t*)c->st.snap, valid, tf, c->P, c->T, \
+                     (long long)c->stride, lr, partials_fused, step_k, c->err
             if (c->variant == 0) {
+                // started while the kernel before it (the decision kernel, or the Top-K sequence)
+                // drains: it waits on the device before it reads anything that kernel writes
                 if (carry)
-                    k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>
-                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
+                    EG_CUDA(c, launch_pdl(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
+                                          dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
                 else
-                    k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>
-                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS);
+                    EG_CUDA(c, launch_pdl(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
+                                          dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
             } else {
                 if (carry)
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, true, false>
