@@ -199,7 +199,9 @@ enum { EG_FUSED_PIPELINED = 0, EG_FUSED_REGISTER = 1, EG_FUSED_AUTO = 2 };
 eg_status eg_set_fused_kernel(eg_ctx* ctx, int kind);
 
 /* Per-kernel timing for measurements (off by default).  When on, eg_step brackets each
- * kernel group with a pair of CUDA events recorded on the step's own stream; eg_kernel_times
+ * kernel group with a pair of CUDA events recorded on the step's own stream (and launches the
+ * kernels one strictly after the other, so that every duration is the kernel's own: a step is
+ * then a few percent slower than without timing); eg_kernel_times
  * synchronises, adds up the elapsed milliseconds per group since the last call into
  * ms_host[EG_KERNEL_GROUPS], the number of timed sections into
  * sections_host[EG_KERNEL_GROUPS], and forgets them.  At most 32768 sections are kept

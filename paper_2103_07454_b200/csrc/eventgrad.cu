@@ -246,8 +246,8 @@ constexpr size_t kMaxTimedPairs = 1 << 15;
 // Launch with the programmatic-serialization attribute: the kernel may begin while its
 // predecessor in the stream finishes; it calls pdl_wait() before it depends on that kernel.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                       Args... args) {
+cudaError_t launch_pdl(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -257,7 +257,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = overlap ? 1 : 0;   // per-kernel timing wants every kernel's duration to be its own
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -645,7 +645,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         ++launches;
     } else {
         TimedSection ts(c, stream, EG_KERNEL_DECIDE);
-        EG_CUDA(c, launch_pdl(k_decide, dim3((c->P * tcount + kWarps - 1) / kWarps), dim3(kThreads), 0, stream,
+        EG_CUDA(c, launch_pdl(!c->timing, k_decide, dim3((c->P * tcount + kWarps - 1) / kWarps), dim3(kThreads), 0, stream,
                               partials, (const int*)tp.seg_begin, tp.n_tiles, dp, c->st,
                               (const long long*)c->d_numel, (const long long*)c->d_kcount, c->outbox_count,
                               c->ctr, (const long long*)c->step_k,
@@ -720,10 +720,10 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                 // started while the kernel before it (the decision kernel, or the Top-K sequence)
                 // drains: it waits on the device before it reads anything that kernel writes
                 if (carry)
-                    EG_CUDA(c, launch_pdl(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
+                    EG_CUDA(c, launch_pdl(!c->timing, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
                                           dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
                 else
-                    EG_CUDA(c, launch_pdl(k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
+                    EG_CUDA(c, launch_pdl(!c->timing, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
                                           dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
             } else {
                 if (carry)
