@@ -111,7 +111,7 @@ typedef struct ego_ctx {
     int own_last_sent;    /* 1: the replica's own term of the average is x_hat_i, i.e.
                              Eq. (dist_sgd_event) read literally (X_hat W) */
     int change_of_norm;   /* 1: the tested quantity is | ||x|| - ||x|| at the last event |
-                             ("the norm of a parameter has changed by some threshold") */
+                             (the change-of-norm reading of the prose of Section 4) */
     double *sent_norm;    /* [P*T] ||x|| at the last event (0 before the first) */
     int hops;             /* ring neighbours on each side (1 = the paper's ring) */
     /* intermittent delivery (Section 7 remarks on the "stochastic nature of the MPI one-sided
@@ -123,6 +123,8 @@ typedef struct ego_ctx {
     uint64_t arrivals;
     double cap_alpha, cap_beta; /* bound g(k) = alpha * beta^k on the squared threshold
                                    (Assumption 1, Corollary 2); alpha <= 0: no bound */
+    double cap_g;               /* g(k) of the current iteration, carried as the geometric
+                                   sequence it is: g(0) = alpha, g(k+1) = beta * g(k) */
     /* heavy-ball momentum (an extension to another training algorithm, Introduction) */
     float *vel;           /* [P][N] velocity of every replica, fp32 like the parameters; NULL: off */
     double mu;            /* momentum coefficient */
@@ -141,6 +143,7 @@ void ego_destroy(ego_ctx *c) {
 void ego_reset(ego_ctx *c) {
     int64_t S = (int64_t)c->P * c->T;
     c->k = 0;
+    c->cap_g = c->cap_alpha;
     c->messages = c->bytes = c->events = 0;
     c->arrivals = 0;
     if (c->mailbox) {
@@ -225,9 +228,14 @@ void ego_set_variant(ego_ctx *c, int own_last_sent, int change_of_norm) {
     c->change_of_norm = change_of_norm != 0;
 }
 
+/* Bound sqrt(g(k)) on the thresholds, g the geometric sequence of Corollary 2 with first term
+ * alpha and ratio beta.  The sequence is evaluated term by term (one multiplication per
+ * iteration); set in the middle of a run it starts from the term of the current iteration. */
 void ego_set_threshold_cap(ego_ctx *c, double alpha, double beta) {
     c->cap_alpha = alpha;
     c->cap_beta = beta;
+    c->cap_g = alpha;
+    for (int64_t q = 0; q < c->k; ++q) c->cap_g = c->cap_g * beta;
 }
 
 int ego_set_hops(ego_ctx *c, int hops) {
@@ -328,7 +336,7 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
      * g(k) = alpha * beta^k of Corollary 2) */
     double thr = c->delta[s];
     if (c->cap_alpha > 0.0) {
-        const double cap = sqrt(c->cap_alpha * pow(c->cap_beta, (double)c->k));
+        const double cap = sqrt(c->cap_g);
         if (cap < thr) thr = cap;
     }
     c->norm[s] = d;
@@ -485,6 +493,7 @@ void ego_step_masked(ego_ctx *c, float *x, const float *g, float lr, const uint8
         phase_b_segment(c, x, g, lr, (int)(s / c->T), (int)(s % c->T));
 
     c->k += 1;
+    if (c->cap_alpha > 0.0) c->cap_g = c->cap_g * c->cap_beta; /* g(k+1) = beta * g(k) */
 }
 
 void ego_step(ego_ctx *c, float *x, const float *g, float lr) { ego_step_masked(c, x, g, lr, NULL); }
@@ -510,6 +519,7 @@ const int *ego_history_len(const ego_ctx *c) { return c->hist_len; }
 float *ego_xhat(ego_ctx *c) { return c->xhat; }
 float *ego_received(ego_ctx *c) { return c->mailbox ? c->mailbox : c->xhat; }
 const uint8_t *ego_pending(const ego_ctx *c) { return c->pending; }
+const uint8_t *ego_received_once(const ego_ctx *c) { return c->mailbox ? c->recv_valid : c->valid; }
 uint64_t ego_arrivals(const ego_ctx *c) { return c->arrivals; }
 int64_t ego_topk_count(const ego_ctx *c, int t) { return c->Kt[t]; }
 int32_t ego_outbox(const ego_ctx *c, int i, int t, const int32_t **idx, const float **val) {

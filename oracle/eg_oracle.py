@@ -59,6 +59,8 @@ def _load():
         lib.ego_received.argtypes = [C.c_void_p]
         lib.ego_pending.restype = C.c_void_p
         lib.ego_pending.argtypes = [C.c_void_p]
+        lib.ego_received_once.restype = C.c_void_p
+        lib.ego_received_once.argtypes = [C.c_void_p]
         lib.ego_arrivals.restype = C.c_uint64
         lib.ego_arrivals.argtypes = [C.c_void_p]
         lib.ego_stats.argtypes = [C.c_void_p] + [C.POINTER(C.c_uint64)] * 3
@@ -135,6 +137,10 @@ class Oracle:
     def reset(self):
         self._lib.ego_reset(self._h)
 
+    def set_threshold_cap(self, alpha: float, beta: float):
+        """Bound sqrt(alpha * beta^k) on the thresholds from the current iteration on."""
+        self._lib.ego_set_threshold_cap(self._h, float(alpha), float(beta))
+
     def set_threads(self, n: int):
         self._lib.ego_set_threads(self._h, int(n))
 
@@ -164,6 +170,10 @@ class Oracle:
         if not p:
             return np.zeros((self.P, self.T), np.uint8)
         return _view(p, np.uint8, self.S).reshape(self.P, self.T).copy()
+
+    def received_once(self):
+        """Per (replica, tensor): the neighbours have received this tensor at least once."""
+        return _view(self._lib.ego_received_once(self._h), np.uint8, self.S).reshape(self.P, self.T).copy()
 
     @property
     def arrivals(self) -> int:

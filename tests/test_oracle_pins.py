@@ -310,6 +310,36 @@ def test_geometric_bound_on_the_threshold():
     assert fired == [0, 1, 0, 0, 1]
 
 
+def test_geometric_bound_stays_on_the_exact_sequence():
+    """The bound is carried as the geometric sequence it is, g(0) = alpha, g(k+1) = beta g(k), one
+    rounding per term.  Against alpha * beta^k in exact rational arithmetic (a double is a dyadic
+    rational) the k-th term is off by at most k roundings; the tested threshold is its square
+    root.  A bound that is set at iteration k0 continues with the k0-th term of the sequence."""
+    from fractions import Fraction
+    alpha, beta, steps = 3.7, 0.93, 60
+    o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=float("inf"), force_first_event=False,
+                  threshold_cap=(alpha, beta))
+    late = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=float("inf"), force_first_event=False)
+    x = np.ones((1, 2), np.float32)
+    exact = Fraction(alpha)
+    for k in range(steps):
+        if k == 17:
+            late.set_threshold_cap(alpha, beta)
+        o.step(x, np.zeros_like(x), 1.0)
+        late.step(x.copy(), np.zeros_like(x), 1.0)
+        thr = o.thresholds_used()[0, 0]
+        rel = abs(Fraction(thr) ** 2 / exact - 1)
+        assert rel <= (k + 2) * 2.0 ** -52, (k, float(rel))
+        if k >= 17:
+            assert late.thresholds_used()[0, 0] == thr
+        else:
+            assert late.thresholds_used()[0, 0] == float("inf")
+        exact *= Fraction(beta)
+    o.reset()
+    o.step(x, np.zeros_like(x), 1.0)
+    assert o.thresholds_used()[0, 0] == np.sqrt(alpha)
+
+
 def test_fixed_threshold_never_adapts():
     o = eo.Oracle(1, [2], mode=eo.FIXED, delta_fixed=2.0, force_first_event=False)
     x = np.zeros((1, 2), np.float32)
