@@ -33,7 +33,10 @@
  *    calls that read results back (eg_stats, eg_last_*, eg_export_state, eg_step_host)
  *    synchronise that stream.
  *  - One context belongs to one device (the one current at eg_create) and is used from one
- *    stream at a time.
+ *    stream at a time: eg_step on another stream than the previous step's, while that stream
+ *    still has unfinished work, returns EG_ERR_STATE (synchronise it first, or order the two
+ *    streams and wait).  Ordering against the caller's other work on the stream is the
+ *    caller's job.
  *  - Every function returns an eg_status; nothing throws, aborts or traps.  A device-side
  *    problem (an index outside its table, a bounded wait that ran out) sets an error word that
  *    the next synchronising call returns as EG_ERR_INTERNAL or EG_ERR_TIMEOUT.
@@ -96,7 +99,8 @@ typedef struct {
 eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_numel, int T,
                     const eg_threshold_params* thr, const eg_topk_params* topk);
 
-/* Layout chosen by the library: tensor_offset_host[T] (elements, within one replica) and
+/* Layout chosen by the library for the parameters of one replica (the N parameters every PE
+ * holds, Section 3): tensor_offset_host[T] (elements, within one replica) and
  * *replica_stride_host (elements).  Either pointer may be NULL. */
 eg_status eg_layout(const eg_ctx* ctx, int64_t* tensor_offset_host, int64_t* replica_stride_host);
 
@@ -129,8 +133,8 @@ eg_status eg_set_carry_norm(eg_ctx* ctx, int enabled);
  *                 taken literally.
  *  trigger_metric EG_TRIGGER_NORM_OF_CHANGE (default): d = || x - x_hat || (the displayed
  *                 trigger condition).  EG_TRIGGER_CHANGE_OF_NORM: d = | ||x|| - ||x at the
- *                 last event|| | (Section 4 prose: "when the norm of a particular parameter
- *                 has changed by some threshold"); the norm pass then reads x only.
+ *                 last event|| | (the change-of-norm reading of the prose of Section 4); the
+ *                 norm pass then reads x only.
  * Allowed before the first step of a context or right after eg_reset (EG_ERR_STATE later). */
 enum { EG_OWN_CURRENT = 0, EG_OWN_LAST_SENT = 1 };
 enum { EG_TRIGGER_NORM_OF_CHANGE = 0, EG_TRIGGER_CHANGE_OF_NORM = 1 };
@@ -148,7 +152,7 @@ eg_status eg_set_variant(eg_ctx* ctx, int own_term, int trigger_metric);
  * eg_step) delivers everything outstanding.  eg_enable_delivery_masks allocates the second
  * copy (P*replica_stride floats) and synchronises; everything sent until then counts as
  * arrived.  Not available together with EG_OWN_LAST_SENT, the carried norm is not used while
- * it is on, and a context with it enabled cannot be checkpointed (EG_ERR_STATE).
+ * it is on.
  * eg_read_received copies the received copies to the host ([P][replica_stride] fp32; equal to
  * eg_read_mailboxes under synchronous delivery); eg_delivery_status returns the per-(replica,
  * tensor) "in flight" flags (host, P*T bytes) and the number of arrivals so far. */
@@ -160,10 +164,12 @@ eg_status eg_delivery_status(eg_ctx* ctx, uint8_t* pending_host, uint64_t* arriv
 
 /* Bound on the thresholds (Assumption 1 of Section 5, with the geometric sequence
  * g(k) = alpha * beta^k of Corollary 2): the threshold a tensor is tested against in iteration
- * k becomes min(delta, sqrt(alpha * beta^k)); the adaptive delta itself is left as computed.
- * alpha <= 0 removes the bound (default).  The bound of a step is evaluated on the host when
- * eg_step is called (from the host's copy of the iteration counter) and passed to the device
- * as a kernel argument. */
+ * k becomes min(delta, sqrt(g(k))); the adaptive delta itself is left as computed.
+ * alpha <= 0 removes the bound (default).  g lives on the device and is carried as the geometric
+ * sequence it is -- g(0) = alpha, g(k+1) = beta * g(k), one fp64 multiplication per iteration,
+ * made by the kernels of the step -- so a step recorded into a CUDA graph keeps the right bound
+ * on every replay.  The call synchronises the context's stream and starts the sequence at the
+ * term of the iteration the context has reached; eg_reset restarts it at alpha. */
 eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
 
 /* Heavy-ball momentum.  The Introduction says that event-triggered communication extends to
@@ -177,10 +183,9 @@ eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
  * (EG_ERR_INVALID otherwise).  Available with the default readings on the nearest-neighbour ring
  * and the default kernel choice, dense or Top-K (EG_ERR_STATE with eg_set_variant choices,
  * EG_TOPO_RING_HOPS(m > 1), intermittent delivery or EG_FUSED_REGISTER).  enabled = 0 returns to
- * the plain update and keeps the buffer.  The velocity is optimizer state like the parameters
- * themselves and not part of eg_export_state: eg_read_velocity / eg_write_velocity copy it to /
- * from a host buffer of P*replica_stride floats (both synchronise; EG_ERR_STATE before the
- * first enabling call). */
+ * the plain update and keeps the buffer.  The velocities are part of eg_export_state once the
+ * buffer exists; eg_read_velocity / eg_write_velocity copy them to / from a host buffer of
+ * P*replica_stride floats (both synchronise; EG_ERR_STATE before the first enabling call). */
 eg_status eg_set_momentum(eg_ctx* ctx, int enabled, double mu);
 eg_status eg_read_velocity(eg_ctx* ctx, float* velocity_host);
 eg_status eg_write_velocity(eg_ctx* ctx, const float* velocity_host);
@@ -216,8 +221,9 @@ eg_status eg_kernel_times(eg_ctx* ctx, double* ms_host, uint64_t* sections_host)
 eg_status eg_stats(eg_ctx* ctx, uint64_t* messages_sent_host, uint64_t* bytes_sent_host);
 eg_status eg_event_count(eg_ctx* ctx, uint64_t* events_host);
 
-/* Decisions of the most recent step, host arrays of P*T entries indexed [i*T + t]:
- * flags (1 = event), norms (d), thresholds (the delta that d was compared with).
+/* Decisions of the most recent step (trigger condition of Section 4), host arrays of P*T
+ * entries indexed [i*T + t]: flags (1 = event), norms (d), thresholds (the delta that d was
+ * compared with).
  * Any pointer may be NULL.  Synchronises. */
 eg_status eg_last_decisions(eg_ctx* ctx, uint8_t* flags_host, double* norms_host,
                             double* thresholds_host);
@@ -236,8 +242,8 @@ eg_status eg_topk_count(const eg_ctx* ctx, int t, int64_t* k_t_host);
 /* Copies the mailboxes x_hat ([P][replica_stride] fp32) into a host buffer. Synchronises. */
 eg_status eg_read_mailboxes(eg_ctx* ctx, float* xhat_host);
 
-/* After training: the model averaged over all replicas ("Obtain averaged model from all
- * PEs", last line of Algorithms A and B): avg_dev[e] = (1/P) sum_i params[i][e] for every
+/* After training: the model averaged over all replicas (the final averaging step of
+ * Algorithms A and B): avg_dev[e] = (1/P) sum_i params[i][e] for every
  * element of the replica layout (device buffer of replica_stride floats), fp64 sum in
  * ascending i, rounded once.  consensus_host, if not NULL, receives
  * sum_i || x_i - mean ||^2 (the consensus distance bounded in the appendix) and makes the
@@ -246,9 +252,13 @@ eg_status eg_average_model(eg_ctx* ctx, const float* params, float* avg_dev,
                            double* consensus_host, void* stream);
 
 /* Checkpoint: eg_export_state with host_buf == NULL stores the needed size in *bytes;
- * otherwise writes the state (iteration counter, counters, trigger state, mailboxes) and
- * the size.  eg_import_state restores it into a context created with the same arguments
- * (EG_ERR_INVALID otherwise). */
+ * otherwise writes the state and the size: iteration counter, counters, trigger state (Eq.
+ * (thres): thresholds, last-event iterations, slope histories), mailboxes, and, where the
+ * context has them, the delivery state (received copies, what is in flight, arrival count) and
+ * the velocities.  eg_import_state restores it into a context created with the same arguments
+ * and configured alike -- ring size, tensors, neighbourhood, threshold parameters, Top-K
+ * fraction, readings (eg_set_variant), threshold bound, delivery masks enabled or not,
+ * momentum buffer and coefficient -- and returns EG_ERR_INVALID otherwise. */
 eg_status eg_export_state(eg_ctx* ctx, void* host_buf, size_t* bytes);
 eg_status eg_import_state(eg_ctx* ctx, const void* host_buf, size_t bytes);
 
@@ -272,7 +282,8 @@ eg_status eg_import_state(eg_ctx* ctx, const void* host_buf, size_t bytes);
  * `stream` and returns; it never synchronises.
  *
  * Limits, checked before anything is launched (EG_ERR_INVALID): T <= EG_STATIC_MAX_TENSORS,
- * and P * sum_t ceil(n_t / 4096) <= EG_STATIC_MAX_PARTIALS.
+ * P <= 65535, every tensor inside its replica (offset + n_t <= replica_stride), and
+ * P * sum_t ceil(n_t / 4096) <= EG_STATIC_MAX_PARTIALS.
  *
  * The first call on each device looks up the device address of the scratch array (a runtime
  * query, no allocation); make that first call outside any stream capture.  All calls on one
@@ -294,7 +305,8 @@ eg_status eg_change_norms_static(const float* x_dev, const float* xhat_dev, int 
  * EG_ERR_TIMEOUT until eg_reset clears the error word.  The context stays usable. */
 eg_status eg_selftest_wait_timeout(eg_ctx* ctx, void* stream);
 
-/* Back to iteration 0 with empty mailboxes, initial thresholds and zero counters. */
+/* Back to iteration 0 of Algorithm B: empty mailboxes (X_0 = 0, Assumption 2), initial
+ * thresholds, zero counters, zero velocities, the threshold bound back at its first term. */
 eg_status eg_reset(eg_ctx* ctx);
 void eg_destroy(eg_ctx* ctx);
 
@@ -307,6 +319,16 @@ void eg_debug_fail_allocation(int nth);
 /* Tracing: with EG_NVTX set (to anything but 0) in the environment when a context is created,
  * eg_step wraps the launches of every kernel group in a named NVTX range ("eventgrad:norm",
  * ":decide", ":topk", ":fused"); without a profiler attached the ranges cost nothing. */
+
+/* Device-side checks.  Kernels never trap: a problem found on the device sets a bit of the
+ * context's error word, the affected access is skipped, and the next call that synchronises
+ * returns eg_status_of_error_word(word): EG_ERR_TIMEOUT when a bounded wait ran out (bit 8),
+ * EG_ERR_INTERNAL when a Top-K entry pointed outside its message (bit 2) or -- in the
+ * bounds-checked build of the library, compiled with -DEG_DEBUG (eg_debug_build() == 1) -- when
+ * an index left its table (bit 4: tile records, per-replica modes, pipeline stages, partial sums,
+ * entry slots are all checked before use there); EG_OK for 0.  eg_reset clears the word. */
+eg_status eg_status_of_error_word(unsigned int word);
+int eg_debug_build(void);
 
 const char* eg_strerror(eg_status s);
 /* cudaError_t of the most recent failed CUDA call of this context (0 if none). */

@@ -29,7 +29,7 @@ EXPORTS = [
     "eg_set_timing", "eg_kernel_times", "eg_set_fused_kernel", "eg_change_norms_static", "eg_set_variant", "eg_set_threshold_cap",
     "eg_enable_delivery_masks", "eg_step_masked", "eg_read_received", "eg_delivery_status",
     "eg_selftest_wait_timeout", "eg_set_momentum", "eg_read_velocity", "eg_write_velocity",
-    "eg_debug_fail_allocation",
+    "eg_debug_fail_allocation", "eg_status_of_error_word", "eg_debug_build",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -104,6 +104,8 @@ def load_library() -> C.CDLL:
     lib.eg_destroy.restype = None
     lib.eg_strerror.argtypes = [C.c_int]
     lib.eg_strerror.restype = C.c_char_p
+    lib.eg_status_of_error_word.argtypes = [C.c_uint]
+    lib.eg_debug_build.argtypes = []
     lib.eg_last_cuda_error.argtypes = [vp]
     lib.eg_last_launch_count.argtypes = [vp]
     _lib = lib
@@ -272,9 +274,13 @@ class EventGrad:
                                                    C.byref(n)), self._h, "eg_last_outbox")
         return idx[:n.value].copy(), val[:n.value].copy()
 
-    def mailboxes(self) -> torch.Tensor:
-        """Host copy of x_hat in the library's layout ``[P, replica_stride]``."""
-        out = torch.empty((self.P, self.replica_stride), dtype=torch.float32)
+    def mailboxes(self, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Host copy of x_hat in the library's layout ``[P, replica_stride]`` (into ``out``, a
+        contiguous fp32 host tensor of that shape, when given)."""
+        if out is None:
+            out = torch.empty((self.P, self.replica_stride), dtype=torch.float32)
+        assert (not out.is_cuda and out.dtype == torch.float32 and out.is_contiguous()
+                and out.shape == (self.P, self.replica_stride))
         _check(self._lib, self._lib.eg_read_mailboxes(self._h, out.data_ptr()), self._h,
                "eg_read_mailboxes")
         return out

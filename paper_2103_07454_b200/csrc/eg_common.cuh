@@ -22,7 +22,40 @@ struct TileTable {
     const int* length;           // [n_tiles] elements in the tile
     const int* seg_begin;        // [T+1] first tile of every tensor
     int n_tiles;
+    unsigned int* err;           // the context's error word (bounds-checked build)
 };
+
+// Bits of a context's error word (set by kernels, read by the calls that synchronise).
+constexpr unsigned kErrTopkSlot = 2u;      // a Top-K entry pointed outside its message or tile
+constexpr unsigned kErrBounds = 4u;        // bounds-checked build: an index left its table
+constexpr unsigned kErrWaitTimeout = 8u;   // a bounded wait on a shared-memory barrier ran out
+
+// Bounds-checked build (-DEG_DEBUG): every index a kernel forms into a table -- tile records,
+// per-replica modes, pipeline stages, partial sums, entry slots -- is compared with the table's
+// size first.  A miss sets kErrBounds in the error word and the access is skipped; nothing traps.
+// In the normal build the checks compile to nothing.
+#ifdef EG_DEBUG
+__device__ __forceinline__ bool index_ok(unsigned int* err, long long idx, long long n) {
+    if (idx >= 0 && idx < n) return true;
+    if (err) atomicOr(err, kErrBounds);
+    return false;
+}
+#define EG_INDEX_OK(err, idx, n) ::eg::index_ok((err), (long long)(idx), (long long)(n))
+#else
+#define EG_INDEX_OK(err, idx, n) true
+#endif
+
+// The record of tile `tile` lies inside its table and describes elements inside one replica.
+__device__ __forceinline__ bool tile_ok(const TileTable& tt, int tile, int T, long long stride, int tile_elems) {
+#ifdef EG_DEBUG
+    if (!EG_INDEX_OK(tt.err, tile, tt.n_tiles)) return false;
+    return EG_INDEX_OK(tt.err, tt.tensor[tile], T) && EG_INDEX_OK(tt.err, tt.length[tile] - 1, tile_elems) &&
+           EG_INDEX_OK(tt.err, tt.offset[tile] + tt.length[tile] - 1, stride);
+#else
+    (void)tt; (void)tile; (void)T; (void)stride; (void)tile_elems;
+    return true;
+#endif
+}
 
 // Per-(replica, tensor) trigger state and the decisions of the current step, all [P*T].
 struct SegState {

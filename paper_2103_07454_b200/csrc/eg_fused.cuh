@@ -58,6 +58,7 @@ k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ 
     double* s_red = reinterpret_cast<double*>(smem + ((2 * P + 15) & ~15));
 
     const int tile = blockIdx.x, tid = threadIdx.x;
+    if (!tile_ok(tt, tile, T, stride, kThreads * 4 * VPT)) return;   // bounds-checked build only
     const int t = tt.tensor[tile];
     const int len = tt.length[tile];
     const long long off = tt.offset[tile];
@@ -123,6 +124,7 @@ k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ 
             for (int v = 0; v < VPT; ++v) { x_nxt[v] = g_nxt[v] = zero4; h_nxt[v] = h_first[v]; }
         }
         const int jl = (j == 0) ? P - 1 : j - 1, jr = (j + 1 == P) ? 0 : j + 1;
+        if (!EG_INDEX_OK(tt.err, jl, P) || !EG_INDEX_OK(tt.err, jr, P)) break;
         const bool ul = has_left && s_valid[jl] != 0;
         const bool ur = has_right && s_valid[jr] != 0;
         const double w = __ddiv_rn(1.0, (double)(1 + (ul ? 1 : 0) + (ur ? 1 : 0)));

@@ -34,6 +34,7 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
     __shared__ double s_w[2 * kMaxHops + 1];                      // 1 / (1 + number heard from)
 
     const int tile = blockIdx.x, tid = threadIdx.x;
+    if (!tile_ok(tt, tile, T, stride, kThreads * 4)) return;     // bounds-checked build only
     const int t = tt.tensor[tile];
     const int len = tt.length[tile];
     const long long off = tt.offset[tile];
@@ -180,6 +181,7 @@ k_fused_hops_staged(float* x, const float* __restrict__ g, float* xhat,
     __shared__ double s_w[2 * M + 1];         // 1 / (1 + number heard from)
 
     const int tile = blockIdx.x, tid = threadIdx.x;
+    if (!tile_ok(tt, tile, T, stride, kThreads * 4)) return;     // bounds-checked build only
     const int t = tt.tensor[tile];
     const int len = tt.length[tile];
     const long long off = tt.offset[tile];

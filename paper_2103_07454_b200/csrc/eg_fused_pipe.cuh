@@ -30,7 +30,6 @@ constexpr int kPipeStages = EG_PIPE_STAGES;
 constexpr int kPipeConsumers = EG_PIPE_CONSUMERS; // consumer threads (+ one producer warp)
 constexpr int kPipeThreads = kPipeConsumers + 32;
 constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
-constexpr unsigned kErrPipeTimeout = 8u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -90,7 +89,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
         if (*s_abort) return false;
         if (clock64() - t0 > limit_cycles) {
             *s_abort = 1;
-            atomicOr(err, kErrPipeTimeout);
+            atomicOr(err, kErrWaitTimeout);
             return false;
         }
     }
@@ -168,6 +167,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
     double* s_part = reinterpret_cast<double*>(s_mode + ((P + 15) & ~15));   // [STAGES][CWARPS * 8]
 
     const int tile = blockIdx.x, tid = threadIdx.x;
+    if (!tile_ok(tt, tile, T, stride, TILE)) return;       // bounds-checked build only; the same in every thread
     const int t = tt.tensor[tile];
     const int len = tt.length[tile];
     const long long off = tt.offset[tile];
@@ -212,7 +212,8 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             if (CWARPS == 2 && pl >= 16) r = 0.0;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) r = __dadd_rn(r, __shfl_xor_sync(0xffffffffu, r, o));
-            if (pl == 0) partials[(long long)j * tt.n_tiles + tile] = r;
+            if (pl == 0 && EG_INDEX_OK(err, j, P) && EG_INDEX_OK(err, slot, STAGES))
+                partials[(long long)j * tt.n_tiles + tile] = r;
         };
         if (CARRY || tid == CONSUMERS) {
             const float* xp = x + off;
@@ -236,7 +237,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     if (!alive) break;
                     if (CARRY) reduce_slot(s, j - STAGES);     // before the stage is filled again
                 }
-                if (pl == 0) {
+                if (pl == 0 && EG_INDEX_OK(err, s, STAGES) && EG_INDEX_OK(err, j, P)) {
                     float* st = stages + s * (kArr * TILE);
                     const bool cx = (s_mode[j] & kCx) != 0;
                     const bool is_last = last_opt && (j == P - 1);
@@ -300,6 +301,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         auto one_replica = [&](const int j, double (&hA)[COLS][4], double (&hB)[COLS][4],
                                double (&hC)[COLS][4]) -> bool {
             const bool more = j + 1 < P;
+            if (!EG_INDEX_OK(err, s, STAGES) || !EG_INDEX_OK(err, s1, STAGES) || !EG_INDEX_OK(err, j, P)) return false;
             if (more) {
                 ok = mbar_wait_bounded(&full[s1], parity1, s_abort, err);
                 if (!ok) return false;

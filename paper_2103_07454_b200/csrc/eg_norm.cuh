@@ -28,6 +28,7 @@ k_norm_partial(const float* __restrict__ x, const float* __restrict__ xhat, Tile
                long long stride, double* __restrict__ partials, int variant) {
     __shared__ double s_warp[kWarps];
     const int tile = blockIdx.x, i = blockIdx.y;
+    if (!tile_ok(tt, tile, 0x7fffffff, stride, kNormTile)) return;   // bounds-checked build only
     const int len = tt.length[tile];
     const long long base = (long long)i * stride + tt.offset[tile];
     constexpr int kIter = kNormTile / (kThreads * 4);
@@ -61,8 +62,14 @@ struct DecideParams {
     int topk;                 // Top-K messages enabled
     int degree;               // distinct ring neighbours of every replica
     int variant;              // kChangeOfNorm: d = | sqrt(sum) - sent_norm |
-    double cap;               // bound sqrt(g(k)) on the threshold of this step (+inf: none)
+    // Bound sqrt(g(k)) on the threshold of a step (Assumption 1 with the geometric sequence
+    // g(k) = alpha * beta^k of Corollary 2).  The sequence lives on the device and advances
+    // with the iteration counter: iteration k reads cap_g[k & 1], the thread that opens the
+    // iteration's decisions writes beta * cap_g[k & 1] into the other slot.  nullptr: no bound.
+    double* cap_g;
+    double cap_beta;
     int t0, tn;               // tensors [t0, t0 + tn) are decided by this launch
+    unsigned int* err;        // the context's error word (bounds-checked build)
 };
 
 // Intermittent delivery: which outstanding messages arrive in this step.
@@ -94,15 +101,20 @@ __device__ __forceinline__ double segment_sum(const double* __restrict__ p, int 
     return acc;
 }
 
+// Bound on the thresholds of iteration k (+inf: none).
+__device__ __forceinline__ double iteration_cap(const DecideParams& dp, long long k) {
+    return dp.cap_g ? __dsqrt_rn(dp.cap_g[k & 1]) : __longlong_as_double(0x7ff0000000000000ll);
+}
+
 // The decision of segment s = (replica, tensor t) in iteration k from `acc`, the sum of its
 // partials: test, threshold update, message accounting, flags (one thread).
 __device__ __forceinline__ void
-decide_segment(double acc, long long s, int t, long long k, const DecideParams& dp, const SegState& st,
+decide_segment(double acc, long long s, int t, long long k, double cap, const DecideParams& dp, const SegState& st,
                const long long* __restrict__ numel, const long long* __restrict__ topk_count,
                int* __restrict__ outbox_count, Counters* ctr, const DeliveryState& dl) {
     const double root = __dsqrt_rn(acc);
     const double d = (dp.variant & kChangeOfNorm) ? fabs(__dsub_rn(root, st.sent_norm[s])) : root;
-    const double thr = fmin(st.delta[s], dp.cap);
+    const double thr = fmin(st.delta[s], cap);
     st.norm[s] = d;
     st.thr_used[s] = thr;
     const bool fire = (dp.force_first && k == 0) || (d >= thr);
@@ -115,6 +127,7 @@ decide_segment(double acc, long long s, int t, long long k, const DecideParams& 
             const double slope = __ddiv_rn(d, (double)(k - st.khat[s]));
             double* h = st.hist + s * dp.H;
             int n = st.hist_len[s];
+            if (!EG_INDEX_OK(dp.err, n, dp.H + 1)) n = dp.H;
             if (n == dp.H) {
                 for (int q = 1; q < dp.H; ++q) h[q - 1] = h[q];
                 n = dp.H - 1;
@@ -175,11 +188,17 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     if (w >= (long long)dp.P * dp.tn) return;
     const int i = (int)(w / dp.tn), t = dp.t0 + (int)(w % dp.tn);
     const long long s = (long long)i * dp.T + t;
+    if (!EG_INDEX_OK(dp.err, t, dp.T) || !EG_INDEX_OK(dp.err, seg_begin[t + 1] - 1, n_tiles) ||
+        !EG_INDEX_OK(dp.err, seg_begin[t], seg_begin[t + 1]))
+        return;                                               // bounds-checked build only
     const double acc = segment_sum(partials + (long long)i * n_tiles, seg_begin[t], seg_begin[t + 1], lane);
     if (lane != 0) return;
     const long long k = *step_k;
     if (w == 0 && st.sparse_steps) st.sparse_steps[(k + 1) & 1] = 0;   // the next iteration's count starts at zero
-    decide_segment(acc, s, t, k, dp, st, numel, topk_count, outbox_count, ctr, dl);
+    const double cap = iteration_cap(dp, k);
+    // next term of the sequence, once per iteration (the launch that holds tensor 0)
+    if (w == 0 && dp.t0 == 0 && dp.cap_g) dp.cap_g[(k + 1) & 1] = __dmul_rn(dp.cap_g[k & 1], dp.cap_beta);
+    decide_segment(acc, s, t, k, cap, dp, st, numel, topk_count, outbox_count, ctr, dl);
 }
 
 }  // namespace eg

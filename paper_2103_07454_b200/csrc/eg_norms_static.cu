@@ -100,13 +100,14 @@ extern "C" eg_status eg_change_norms_static(const float* x_dev, const float* xha
                                             const int64_t* layer_numel_host, int T, double* norms_dev,
                                             void* stream_v) {
     if (!x_dev || !xhat_dev || !tensor_offset_host || !layer_numel_host || !norms_dev) return EG_ERR_INVALID;
-    if (P < 1 || T < 1 || T > kStaticMaxTensors || replica_stride < 1) return EG_ERR_INVALID;
+    // P is the second grid dimension of the first kernel
+    if (P < 1 || P > 65535 || T < 1 || T > kStaticMaxTensors || replica_stride < 1) return EG_ERR_INVALID;
     if (((uintptr_t)x_dev & 15u) || ((uintptr_t)xhat_dev & 15u) || (replica_stride & 3)) return EG_ERR_INVALID;
     StaticTable tab;
     long long tiles = 0;
     for (int t = 0; t < T; ++t) {
         const int64_t n = layer_numel_host[t], o = tensor_offset_host[t];
-        if (n < 1 || n > 0x7fffffffll || o < 0 || (o & 3) || o + n > replica_stride) return EG_ERR_INVALID;
+        if (n < 1 || n > 0x7fffffffll || o < 0 || (o & 3) || o > replica_stride - n) return EG_ERR_INVALID;
         tab.offset[t] = o;
         tab.numel[t] = (int)n;
         tab.tile_begin[t] = (int)tiles;
@@ -131,10 +132,19 @@ extern "C" eg_status eg_change_norms_static(const float* x_dev, const float* xha
         scratch = g_scratch_addr[dev];
     }
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-    k_static_norm_partial<<<dim3((unsigned)tiles, (unsigned)P), kThreads, 0, stream>>>(
-        x_dev, xhat_dev, tab, (long long)replica_stride, (int)tiles, scratch);
+    // The status of each launch is taken from the launch itself, so that an error left behind
+    // by an unrelated earlier call is neither reported here nor cleared.
+    long long stride_ll = (long long)replica_stride;
+    int n_tiles = (int)tiles;
+    void* args1[] = {&x_dev, &xhat_dev, &tab, &stride_ll, &n_tiles, &scratch};
+    if (cudaLaunchKernel((const void*)k_static_norm_partial, dim3((unsigned)tiles, (unsigned)P), dim3(kThreads),
+                         args1, 0, stream) != cudaSuccess)
+        return EG_ERR_CUDA;          // the second kernel is not launched on stale partial sums
     const long long S = (long long)P * T;
-    k_static_norm_final<<<(unsigned)((S + kWarps - 1) / kWarps), kThreads, 0, stream>>>(
-        scratch, tab, P, (int)tiles, norms_dev);
-    return cudaGetLastError() == cudaSuccess ? EG_OK : EG_ERR_CUDA;
+    const double* scratch_c = scratch;
+    void* args2[] = {&scratch_c, &tab, &P, &n_tiles, &norms_dev};
+    if (cudaLaunchKernel((const void*)k_static_norm_final, dim3((unsigned)((S + kWarps - 1) / kWarps)),
+                         dim3(kThreads), args2, 0, stream) != cudaSuccess)
+        return EG_ERR_CUDA;
+    return EG_OK;
 }

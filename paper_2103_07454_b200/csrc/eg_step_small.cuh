@@ -64,11 +64,13 @@ k_step_small(float* __restrict__ x, const float* __restrict__ g, float* __restri
     double* s_red = reinterpret_cast<double*>(tail + 64);                // [P][kWarps]
 
     const int tile = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (!tile_ok(tt, tile, dp.T, stride, kSmallTile) || !EG_INDEX_OK(err, P - 1, PMAX)) return;   // bounds-checked build only
     const int t = tt.tensor[tile];
     const int len = tt.length[tile];
     const long long off = tt.offset[tile];
     const uint32_t copy_bytes = (uint32_t)(((len + 3) & ~3) * 4);
     const long long k = *step_k;
+    const double cap = iteration_cap(dp, k);
 
     if (tid == 0) {
         mbar_init(bar, 1);
@@ -105,6 +107,7 @@ k_step_small(float* __restrict__ x, const float* __restrict__ g, float* __restri
         p_in = (k & 1) ? sa.carried[1] : sa.carried[0]; p_stride = tt.n_tiles;
         q0 = r_fused.x; q1 = r_fused.y;
     }
+    if (!EG_INDEX_OK(err, q0, p_stride) || !EG_INDEX_OK(err, q1 - 1, p_stride)) return;   // ranges of partial sums
     double mine[(kSmallMaxP + kWarps - 1) / kWarps];     // lane 0: the sums this warp took
 #pragma unroll
     for (int r = 0; r < (kSmallMaxP + kWarps - 1) / kWarps; ++r) {
@@ -117,7 +120,7 @@ k_step_small(float* __restrict__ x, const float* __restrict__ g, float* __restri
             const double acc = segment_sum(p_in + (long long)j * p_stride, q0, q1, lane);
             mine[r] = acc;
             if (lane == 0) {
-                const bool fire = (dp.force_first && k == 0) || (__dsqrt_rn(acc) >= fmin(delta, dp.cap));
+                const bool fire = (dp.force_first && k == 0) || (__dsqrt_rn(acc) >= fmin(delta, cap));
                 s_mode[j] = (uint8_t)((fire ? 1 : 0) | ((fire || was_valid != 0) ? 2 : 0));
             }
         }
@@ -215,7 +218,7 @@ k_step_small(float* __restrict__ x, const float* __restrict__ g, float* __restri
             for (int r = 0; r < (kSmallMaxP + kWarps - 1) / kWarps; ++r) {
                 const int j = warp + r * kWarps;
                 if (j < P)
-                    decide_segment(mine[r], (long long)j * dp.T + t, t, k, dp, st, numel, nullptr, nullptr, ctr,
+                    decide_segment(mine[r], (long long)j * dp.T + t, t, k, cap, dp, st, numel, nullptr, nullptr, ctr,
                                    DeliveryState{nullptr, nullptr, nullptr, nullptr, nullptr, 0});
             }
         }
@@ -225,6 +228,7 @@ k_step_small(float* __restrict__ x, const float* __restrict__ g, float* __restri
     if (tid == 0) {
         __threadfence();
         if (atomicAdd(sa.done, 1) == (int)gridDim.x - 1) {   // last CTA of the launch
+            if (dp.cap_g) dp.cap_g[(k + 1) & 1] = __dmul_rn(dp.cap_g[k & 1], dp.cap_beta);
             *step_k = k + 1;
             *sa.done = 0;
         }

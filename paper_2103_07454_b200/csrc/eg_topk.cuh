@@ -10,9 +10,9 @@
 //                             in index order, into an entry buffer as (20 low key bits, position,
 //                             value of x); digit 1 of the undecided ones (top digit == b0) is
 //                             histogrammed on the way
-//   digit 2, per-tile counts, ordered compaction into the outbox and delivery into x_hat:
-//                             from the entries only (K_t plus the population of one bin: a few
-//                             percent of the tensor)
+//   digit 2 together with per-tile counts, then ordered compaction into the outbox and delivery
+//   into x_hat:               two walks over the entries only (K_t plus the population of one
+//                             bin: a few percent of the tensor)
 // so a sparse message costs two passes over its tensor.  The host knows nothing about the
 // decisions: a planning phase turns the device-side `sparse` flags into a compact list of work
 // tiles and every other phase runs a fixed-size grid over that list.  All phases can run in one
@@ -24,20 +24,20 @@
 
 namespace eg {
 
-constexpr int kTopkGrid = 148 * 8;      // CTAs of the tile kernels (they loop over the work list)
-constexpr int kTopkSegGrid = 148 * 4;   // CTAs of the per-segment kernels
+constexpr int kTopkCtasPerSm = 8;      // CTAs per multiprocessor of the tile kernels (they loop over the work list)
+constexpr int kTopkSegCtasPerSm = 4;   // ... of the per-segment kernels
 
 struct TopkPlan {
     int n_sparse;       // segments that send a sparse message in this step
     int total_tiles;    // their tiles
-    int chunk;          // work tiles per planned share (kTopkGrid shares, or one per CTA of the single launch)
+    int chunk;          // work tiles per planned share (one share per CTA of the tile phases)
 };
 
 struct TopkState {
     TopkPlan* plan;
     int* sp_seg;               // [P*T] segment id of the q-th sparse segment
     int* sp_begin;             // [P*T+1] first work tile of the q-th sparse segment
-    int* cta_q;                // [kTopkGrid] sparse slot that holds the first work tile of CTA c's share
+    int* cta_q;                // [CTAs of the tile phases] sparse slot that holds the first work tile of CTA c's share
     unsigned int* hist;        // [P*T][kMaxBins]
     unsigned int* prefix;      // [P*T] key bits resolved so far (after the last digit: tau)
     unsigned int* remaining;   // [P*T] rank still to resolve (after the last digit: number of
@@ -134,6 +134,7 @@ struct WorkCursor {
         changed = false;
         while (w >= end) {
             ++q;
+            if (!EG_INDEX_OK(tt.err, q, tk.plan->n_sparse)) { changed = true; break; }   // (the loop would not end)
             begin = tk.sp_begin[q];
             end = tk.sp_begin[q + 1];
             changed = true;
@@ -272,9 +273,12 @@ __device__ __forceinline__ int sub_offset(int len, int w) { return min(len, w * 
 // tile's slice of the entry buffer, IN ASCENDING INDEX ORDER inside each warp's sub-slice (the
 // later phases rely on that order: concatenating the sub-slices of a tensor's tiles lists its
 // entries by index).  Digit 1 of the undecided entries is histogrammed on the way.  Nothing is
-// shared between warps except that histogram: a lane marks its elements in four 4-bit masks,
-// one warp scan of the four packed 8-bit counts (a chunk holds 128 elements, so a field cannot
-// overflow) gives every lane its first slot in each chunk.
+// shared between warps except that histogram.  Entries are few (a few percent of the elements),
+// so the pass is split: first every lane only MARKS its sixteen elements in a bit mask (a chunk
+// holds 128 elements, so one warp scan of the four packed 8-bit counts gives every lane its
+// first slot in each chunk); then a lane walks the set bits of its mask -- usually none, one or
+// two -- and builds each entry from the element itself, which it reads again (the line has just
+// been fetched by this warp, so the second read is served by the caches).
 __device__ __forceinline__ void
 topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
                long long stride, TopkState tk) {
@@ -285,6 +289,7 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
     for (int b = threadIdx.x; b < kBins1; b += kThreads) s_hist[b] = 0;
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int mine = warp * kWarpSpan + lane * 4;      // this lane's first element of the tile
     WorkCursor cur;
     cur.init(tk, tt, T, r.q);
     unsigned int b0 = 0;
@@ -295,21 +300,22 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
         const int i = cur.i;
         const int len = tt.length[tile];
         const long long base = (long long)i * stride + tt.offset[tile];
-        unsigned int key[4 * kSubChunks];
-        float val[4 * kSubChunks];
+        float4 a[kSubChunks], b[kSubChunks];
+#pragma unroll
+        for (int j = 0; j < kSubChunks; ++j) {
+            const int local = mine + j * 128;
+            a[j] = b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (local < len) { a[j] = ld_stream(x + base + local); b[j] = ld_stream(xhat + base + local); }
+        }
         unsigned int mask = 0, packed = 0;      // bit 4j+c: element c of chunk j is an entry
 #pragma unroll
         for (int j = 0; j < kSubChunks; ++j) {
-            const int local = warp * kWarpSpan + j * 128 + lane * 4;
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-            if (local < len) { a = ld_stream(x + base + local); b = ld_stream(xhat + base + local); }
-            key[4 * j + 0] = rank_key(a.x, b.x); key[4 * j + 1] = rank_key(a.y, b.y);
-            key[4 * j + 2] = rank_key(a.z, b.z); key[4 * j + 3] = rank_key(a.w, b.w);
-            val[4 * j + 0] = a.x; val[4 * j + 1] = a.y; val[4 * j + 2] = a.z; val[4 * j + 3] = a.w;
-            const int nel = len - local;          // live elements of this float4 (<= 0: none)
+            const int nel = len - (mine + j * 128);   // live elements of this float4 (<= 0: none)
             unsigned int m = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) m |= (c < nel && (key[4 * j + c] >> 20) >= b0) ? (1u << c) : 0u;
+            m |= (0 < nel && (rank_key(a[j].x, b[j].x) >> 20) >= b0) ? 1u : 0u;
+            m |= (1 < nel && (rank_key(a[j].y, b[j].y) >> 20) >= b0) ? 2u : 0u;
+            m |= (2 < nel && (rank_key(a[j].z, b[j].z) >> 20) >= b0) ? 4u : 0u;
+            m |= (3 < nel && (rank_key(a[j].w, b[j].w) >> 20) >= b0) ? 8u : 0u;
             mask |= m << (4 * j);
             packed |= (unsigned int)__popc(m) << (8 * j);
         }
@@ -321,23 +327,32 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
         }
         const unsigned int tot = __shfl_sync(0xffffffffu, inc, 31);
         const unsigned int excl = inc - packed;
-        uint2* ent = tk.ent + base + sub_offset(len, warp);
+        // first slot of this lane in each chunk, 10 bits each (a sub-slice holds at most 512 entries)
+        unsigned long long first = 0;
         unsigned int chunk_first = 0;
 #pragma unroll
         for (int j = 0; j < kSubChunks; ++j) {
-            unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (mask & (1u << (4 * j + c))) {
-                    const unsigned int k = key[4 * j + c];
-                    const bool sure = (k >> 20) > b0;
-                    ent[pos++] = make_uint2((sure ? kEntSure : 0u) | ((k & 0xfffffu) << 9) |
-                                                (unsigned int)(j * 128 + lane * 4 + c),
-                                            __float_as_uint(val[4 * j + c]));
-                    if (!sure) atomicAdd(&s_hist[(k >> 10) & (kBins1 - 1)], 1u);
-                }
-            }
+            first |= (unsigned long long)(chunk_first + ((excl >> (8 * j)) & 0xffu)) << (10 * j);
             chunk_first += (tot >> (8 * j)) & 0xffu;
+        }
+        uint2* ent = tk.ent + base + sub_offset(len, warp);
+        const float* xs = x + base + mine;
+        const float* hs = xhat + base + mine;
+        unsigned int todo = mask;
+        while (todo) {
+            const int bit = __ffs(todo) - 1;
+            todo &= todo - 1u;
+            const int j = bit >> 2, e = j * 128 + (bit & 3);       // element mine + e of the tile
+            const float xv = xs[e];
+            const unsigned int k = rank_key(xv, hs[e]);
+            const bool sure = (k >> 20) > b0;
+            // slot: the lane's first slot in the chunk plus its own earlier entries of that chunk
+            const unsigned int pos = (unsigned int)((first >> (10 * j)) & 0x3ffu) +
+                                     __popc(mask & ((1u << bit) - 1u) & (0xfu << (4 * j)));
+            if (!EG_INDEX_OK(tt.err, pos, kWarpSpan) || !EG_INDEX_OK(tt.err, sub_offset(len, warp) + pos, len)) continue;
+            ent[pos] = make_uint2((sure ? kEntSure : 0u) | ((k & 0xfffffu) << 9) | (unsigned int)(lane * 4 + e),
+                                  __float_as_uint(xv));
+            if (!sure) atomicAdd(&s_hist[(k >> 10) & (kBins1 - 1)], 1u);
         }
         if (lane == 0) tk.tile_cand[((long long)i * tt.n_tiles + tile) * kSubSlices + warp] = (int)chunk_first;
         if (w + 1 == r.w1 || w + 1 >= cur.end) {   // last tile of this segment here
@@ -378,47 +393,25 @@ struct WarpWalk {
 };
 
 // The entries of one tile: sub-slice u (the elements [512 u, 512 u + 512) of the tile, in index
-// order) holds n[u] entries starting at place min(len, 512 u) of the tile's slice.  The phases
-// below walk four sub-slices side by side -- round r touches entries 32 r + lane of each of
-// them, four independent loads per lane -- because a tile rarely holds more than a few
-// dozen entries per sub-slice and a walk one after the other would wait for memory eight times
-// instead of twice.
-constexpr int kSubGroup = 4;        // sub-slices walked side by side
-struct TileEntries {
-    int n[kSubSlices];
-    const uint2* slice;
-    int len;
-    long long slot;                 // first of the tile's eight per-sub-slice records
-    // `mine`: lane u < 8 brings the entry count of sub-slice u (see TileFeed)
-    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, long long stride,
-                                         const WarpTile& z, int mine) {
-        slot = ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices;
-#pragma unroll
-        for (int u = 0; u < kSubSlices; ++u) n[u] = __shfl_sync(0xffffffffu, mine, u);
-        slice = tk.ent + (long long)z.i * stride + tt.offset[z.tile];
-        len = tt.length[z.tile];
-    }
-    __device__ __forceinline__ const uint2* sub(int u) const { return slice + min(len, u * kWarpSpan); }
-    // largest entry count among the sub-slices u0 .. u0 + kSubGroup - 1
-    __device__ __forceinline__ int most_of(int u0) const {
-        int m = 0;
-#pragma unroll
-        for (int v = 0; v < kSubGroup; ++v) m = max(m, n[u0 + v]);
-        return m;
-    }
-};
+// order) holds n_u entries starting at place min(len, 512 u) of the tile's slice.  A tile
+// rarely holds more than a dozen entries per sub-slice, so the phases below read all eight
+// sub-slices at once: lane 4 u + r takes the entries r, r + 4, r + 8, ... of sub-slice u, four
+// of them (kRounds) per trip to memory, and every lane has its loads in flight together.
+constexpr int kRounds = 4;          // entries per lane and trip
+constexpr int kGroupLanes = 4;      // lanes per sub-slice
+static_assert(kSubSlices * kGroupLanes == 32, "one warp covers the eight sub-slices of a tile");
 
 // A warp's tiles, one ahead: while a tile is worked on, the entry counts of the warp's next
-// tile are already on their way, so a tile costs one wait less.
+// tile are already on their way, so a tile costs one wait less.  Every lane gets the count of
+// its own sub-slice.
 struct TileFeed {
     WarpWalk walk;
     WarpTile ahead;
     int ahead_mine;
     bool have;
     __device__ __forceinline__ int fetch(const TopkState& tk, const TileTable& tt) const {
-        const int lane = threadIdx.x & 31;
-        return (lane < kSubSlices)
-                   ? tk.tile_cand[((long long)ahead.i * tt.n_tiles + ahead.tile) * kSubSlices + lane] : 0;
+        const int u = (threadIdx.x & 31) / kGroupLanes;
+        return tk.tile_cand[((long long)ahead.i * tt.n_tiles + ahead.tile) * kSubSlices + u];
     }
     __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int shares) {
         walk.init(tk, tt, T, shares);
@@ -435,87 +428,94 @@ struct TileFeed {
     }
 };
 
-// Digit 2 over the entries: one warp per tile, global histogram updated directly (only the
-// undecided entries that match the 21 resolved bits take part: about one in a thousand).
+// (greater, equal) counts of a tile's eight sub-slices from per-lane counts: sums over the four
+// lanes of every sub-slice, stores the eight packed pairs and the tile's totals.
 __device__ __forceinline__ void
-topk_hist_cand(TileTable tt, int T, long long stride, TopkState tk, int shares = 1) {
+store_tile_counts(const TopkState& tk, long long slot, long long tile_index, unsigned int gt, unsigned int eq) {
     const int lane = threadIdx.x & 31;
+    unsigned int both = gt | (eq << 16);            // a sub-slice holds at most 512 entries
+    both += __shfl_xor_sync(0xffffffffu, both, 1);
+    both += __shfl_xor_sync(0xffffffffu, both, 2);
+    if ((lane & (kGroupLanes - 1)) == 0) tk.tile_sub[slot + lane / kGroupLanes] = both;
+    unsigned int all_gt = both & 0xffffu, all_eq = both >> 16;     // a tile holds at most 4096
+    all_gt += __shfl_xor_sync(0xffffffffu, all_gt, 4); all_eq += __shfl_xor_sync(0xffffffffu, all_eq, 4);
+    all_gt += __shfl_xor_sync(0xffffffffu, all_gt, 8); all_eq += __shfl_xor_sync(0xffffffffu, all_eq, 8);
+    all_gt += __shfl_xor_sync(0xffffffffu, all_gt, 16); all_eq += __shfl_xor_sync(0xffffffffu, all_eq, 16);
+    if (lane == 0) tk.tile_count[tile_index] = make_uint2(all_gt, all_eq);
+}
+
+// Digit 2 over the entries, and the counts the compaction needs.  One warp per tile.  With the 21
+// key bits resolved so far an entry is greater than tau for sure (a larger top digit, or the
+// same top digit and a larger digit 1), smaller for sure, or OPEN (both digits equal: digit 2
+// decides).  Open entries -- about one in a thousand -- go into the digit-2 histogram.  Per
+// sub-slice and per tile the kernel stores (greater for sure, open); for a tile without open
+// entries these are already its final (greater than tau, equal to tau) counts, the few tiles
+// that have some are counted again once tau is complete (topk_scan).
+__device__ __forceinline__ void
+topk_digit2(TileTable tt, int T, long long stride, TopkState tk, int shares = 1) {
+    const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
     TileFeed feed;
     feed.init(tk, tt, T, shares);
     WarpTile z;
-    int mine_n;
+    int n;                               // entries of this lane's sub-slice
     int s_now = -1;
     unsigned int want = 0;
-    while (feed.next(tk, tt, T, z, mine_n)) {
-        if (z.s != s_now) { s_now = z.s; want = tk.prefix[z.s] & ((1u << kDigitBits1) - 1); }   // digit 1 of tau
-        unsigned int* gh = tk.hist + (long long)z.s * kMaxBins;
-        TileEntries te;
-        te.init(tk, tt, stride, z, mine_n);
+    unsigned int* gh = nullptr;
+    while (feed.next(tk, tt, T, z, n)) {
+        if (z.s != s_now) {
+            s_now = z.s;
+            want = tk.prefix[z.s] & ((1u << kDigitBits1) - 1);      // digit 1 of tau
+            gh = tk.hist + (long long)z.s * kMaxBins;
+        }
+        const int len = tt.length[z.tile];
+        const uint2* sub = tk.ent + (long long)z.i * stride + tt.offset[z.tile] + min(len, u * kWarpSpan);
+        unsigned int gt = 0, open = 0;
+        for (int f0 = r; __any_sync(0xffffffffu, f0 - r < n); f0 += kRounds * kGroupLanes) {
+            unsigned int meta[kRounds];
 #pragma unroll
-        for (int u0 = 0; u0 < kSubSlices; u0 += kSubGroup) {
-            for (int f = lane; f - lane < te.most_of(u0); f += 32) {
-                unsigned int meta[kSubGroup];
+            for (int q = 0; q < kRounds; ++q) {
+                const int f = f0 + q * kGroupLanes;
+                meta[q] = (f < n) ? sub[f].x : 0u;
+            }
 #pragma unroll
-                for (int v = 0; v < kSubGroup; ++v) meta[v] = (f < te.n[u0 + v]) ? te.sub(u0 + v)[f].x : kEntSure;
-#pragma unroll
-                for (int v = 0; v < kSubGroup; ++v) {
-                    const unsigned int low = ent_low20(meta[v]);
-                    if (!ent_sure(meta[v]) && (low >> kDigitBits2) == want)
-                        atomicAdd(&gh[low & ((1u << kDigitBits2) - 1)], 1u);
+            for (int q = 0; q < kRounds; ++q) {
+                const bool live = f0 + q * kGroupLanes < n;
+                const unsigned int low = ent_low20(meta[q]), d1 = low >> kDigitBits2;
+                if (live && (ent_sure(meta[q]) || d1 > want)) ++gt;
+                if (live && !ent_sure(meta[q]) && d1 == want) {
+                    ++open;
+                    atomicAdd(&gh[low & ((1u << kDigitBits2) - 1)], 1u);
                 }
             }
         }
+        store_tile_counts(tk, ((long long)z.i * tt.n_tiles + z.tile) * kSubSlices,
+                          (long long)z.i * tt.n_tiles + z.tile, gt, open);
     }
 }
 
-// Per tile and per sub-slice: keys greater than / equal to tau, from the entries.  One warp per
-// tile.  tile_sub gets the eight (greater | equal << 16) pairs, tile_count the tile's totals.
+// (greater than tau, equal to tau) per sub-slice and per tile, counted from the entries of one tile
+// by one warp with all 31 bits of tau known.
 __device__ __forceinline__ void
-topk_count(TileTable tt, int T, long long stride, TopkState tk, int shares = 1) {
-    const int lane = threadIdx.x & 31;
-    TileFeed feed;
-    feed.init(tk, tt, T, shares);
-    WarpTile z;
-    int mine_n;
-    int s_now = -1;
-    unsigned int tau20 = 0;
-    while (feed.next(tk, tt, T, z, mine_n)) {
-        if (z.s != s_now) { s_now = z.s; tau20 = tk.prefix[z.s] & 0xfffffu; }
-        TileEntries te;
-        te.init(tk, tt, stride, z, mine_n);
-        unsigned int mine = 0, all_gt = 0, all_eq = 0;
-#pragma unroll
-        for (int u0 = 0; u0 < kSubSlices; u0 += kSubGroup) {
-            unsigned int gt[kSubGroup], eq[kSubGroup];        // the same in every lane
-#pragma unroll
-            for (int v = 0; v < kSubGroup; ++v) gt[v] = eq[v] = 0;
-            for (int f = lane; f - lane < te.most_of(u0); f += 32) {
-                unsigned int meta[kSubGroup];
-#pragma unroll
-                for (int v = 0; v < kSubGroup; ++v) meta[v] = (f < te.n[u0 + v]) ? te.sub(u0 + v)[f].x : 0u;
-#pragma unroll
-                for (int v = 0; v < kSubGroup; ++v) {
-                    const bool live = f < te.n[u0 + v];
-                    const unsigned int low = ent_low20(meta[v]);
-                    gt[v] += __popc(__ballot_sync(0xffffffffu, live && (ent_sure(meta[v]) || low > tau20)));
-                    eq[v] += __popc(__ballot_sync(0xffffffffu, live && !ent_sure(meta[v]) && low == tau20));
-                }
-            }
-#pragma unroll
-            for (int v = 0; v < kSubGroup; ++v) {
-                if (lane == u0 + v) mine = gt[v] | (eq[v] << 16);
-                all_gt += gt[v];
-                all_eq += eq[v];
-            }
-        }
-        if (lane < kSubSlices) tk.tile_sub[te.slot + lane] = mine;
-        if (lane == 0) tk.tile_count[(long long)z.i * tt.n_tiles + z.tile] = make_uint2(all_gt, all_eq);
+count_tile_exact(const TileTable& tt, long long stride, const TopkState& tk, int i, int tile, unsigned int tau20) {
+    const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
+    const long long index = (long long)i * tt.n_tiles + tile;
+    const int n = tk.tile_cand[index * kSubSlices + u];
+    const int len = tt.length[tile];
+    const uint2* sub = tk.ent + (long long)i * stride + tt.offset[tile] + min(len, u * kWarpSpan);
+    unsigned int gt = 0, eq = 0;
+    for (int f = r; f < n; f += kGroupLanes) {
+        const unsigned int meta = sub[f].x, low = ent_low20(meta);
+        if (ent_sure(meta) || low > tau20) ++gt;
+        else if (low == tau20) ++eq;
     }
+    store_tile_counts(tk, index * kSubSlices, index, gt, eq);
 }
 
-// One CTA per sparse segment: exclusive prefix of the tile counts, in tile order.
+// One CTA per sparse segment.  First the tiles that held open entries are counted again, now
+// that tau is complete (a handful per tensor, unless many keys tie); then the exclusive prefix
+// of the tile counts, in tile order.
 __device__ __forceinline__ void
-topk_scan(TileTable tt, int T, TopkState tk) {
+topk_scan(TileTable tt, int T, long long stride, TopkState tk) {
     __shared__ unsigned int s_gt[kWarps], s_eq[kWarps];
     __shared__ unsigned int s_run[2];
     const int nq = tk.plan->n_sparse;
@@ -525,8 +525,19 @@ topk_scan(TileTable tt, int T, TopkState tk) {
         const int i = s / T, t = s - i * T;
         const int q0 = tt.seg_begin[t], q1 = tt.seg_begin[t + 1];
         uint2* tc = tk.tile_count + (long long)i * tt.n_tiles;
+        const unsigned int tau20 = tk.prefix[s] & 0xfffffu;
+        for (int c0 = q0; c0 < q1; c0 += 32 * kWarps) {
+            // a lane looks at one tile; the warp then counts the marked ones together, one by one
+            const int z = c0 + warp * 32 + lane;
+            unsigned int marked = __ballot_sync(0xffffffffu, z < q1 && tc[z].y != 0u);
+            while (marked) {
+                const int l = __ffs(marked) - 1;
+                marked &= marked - 1u;
+                count_tile_exact(tt, stride, tk, i, c0 + warp * 32 + l, tau20);
+            }
+        }
         if (threadIdx.x == 0) s_run[0] = s_run[1] = 0;
-        __syncthreads();
+        __syncthreads();            // the recounted pairs are visible to the whole CTA
         for (int c0 = q0; c0 < q1; c0 += kThreads) {
             const int z = c0 + threadIdx.x;
             uint2 v = make_uint2(0, 0);
@@ -554,27 +565,29 @@ topk_scan(TileTable tt, int T, TopkState tk) {
     }
 }
 
-// Pass C: ordered compaction of the selected entries into the outbox, and delivery: the same
+// Ordered compaction of the selected entries into the outbox, and delivery: the same
 // (index, value) pairs are written into the mailbox x_hat, which is what the receivers hold
 // once the message has arrived.  Works from the entries alone (a few percent of the tensor);
 // x and x_hat are not read again.
 // An entry is selected if key > tau, or key == tau and fewer than `remaining` equal keys
 // precede it in the tensor.  Its slot is (#greater before it) + min(#equal before it, remaining).
-// One warp per tile walks the tile's entries in index order, 32 at a time; ballots give every
-// lane the number of greater / equal entries before its own.
+// One warp per tile; within a sub-slice the entries are taken in index order, four at a time by
+// the four lanes of the sub-slice, and ballots give every lane the number of greater / equal
+// entries before its own.
 __device__ __forceinline__ void
 topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, unsigned int* __restrict__ err,
            int shares = 1) {
-    const int lane = threadIdx.x & 31;
-    const unsigned int below = (1u << lane) - 1u;
+    const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
+    const unsigned int group = (unsigned int)((1u << kGroupLanes) - 1u) << (u * kGroupLanes);   // lanes of this sub-slice
+    const unsigned int lower = ((1u << r) - 1u) << (u * kGroupLanes);                            // ... before this lane
     TileFeed feed;
     feed.init(tk, tt, T, shares);
     WarpTile z;
-    int mine_n;
+    int n;
     int s_now = -1;
     unsigned int tau20 = 0, take = 0, K = 0;
     int2* out = nullptr;
-    while (feed.next(tk, tt, T, z, mine_n)) {
+    while (feed.next(tk, tt, T, z, n)) {
         if (z.s != s_now) {
             s_now = z.s;
             tau20 = tk.prefix[z.s] & 0xfffffu;
@@ -582,50 +595,50 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, uns
             K = (unsigned int)tk.count[z.t];
             out = tk.outbox + (long long)z.i * tk.out_stride + tk.out_off[z.t];
         }
-        TileEntries te;
-        te.init(tk, tt, stride, z, mine_n);
-        const uint2 before = tk.tile_count[(long long)z.i * tt.n_tiles + z.tile];
-        const unsigned int sub_mine = (lane < kSubSlices) ? tk.tile_sub[te.slot + lane] : 0u;
+        const long long index = (long long)z.i * tt.n_tiles + z.tile;
+        const uint2 before = tk.tile_count[index];
+        const unsigned int sub_mine = tk.tile_sub[index * kSubSlices + u];
+        const int len = tt.length[z.tile];
         const long long base = (long long)z.i * stride + tt.offset[z.tile];
+        const uint2* sub = tk.ent + base + min(len, u * kWarpSpan);
         const int first = (z.tile - tt.seg_begin[z.t]) * kNormTile;   // index of the tile's first element
-        unsigned int gt_before = before.x, eq_before = before.y;   // entries before sub-slice u0, whole tensor
+        // selected entries of the whole tensor before this sub-slice: the tile's prefix plus the
+        // sub-slices before it (all four lanes of a sub-slice hold the same pair)
+        unsigned int inc = sub_mine;
 #pragma unroll
-        for (int u0 = 0; u0 < kSubSlices; u0 += kSubGroup) {
-            unsigned int run_gt[kSubGroup], run_eq[kSubGroup];     // the same in every lane
+        for (int o = kGroupLanes; o < 32; o <<= 1) {
+            const unsigned int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        unsigned int run_gt = before.x + ((inc - sub_mine) & 0xffffu);
+        unsigned int run_eq = before.y + ((inc - sub_mine) >> 16);
+        for (int f0 = r; __any_sync(0xffffffffu, f0 - r < n); f0 += kRounds * kGroupLanes) {
+            uint2 e[kRounds];
 #pragma unroll
-            for (int v = 0; v < kSubGroup; ++v) {
-                const unsigned int packed = __shfl_sync(0xffffffffu, sub_mine, u0 + v);
-                run_gt[v] = gt_before;
-                run_eq[v] = eq_before;
-                gt_before += packed & 0xffffu;
-                eq_before += packed >> 16;
+            for (int q = 0; q < kRounds; ++q) {
+                const int f = f0 + q * kGroupLanes;
+                e[q] = (f < n) ? sub[f] : make_uint2(0u, 0u);
             }
-            for (int f = lane; f - lane < te.most_of(u0); f += 32) {
-                uint2 e[kSubGroup];
 #pragma unroll
-                for (int v = 0; v < kSubGroup; ++v)
-                    e[v] = (f < te.n[u0 + v]) ? te.sub(u0 + v)[f] : make_uint2(0u, 0u);
-#pragma unroll
-                for (int v = 0; v < kSubGroup; ++v) {
-                    const bool live = f < te.n[u0 + v];
-                    const unsigned int low = ent_low20(e[v].x);
-                    const bool g = live && (ent_sure(e[v].x) || low > tau20);
-                    const bool q = live && !ent_sure(e[v].x) && low == tau20;
-                    const unsigned int bg = __ballot_sync(0xffffffffu, g), bq = __ballot_sync(0xffffffffu, q);
-                    const unsigned int my_gt = run_gt[v] + __popc(bg & below), my_eq = run_eq[v] + __popc(bq & below);
-                    if (g || (q && my_eq < take)) {
-                        const unsigned int slot = my_gt + min(my_eq, take);
-                        const int local = (u0 + v) * kWarpSpan + (int)(e[v].x & 0x1ffu);
-                        if (slot < K && local < te.len) {
-                            out[slot] = make_int2(first + local, (int)e[v].y);
-                            xhat[base + local] = __uint_as_float(e[v].y);
-                        } else {
-                            atomicOr(err, 2u);
-                        }
+            for (int q = 0; q < kRounds; ++q) {
+                const bool live = f0 + q * kGroupLanes < n;
+                const unsigned int low = ent_low20(e[q].x);
+                const bool g = live && (ent_sure(e[q].x) || low > tau20);
+                const bool same = live && !ent_sure(e[q].x) && low == tau20;
+                const unsigned int bg = __ballot_sync(0xffffffffu, g), bq = __ballot_sync(0xffffffffu, same);
+                const unsigned int my_gt = run_gt + __popc(bg & lower), my_eq = run_eq + __popc(bq & lower);
+                if (g || (same && my_eq < take)) {
+                    const unsigned int slot = my_gt + min(my_eq, take);
+                    const int local = u * kWarpSpan + (int)(e[q].x & 0x1ffu);
+                    if (slot < K && local < len) {
+                        out[slot] = make_int2(first + local, (int)e[q].y);
+                        xhat[base + local] = __uint_as_float(e[q].y);
+                    } else {
+                        atomicOr(err, kErrTopkSlot);
                     }
-                    run_gt[v] += __popc(bg);
-                    run_eq[v] += __popc(bq);
                 }
+                run_gt += __popc(bg & group);
+                run_eq += __popc(bq & group);
             }
         }
     }
@@ -635,7 +648,8 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, uns
 // Launch forms.  k_topk_all runs the whole sequence in ONE cooperative launch with grid-wide
 // barriers between the phases, and every CTA leaves after the first barrier when no segment
 // sends a sparse message in this step -- a quiet step then costs one launch instead of ten.
-// The single-phase kernels below are the fallback where a cooperative launch is not available.
+// The single-phase kernels below are used for large problems and where a cooperative launch is
+// not available.
 // ---------------------------------------------------------------------------------------
 struct TopkArgs {
     const float* x;
@@ -648,6 +662,7 @@ struct TopkArgs {
     unsigned int* err;
     const unsigned int* sparse_steps;   // [2] sparse messages decided in the iteration of this parity
     const long long* step_k;
+    int plan_ctas;                      // CTAs of the tile phases when they are launched one by one
 };
 
 __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
@@ -666,41 +681,49 @@ __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     grid.sync();
     topk_pick(a.T, a.tk, 1);
     grid.sync();
-    topk_hist_cand(a.tt, a.T, a.stride, a.tk);
+    topk_digit2(a.tt, a.T, a.stride, a.tk);
     grid.sync();
     topk_pick(a.T, a.tk, 2);
     grid.sync();
-    topk_count(a.tt, a.T, a.stride, a.tk);
-    grid.sync();
-    topk_scan(a.tt, a.T, a.tk);
+    topk_scan(a.tt, a.T, a.stride, a.tk);
     grid.sync();
     topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
 }
 
+// Every single-phase kernel may be launched while the kernel before it drains (programmatic
+// dependent launch): it lets its own successor do the same and then waits for its predecessor
+// before it reads anything.
 __global__ void __launch_bounds__(kThreads) k_topk_plan(TopkArgs a) {
-    topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, kTopkGrid);   // every tile phase runs kTopkGrid CTAs
+    pdl_release(); pdl_wait();
+    topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, a.plan_ctas);
 }
 __global__ void __launch_bounds__(kThreads) k_topk_hist(TopkArgs a) {
+    pdl_release(); pdl_wait();
     topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
 }
-__global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int digit) { topk_pick(a.T, a.tk, digit); }
+__global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int digit) {
+    pdl_release(); pdl_wait();
+    topk_pick(a.T, a.tk, digit);
+}
 #ifndef EG_COLLECT_MINB
 #define EG_COLLECT_MINB 4
 #endif
 __global__ void __launch_bounds__(kThreads, EG_COLLECT_MINB) k_topk_collect(TopkArgs a) {
+    pdl_release(); pdl_wait();
     topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
 }
-// The phases that work from the entries keep more registers than the streaming passes: they
-// run half the planned CTAs, each taking two planned shares.
+// The phases that work from the entries run half the planned CTAs, each taking two planned shares.
 constexpr int kEntryShares = 2;
-__global__ void __launch_bounds__(kThreads, 4) k_topk_hist_cand(TopkArgs a) {
-    topk_hist_cand(a.tt, a.T, a.stride, a.tk, kEntryShares);
+__global__ void __launch_bounds__(kThreads, 4) k_topk_digit2(TopkArgs a) {
+    pdl_release(); pdl_wait();
+    topk_digit2(a.tt, a.T, a.stride, a.tk, kEntryShares);
 }
-__global__ void __launch_bounds__(kThreads, 4) k_topk_count(TopkArgs a) {
-    topk_count(a.tt, a.T, a.stride, a.tk, kEntryShares);
+__global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) {
+    pdl_release(); pdl_wait();
+    topk_scan(a.tt, a.T, a.stride, a.tk);
 }
-__global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) { topk_scan(a.tt, a.T, a.tk); }
 __global__ void __launch_bounds__(kThreads, 4) k_topk_write(TopkArgs a) {
+    pdl_release(); pdl_wait();
     topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.err, kEntryShares);
 }
 

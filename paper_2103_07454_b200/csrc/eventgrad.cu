@@ -29,7 +29,7 @@ using PipeLayout = PipeSmem<kPipeTile, kPipeStages>;
 constexpr int kMomStages = 4;                         // four tiles per stage: same footprint as 5 x 3
 using MomLayout = PipeSmem<kPipeTile, kMomStages, 4>;
 static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
-constexpr uint64_t kStateMagic = 0x4547535441544532ull;  // "EGSTATE2"
+constexpr uint64_t kStateMagic = 0x4547535441544533ull;  // "EGSTATE3"
 
 struct HostTiles {
     std::vector<int> tensor, length, seg_begin;
@@ -40,7 +40,7 @@ struct DeviceTiles {
     int *tensor = nullptr, *length = nullptr, *seg_begin = nullptr;
     long long* offset = nullptr;
     int n_tiles = 0;
-    TileTable view() const { return TileTable{tensor, offset, length, seg_begin, n_tiles}; }
+    TileTable view(unsigned int* err) const { return TileTable{tensor, offset, length, seg_begin, n_tiles, err}; }
 };
 
 }  // namespace
@@ -85,7 +85,10 @@ struct eg_ctx {
     int topk_coop_grid = 0;   // CTAs of the one-launch Top-K kernel; 0: use the ten single-phase launches
     int variant = 0;
     double cap_alpha = 0.0, cap_beta = 1.0;   // bound alpha*beta^k on the squared threshold
-    long long host_k = 0;                     // host copy of the iteration counter
+    double* cap_g = nullptr;                  // [2] device: g(k) at [k & 1], advanced by the kernels
+    int sms = 148;                            // multiprocessors of the context's device
+    int topk_grid = 0, topk_seg_grid = 0;     // CTAs of the Top-K tile / segment phases
+    bool last_capturing = false;              // the most recent step was recorded into a graph
     // sub-range of the step that eg_step_masked launches (eg_step_host pipelines groups of
     // tensors); the default is everything
     std::vector<int> seg_begin_norm, seg_begin_fused;   // host copies, [T+1]
@@ -106,6 +109,8 @@ struct eg_ctx {
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
     bool nvtx = false;      // EG_NVTX in the environment at eg_create: named ranges around the kernel groups
+    bool topk_pdl = false;  // EG_TOPK_PDL in the environment at eg_create: dependent launches inside the Top-K sequence too
+    bool no_pdl = false;    // EG_NO_PDL in the environment at eg_create: every kernel starts after its predecessor has ended
     std::vector<cudaEvent_t> ev_pool;      // pairs
     std::vector<int> ev_kind;              // kernel group of every recorded pair
     size_t ev_used = 0;
@@ -227,9 +232,26 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->small_done, 0, sizeof(int)));
     }
     if (c->vel) EG_CUDA(c, cudaMemset(c->vel, 0, (size_t)c->P * c->stride * sizeof(float)));
+    {
+        const double g0[2] = {c->cap_alpha, c->cap_alpha};   // iteration 0 reads slot 0
+        EG_CUDA(c, cudaMemcpy(c->cap_g, g0, sizeof(g0), cudaMemcpyHostToDevice));
+    }
     c->carried_valid = false;
     c->stepped = false;
-    c->host_k = 0;
+    return EG_OK;
+}
+
+// g(k) = alpha * beta^k as the kernels carry it: k multiplications, one rounding each.
+double cap_term(double alpha, double beta, long long k) {
+    double g = alpha;
+    for (long long q = 0; q < k; ++q) g = g * beta;
+    return g;
+}
+
+// Puts the term of iteration k where that iteration will read it.
+eg_status upload_cap(eg_ctx* c, long long k) {
+    const double g = cap_term(c->cap_alpha, c->cap_beta, k);
+    EG_CUDA(c, cudaMemcpy(c->cap_g + (k & 1), &g, sizeof(g), cudaMemcpyHostToDevice));
     return EG_OK;
 }
 
@@ -237,8 +259,7 @@ eg_status sync_and_check(eg_ctx* c) {
     EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
     unsigned int e = 0;
     EG_CUDA(c, cudaMemcpy(&e, c->err, sizeof(e), cudaMemcpyDeviceToHost));
-    if (e & kErrPipeTimeout) return EG_ERR_TIMEOUT;   // a bounded device-side wait gave up
-    return e ? EG_ERR_INTERNAL : EG_OK;
+    return eg_status_of_error_word(e);
 }
 
 constexpr size_t kMaxTimedPairs = 1 << 15;
@@ -366,6 +387,19 @@ const char* eg_strerror(eg_status s) {
     return "unknown status";
 }
 
+eg_status eg_status_of_error_word(unsigned int word) {
+    if (word & kErrWaitTimeout) return EG_ERR_TIMEOUT;   // a bounded device-side wait gave up
+    return word ? EG_ERR_INTERNAL : EG_OK;               // kErrBounds, kErrTopkSlot
+}
+
+int eg_debug_build(void) {
+#ifdef EG_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 int eg_last_cuda_error(const eg_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 int eg_last_launch_count(const eg_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 
@@ -404,8 +438,14 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     auto fail = [&](eg_status code) { eg_destroy(c); return code; };
     if (cudaGetDevice(&c->device) != cudaSuccess) return fail(EG_ERR_CUDA);
     { const char* e = getenv("EG_NVTX"); c->nvtx = e && *e && *e != '0'; }
+    { const char* e = getenv("EG_NO_PDL"); c->no_pdl = e && *e && *e != '0'; }
+    { const char* e = getenv("EG_TOPK_PDL"); c->topk_pdl = e && *e && *e != '0'; }
     c->P = P; c->T = T; c->H = thr->history_len; c->thr = *thr;
     if (topk) c->topk = *topk;
+    if (cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->sms < 1)
+        return fail(EG_ERR_CUDA);
+    c->topk_grid = c->sms * kTopkCtasPerSm;       // the tile phases loop over the work list
+    c->topk_seg_grid = c->sms * kTopkSegCtasPerSm;
     c->hops = topology + 1;                       // EG_TOPO_RING_HOPS(m) == m - 1
     c->degree = std::min(2 * c->hops, P - 1);     // distinct neighbours of every replica
     // layout: every tensor starts on a 128-byte boundary
@@ -447,7 +487,7 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     EG_ALLOC(c->st.hist_len, S); EG_ALLOC(c->st.valid, S); EG_ALLOC(c->st.flag, S);
     EG_ALLOC(c->st.snap, S); EG_ALLOC(c->st.sparse, S); EG_ALLOC(c->st.norm, S);
     EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S); EG_ALLOC(c->st.sent_norm, S);
-    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 2);
+    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 2); EG_ALLOC(c->cap_g, 2);
     EG_ALLOC(c->outbox_count, S);
     if (c->topk.enabled) EG_ALLOC(c->st.sparse_steps, 2);
     EG_ALLOC(c->cons_partials, (size_t)c->tiles_fused.n_tiles + 1);
@@ -461,20 +501,20 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         EG_ALLOC(c->tk.plan, 1);
         EG_ALLOC(c->tk.sp_seg, S);
         EG_ALLOC(c->tk.sp_begin, S + 1);
-        EG_ALLOC(c->tk.cta_q, kTopkGrid);
+        EG_ALLOC(c->tk.cta_q, c->topk_grid);
         EG_ALLOC(c->tk.outbox, (size_t)P * c->out_stride);
         {
             // one cooperative launch needs all its CTAs resident at the same time
-            int coop = 0, per_sm = 0, sms = 0;
+            int coop = 0, per_sm = 0;
+            const int sms = c->sms;
             if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) == cudaSuccess && coop &&
-                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess &&
                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_topk_all, kThreads, 0) == cudaSuccess &&
                 per_sm > 0)
                 c->topk_coop_grid = std::min(per_sm, 4) * sms;
             // Measured: the single launch saves about 40 us in a step without sparse messages but
-            // is about 20 % slower than the ten launches when most tensors send (it runs every
+            // is about 20 % slower than the separate launches when most tensors send (it runs every
             // phase at the occupancy of the largest one), so it is used where launch overhead
-            // is visible: small problems.  EG_TOPK_SEPARATE_LAUNCHES forces the ten launches.
+            // is visible: small problems.  EG_TOPK_SEPARATE_LAUNCHES forces the separate launches.
             if ((long long)P * c->tiles_norm.n_tiles > 65536 || getenv("EG_TOPK_SEPARATE_LAUNCHES"))
                 c->topk_coop_grid = 0;
         }
@@ -520,10 +560,10 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     {
         // one launch per iteration where a few hundred CTAs cover the whole parameter set
         // ... and all of them are resident at the same time (a second wave would double the latency)
-        int sms = 0, max_smem = 0, per_sm = 0;
+        int max_smem = 0, per_sm = 0;
+        const int sms = c->sms;
         const void* fn = small_kernel(P);
         if (fn && !c->topk.enabled && c->hops == 1 &&
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess &&
             cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) == cudaSuccess &&
             small_smem_bytes(P) <= (size_t)max_smem &&
             cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)small_smem_bytes(P)) ==
@@ -586,9 +626,24 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     DeviceGuard guard(c->device);
     if (!guard.ok) return EG_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    // One stream at a time: moving to another stream is allowed only once the stream of the
+    // previous call has run dry.  Nothing can be asked while a graph is being recorded (on the
+    // new stream or on the previous one): the caller ends the recording before moving on.
+    bool capturing = false;
+    {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) { (void)cudaGetLastError(); cs = cudaStreamCaptureStatusNone; }
+        capturing = cs != cudaStreamCaptureStatusNone;
+    }
+    if (c->stepped && stream != c->last_stream && !c->last_capturing && !capturing) {
+        const cudaError_t q = cudaStreamQuery(c->last_stream);
+        if (q == cudaErrorNotReady) return EG_ERR_STATE;
+        if (q != cudaSuccess) (void)cudaGetLastError();
+    }
+    c->last_capturing = capturing;
     c->last_stream = stream;
     int launches = 0;
-    const TileTable tn_all = c->tiles_norm.view(), tf_all = c->tiles_fused.view();
+    const TileTable tn_all = c->tiles_norm.view(c->err), tf_all = c->tiles_fused.view(c->err);
     const int S = c->P * c->T;
     // tensors [t0, t0 + tcount) of this launch and their tiles in both tile tables
     const int t0 = c->range_tn ? c->range_t0 : 0, tcount = c->range_tn ? c->range_tn : c->T;
@@ -622,9 +677,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     // a2 + a6: decision, threshold update, counters
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
                     c->topk.enabled, c->degree, c->variant,
-                    c->cap_alpha > 0.0 ? std::sqrt(c->cap_alpha * std::pow(c->cap_beta, (double)c->host_k))
-                                       : HUGE_VAL,
-                    t0, tcount};
+                    c->cap_alpha > 0.0 ? c->cap_g : nullptr, c->cap_beta, t0, tcount, c->err};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf_all : tn_all;
     if (small) {
@@ -645,7 +698,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         ++launches;
     } else {
         TimedSection ts(c, stream, EG_KERNEL_DECIDE);
-        EG_CUDA(c, launch_pdl(!c->timing, k_decide, dim3((c->P * tcount + kWarps - 1) / kWarps), dim3(kThreads), 0, stream,
+        EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_decide, dim3((c->P * tcount + kWarps - 1) / kWarps), dim3(kThreads), 0, stream,
                               partials, (const int*)tp.seg_begin, tp.n_tiles, dp, c->st,
                               (const long long*)c->d_numel, (const long long*)c->d_kcount, c->outbox_count,
                               c->ctr, (const long long*)c->step_k,
@@ -657,24 +710,29 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     if (c->topk.enabled && !small) {
         TimedSection ts(c, stream, EG_KERNEL_TOPK);
         TopkArgs ta{params, c->xhat, tn, S, c->T, c->stride, c->st.sparse, c->tk, c->err, c->st.sparse_steps,
-                    c->step_k};
+                    c->step_k, c->topk_grid};
+        const int tile_grid = c->topk_grid, seg_grid = c->topk_seg_grid;
         if (c->topk_coop_grid > 0) {
             void* args[] = {&ta};
             EG_CUDA(c, cudaLaunchCooperativeKernel((const void*)k_topk_all, dim3(c->topk_coop_grid),
                                                    dim3(kThreads), args, 0, stream));
             launches += 1;
         } else {
-            k_topk_plan<<<1, kThreads, 0, stream>>>(ta);
-            k_topk_hist<<<kTopkGrid, kThreads, 0, stream>>>(ta);
-            k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(ta, 0);
-            k_topk_collect<<<kTopkGrid, kThreads, 0, stream>>>(ta);
-            k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(ta, 1);
-            k_topk_hist_cand<<<kTopkGrid / kEntryShares, kThreads, 0, stream>>>(ta);
-            k_topk_pick<<<kTopkSegGrid, kThreads, 0, stream>>>(ta, 2);
-            k_topk_count<<<kTopkGrid / kEntryShares, kThreads, 0, stream>>>(ta);
-            k_topk_scan<<<kTopkSegGrid, kThreads, 0, stream>>>(ta);
-            k_topk_write<<<kTopkGrid / kEntryShares, kThreads, 0, stream>>>(ta);
-            launches += 10;
+            // Nine launches.  They can be started as dependent launches (each waits on the device,
+            // first thing it does, for the kernel before it), but measured on 64 x 25.6 M elements
+            // that made the sequence 30 % slower, so it is only done on request (EG_TOPK_PDL).
+            const bool pdl = !c->timing && !c->no_pdl && c->topk_pdl;
+            const dim3 tile_blocks(tile_grid), entry_blocks(tile_grid / kEntryShares), seg_blocks(seg_grid);
+            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, dim3(1), dim3(kThreads), 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, dim3(kThreads), 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, dim3(kThreads), 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, tile_blocks, dim3(kThreads), 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, dim3(kThreads), 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_digit2, entry_blocks, dim3(kThreads), 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, dim3(kThreads), 0, stream, ta, 2));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_scan, seg_blocks, dim3(kThreads), 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_write, entry_blocks, dim3(kThreads), 0, stream, ta));
+            launches += 9;
         }
     }
     // a3 + a5: dense snapshot, consensus average, SGD
@@ -720,10 +778,10 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                 // started while the kernel before it (the decision kernel, or the Top-K sequence)
                 // drains: it waits on the device before it reads anything that kernel writes
                 if (carry)
-                    EG_CUDA(c, launch_pdl(!c->timing, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
+                    EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
                                           dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
                 else
-                    EG_CUDA(c, launch_pdl(!c->timing, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
+                    EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
                                           dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
             } else {
                 if (carry)
@@ -747,7 +805,6 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     c->carried_valid = carry && whole;
     c->carried_params = params;
     c->stepped = true;
-    if (c->range_last) c->host_k += 1;
     c->last_launches = launches;
     EG_CUDA(c, cudaGetLastError());
     return EG_OK;
@@ -1000,9 +1057,15 @@ eg_status eg_selftest_wait_timeout(eg_ctx* c, void* stream_v) {
 
 eg_status eg_set_threshold_cap(eg_ctx* c, double alpha, double beta) {
     if (!c || std::isnan(alpha) || std::isnan(beta) || (alpha > 0.0 && !(beta > 0.0))) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return EG_ERR_CUDA;
+    // the sequence continues from the term of the iteration the device has reached
+    EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    long long k = 0;
+    EG_CUDA(c, cudaMemcpy(&k, c->step_k, sizeof(k), cudaMemcpyDeviceToHost));
     c->cap_alpha = alpha;
     c->cap_beta = beta;
-    return EG_OK;
+    return upload_cap(c, k);
 }
 
 eg_status eg_set_fused_kernel(eg_ctx* c, int kind) {
@@ -1182,8 +1245,8 @@ eg_status eg_average_model(eg_ctx* c, const float* params, float* avg_dev, doubl
     if (!c || !params || !avg_dev) return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-    const TileTable tf = c->tiles_fused.view();
-    const int grid = std::min(tf.n_tiles, 148 * 8);
+    const TileTable tf = c->tiles_fused.view(c->err);
+    const int grid = std::min(tf.n_tiles, c->sms * 8);
     k_average_model<<<grid, kThreads, 0, stream>>>(params, avg_dev, tf, c->P, c->stride,
                                                    consensus_host ? c->cons_partials : nullptr);
     if (consensus_host) {
@@ -1199,39 +1262,61 @@ eg_status eg_average_model(eg_ctx* c, const float* params, float* avg_dev, doubl
 // ---------------------------------------------------------------------------------------
 // checkpoint
 // ---------------------------------------------------------------------------------------
+// Everything a context needs to continue a run: the header names the context the state belongs
+// to (an import into a context created or configured differently is refused), then the
+// iteration counter and counters, the trigger state, the mailboxes, and -- when the context
+// has them -- the delivery state (received copies, messages in flight) and the velocities.
 struct StateHeader {
     uint64_t magic;
     int64_t P, T, H, stride, n_total, topk, k_num, k_den, variant;
     int64_t step;
     uint64_t messages, bytes, events;
+    int64_t hops, mode, force_first, delivery, velocity;
+    double horizon, delta_init, delta_fixed, cap_alpha, cap_beta, mu;
+    uint64_t arrivals;
 };
 
 static size_t state_bytes(const eg_ctx* c) {
-    const size_t S = (size_t)c->P * c->T;
-    return sizeof(StateHeader) + S * (2 * sizeof(double) + sizeof(long long) + sizeof(int) + 1 +
-                                      sizeof(unsigned long long)) +
-           S * c->H * sizeof(double) + (size_t)c->P * c->stride * sizeof(float);
+    const size_t S = (size_t)c->P * c->T, n = (size_t)c->P * c->stride * sizeof(float);
+    size_t b = sizeof(StateHeader) + S * (2 * sizeof(double) + sizeof(long long) + sizeof(int) + 1 +
+                                          sizeof(unsigned long long)) +
+               S * c->H * sizeof(double) + n;
+    if (c->async) b += n + 2 * S;
+    if (c->vel) b += n;
+    return b;
+}
+
+static StateHeader state_header(const eg_ctx* c) {
+    StateHeader h{};
+    h.magic = kStateMagic; h.P = c->P; h.T = c->T; h.H = c->H; h.stride = c->stride;
+    h.n_total = c->n_total; h.topk = c->topk.enabled; h.k_num = c->topk.k_num; h.k_den = c->topk.k_den;
+    h.variant = c->variant; h.hops = c->hops; h.mode = c->thr.mode; h.force_first = c->thr.force_first_event;
+    h.delivery = c->async ? 1 : 0; h.velocity = c->vel ? 1 : 0;
+    h.horizon = c->thr.horizon; h.delta_init = c->thr.delta_init; h.delta_fixed = c->thr.delta_fixed;
+    h.cap_alpha = c->cap_alpha; h.cap_beta = c->cap_beta; h.mu = c->momentum ? c->mu : 0.0;
+    return h;
 }
 
 eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
     if (!c || !bytes) return EG_ERR_INVALID;
-    if (c->async) return EG_ERR_STATE;   // messages in flight are not part of a checkpoint
     const size_t need = state_bytes(c);
     if (!host_buf) { *bytes = need; return EG_OK; }
     if (*bytes < need) { *bytes = need; return EG_ERR_INVALID; }
     DeviceGuard guard(c->device);
     eg_status s = sync_and_check(c);
     if (s != EG_OK) return s;
-    const size_t S = (size_t)c->P * c->T;
-    StateHeader h{};
+    const size_t S = (size_t)c->P * c->T, n = (size_t)c->P * c->stride * sizeof(float);
+    StateHeader h = state_header(c);
     Counters ctr{};
     long long k = 0;
     EG_CUDA(c, cudaMemcpy(&ctr, c->ctr, sizeof(ctr), cudaMemcpyDeviceToHost));
     EG_CUDA(c, cudaMemcpy(&k, c->step_k, sizeof(k), cudaMemcpyDeviceToHost));
-    h.magic = kStateMagic; h.P = c->P; h.T = c->T; h.H = c->H; h.stride = c->stride;
-    h.n_total = c->n_total; h.topk = c->topk.enabled; h.k_num = c->topk.k_num; h.k_den = c->topk.k_den;
-    h.variant = c->variant;
     h.step = k; h.messages = ctr.messages; h.bytes = ctr.bytes; h.events = ctr.events;
+    if (c->async) {
+        unsigned long long a = 0;
+        EG_CUDA(c, cudaMemcpy(&a, c->arrivals, sizeof(a), cudaMemcpyDeviceToHost));
+        h.arrivals = a;
+    }
     char* p = static_cast<char*>(host_buf);
     memcpy(p, &h, sizeof(h)); p += sizeof(h);
 #define EG_PULL(ptr, nbytes)                                                     \
@@ -1243,7 +1328,13 @@ eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
     EG_PULL(c->st.events, S * sizeof(unsigned long long));
     EG_PULL(c->st.hist, S * c->H * sizeof(double));
     EG_PULL(c->st.sent_norm, S * sizeof(double));
-    EG_PULL(c->xhat, (size_t)c->P * c->stride * sizeof(float));
+    EG_PULL(c->xhat, n);
+    if (c->async) {
+        EG_PULL(c->mailbox, n);
+        EG_PULL(c->pending, S);
+        EG_PULL(c->recv_valid, S);
+    }
+    if (c->vel) { EG_PULL(c->vel, n); }
 #undef EG_PULL
     *bytes = need;
     return EG_OK;
@@ -1251,18 +1342,23 @@ eg_status eg_export_state(eg_ctx* c, void* host_buf, size_t* bytes) {
 
 eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
     if (!c || !host_buf || bytes < state_bytes(c)) return EG_ERR_INVALID;
-    if (c->async) return EG_ERR_STATE;
     StateHeader h;
     memcpy(&h, host_buf, sizeof(h));
-    if (h.magic != kStateMagic || h.P != c->P || h.T != c->T || h.H != c->H || h.stride != c->stride ||
-        h.n_total != c->n_total || h.topk != c->topk.enabled || h.variant != c->variant ||
-        (h.topk && (h.k_num != c->topk.k_num || h.k_den != c->topk.k_den)))
+    const StateHeader w = state_header(c);
+    // doubles are compared by their bits: a checkpoint belongs to exactly the rules it was made under
+    auto same = [](double a, double b) { return memcmp(&a, &b, sizeof(double)) == 0; };
+    if (h.magic != w.magic || h.P != w.P || h.T != w.T || h.H != w.H || h.stride != w.stride ||
+        h.n_total != w.n_total || h.topk != w.topk || h.variant != w.variant ||
+        (h.topk && (h.k_num != w.k_num || h.k_den != w.k_den)) || h.hops != w.hops || h.mode != w.mode ||
+        h.force_first != w.force_first || h.delivery != w.delivery || h.velocity != w.velocity ||
+        !same(h.horizon, w.horizon) || !same(h.delta_init, w.delta_init) || !same(h.delta_fixed, w.delta_fixed) ||
+        !same(h.cap_alpha, w.cap_alpha) || !same(h.cap_beta, w.cap_beta) || !same(h.mu, w.mu) || h.step < 0)
         return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
     EG_CUDA(c, cudaStreamSynchronize(c->last_stream));
     eg_status s = init_state(c);
     if (s != EG_OK) return s;
-    const size_t S = (size_t)c->P * c->T;
+    const size_t S = (size_t)c->P * c->T, n = (size_t)c->P * c->stride * sizeof(float);
     Counters ctr{h.messages, h.bytes, h.events, 0};
     long long k = h.step;
     EG_CUDA(c, cudaMemcpy(c->ctr, &ctr, sizeof(ctr), cudaMemcpyHostToDevice));
@@ -1277,13 +1373,20 @@ eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
     EG_PUSH(c->st.events, S * sizeof(unsigned long long));
     EG_PUSH(c->st.hist, S * c->H * sizeof(double));
     EG_PUSH(c->st.sent_norm, S * sizeof(double));
-    EG_PUSH(c->xhat, (size_t)c->P * c->stride * sizeof(float));
+    EG_PUSH(c->xhat, n);
+    if (c->async) {
+        EG_PUSH(c->mailbox, n);
+        EG_PUSH(c->pending, S);
+        EG_PUSH(c->recv_valid, S);
+        const unsigned long long a = h.arrivals;
+        EG_CUDA(c, cudaMemcpy(c->arrivals, &a, sizeof(a), cudaMemcpyHostToDevice));
+    }
+    if (c->vel) { EG_PUSH(c->vel, n); }
 #undef EG_PUSH
     EG_CUDA(c, cudaDeviceSynchronize());
     c->carried_valid = false;
     c->stepped = h.step > 0;
-    c->host_k = h.step;
-    return EG_OK;
+    return upload_cap(c, h.step);
 }
 
 }  // extern "C"

@@ -14,6 +14,7 @@ the whole configuration.
 from __future__ import annotations
 
 import os
+import time
 from dataclasses import dataclass, field
 from typing import List, Optional, Sequence
 
@@ -47,6 +48,7 @@ class Report:
     max_norm_rel: float = 0.0
     params_bit_exact: bool = True
     launches: int = 0
+    seconds: dict = field(default_factory=lambda: {"inputs": 0.0, "oracle": 0.0, "compare": 0.0})
 
 
 def oracle_threads() -> int:
@@ -58,10 +60,27 @@ def _columns(numel: Sequence[int], tensors: Sequence[int]) -> np.ndarray:
     return np.concatenate([np.arange(off[t], off[t] + numel[t]) for t in tensors])
 
 
-HEADER_WORDS = 14  # checkpoint header: magic, P, T, H, stride, N, topk, k_num, k_den, variant, step, 3 counters
+def _counters_from_events(events: np.ndarray, numel, k_t, degree: int) -> dict:
+    """Message, byte and event totals implied by the number of events of every (replica,
+    tensor): `degree` messages per event, 4 n_t bytes for a dense message, 8 K_t for a Top-K
+    message, the first message of a tensor always being dense."""
+    ev = np.asarray(events, dtype=np.int64)
+    n = np.asarray(numel, dtype=np.int64)[None, :]
+    if k_t is None:
+        payload = 4 * n * ev
+    else:
+        kt = np.asarray(k_t, dtype=np.int64)[None, :]
+        payload = np.where(ev > 0, 4 * n + 8 * kt * (ev - 1), 0)
+    return {"messages": int(degree * ev.sum()), "bytes": int(degree * payload.sum()), "events": int(ev.sum())}
 
 
-def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np.ndarray):
+# Checkpoint header, 8-byte words: magic, P, T, H, stride, N, topk, k_num, k_den, variant, step,
+# 3 counters, hops, mode, force_first, delivery, velocity, 6 doubles (horizon, delta_init,
+# delta_fixed, bound alpha / beta, mu), arrivals.
+HEADER_WORDS = 26
+
+
+def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np.ndarray, delivery: bool = False):
     """After a reported near-threshold disagreement: overwrite the CUDA context's state and
     parameters with the oracle's (through the checkpoint interface) so the comparison of the
     following steps stays meaningful."""
@@ -71,6 +90,7 @@ def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np
     st = o.stats()
     head[10] = o.iteration
     head[11:14] = [st["messages"], st["bytes"], st["events"]]
+    head[25] = o.arrivals
     pos = HEADER_WORDS * 8
 
     def put(arr, dtype):
@@ -78,6 +98,11 @@ def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np
         raw = np.ascontiguousarray(arr, dtype=dtype).tobytes()
         blob[pos:pos + len(raw)] = raw
         pos += len(raw)
+
+    def put_layout(packed):
+        padded = torch.zeros((eg.P, eg.replica_stride), dtype=torch.float32)
+        eg.pack_into(padded, torch.from_numpy(packed))
+        put(padded.numpy(), np.float32)
 
     hist, hist_len = o.history()
     put(o.thresholds(), np.float64)
@@ -87,16 +112,16 @@ def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np
     put(o.segment_events(), np.uint64)
     put(hist, np.float64)
     put(o.sent_norms(), np.float64)
-    xhat = torch.zeros((eg.P, eg.replica_stride), dtype=torch.float32)
-    eg.pack_into(xhat, torch.from_numpy(o.xhat()))
-    put(xhat.numpy(), np.float32)
+    put_layout(o.xhat())
+    if delivery:
+        put_layout(o.received())
+        put(o.pending(), np.uint8)
+        put(o.received_once(), np.uint8)
+    if o.velocity() is not None:
+        put_layout(o.velocity())
     assert pos == len(blob)
     eg.import_state(bytes(blob))
     eg.pack_into(x_dev, torch.from_numpy(x_host).to(x_dev.device))
-    if o.velocity() is not None:
-        vel = torch.zeros((eg.P, eg.replica_stride), dtype=torch.float32)
-        eg.pack_into(vel, torch.from_numpy(o.velocity()))
-        eg.write_velocity(vel)
 
 
 def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "workload",
@@ -109,7 +134,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     full = tensors is None
     tensors = list(range(wl.T)) if full else list(tensors)
     sub_numel = [wl.numel[t] for t in tensors]
-    cols = None if full else torch.from_numpy(_columns(wl.numel, tensors)).to(gen_device)
+    cols = None if full else torch.from_numpy(_columns(wl.numel, tensors)).to(dev)
 
     okw = dict(horizon=wl.horizon, history_len=wl.history_len, delta_init=wl.delta_init,
                topk=wl.topk, threads=oracle_threads())
@@ -138,39 +163,84 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     if okw.get("momentum") is not None:
         eg.set_momentum(okw["momentum"])
 
-    x0 = W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)
+    x0 = (W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)).to(dev)
     x_dev = eg.to_layout(x0)
     x_host = (x0 if full else x0[:, cols]).cpu().numpy().copy()
-    g_dev = eg.empty_params()
     del x0
+    ncol = x_host.shape[1]
+    # Large runs move their data between device and host through page-locked buffers, and the
+    # inputs of iteration k+1 are produced on the device while the oracle works on iteration k.
+    big = wl.P * ncol >= (1 << 24)
+    g_devs = [eg.empty_params(), eg.empty_params()]
+    g_pins = [torch.empty((wl.P, ncol), dtype=torch.float32, pin_memory=big) for _ in range(2)]
+    chk_pin = torch.empty((wl.P, ncol), dtype=torch.float32, pin_memory=True) if big else None
+    box_pin = torch.empty((wl.P, eg.replica_stride), dtype=torch.float32, pin_memory=True) if big else None
     rep = Report()
     sub_off = np.concatenate([[0], np.cumsum(sub_numel)])
+    degree = min(2 * int(okw.get("hops", 1)), wl.P - 1)
+    all_kt = [eg.topk_count(t) for t in range(wl.T)] if wl.topk else None
+    sub_kt = [all_kt[t] for t in tensors] if wl.topk else None
     rng = np.random.default_rng(7)
 
     def gpu_sub(padded: torch.Tensor) -> np.ndarray:
+        """The oracle's tensors of a device array in the library's layout, packed, on the host."""
         parts = [padded[:, eg.tensor_offset[t]:eg.tensor_offset[t] + wl.numel[t]] for t in tensors]
-        return torch.cat(parts, dim=1).cpu().numpy()
+        packed = torch.cat(parts, dim=1)
+        if chk_pin is None:
+            return packed.cpu().numpy()
+        chk_pin.copy_(packed)
+        return chk_pin.numpy()
 
-    for k in range(steps):
+    def host_sub(padded: np.ndarray, packed: np.ndarray) -> bool:
+        """Bit equality of the oracle's tensors of a host array in the library's layout with a packed array."""
+        return all(np.array_equal(padded[:, eg.tensor_offset[t]:eg.tensor_offset[t] + wl.numel[t]].view(np.uint32),
+                                  packed[:, sub_off[q]:sub_off[q + 1]].view(np.uint32))
+                   for q, t in enumerate(tensors))
+
+    def produce(k):
+        """Inputs of iteration k: gradients in the library's layout on the device, and the
+        oracle's columns of them on the host (ready once the returned event has completed)."""
+        slot = k & 1
         g = wl.grads(k, gen_device)
         if grad_hook is not None:
             g = grad_hook(k, g)
-        eg.pack_into(g_dev, g.to(dev))
-        g_host = (g if full else g[:, cols]).cpu().numpy()
-        del g
+        g = g.to(dev)
+        eg.pack_into(g_devs[slot], g)
+        g_pins[slot].copy_(g if full else g[:, cols], non_blocking=True)
+        ready = torch.cuda.Event()
+        ready.record()
+        return g_devs[slot], g_pins[slot].numpy(), ready
+
+    t_mark = time.perf_counter()
+
+    def lap(name):
+        nonlocal t_mark
+        now = time.perf_counter()
+        rep.seconds[name] += now - t_mark
+        t_mark = now
+
+    ahead = produce(0)
+    for k in range(steps):
+        g_dev, g_host, ready = ahead
+        ready.synchronize()
         sent_pre = o.sent_norms() if okw.get("change_of_norm") else None
         mask = None if deliver_fn is None else deliver_fn(k)          # [P, T] uint8 or None
-        o.step(x_host, np.ascontiguousarray(g_host), wl.lr,
-               deliver=None if mask is None else np.ascontiguousarray(mask[:, tensors]))
         if deliver_fn is None:
             eg.step(x_dev, g_dev, wl.lr)
         else:
             eg.step_masked(x_dev, g_dev, wl.lr,
                            None if mask is None else torch.from_numpy(np.ascontiguousarray(mask)).to(dev))
+        if k + 1 < steps:
+            ahead = produce(k + 1)          # enqueued behind the step; runs while the oracle works
+        lap("inputs")
+        o.step(x_host, g_host, wl.lr,
+               deliver=None if mask is None else np.ascontiguousarray(mask[:, tensors]))
+        lap("oracle")
         rep.launches += eg.last_launch_count
         rep.steps += 1
         if (k % check_every) and k != steps - 1 and k >= 8:
             continue        # the first steps (where most events happen) are always checked
+        # (what follows synchronises with the device; its time is booked under "compare")
 
         f_g, d_g, thr_g = eg.last_decisions()
         f_g, d_g, thr_g = f_g[:, tensors], d_g[:, tensors], thr_g[:, tensors]
@@ -196,7 +266,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             assert near[bad].all(), f"trigger flags differ away from the threshold, step {k}"
             rep.near_threshold += [(k, int(i), int(tensors[t])) for i, t in zip(*np.nonzero(bad))]
             assert full, "near-threshold disagreement in a tensor-subset run cannot be re-synchronised"
-            resynchronise(eg, o, x_dev, x_host)
+            resynchronise(eg, o, x_dev, x_host, delivery=deliver_fn is not None)
             continue
         rep.events += int(f_o.sum())
 
@@ -205,6 +275,15 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             assert so == sg, f"counters, step {k}: oracle {so} cuda {sg}"
         _, ev_g = eg.thresholds()
         assert np.array_equal(ev_g[:, tensors], o.segment_events()), f"per-tensor events, step {k}"
+        if not full:
+            # The oracle's counters cover its tensors only.  Both totals follow from the events
+            # per (replica, tensor) -- every event is one message per distinct neighbour, the
+            # first message of a tensor is dense, later ones carry K_t pairs under Top-K -- so
+            # the oracle's counters must equal that sum over its tensors and the library's the
+            # same sum over all tensors, the per-tensor events of the sample being equal.
+            so, sg = o.stats(), eg.stats()
+            assert so == _counters_from_events(o.segment_events(), sub_numel, sub_kt, degree), f"step {k}"
+            assert sg == _counters_from_events(ev_g, wl.numel, all_kt, degree), f"counters, step {k}"
         dl_g, _ = eg.thresholds()
         dl_g, dl_o = dl_g[:, tensors], o.thresholds()
         fin = np.isfinite(dl_o)
@@ -228,8 +307,11 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             err = np.abs(x_g.astype(np.float64) - x_host) / np.maximum(np.abs(x_host), 1e-30)
             rep.max_param_rel = max(rep.max_param_rel, float(err.max()))
             assert rep.max_param_rel <= PARAM_RTOL, f"parameters, step {k}: rel err {rep.max_param_rel}"
-        xh_g = gpu_sub(eg.mailboxes().to(dev))
-        assert np.array_equal(xh_g.view(np.uint32), o.xhat().view(np.uint32)), f"mailboxes, step {k}"
+        if box_pin is None:
+            xh_g = gpu_sub(eg.mailboxes().to(dev))
+            assert np.array_equal(xh_g.view(np.uint32), o.xhat().view(np.uint32)), f"mailboxes, step {k}"
+        else:
+            assert host_sub(eg.mailboxes(out=box_pin).numpy(), o.xhat()), f"mailboxes, step {k}"
         if okw.get("momentum") is not None:
             v_g = gpu_sub(eg.velocity().to(dev))
             assert np.array_equal(v_g.view(np.uint32), o.velocity().view(np.uint32)), f"velocity, step {k}"
@@ -240,6 +322,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             assert np.array_equal(pend[:, tensors], o.pending()), f"in flight, step {k}"
             if full:
                 assert arrivals == o.arrivals, f"arrivals, step {k}"
+        lap("compare")
 
     eg.close()
     o.close()

@@ -173,9 +173,91 @@ def test_delivery_masks_enabled_mid_run_and_refusals():
         assert np.array_equal(eg.last_decisions()[0], o.flags())
     assert np.array_equal(eg.from_layout(xd).cpu().numpy(), xh)
     assert np.array_equal(eg.from_layout(eg.received()).numpy(), o.received())
-    with pytest.raises(B.EventGradError):
-        eg.export_state()                          # messages in flight are not checkpointed
     eg.close()
+
+
+def test_checkpoint_with_messages_in_flight_and_velocities():
+    """A checkpoint carries the delivery state (received copies, what is still in flight, the
+    arrival count) and the velocities: a context restored from it continues bit for bit."""
+    wl = W.synthetic(5, [5, 1000, 4097], steps=12, lr=0.1, grad_sigma=0.01, history_len=2)
+    rng = np.random.default_rng(11)
+    masks = [torch.from_numpy((rng.random((5, wl.T)) < 0.4).astype(np.uint8)).cuda() for _ in range(wl.steps)]
+    g = None
+
+    def run(eg, x, k0, k1):
+        for k in range(k0, k1):
+            eg.step_masked(x, eg.to_layout(wl.grads(k, "cuda")), wl.lr, masks[k])
+
+    a = B.from_workload(wl)
+    a.enable_delivery_masks()
+    xa = a.to_layout(W.distinct_init_params(wl, "cuda"))
+    run(a, xa, 0, 6)
+    assert a.delivery_status()[0].any()            # something is in flight at the checkpoint
+    blob, x_mid = a.export_state(), xa.clone()
+    run(a, xa, 6, 12)
+    b = B.from_workload(wl)
+    with pytest.raises(B.EventGradError):
+        b.import_state(blob)                       # not a context with delivery masks
+    b.enable_delivery_masks()
+    b.import_state(blob)
+    xb = x_mid.clone()
+    run(b, xb, 6, 12)
+    assert torch.equal(xa, xb) and a.stats() == b.stats()
+    assert torch.equal(a.received(), b.received()) and torch.equal(a.mailboxes(), b.mailboxes())
+    pa, pb = a.delivery_status(), b.delivery_status()
+    assert np.array_equal(pa[0], pb[0]) and pa[1] == pb[1]
+    a.close(); b.close()
+
+    # momentum: the velocities travel with the state
+    a, b = B.from_workload(wl), B.from_workload(wl)
+    a.set_momentum(0.9)
+    xa = a.to_layout(W.distinct_init_params(wl, "cuda"))
+    for k in range(6):
+        a.step(xa, a.to_layout(wl.grads(k, "cuda")), wl.lr)
+    blob, xb = a.export_state(), xa.clone()
+    with pytest.raises(B.EventGradError):
+        b.import_state(blob)                       # no velocity buffer there
+    b.set_momentum(0.5)
+    with pytest.raises(B.EventGradError):
+        b.import_state(blob)                       # another coefficient
+    b.set_momentum(0.9)
+    b.import_state(blob)
+    for k in range(6, 12):
+        gk = a.to_layout(wl.grads(k, "cuda"))
+        a.step(xa, gk, wl.lr)
+        b.step(xb, gk, wl.lr)
+    assert torch.equal(xa, xb) and torch.equal(a.velocity(), b.velocity()) and a.stats() == b.stats()
+    a.close(); b.close()
+
+
+def test_checkpoint_is_refused_by_a_differently_configured_context():
+    wl = W.synthetic(6, [5, 1000, 4097], steps=4, lr=0.1, grad_sigma=0.01, history_len=2)
+    src = B.from_workload(wl)
+    src.set_threshold_cap(1e-3, 0.9)
+    x = src.to_layout(W.distinct_init_params(wl, "cuda"))
+    for k in range(3):
+        src.step(x, src.to_layout(wl.grads(k, "cuda")), wl.lr)
+    blob = src.export_state()
+    same = B.from_workload(wl)
+    same.set_threshold_cap(1e-3, 0.9)
+    same.import_state(blob)
+    others = [B.from_workload(wl, hops=2), B.from_workload(wl, horizon=2.0), B.from_workload(wl, delta_init=0.5),
+              B.from_workload(wl, mode=B.THRESH_FIXED, delta_fixed=0.1), B.from_workload(wl, force_first_event=False),
+              B.from_workload(wl), B.from_workload(wl)]
+    others[-1].set_threshold_cap(1e-3, 0.8)
+    for other in others:
+        with pytest.raises(B.EventGradError):
+            other.import_state(blob)
+        other.close()
+    # the bound continues from the restored iteration
+    y = x.clone()
+    g = src.to_layout(wl.grads(3, "cuda"))
+    src.step(x, g, wl.lr)
+    same.step(y, g, wl.lr)
+    assert torch.equal(x, y)
+    for a, b in zip(src.last_decisions(), same.last_decisions()):
+        assert np.array_equal(a, b)
+    src.close(); same.close()
 
 
 def test_variant_with_topk():
@@ -275,12 +357,12 @@ def test_topk_degenerate_all_keys_equal(separate, monkeypatch):
 
 
 def test_topk_with_separate_launches(monkeypatch):
-    """The ten single-phase Top-K launches (fallback where a cooperative launch is unavailable)."""
+    """The nine single-phase Top-K launches (fallback where a cooperative launch is unavailable)."""
     monkeypatch.setenv("EG_TOPK_SEPARATE_LAUNCHES", "1")
     wl = W.synthetic(3, RAGGED, steps=10, lr=0.1, grad_sigma=0.01, topk=(10, 100))
     rep = lockstep(wl, init="distinct", outbox_samples=64)
     assert rep.params_bit_exact and rep.sparse_checked > 5
-    assert rep.launches == 10 * 13
+    assert rep.launches == 10 * 12
 
 
 @pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
@@ -382,13 +464,23 @@ def test_config2_resnet20(carry, kernel):
         assert rep.launches == (wl.steps + 1 if carry else 2 * wl.steps)
 
 
+def _report(name, rep):
+    """What a configured run did, on the test log (shown with -s or on failure)."""
+    print(f"{name}: steps {rep.steps}, events {rep.events}, sparse messages checked {rep.sparse_checked}, "
+          f"largest norm error {rep.max_norm_rel:.2e} of its tolerance, parameters bit-exact {rep.params_bit_exact}, "
+          f"decisions within 1e-6 of the threshold that differed {rep.near_threshold}; seconds spent on "
+          + ", ".join(f"{k} {v:.1f}" for k, v in rep.seconds.items()))
+
+
 @pytest.mark.parametrize("carry", [False, True])
 def test_config3_resnet18_p16(carry):
+    """Configuration 3 as configured: 100 iterations, all 62 tensors, both norm variants."""
     (wl,) = W.config(3)
-    steps = wl.steps if (carry or os.environ.get("EG_FULL")) else 30
-    rep = lockstep(wl, steps=steps, carry=carry, check_every=5)
+    rep = lockstep(wl, carry=carry, check_every=5)
+    _report(f"{wl.name} carry={carry}", rep)
+    assert rep.steps == wl.steps == 100
     assert rep.params_bit_exact and not rep.near_threshold
-    assert rep.launches == (steps * 2 + 1 if carry else steps * 3)
+    assert rep.launches == (wl.steps * 2 + 1 if carry else wl.steps * 3)
 
 
 def _sample_tensors(wl, n_small=6, n_mid=3, n_big=2):
@@ -398,21 +490,40 @@ def _sample_tensors(wl, n_small=6, n_mid=3, n_big=2):
     return sorted(set(int(t) for t in pick))
 
 
+def _size_classes_and_boosted(wl):
+    """Tensors the oracle follows at configuration 5: the first tensor of every distinct size
+    (all 22 size classes of ResNet-50, the 2048 x 1000 classifier among them) and every tensor
+    whose gradients are scaled by ten (t mod 10 == 0): 35 of 161 tensors, 43 % of the elements."""
+    first = {}
+    for t, n in enumerate(wl.numel):
+        first.setdefault(n, t)
+    return sorted(set(first.values()) | set(range(0, wl.T, 10)))
+
+
 @pytest.mark.parametrize("which", [0, 1])
 def test_config4_resnet18_topk(which):
+    """Configuration 4 as configured: 100 iterations at K = 1 % and K = 10 %, the oracle follows
+    all 62 tensors, so the message and byte counters are compared as well."""
     wl = W.config(4)[which]
-    steps = wl.steps if os.environ.get("EG_FULL") else 40
-    rep = lockstep(wl, steps=steps, tensors=_sample_tensors(wl), check_every=4, outbox_samples=12)
-    assert rep.params_bit_exact and rep.sparse_checked > 10
+    rep = lockstep(wl, check_every=5, outbox_samples=12)
+    _report(wl.name, rep)
+    assert rep.steps == wl.steps == 100
+    assert rep.params_bit_exact and not rep.near_threshold and rep.sparse_checked > 10
 
 
 @pytest.mark.parametrize("which", [0, 1])
 def test_config5_resnet50_p64(which):
+    """Configuration 5 as configured: 50 iterations, dense (carried norm) and K = 1 % (two-pass);
+    the library runs all 161 tensors of the 64 replicas, the oracle a 35-tensor sample."""
     wl = W.config(5)[which]
-    steps = wl.steps if os.environ.get("EG_FULL") else 12
-    rep = lockstep(wl, steps=steps, tensors=_sample_tensors(wl, 6, 3, 1), check_every=4,
-                   outbox_samples=12, carry=(which == 0))
-    assert rep.params_bit_exact
+    tensors = _size_classes_and_boosted(wl)
+    assert len(tensors) == 35 and wl.numel.index(2048 * 1000) in tensors
+    rep = lockstep(wl, tensors=tensors, check_every=5, outbox_samples=12, carry=(which == 0))
+    _report(wl.name, rep)
+    assert rep.steps == wl.steps == 50
+    assert rep.params_bit_exact and not rep.near_threshold
+    if which == 1:
+        assert rep.sparse_checked > 10
 
 
 def test_checkpoint_roundtrip_and_reset():
@@ -516,6 +627,89 @@ def test_steps_replayed_from_a_cuda_graph_match_direct_calls():
         eg.close()
     assert torch.equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
     assert all(np.array_equal(a, b) for a, b in zip(outs[0][2], outs[1][2]))
+
+
+@pytest.mark.parametrize("what", ["pipelined_carry_cap", "small_cap", "topk_cap", "two_pass"])
+def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(what):
+    """Replays of one captured eg_step against direct calls and the oracle, for the launch forms a
+    step can take: decision + pipelined kernel started as dependent launches (carried norm), the
+    single-launch kernel, norm + decision + pipelined kernel, and the cooperative Top-K launch;
+    with a geometric bound on the thresholds, whose sequence advances on the device."""
+    from oracle import eg_oracle as eo
+    topk = (10, 100) if what == "topk_cap" else None
+    wl = W.synthetic(4, [5, 1000, 4097, 70000], steps=9, lr=0.1, grad_sigma=0.01, topk=topk)
+    kernel = B.FUSED_AUTO if what == "small_cap" else B.FUSED_PIPELINED
+    cap = None if what == "two_pass" else (4e-3, 0.6)
+    carry = what != "two_pass"
+    outs = []
+    for use_graph in (False, True):
+        eg = B.from_workload(wl)
+        eg.set_carry_norm(carry)
+        eg.set_fused_kernel(kernel)
+        if cap:
+            eg.set_threshold_cap(*cap)
+        x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+        grad = eg.to_layout(wl.grads(0, "cuda"))
+        eg.step(x, grad, wl.lr)
+        if use_graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                eg.step(x, grad, wl.lr)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                eg.step(x, grad, wl.lr)
+            for _ in range(7):
+                g.replay()
+        else:
+            for _ in range(8):
+                eg.step(x, grad, wl.lr)
+        torch.cuda.synchronize()
+        outs.append((x.clone(), eg.stats(), eg.last_decisions(), eg.mailboxes()))
+        eg.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    assert torch.equal(outs[0][3], outs[1][3])
+    assert all(np.array_equal(a, b) for a, b in zip(outs[0][2], outs[1][2]))
+    # and the oracle, fed the same gradient nine times
+    o = eo.from_workload(wl, threshold_cap=cap) if cap else eo.from_workload(wl)
+    xh = W.distinct_init_params(wl).numpy().copy()
+    gh = wl.grads(0).numpy()
+    for _ in range(9):
+        o.step(xh, gh, wl.lr)
+    eg = B.from_workload(wl)
+    assert np.array_equal(eg.from_layout(outs[1][0]).cpu().numpy(), xh)
+    assert outs[1][1] == o.stats()
+    assert np.array_equal(outs[1][2][0], o.flags())
+    if cap:
+        assert 0 < outs[1][1]["events"] < 9 * 4 * wl.T
+    eg.close()
+
+
+def test_one_stream_at_a_time():
+    """A context moves to another stream only once the stream of its previous step has run dry."""
+    wl = W.synthetic(3, [7, 3000], steps=3, lr=0.1, grad_sigma=0.01)
+    eg, ref = B.from_workload(wl), B.from_workload(wl)
+    x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+    y = x.clone()
+    g = eg.to_layout(wl.grads(0, "cuda"))
+    a, b = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    eg.step(x, g, wl.lr, stream=a)
+    with torch.cuda.stream(a):
+        torch.cuda._sleep(400_000_000)             # keeps stream a busy for a fraction of a second
+    with pytest.raises(B.EventGradError, match="not allowed"):
+        eg.step(x, g, wl.lr, stream=b)
+    eg.step(x, g, wl.lr, stream=a)                 # the same stream is always fine
+    a.synchronize()
+    eg.step(x, g, wl.lr, stream=b)
+    b.synchronize()
+    for _ in range(3):
+        ref.step(y, g, wl.lr)
+    torch.cuda.synchronize()
+    assert torch.equal(x, y) and eg.stats() == ref.stats()
+    eg.close(); ref.close()
 
 
 def test_average_model_and_consensus():

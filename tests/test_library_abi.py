@@ -34,6 +34,17 @@ def test_status_strings():
     assert lib.eg_last_cuda_error(None) == 0
 
 
+def test_error_word_decoding():
+    """What the synchronising calls make of the device-side error word: a bounded wait that ran
+    out is a time-out, a failed index check or a misplaced Top-K entry an internal error."""
+    lib = binding.load_library()
+    assert lib.eg_status_of_error_word(0) == 0
+    assert lib.eg_status_of_error_word(2) == 6 and lib.eg_status_of_error_word(4) == 6
+    assert lib.eg_status_of_error_word(8) == 5 and lib.eg_status_of_error_word(8 | 4 | 2) == 5
+    assert lib.eg_strerror(5) == b"timeout"
+    assert lib.eg_debug_build() in (0, 1)
+
+
 def test_create_rejects_bad_arguments_before_touching_the_device():
     lib = binding.load_library()
     h = ctypes.c_void_p()

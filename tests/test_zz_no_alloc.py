@@ -76,3 +76,10 @@ def test_static_norms_unpadded_layout_and_limits():
                                       out.data_ptr(), None) == 1
     assert lib.eg_change_norms_static(None, h.data_ptr(), 1, 8, offs_c, (i64 * 1)(8), 1,
                                       out.data_ptr(), None) == 1      # NULL input
+    # more replicas than a grid dimension holds: refused before anything is launched
+    assert lib.eg_change_norms_static(x.data_ptr(), h.data_ptr(), 65536, 4, offs_c, (i64 * 1)(4), 1,
+                                      out.data_ptr(), None) == 1
+    # an offset that would overflow the bounds check
+    assert lib.eg_change_norms_static(x.data_ptr(), h.data_ptr(), 1, 8, (i64 * 1)(2 ** 63 - 4), (i64 * 1)(8), 1,
+                                      out.data_ptr(), None) == 1
+    torch.cuda.synchronize()
