@@ -239,6 +239,18 @@ eg_status eg_last_outbox(eg_ctx* ctx, int i, int t, int32_t* idx_host, float* va
                          int32_t* count_host);
 eg_status eg_topk_count(const eg_ctx* ctx, int t, int64_t* k_t_host);
 
+/* How the Top-K entries are found (Top-K paragraph of Section 7; the result is always the exact
+ * K_t largest |x - x_hat|, ties to the lower index).  For a large tensor the library first
+ * guesses, from a sample of the tensor, a magnitude bin at or below that of the K_t-th largest
+ * entry, collects everything at or above it in one pass and finishes the selection exactly on
+ * what it collected; when the guess turns out wrong (too few collected, or far too many) that
+ * tensor is selected again without guessing, at the cost of two more passes over it.
+ * eg_topk_repeat_count returns how many sparse messages took that second route since the
+ * context was created or reset (synchronises).  EG_TOPK_GUESS_MARGIN in the environment at
+ * eg_create sets the safety margin of the guess in standard deviations of the sampled count
+ * (default 5; a negative value makes every guess fail, which exercises the second route). */
+eg_status eg_topk_repeat_count(eg_ctx* ctx, uint64_t* repeats_host);
+
 /* Copies the mailboxes x_hat ([P][replica_stride] fp32) into a host buffer. Synchronises. */
 eg_status eg_read_mailboxes(eg_ctx* ctx, float* xhat_host);
 

@@ -30,6 +30,7 @@ EXPORTS = [
     "eg_enable_delivery_masks", "eg_step_masked", "eg_read_received", "eg_delivery_status",
     "eg_selftest_wait_timeout", "eg_set_momentum", "eg_read_velocity", "eg_write_velocity",
     "eg_debug_fail_allocation", "eg_status_of_error_word", "eg_debug_build",
+    "eg_topk_repeat_count",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -61,11 +62,13 @@ def load_library() -> C.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
+    # EG_LIBRARY names another build of the same library (the bounds-checked one, for instance)
+    path = os.environ.get("EG_LIBRARY") or LIB_PATH
+    if not os.path.exists(path):
         raise EventGradError(
-            f"{LIB_PATH} not found: build it with `python -m paper_2103_07454_b200.build`; "
+            f"{path} not found: build it with `python -m paper_2103_07454_b200.build`; "
             "this package has no CPU fallback")
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     vp, i64p, u64p = C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_uint64)
     lib.eg_create.argtypes = [C.POINTER(vp), C.c_int, C.c_int, i64p, C.c_int,
                               C.POINTER(ThresholdParams), C.POINTER(TopkParams)]
@@ -106,6 +109,7 @@ def load_library() -> C.CDLL:
     lib.eg_strerror.restype = C.c_char_p
     lib.eg_status_of_error_word.argtypes = [C.c_uint]
     lib.eg_debug_build.argtypes = []
+    lib.eg_topk_repeat_count.argtypes = [vp, u64p]
     lib.eg_last_cuda_error.argtypes = [vp]
     lib.eg_last_launch_count.argtypes = [vp]
     _lib = lib
@@ -265,6 +269,12 @@ class EventGrad:
         k = C.c_int64()
         _check(self._lib, self._lib.eg_topk_count(self._h, t, C.byref(k)), self._h, "eg_topk_count")
         return int(k.value)
+
+    def topk_repeat_count(self) -> int:
+        """Sparse messages whose guessed bin failed and that were selected again exactly."""
+        n = C.c_uint64()
+        _check(self._lib, self._lib.eg_topk_repeat_count(self._h, C.byref(n)), self._h, "eg_topk_repeat_count")
+        return int(n.value)
 
     def last_outbox(self, i: int, t: int):
         cap = max(1, self.topk_count(t))

@@ -3,20 +3,28 @@
 // index), pack them as (index, value) in ascending index order into the replica's outbox,
 // and deliver them into the mailbox x_hat.
 //
-// The rank key is the bit pattern of |x - x_hat| (fp32), which orders like the magnitude.
-// The K_t-th largest key tau is found by radix select over three digits (11 + 10 + 10 bits):
-//   pass A  (reads x, x_hat)  histogram of the top digit                     -> bin b0
-//   pass B  (reads x, x_hat)  every element whose top digit is >= b0 is copied, tile by tile and
-//                             in index order, into an entry buffer as (20 low key bits, position,
-//                             value of x); digit 1 of the undecided ones (top digit == b0) is
-//                             histogrammed on the way
+// The rank key is the bit pattern of |x - x_hat| (fp32), which orders like the magnitude; its
+// top digit is bits 30..20 (11 bits), digit 1 bits 19..10, digit 2 bits 9..0.  The K_t-th
+// largest key tau is found exactly, in ONE pass over the tensor plus work on a few percent of it:
+//   guess    a histogram of the top digit over a pseudo-random SAMPLE of the tensor's tiles
+//            (one in 2 ... 16 for large tensors, all of them for small ones) gives a bin
+//            b' that lies, with a safety margin, at or below the bin of tau;
+//   collect  (reads x, x_hat once) every element whose top digit is >= b' is copied, tile by
+//            tile and in index order, into an entry buffer as (top digit - b', 20 low key
+//            bits, position, value of x); the entries are counted per top digit, and digit 1 of
+//            the entries in the two lowest bins is histogrammed on the way;
+//   resolve  the exact counts of the collected bins give the bin of tau (no sampling involved
+//            any more: every element at or above b' is an entry) and the rank inside it; then
+//            digit 1 from its histogram;
 //   digit 2 together with per-tile counts, then ordered compaction into the outbox and delivery
-//   into x_hat:               two walks over the entries only (K_t plus the population of one
-//                             bin: a few percent of the tensor)
-// so a sparse message costs two passes over its tensor.  The host knows nothing about the
-// decisions: a planning phase turns the device-side `sparse` flags into a compact list of work
-// tiles and every other phase runs a fixed-size grid over that list.  All phases can run in one
-// cooperative launch (k_topk_all, bottom of this file).
+//            into x_hat: two walks over the entries only.
+// Where the guess fails -- fewer than K_t elements at or above b', or tau more than one bin
+// above b' -- the segment is selected again the plain way: full histogram of the top digit,
+// exact bin, collect.  With all tiles sampled the guess IS the exact bin, so small tensors and
+// the repeat path are the two-pass radix select without any guessing.
+// The host knows nothing about the decisions: a planning phase turns the device-side `sparse`
+// flags into a compact list of work tiles and every other phase runs a fixed-size grid over that
+// list.  All phases can run in one cooperative launch (k_topk_all, bottom of this file).
 #pragma once
 #include <cooperative_groups.h>
 
@@ -27,21 +35,40 @@ namespace eg {
 constexpr int kTopkCtasPerSm = 8;      // CTAs per multiprocessor of the tile kernels (they loop over the work list)
 constexpr int kTopkSegCtasPerSm = 4;   // ... of the per-segment kernels
 
+// The work tiles of a list are cut into chunks of equal size, kFine of them for every CTA of the
+// tile phases: a phase whose tiles all cost the same gives a CTA kFine consecutive chunks, the
+// sampling phase (whose tiles do not) deals the chunks out round-robin.
+constexpr int kFine = 8;
 struct TopkPlan {
-    int n_sparse;       // segments that send a sparse message in this step
+    int n_sparse;       // segments on the list
     int total_tiles;    // their tiles
-    int chunk;          // work tiles per planned share (one share per CTA of the tile phases)
+    int chunk;          // work tiles per chunk
+    int n_chunks;       // chunks planned
 };
 
-struct TopkState {
+// A list of segments to select from and of their tiles.  List 0: the segments that send a sparse
+// message in this iteration; list 1: those of them that are selected again without guessing.
+struct WorkList {
     TopkPlan* plan;
-    int* sp_seg;               // [P*T] segment id of the q-th sparse segment
-    int* sp_begin;             // [P*T+1] first work tile of the q-th sparse segment
-    int* cta_q;                // [CTAs of the tile phases] sparse slot that holds the first work tile of CTA c's share
+    int* sp_seg;               // [P*T] segment id of the q-th listed segment
+    int* sp_begin;             // [P*T+1] first work tile of the q-th listed segment
+    int* cta_q;                // [chunks] list slot that holds the first work tile of chunk c
+};
+
+constexpr int kOffBins = 8;                // top digits b' .. b'+6 are told apart, anything above counts as b'+7
+constexpr int kOffHist = 2;                // digit 1 is histogrammed for top digits b' and b'+1
+
+struct TopkState {
+    WorkList list[2];
     unsigned int* hist;        // [P*T][kMaxBins]
-    unsigned int* prefix;      // [P*T] key bits resolved so far (after the last digit: tau)
-    unsigned int* remaining;   // [P*T] rank still to resolve (after the last digit: number of
+    unsigned int* prefix;      // [P*T] b' after the guess; key bits resolved so far afterwards (at the end: tau)
+    unsigned int* remaining;   // [P*T] rank still to resolve (at the end: number of
                                //       entries equal to tau that are part of the message)
+    unsigned int* offcnt;      // [P*T][kOffBins] entries per top digit, relative to b'
+    uint8_t* offsel;           // [P*T] top digit of tau, relative to b'
+    uint8_t* redo;             // [P*T] the guess failed: select again without guessing
+    unsigned int* redo_count;  // number of such segments in this iteration
+    unsigned long long* redo_total;   // ... since the context was created or reset
     uint2* ent;                // [P][stride] entries (meta, value bits) of a tile, at the tile's own offset
     int* tile_cand;            // [P][n_tiles][8] entries stored by each warp for the tile
     unsigned int* tile_sub;    // [P][n_tiles][8] of those, (greater than tau) | (equal to tau) << 16
@@ -49,7 +76,9 @@ struct TopkState {
     int2* outbox;              // [P][sum K_t] (index, value bits)
     const long long* out_off;  // [T] start of tensor t inside one replica's outbox
     const long long* count;    // [T] K_t
+    const long long* numel;    // [T] n_t
     long long out_stride;      // sum K_t
+    float guess_margin;        // safety margin of the guess, in standard deviations of the sampled count
 };
 
 __device__ __forceinline__ unsigned int rank_key(float a, float b) {
@@ -59,17 +88,20 @@ __device__ __forceinline__ unsigned int rank_key(float a, float b) {
 // digit 0: bits 30..20, digit 1: bits 19..10, digit 2: bits 9..0
 __device__ __forceinline__ int digit_bits(int digit) { return digit == 0 ? kDigitBits0 : kDigitBits1; }
 
-// One CTA (of kThreads threads): compact list of the sparse segments and of their tiles, in
-// segment order.
-__device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restrict__ sparse,
+// One CTA (of kThreads threads): compact list of the flagged segments and of their tiles, in
+// segment order.  `main_list`: also forget the previous iteration's repeat requests.
+__device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restrict__ flagged,
                                           const int* __restrict__ seg_begin, const TopkState& tk,
-                                          int n_cta) {
+                                          const WorkList& wl, int n_cta, bool main_list) {
     __shared__ int s_cnt[kThreads], s_tiles[kThreads];
     const int per = (S + kThreads - 1) / kThreads;
     const int lo = threadIdx.x * per, hi = min(S, lo + per);
     int cnt = 0, tiles = 0;
-    for (int s = lo; s < hi; ++s)
-        if (sparse[s]) { const int t = s % T; ++cnt; tiles += seg_begin[t + 1] - seg_begin[t]; }
+    for (int s = lo; s < hi; ++s) {
+        if (flagged[s]) { const int t = s % T; ++cnt; tiles += seg_begin[t + 1] - seg_begin[t]; }
+        if (main_list) tk.redo[s] = 0;
+    }
+    if (main_list && threadIdx.x == 0) *tk.redo_count = 0u;
     s_cnt[threadIdx.x] = cnt;
     s_tiles[threadIdx.x] = tiles;
     __syncthreads();
@@ -82,65 +114,71 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
         s_tiles[threadIdx.x] += b;
         __syncthreads();
     }
-    // the tile phases give CTA c the work tiles [c * chunk, (c + 1) * chunk): note for every c
-    // the sparse slot its first tile falls into, so that no phase has to search for it
-    const int chunk = (s_tiles[kThreads - 1] + n_cta - 1) / n_cta;
-    if (threadIdx.x == 0) tk.plan->chunk = chunk;
+    // chunk c holds the work tiles [c * chunk, (c + 1) * chunk): note for every c the list slot
+    // its first tile falls into, so that no phase has to search for it
+    n_cta *= kFine;
+    const int chunk = max(1, (s_tiles[kThreads - 1] + n_cta - 1) / n_cta);
+    if (threadIdx.x == 0) { wl.plan->chunk = chunk; wl.plan->n_chunks = n_cta; }
     int q = s_cnt[threadIdx.x] - cnt, w = s_tiles[threadIdx.x] - tiles;
     for (int s = lo; s < hi; ++s)
-        if (sparse[s]) {
+        if (flagged[s]) {
             const int t = s % T;
             const int w_end = w + seg_begin[t + 1] - seg_begin[t];
-            tk.sp_seg[q] = s;
-            tk.sp_begin[q] = w;
-            for (int c = (w + chunk - 1) / chunk; c < n_cta && c * chunk < w_end; ++c) tk.cta_q[c] = q;
+            wl.sp_seg[q] = s;
+            wl.sp_begin[q] = w;
+            for (int c = (w + chunk - 1) / chunk; c < n_cta && c * chunk < w_end; ++c) wl.cta_q[c] = q;
             ++q;
             w = w_end;
         }
     if (threadIdx.x == kThreads - 1) {
-        tk.plan->n_sparse = s_cnt[threadIdx.x];
-        tk.plan->total_tiles = s_tiles[threadIdx.x];
-        tk.sp_begin[s_cnt[threadIdx.x]] = s_tiles[threadIdx.x];
+        wl.plan->n_sparse = s_cnt[threadIdx.x];
+        wl.plan->total_tiles = s_tiles[threadIdx.x];
+        wl.sp_begin[s_cnt[threadIdx.x]] = s_tiles[threadIdx.x];
     }
+    __syncthreads();      // the shared arrays may be used again by a second call
 }
 
-// Contiguous share of the work-tile list for this CTA and the sparse slot of its first tile.
+// A run of work tiles and the list slot of its first tile.
 struct WorkRange {
     int w0, w1, q;
 };
-// `shares`: planned shares per CTA (a phase may run with a grid `shares` times smaller than planned).
-__device__ __forceinline__ WorkRange work_range(const TopkState& tk, int shares = 1) {
-    const int total = tk.plan->total_tiles;
-    const int chunk = tk.plan->chunk;
+// The chunks [first, first + count) of the list.
+__device__ __forceinline__ WorkRange chunk_range(const WorkList& wl, int first, int count) {
+    const int total = wl.plan->total_tiles;
+    const int chunk = wl.plan->chunk;
     WorkRange r;
-    r.w0 = min(total, (int)blockIdx.x * shares * chunk);
-    r.w1 = min(total, r.w0 + shares * chunk);
-    r.q = (r.w0 < r.w1) ? tk.cta_q[blockIdx.x * shares] : 0;
+    r.w0 = (int)min((long long)total, (long long)first * chunk);
+    r.w1 = (int)min((long long)total, (long long)r.w0 + (long long)count * chunk);
+    r.q = (r.w0 < r.w1) ? wl.cta_q[first] : 0;
     return r;
+}
+// Contiguous share of this CTA.  `shares`: planned shares per CTA (a phase may run with a grid
+// `shares` times smaller than planned).
+__device__ __forceinline__ WorkRange work_range(const WorkList& wl, int shares = 1) {
+    return chunk_range(wl, (int)blockIdx.x * shares * kFine, shares * kFine);
 }
 
 // Walks a CTA's share of the work list.  Segment-level values are re-read only when the
 // segment changes, so consecutive tiles of one tensor cost two dependent loads, not six.
 struct WorkCursor {
     int q, end, s, i, t, first_tile, begin;
-    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int q0) {
+    __device__ __forceinline__ void init(int q0) {
         q = q0 - 1;
         end = -1;
-        (void)tk; (void)tt; (void)T;
     }
     // returns the tile id of work item w; `changed` tells whether a new segment started
-    __device__ __forceinline__ int advance(const TopkState& tk, const TileTable& tt, int T, int w,
+    __device__ __forceinline__ int advance(const WorkList& wl, const TileTable& tt, int T, int w,
                                            bool& changed) {
         changed = false;
         while (w >= end) {
             ++q;
-            if (!EG_INDEX_OK(tt.err, q, tk.plan->n_sparse)) { changed = true; break; }   // (the loop would not end)
-            begin = tk.sp_begin[q];
-            end = tk.sp_begin[q + 1];
+            if (!EG_INDEX_OK(tt.err, q, wl.plan->n_sparse)) { changed = true; break; }   // (the loop would not end)
+            begin = wl.sp_begin[q];
+            end = wl.sp_begin[q + 1];
             changed = true;
         }
         if (changed) {
-            s = tk.sp_seg[q];
+            s = wl.sp_seg[q];
             i = s / T;
             t = s - i * T;
             first_tile = tt.seg_begin[t];
@@ -149,105 +187,196 @@ struct WorkCursor {
     }
 };
 
-// Pass A: histogram of the top digit of every key of the work tiles.
+// ---------------------------------------------------------------------------------------
+// The sample.  Of a tensor with K_t wanted entries one tile (4096 consecutive elements) in
+// 2^shift is looked at, chosen by a hash of the tile's number (the first tile always), so that
+// about 600 of the wanted entries fall into the sample whatever the size of the tensor (the
+// relative error of a count of 600 is 4 %).  Whole tiles, because a tile that is skipped costs
+// nothing, while a tile of which only some lines are read costs as much time as a whole one.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int sample_shift(long long k_t) {
+    int sh = 0;
+    while (sh < 4 && (k_t >> (sh + 1)) >= 600) ++sh;
+    return sh;
+}
+__device__ __forceinline__ bool tile_sampled(unsigned int tile_in_tensor, unsigned int salt, int shift) {
+    unsigned int h = (tile_in_tensor + salt * 0x9E3779B1u) * 0x85EBCA77u;
+    h ^= h >> 15;
+    h *= 0xC2B2AE3Du;
+    h ^= h >> 13;
+    return tile_in_tensor == 0u || (h & ((1u << shift) - 1u)) == 0u;
+}
+
+// Histogram of the top digit of the keys of the work tiles: of the sampled tiles only (`sampled`),
+// or of every element.
 __device__ __forceinline__ void
 topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
-            long long stride, TopkState tk) {
+          long long stride, const TopkState& tk, const WorkList& wl, bool sampled) {
     __shared__ unsigned int s_hist[kMaxBins];
-    WorkRange r = work_range(tk);
-    if (r.w0 >= r.w1) return;
     for (int b = threadIdx.x; b < kMaxBins; b += kThreads) s_hist[b] = 0;
     __syncthreads();
-    WorkCursor cur;
-    cur.init(tk, tt, T, r.q);
-    for (int w = r.w0; w < r.w1; ++w) {
-        bool changed;
-        const int tile = cur.advance(tk, tt, T, w, changed);
-        const int len = tt.length[tile];
-        const long long base = (long long)cur.i * stride + tt.offset[tile];
-        for (int local = threadIdx.x * 4; local < len; local += kThreads * 4) {
-            const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
-            const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
-                                       rank_key(a.w, b.w)};
-            const int nel = min(4, len - local);
+    // every tile costs the same when all are read: one contiguous share; sampled: the chunks are
+    // dealt out round-robin, because the fraction that is read differs from tensor to tensor
+    const int n_chunks = wl.plan->n_chunks;
+    const int step = sampled ? (int)gridDim.x : n_chunks;
+    for (int first = sampled ? (int)blockIdx.x : (int)blockIdx.x * kFine; first < n_chunks; first += step) {
+        const WorkRange r = chunk_range(wl, first, sampled ? 1 : kFine);
+        if (r.w0 >= r.w1) break;
+        WorkCursor cur;
+        cur.init(r.q);
+        int shift = 0;
+        bool any = false;                     // something of the current segment sits in s_hist
+        for (int w = r.w0; w < r.w1; ++w) {
+            bool changed;
+            const int tile = cur.advance(wl, tt, T, w, changed);
+            if (changed) shift = sampled ? sample_shift(tk.count[cur.t]) : 0;
+            if (shift == 0 || tile_sampled((unsigned int)(tile - cur.first_tile), (unsigned int)cur.s, shift)) {
+                any = true;
+                const int len = tt.length[tile];
+                const long long base = (long long)cur.i * stride + tt.offset[tile];
+                for (int local = threadIdx.x * 4; local < len; local += kThreads * 4) {
+                    const float4 a = ld_stream(x + base + local), b = ld_stream(xhat + base + local);
+                    const unsigned int k[4] = {rank_key(a.x, b.x), rank_key(a.y, b.y), rank_key(a.z, b.z),
+                                               rank_key(a.w, b.w)};
+                    const int nel = min(4, len - local);
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (c < nel) atomicAdd(&s_hist[k[c] >> 20], 1u);
-        }
-        // flush when the next tile belongs to another segment (or this was the last one)
-        if (w + 1 == r.w1 || w + 1 >= cur.end) {
-            __syncthreads();
-            unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
-            for (int b = threadIdx.x; b < kMaxBins; b += kThreads) {
-                const unsigned int v = s_hist[b];
-                if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
+                    for (int c = 0; c < 4; ++c)
+                        if (c < nel) atomicAdd(&s_hist[k[c] >> 20], 1u);
+                }
             }
-            __syncthreads();
+            // flush when the next tile belongs to another segment (or this was the last one)
+            if ((w + 1 == r.w1 || w + 1 >= cur.end) && any) {
+                __syncthreads();
+                unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
+                for (int b = threadIdx.x; b < kMaxBins; b += kThreads) {
+                    const unsigned int v = s_hist[b];
+                    if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
+                }
+                __syncthreads();
+                any = false;
+            }
         }
     }
 }
 
-// One warp per sparse segment: pick the bin that holds the wanted rank, counting from the
-// largest key downwards; clear the histogram for the next digit.  The histogram is walked in
+// One warp: the bin of a histogram of `nbins` bins (a multiple of 1024) that holds rank `rem`,
+// counting from the highest bin downwards; the histogram is cleared on the way.  It is walked in
 // blocks of 1024 bins from the top; a lane owns 32 consecutive bins of a block (eight 16-byte
 // loads, all in flight together), one warp scan places the rank in a lane, which then walks
-// its own bins.
-__device__ __forceinline__ void
-topk_pick(int T, TopkState tk, int digit) {
+// its own bins.  Returns false when the histogram holds fewer than `rem` keys.  `bin` and
+// `above_out` (keys in the bins above the chosen one) are valid in every lane.
+__device__ __forceinline__ bool
+pick_bin(unsigned int* gh, int nbins, unsigned int rem, unsigned int& bin, unsigned int& above_out) {
     constexpr int kBlock = 1024, kPer = kBlock / 32;
-    const int nq = tk.plan->n_sparse;
+    const int lane = threadIdx.x & 31;
+    unsigned int above_blocks = 0;      // keys in the blocks already walked
+    bool found = false;                 // the same in every lane
+    unsigned int my_bin = 0, my_above = 0;
+    int owner = 0;
+    for (int blk = nbins / kBlock - 1; blk >= 0; --blk) {
+        uint4* g4 = reinterpret_cast<uint4*>(gh + blk * kBlock + lane * kPer);
+        if (found) {                    // only the clearing is left
+#pragma unroll
+            for (int j = 0; j < kPer / 4; ++j) g4[j] = make_uint4(0u, 0u, 0u, 0u);
+            continue;
+        }
+        unsigned int c[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer / 4; ++j) {
+            const uint4 v = g4[j];
+            c[4 * j] = v.x; c[4 * j + 1] = v.y; c[4 * j + 2] = v.z; c[4 * j + 3] = v.w;
+        }
+#pragma unroll
+        for (int j = 0; j < kPer / 4; ++j) g4[j] = make_uint4(0u, 0u, 0u, 0u);
+        unsigned int mine = 0;
+#pragma unroll
+        for (int z = 0; z < kPer; ++z) mine += c[z];
+        unsigned int inc = mine;        // inclusive sum over this and the higher lanes
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int v = __shfl_down_sync(0xffffffffu, inc, o);
+            if (lane + o < 32) inc += v;
+        }
+        unsigned int above = above_blocks + inc - mine;
+        const bool here = above < rem && rem <= above + mine;
+        if (here) {
+            bool done = false;
+#pragma unroll
+            for (int z = kPer - 1; z >= 0; --z) {
+                if (!done && rem <= above + c[z]) {
+                    my_bin = (unsigned int)(blk * kBlock + lane * kPer + z);
+                    my_above = above;
+                    done = true;
+                }
+                above += c[z];
+            }
+        }
+        const unsigned int where = __ballot_sync(0xffffffffu, here);
+        if (where) { found = true; owner = __ffs(where) - 1; }
+        above_blocks += __shfl_sync(0xffffffffu, inc, 0);
+    }
+    bin = __shfl_sync(0xffffffffu, my_bin, owner);
+    above_out = __shfl_sync(0xffffffffu, my_above, owner);
+    return found;
+}
+
+// One warp per listed segment: digit `digit` (0 or 2) of tau from the segment's histogram.
+// Digit 0 is only taken this way from a histogram over ALL elements of the tensor.
+__device__ __forceinline__ void
+topk_pick(int T, const TopkState& tk, const WorkList& wl, int digit) {
+    const int nq = wl.plan->n_sparse;
     const int nbins = 1 << digit_bits(digit);
     const int lane = threadIdx.x & 31;
     const int nwarps = gridDim.x * kWarps;
     for (int q = blockIdx.x * kWarps + (threadIdx.x >> 5); q < nq; q += nwarps) {
-        const int s = tk.sp_seg[q];
+        const int s = wl.sp_seg[q];
+        const int t = s % T;
+        const unsigned int rem = (digit == 0) ? (unsigned int)tk.count[t] : tk.remaining[s];
+        unsigned int bin, above;
+        const bool found = pick_bin(tk.hist + (long long)s * kMaxBins, nbins, rem, bin, above);
+        if (lane == 0 && found) {
+            const unsigned int old = (digit == 0) ? 0u : tk.prefix[s];
+            tk.prefix[s] = (old << digit_bits(digit)) | bin;
+            tk.remaining[s] = rem - above;
+        }
+    }
+}
+
+// One warp per sparse segment: from the histogram of the sampled tiles, a bin b' that is at or
+// below the bin of the K_t-th largest key unless the sample is off by more than the margin.
+// With m of the tensor's n elements in the sample, the number of sampled elements among the
+// K_t largest has mean K_t m / n and variance about K_t (m / n)(1 - m / n); b' is the bin that
+// holds the sample's rank mean + margin * deviation + 1.  A sample that holds every element
+// (m == n) makes b' the exact bin.  A rank beyond the sample gives b' = 0: everything is collected.
+__device__ __forceinline__ void
+topk_guess(int T, const TopkState& tk, const WorkList& wl) {
+    const int nq = wl.plan->n_sparse;
+    const int lane = threadIdx.x & 31;
+    const int nwarps = gridDim.x * kWarps;
+    for (int q = blockIdx.x * kWarps + (threadIdx.x >> 5); q < nq; q += nwarps) {
+        const int s = wl.sp_seg[q];
         const int t = s % T;
         unsigned int* gh = tk.hist + (long long)s * kMaxBins;
-        const unsigned int rem = (digit == 0) ? (unsigned int)tk.count[t] : tk.remaining[s];
-        unsigned int above_blocks = 0;      // keys in the blocks already walked
-        bool found = false;                 // the same in every lane
-        for (int blk = nbins / kBlock - 1; blk >= 0; --blk) {
-            uint4* g4 = reinterpret_cast<uint4*>(gh + blk * kBlock + lane * kPer);
-            if (found) {                    // only the clearing is left
+        const long long K = tk.count[t], n = tk.numel[t];
+        unsigned int rank = (unsigned int)K;
+        if (sample_shift(K) != 0) {
+            // size of the sample: the tiles are chosen by a hash, so their number varies
+            unsigned int m = 0;
+            const uint4* g4 = reinterpret_cast<const uint4*>(gh);
+            for (int j = lane; j < kMaxBins / 4; j += 32) { const uint4 v = g4[j]; m += v.x + v.y + v.z + v.w; }
 #pragma unroll
-                for (int j = 0; j < kPer / 4; ++j) g4[j] = make_uint4(0u, 0u, 0u, 0u);
-                continue;
+            for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+            if ((long long)m < n) {
+                const float frac = (float)m / (float)n;
+                const float mean = (float)K * frac;
+                const float dev = sqrtf(fmaxf(mean * (1.f - frac), 0.f));
+                const float want = ceilf(mean + tk.guess_margin * dev) + 1.f;
+                rank = (unsigned int)fminf(fmaxf(want, 1.f), 4.0e9f);
             }
-            unsigned int c[kPer];
-#pragma unroll
-            for (int j = 0; j < kPer / 4; ++j) {
-                const uint4 v = g4[j];
-                c[4 * j] = v.x; c[4 * j + 1] = v.y; c[4 * j + 2] = v.z; c[4 * j + 3] = v.w;
-            }
-#pragma unroll
-            for (int j = 0; j < kPer / 4; ++j) g4[j] = make_uint4(0u, 0u, 0u, 0u);
-            unsigned int mine = 0;
-#pragma unroll
-            for (int z = 0; z < kPer; ++z) mine += c[z];
-            unsigned int inc = mine;        // inclusive sum over this and the higher lanes
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned int v = __shfl_down_sync(0xffffffffu, inc, o);
-                if (lane + o < 32) inc += v;
-            }
-            unsigned int above = above_blocks + inc - mine;
-            const bool here = above < rem && rem <= above + mine;
-            if (here) {
-                bool done = false;
-#pragma unroll
-                for (int z = kPer - 1; z >= 0; --z) {
-                    if (!done && rem <= above + c[z]) {
-                        const unsigned int old = (digit == 0) ? 0u : tk.prefix[s];
-                        tk.prefix[s] = (old << digit_bits(digit)) | (unsigned int)(blk * kBlock + lane * kPer + z);
-                        tk.remaining[s] = rem - above;
-                        done = true;
-                    }
-                    above += c[z];
-                }
-            }
-            found = __any_sync(0xffffffffu, here);
-            above_blocks += __shfl_sync(0xffffffffu, inc, 0);
         }
+        unsigned int bin, above;
+        const bool found = pick_bin(gh, kMaxBins, rank, bin, above);
+        if (lane == 0) tk.prefix[s] = found ? bin : 0u;
     }
 }
 
@@ -256,46 +385,47 @@ constexpr int kWarpSpan = kNormTile / kWarps;            // 512 consecutive elem
 constexpr int kSubChunks = kWarpSpan / 128;              // read as 4 chunks of 128 (one float4 per lane)
 static_assert(kWarpSpan == 512 && kSubChunks == 4, "entry words hold a 9-bit position and four 8-bit counts");
 
-// An entry describes one element whose top digit is at least the chosen bin b0:
-//   meta = sure << 29 | (key & 0xfffff) << 9 | position inside the warp's 512 elements
+// An entry describes one element whose top digit is at least b':
+//   meta = min(top digit - b', 7) << 29 | (key & 0xfffff) << 9 | position inside the warp's 512 elements
 //   val  = bits of x at that element
-// `sure` marks a top digit above b0 (the element is part of the message whatever the lower
-// digits say); otherwise the top digit equals b0 and the 20 low key bits decide.
-constexpr unsigned int kEntSure = 1u << 29;
+// Once the bin of tau is known (offsel, relative to b'), an entry with a larger top digit is part
+// of the message whatever its lower digits say, one with a smaller top digit is not, and for the
+// others the 20 low key bits decide.
 __device__ __forceinline__ unsigned int ent_low20(unsigned int meta) { return (meta >> 9) & 0xfffffu; }
-__device__ __forceinline__ bool ent_sure(unsigned int meta) { return (meta & kEntSure) != 0u; }
+__device__ __forceinline__ unsigned int ent_off(unsigned int meta) { return meta >> 29; }
 
 // Warp w of a CTA owns elements [512 w, 512 w + 512) of a tile; its entries start at the same
 // place in the tile's slice of the entry buffer, so the slices can never overlap.
 __device__ __forceinline__ int sub_offset(int len, int w) { return min(len, w * kWarpSpan); }
 
-// Pass B: per tile, every element whose top digit is at least b0 is copied as an entry into the
-// tile's slice of the entry buffer, IN ASCENDING INDEX ORDER inside each warp's sub-slice (the
-// later phases rely on that order: concatenating the sub-slices of a tensor's tiles lists its
-// entries by index).  Digit 1 of the undecided entries is histogrammed on the way.  Nothing is
-// shared between warps except that histogram.  Entries are few (a few percent of the elements),
-// so the pass is split: first every lane only MARKS its sixteen elements in a bit mask (a chunk
-// holds 128 elements, so one warp scan of the four packed 8-bit counts gives every lane its
-// first slot in each chunk); then a lane walks the set bits of its mask -- usually none, one or
-// two -- and builds each entry from the element itself, which it reads again (the line has just
-// been fetched by this warp, so the second read is served by the caches).
+// The collecting pass: per tile, every element whose top digit is at least b' is copied as an
+// entry into the tile's slice of the entry buffer, IN ASCENDING INDEX ORDER inside each warp's
+// sub-slice (the later phases rely on that order: concatenating the sub-slices of a tensor's
+// tiles lists its entries by index).  The entries are counted per top digit and digit 1 of those
+// in the two lowest bins is histogrammed on the way.  Nothing is shared between warps except
+// these counters: a lane marks its elements in four 4-bit masks, one warp scan of the four
+// packed 8-bit counts (a chunk holds 128 elements, so a field cannot overflow) gives every lane
+// its first slot in each chunk.
 __device__ __forceinline__ void
 topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
-               long long stride, TopkState tk) {
+             long long stride, const TopkState& tk, const WorkList& wl) {
     constexpr int kBins1 = 1 << kDigitBits1;
-    __shared__ unsigned int s_hist[kBins1];
-    WorkRange r = work_range(tk);
+    static_assert(kOffHist * kBins1 == kMaxBins, "the digit-1 histograms of two bins share the segment's histogram");
+    __shared__ unsigned int s_hist[kOffHist * kBins1];
+    __shared__ unsigned int s_off[kOffBins];
+    WorkRange r = work_range(wl);
     if (r.w0 >= r.w1) return;
-    for (int b = threadIdx.x; b < kBins1; b += kThreads) s_hist[b] = 0;
+    for (int b = threadIdx.x; b < kOffHist * kBins1; b += kThreads) s_hist[b] = 0;
+    if (threadIdx.x < kOffBins) s_off[threadIdx.x] = 0;
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int mine = warp * kWarpSpan + lane * 4;      // this lane's first element of the tile
     WorkCursor cur;
-    cur.init(tk, tt, T, r.q);
+    cur.init(r.q);
     unsigned int b0 = 0;
     for (int w = r.w0; w < r.w1; ++w) {
         bool changed;
-        const int tile = cur.advance(tk, tt, T, w, changed);
+        const int tile = cur.advance(wl, tt, T, w, changed);
         if (changed) b0 = tk.prefix[cur.s];
         const int i = cur.i;
         const int len = tt.length[tile];
@@ -327,42 +457,102 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
         }
         const unsigned int tot = __shfl_sync(0xffffffffu, inc, 31);
         const unsigned int excl = inc - packed;
-        // first slot of this lane in each chunk, 10 bits each (a sub-slice holds at most 512 entries)
-        unsigned long long first = 0;
+        uint2* ent = tk.ent + base + sub_offset(len, warp);
+        const int room = len - sub_offset(len, warp);      // slots of this sub-slice (bounds-checked build)
         unsigned int chunk_first = 0;
+        auto emit = [&](float xv, float hv, unsigned int pos, unsigned int where) {
+            const unsigned int k = rank_key(xv, hv);
+            const unsigned int off = min((k >> 20) - b0, (unsigned int)(kOffBins - 1));
+            if (!EG_INDEX_OK(tt.err, pos, room)) return;
+            ent[pos] = make_uint2((off << 29) | ((k & 0xfffffu) << 9) | where, __float_as_uint(xv));
+            atomicAdd(&s_off[off], 1u);
+            if (off < (unsigned int)kOffHist) atomicAdd(&s_hist[off * kBins1 + ((k >> 10) & (kBins1 - 1))], 1u);
+        };
 #pragma unroll
         for (int j = 0; j < kSubChunks; ++j) {
-            first |= (unsigned long long)(chunk_first + ((excl >> (8 * j)) & 0xffu)) << (10 * j);
+            const unsigned int m = (mask >> (4 * j)) & 0xfu;
+            if (m) {                                         // few lanes hold an entry in a given chunk
+                unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
+                const unsigned int where = (unsigned int)(j * 128 + lane * 4);
+                if (m & 1u) emit(a[j].x, b[j].x, pos++, where);
+                if (m & 2u) emit(a[j].y, b[j].y, pos++, where + 1);
+                if (m & 4u) emit(a[j].z, b[j].z, pos++, where + 2);
+                if (m & 8u) emit(a[j].w, b[j].w, pos++, where + 3);
+            }
             chunk_first += (tot >> (8 * j)) & 0xffu;
-        }
-        uint2* ent = tk.ent + base + sub_offset(len, warp);
-        const float* xs = x + base + mine;
-        const float* hs = xhat + base + mine;
-        unsigned int todo = mask;
-        while (todo) {
-            const int bit = __ffs(todo) - 1;
-            todo &= todo - 1u;
-            const int j = bit >> 2, e = j * 128 + (bit & 3);       // element mine + e of the tile
-            const float xv = xs[e];
-            const unsigned int k = rank_key(xv, hs[e]);
-            const bool sure = (k >> 20) > b0;
-            // slot: the lane's first slot in the chunk plus its own earlier entries of that chunk
-            const unsigned int pos = (unsigned int)((first >> (10 * j)) & 0x3ffu) +
-                                     __popc(mask & ((1u << bit) - 1u) & (0xfu << (4 * j)));
-            if (!EG_INDEX_OK(tt.err, pos, kWarpSpan) || !EG_INDEX_OK(tt.err, sub_offset(len, warp) + pos, len)) continue;
-            ent[pos] = make_uint2((sure ? kEntSure : 0u) | ((k & 0xfffffu) << 9) | (unsigned int)(lane * 4 + e),
-                                  __float_as_uint(xv));
-            if (!sure) atomicAdd(&s_hist[(k >> 10) & (kBins1 - 1)], 1u);
         }
         if (lane == 0) tk.tile_cand[((long long)i * tt.n_tiles + tile) * kSubSlices + warp] = (int)chunk_first;
         if (w + 1 == r.w1 || w + 1 >= cur.end) {   // last tile of this segment here
             __syncthreads();
             unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
-            for (int b = threadIdx.x; b < kBins1; b += kThreads) {
+            for (int b = threadIdx.x; b < kOffHist * kBins1; b += kThreads) {
                 const unsigned int v = s_hist[b];
                 if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
             }
+            if (threadIdx.x < kOffBins) {
+                const unsigned int v = s_off[threadIdx.x];
+                if (v) { atomicAdd(&tk.offcnt[(long long)cur.s * kOffBins + threadIdx.x], v); s_off[threadIdx.x] = 0; }
+            }
             __syncthreads();
+        }
+    }
+}
+
+// One warp per listed segment, after the collecting pass: the exact counts of the collected bins
+// place tau's top digit (counting K_t entries down from the highest bin) and the rank left
+// inside that bin; digit 1 then comes from the bin's digit-1 histogram.  A segment whose guess
+// did not work out -- fewer than K_t entries, tau in the catch-all bin, or in a bin without a
+// digit-1 histogram -- is marked for the exact repeat instead.  Both histograms and the
+// counters are left cleared.
+__device__ __forceinline__ void
+topk_resolve(int T, const TopkState& tk, const WorkList& wl, bool is_repeat, unsigned int* __restrict__ err) {
+    constexpr int kBins1 = 1 << kDigitBits1;
+    const int nq = wl.plan->n_sparse;
+    const int lane = threadIdx.x & 31;
+    const int nwarps = gridDim.x * kWarps;
+    for (int q = blockIdx.x * kWarps + (threadIdx.x >> 5); q < nq; q += nwarps) {
+        const int s = wl.sp_seg[q];
+        const int t = s % T;
+        unsigned int* oc = tk.offcnt + (long long)s * kOffBins;
+        const unsigned int mine = (lane < kOffBins) ? oc[lane] : 0u;
+        if (lane < kOffBins) oc[lane] = 0u;
+        const unsigned int K = (unsigned int)tk.count[t];
+        unsigned int above = 0;
+        int sel = -1;
+#pragma unroll
+        for (int o = kOffBins - 1; o >= 0; --o) {
+            const unsigned int c = __shfl_sync(0xffffffffu, mine, o);
+            if (sel < 0) {
+                if (K <= above + c) sel = o; else above += c;
+            }
+        }
+        unsigned int* gh = tk.hist + (long long)s * kMaxBins;
+        const bool ok = sel >= 0 && sel < kOffHist;
+        bool found = false;
+        if (ok) {
+            unsigned int bin, above1;
+            const unsigned int rem = K - above;
+            found = pick_bin(gh + sel * kBins1, kBins1, rem, bin, above1);
+            if (lane == 0 && found) {
+                tk.prefix[s] = ((tk.prefix[s] + (unsigned int)sel) << kDigitBits1) | bin;
+                tk.remaining[s] = rem - above1;
+                tk.offsel[s] = (uint8_t)sel;
+            }
+        }
+        // clear what pick_bin has not walked
+        for (int h = 0; h < kOffHist; ++h) {
+            if (ok && h == sel) continue;
+            uint4* g4 = reinterpret_cast<uint4*>(gh + h * kBins1);
+            for (int j = lane; j < kBins1 / 4; j += 32) g4[j] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (lane == 0 && !(ok && found)) {
+            if (is_repeat) {
+                atomicOr(err, kErrTopkSlot);      // an exact bin always resolves
+            } else {
+                tk.redo[s] = 1;
+                atomicAdd(tk.redo_count, 1u);
+                atomicAdd(tk.redo_total, 1ull);
+            }
         }
     }
 }
@@ -377,15 +567,15 @@ struct WarpWalk {
     WorkRange r;
     WorkCursor cur;
     int w;
-    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int shares = 1) {
-        r = work_range(tk, shares);
-        cur.init(tk, tt, T, r.q);
+    __device__ __forceinline__ void init(const WorkList& wl, int shares = 1) {
+        r = work_range(wl, shares);
+        cur.init(r.q);
         w = r.w0 + (int)(threadIdx.x >> 5);
     }
-    __device__ __forceinline__ bool next(const TopkState& tk, const TileTable& tt, int T, WarpTile& z) {
+    __device__ __forceinline__ bool next(const WorkList& wl, const TileTable& tt, int T, WarpTile& z) {
         if (w >= r.w1) return false;
         bool changed;
-        z.tile = cur.advance(tk, tt, T, w, changed);
+        z.tile = cur.advance(wl, tt, T, w, changed);
         z.s = cur.s; z.i = cur.i; z.t = cur.t;
         w += kWarps;
         return true;
@@ -413,16 +603,18 @@ struct TileFeed {
         const int u = (threadIdx.x & 31) / kGroupLanes;
         return tk.tile_cand[((long long)ahead.i * tt.n_tiles + ahead.tile) * kSubSlices + u];
     }
-    __device__ __forceinline__ void init(const TopkState& tk, const TileTable& tt, int T, int shares) {
-        walk.init(tk, tt, T, shares);
-        have = walk.next(tk, tt, T, ahead);
+    __device__ __forceinline__ void init(const TopkState& tk, const WorkList& wl, const TileTable& tt, int T,
+                                         int shares) {
+        walk.init(wl, shares);
+        have = walk.next(wl, tt, T, ahead);
         ahead_mine = have ? fetch(tk, tt) : 0;
     }
-    __device__ __forceinline__ bool next(const TopkState& tk, const TileTable& tt, int T, WarpTile& z, int& mine) {
+    __device__ __forceinline__ bool next(const TopkState& tk, const WorkList& wl, const TileTable& tt, int T,
+                                         WarpTile& z, int& mine) {
         if (!have) return false;
         z = ahead;
         mine = ahead_mine;
-        have = walk.next(tk, tt, T, ahead);
+        have = walk.next(wl, tt, T, ahead);
         ahead_mine = have ? fetch(tk, tt) : 0;
         return true;
     }
@@ -452,19 +644,20 @@ store_tile_counts(const TopkState& tk, long long slot, long long tile_index, uns
 // entries these are already its final (greater than tau, equal to tau) counts, the few tiles
 // that have some are counted again once tau is complete (topk_scan).
 __device__ __forceinline__ void
-topk_digit2(TileTable tt, int T, long long stride, TopkState tk, int shares = 1) {
+topk_digit2(TileTable tt, int T, long long stride, const TopkState& tk, const WorkList& wl, int shares = 1) {
     const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
     TileFeed feed;
-    feed.init(tk, tt, T, shares);
+    feed.init(tk, wl, tt, T, shares);
     WarpTile z;
     int n;                               // entries of this lane's sub-slice
     int s_now = -1;
-    unsigned int want = 0;
+    unsigned int want = 0, sel = 0;
     unsigned int* gh = nullptr;
-    while (feed.next(tk, tt, T, z, n)) {
+    while (feed.next(tk, wl, tt, T, z, n)) {
         if (z.s != s_now) {
             s_now = z.s;
             want = tk.prefix[z.s] & ((1u << kDigitBits1) - 1);      // digit 1 of tau
+            sel = tk.offsel[z.s];
             gh = tk.hist + (long long)z.s * kMaxBins;
         }
         const int len = tt.length[z.tile];
@@ -480,9 +673,9 @@ topk_digit2(TileTable tt, int T, long long stride, TopkState tk, int shares = 1)
 #pragma unroll
             for (int q = 0; q < kRounds; ++q) {
                 const bool live = f0 + q * kGroupLanes < n;
-                const unsigned int low = ent_low20(meta[q]), d1 = low >> kDigitBits2;
-                if (live && (ent_sure(meta[q]) || d1 > want)) ++gt;
-                if (live && !ent_sure(meta[q]) && d1 == want) {
+                const unsigned int off = ent_off(meta[q]), low = ent_low20(meta[q]), d1 = low >> kDigitBits2;
+                if (live && (off > sel || (off == sel && d1 > want))) ++gt;
+                if (live && off == sel && d1 == want) {
                     ++open;
                     atomicAdd(&gh[low & ((1u << kDigitBits2) - 1)], 1u);
                 }
@@ -496,7 +689,8 @@ topk_digit2(TileTable tt, int T, long long stride, TopkState tk, int shares = 1)
 // (greater than tau, equal to tau) per sub-slice and per tile, counted from the entries of one tile
 // by one warp with all 31 bits of tau known.
 __device__ __forceinline__ void
-count_tile_exact(const TileTable& tt, long long stride, const TopkState& tk, int i, int tile, unsigned int tau20) {
+count_tile_exact(const TileTable& tt, long long stride, const TopkState& tk, int i, int tile, unsigned int sel,
+                 unsigned int tau20) {
     const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
     const long long index = (long long)i * tt.n_tiles + tile;
     const int n = tk.tile_cand[index * kSubSlices + u];
@@ -504,9 +698,9 @@ count_tile_exact(const TileTable& tt, long long stride, const TopkState& tk, int
     const uint2* sub = tk.ent + (long long)i * stride + tt.offset[tile] + min(len, u * kWarpSpan);
     unsigned int gt = 0, eq = 0;
     for (int f = r; f < n; f += kGroupLanes) {
-        const unsigned int meta = sub[f].x, low = ent_low20(meta);
-        if (ent_sure(meta) || low > tau20) ++gt;
-        else if (low == tau20) ++eq;
+        const unsigned int meta = sub[f].x, off = ent_off(meta), low = ent_low20(meta);
+        if (off > sel || (off == sel && low > tau20)) ++gt;
+        else if (off == sel && low == tau20) ++eq;
     }
     store_tile_counts(tk, index * kSubSlices, index, gt, eq);
 }
@@ -515,17 +709,17 @@ count_tile_exact(const TileTable& tt, long long stride, const TopkState& tk, int
 // that tau is complete (a handful per tensor, unless many keys tie); then the exclusive prefix
 // of the tile counts, in tile order.
 __device__ __forceinline__ void
-topk_scan(TileTable tt, int T, long long stride, TopkState tk) {
+topk_scan(TileTable tt, int T, long long stride, const TopkState& tk, const WorkList& wl) {
     __shared__ unsigned int s_gt[kWarps], s_eq[kWarps];
     __shared__ unsigned int s_run[2];
-    const int nq = tk.plan->n_sparse;
+    const int nq = wl.plan->n_sparse;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int q = blockIdx.x; q < nq; q += gridDim.x) {
-        const int s = tk.sp_seg[q];
+        const int s = wl.sp_seg[q];
         const int i = s / T, t = s - i * T;
         const int q0 = tt.seg_begin[t], q1 = tt.seg_begin[t + 1];
         uint2* tc = tk.tile_count + (long long)i * tt.n_tiles;
-        const unsigned int tau20 = tk.prefix[s] & 0xfffffu;
+        const unsigned int tau20 = tk.prefix[s] & 0xfffffu, sel = tk.offsel[s];
         for (int c0 = q0; c0 < q1; c0 += 32 * kWarps) {
             // a lane looks at one tile; the warp then counts the marked ones together, one by one
             const int z = c0 + warp * 32 + lane;
@@ -533,7 +727,7 @@ topk_scan(TileTable tt, int T, long long stride, TopkState tk) {
             while (marked) {
                 const int l = __ffs(marked) - 1;
                 marked &= marked - 1u;
-                count_tile_exact(tt, stride, tk, i, c0 + warp * 32 + l, tau20);
+                count_tile_exact(tt, stride, tk, i, c0 + warp * 32 + l, sel, tau20);
             }
         }
         if (threadIdx.x == 0) s_run[0] = s_run[1] = 0;
@@ -575,22 +769,23 @@ topk_scan(TileTable tt, int T, long long stride, TopkState tk) {
 // the four lanes of the sub-slice, and ballots give every lane the number of greater / equal
 // entries before its own.
 __device__ __forceinline__ void
-topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, unsigned int* __restrict__ err,
-           int shares = 1) {
+topk_write(float* xhat, TileTable tt, int T, long long stride, const TopkState& tk, const WorkList& wl,
+           unsigned int* __restrict__ err, int shares = 1) {
     const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
     const unsigned int group = (unsigned int)((1u << kGroupLanes) - 1u) << (u * kGroupLanes);   // lanes of this sub-slice
     const unsigned int lower = ((1u << r) - 1u) << (u * kGroupLanes);                            // ... before this lane
     TileFeed feed;
-    feed.init(tk, tt, T, shares);
+    feed.init(tk, wl, tt, T, shares);
     WarpTile z;
     int n;
     int s_now = -1;
-    unsigned int tau20 = 0, take = 0, K = 0;
+    unsigned int tau20 = 0, take = 0, K = 0, sel = 0;
     int2* out = nullptr;
-    while (feed.next(tk, tt, T, z, n)) {
+    while (feed.next(tk, wl, tt, T, z, n)) {
         if (z.s != s_now) {
             s_now = z.s;
             tau20 = tk.prefix[z.s] & 0xfffffu;
+            sel = tk.offsel[z.s];
             take = tk.remaining[z.s];
             K = (unsigned int)tk.count[z.t];
             out = tk.outbox + (long long)z.i * tk.out_stride + tk.out_off[z.t];
@@ -622,9 +817,9 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, uns
 #pragma unroll
             for (int q = 0; q < kRounds; ++q) {
                 const bool live = f0 + q * kGroupLanes < n;
-                const unsigned int low = ent_low20(e[q].x);
-                const bool g = live && (ent_sure(e[q].x) || low > tau20);
-                const bool same = live && !ent_sure(e[q].x) && low == tau20;
+                const unsigned int off = ent_off(e[q].x), low = ent_low20(e[q].x);
+                const bool g = live && (off > sel || (off == sel && low > tau20));
+                const bool same = live && off == sel && low == tau20;
                 const unsigned int bg = __ballot_sync(0xffffffffu, g), bq = __ballot_sync(0xffffffffu, same);
                 const unsigned int my_gt = run_gt + __popc(bg & lower), my_eq = run_eq + __popc(bq & lower);
                 if (g || (same && my_eq < take)) {
@@ -647,7 +842,7 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, TopkState tk, uns
 // ---------------------------------------------------------------------------------------
 // Launch forms.  k_topk_all runs the whole sequence in ONE cooperative launch with grid-wide
 // barriers between the phases, and every CTA leaves after the first barrier when no segment
-// sends a sparse message in this step -- a quiet step then costs one launch instead of ten.
+// sends a sparse message in this step -- a quiet step then costs one launch.
 // The single-phase kernels below are used for large problems and where a cooperative launch is
 // not available.
 // ---------------------------------------------------------------------------------------
@@ -670,61 +865,90 @@ __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     // a quiet iteration (the decision kernel counted no sparse message) ends here, before any
     // grid-wide barrier: the same answer in every CTA
     if (a.sparse_steps[*a.step_k & 1] == 0) return;
-    if (blockIdx.x == 0) topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, (int)gridDim.x);
+    const WorkList& all = a.tk.list[0];
+    const WorkList& again = a.tk.list[1];
+    if (blockIdx.x == 0) topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, all, (int)gridDim.x, true);
     grid.sync();
-    if (a.tk.plan->n_sparse == 0) return;          // the same for every CTA
-    topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+    if (all.plan->n_sparse == 0) return;          // the same for every CTA
+    topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, all, true);
     grid.sync();
-    topk_pick(a.T, a.tk, 0);
+    topk_guess(a.T, a.tk, all);
     grid.sync();
-    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, all);
     grid.sync();
-    topk_pick(a.T, a.tk, 1);
+    topk_resolve(a.T, a.tk, all, false, a.err);
     grid.sync();
-    topk_digit2(a.tt, a.T, a.stride, a.tk);
+    if (*a.tk.redo_count != 0u) {                  // the same for every CTA
+        if (blockIdx.x == 0) topk_plan(a.S, a.T, a.tk.redo, a.tt.seg_begin, a.tk, again, (int)gridDim.x, false);
+        grid.sync();
+        topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, again, false);
+        grid.sync();
+        topk_pick(a.T, a.tk, again, 0);
+        grid.sync();
+        topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, again);
+        grid.sync();
+        topk_resolve(a.T, a.tk, again, true, a.err);
+        grid.sync();
+    }
+    topk_digit2(a.tt, a.T, a.stride, a.tk, all);
     grid.sync();
-    topk_pick(a.T, a.tk, 2);
+    topk_pick(a.T, a.tk, all, 2);
     grid.sync();
-    topk_scan(a.tt, a.T, a.stride, a.tk);
+    topk_scan(a.tt, a.T, a.stride, a.tk, all);
     grid.sync();
-    topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.err);
+    topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, all, a.err);
 }
 
-// Every single-phase kernel may be launched while the kernel before it drains (programmatic
+// Every single-phase kernel can be launched while the kernel before it drains (programmatic
 // dependent launch): it lets its own successor do the same and then waits for its predecessor
-// before it reads anything.
-__global__ void __launch_bounds__(kThreads) k_topk_plan(TopkArgs a) {
-    pdl_release(); pdl_wait();
-    topk_plan(a.S, a.T, a.sparse, a.tt.seg_begin, a.tk, a.plan_ctas);
+// before it reads anything.  `which` names the work list: 0 for this iteration's sparse
+// segments, 1 for the exact repeat; the kernels of the repeat leave at once when no segment
+// asked for it.
+__device__ __forceinline__ bool topk_enter(const TopkArgs& a, int which) {
+    pdl_release();
+    pdl_wait();
+    return which == 0 || *a.tk.redo_count != 0u;
 }
-__global__ void __launch_bounds__(kThreads) k_topk_hist(TopkArgs a) {
-    pdl_release(); pdl_wait();
-    topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+__global__ void __launch_bounds__(kThreads) k_topk_plan(TopkArgs a, int which) {
+    if (!topk_enter(a, which)) return;
+    topk_plan(a.S, a.T, which ? a.tk.redo : a.sparse, a.tt.seg_begin, a.tk, a.tk.list[which], a.plan_ctas, which == 0);
 }
-__global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int digit) {
-    pdl_release(); pdl_wait();
-    topk_pick(a.T, a.tk, digit);
+__global__ void __launch_bounds__(kThreads) k_topk_hist(TopkArgs a, int which) {
+    if (!topk_enter(a, which)) return;
+    topk_hist(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.tk.list[which], which == 0);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_guess(TopkArgs a) {
+    if (!topk_enter(a, 0)) return;
+    topk_guess(a.T, a.tk, a.tk.list[0]);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int which, int digit) {
+    if (!topk_enter(a, which)) return;
+    topk_pick(a.T, a.tk, a.tk.list[which], digit);
 }
 #ifndef EG_COLLECT_MINB
 #define EG_COLLECT_MINB 4
 #endif
-__global__ void __launch_bounds__(kThreads, EG_COLLECT_MINB) k_topk_collect(TopkArgs a) {
-    pdl_release(); pdl_wait();
-    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk);
+__global__ void __launch_bounds__(kThreads, EG_COLLECT_MINB) k_topk_collect(TopkArgs a, int which) {
+    if (!topk_enter(a, which)) return;
+    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.tk.list[which]);
+}
+__global__ void __launch_bounds__(kThreads) k_topk_resolve(TopkArgs a, int which) {
+    if (!topk_enter(a, which)) return;
+    topk_resolve(a.T, a.tk, a.tk.list[which], which != 0, a.err);
 }
 // The phases that work from the entries run half the planned CTAs, each taking two planned shares.
 constexpr int kEntryShares = 2;
 __global__ void __launch_bounds__(kThreads, 4) k_topk_digit2(TopkArgs a) {
-    pdl_release(); pdl_wait();
-    topk_digit2(a.tt, a.T, a.stride, a.tk, kEntryShares);
+    if (!topk_enter(a, 0)) return;
+    topk_digit2(a.tt, a.T, a.stride, a.tk, a.tk.list[0], kEntryShares);
 }
 __global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) {
-    pdl_release(); pdl_wait();
-    topk_scan(a.tt, a.T, a.stride, a.tk);
+    if (!topk_enter(a, 0)) return;
+    topk_scan(a.tt, a.T, a.stride, a.tk, a.tk.list[0]);
 }
 __global__ void __launch_bounds__(kThreads, 4) k_topk_write(TopkArgs a) {
-    pdl_release(); pdl_wait();
-    topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.err, kEntryShares);
+    if (!topk_enter(a, 0)) return;
+    topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.tk.list[0], a.err, kEntryShares);
 }
 
 }  // namespace eg

@@ -219,6 +219,11 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->tk.hist, 0, S * kMaxBins * sizeof(unsigned int)));
         EG_CUDA(c, cudaMemset(c->tk.prefix, 0, S * sizeof(unsigned int)));
         EG_CUDA(c, cudaMemset(c->tk.remaining, 0, S * sizeof(unsigned int)));
+        EG_CUDA(c, cudaMemset(c->tk.offcnt, 0, S * kOffBins * sizeof(unsigned int)));
+        EG_CUDA(c, cudaMemset(c->tk.offsel, 0, S));
+        EG_CUDA(c, cudaMemset(c->tk.redo, 0, S));
+        EG_CUDA(c, cudaMemset(c->tk.redo_count, 0, sizeof(unsigned int)));
+        EG_CUDA(c, cudaMemset(c->tk.redo_total, 0, sizeof(unsigned long long)));
     }
     if (c->async) {
         EG_CUDA(c, cudaMemset(c->mailbox, 0, (size_t)c->P * c->stride * sizeof(float)));
@@ -498,10 +503,17 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         EG_ALLOC(c->tk.tile_cand, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
         EG_ALLOC(c->tk.tile_sub, (size_t)P * c->tiles_norm.n_tiles * kSubSlices);
         EG_ALLOC(c->tk.ent, (size_t)P * c->stride);
-        EG_ALLOC(c->tk.plan, 1);
-        EG_ALLOC(c->tk.sp_seg, S);
-        EG_ALLOC(c->tk.sp_begin, S + 1);
-        EG_ALLOC(c->tk.cta_q, c->topk_grid);
+        for (int l = 0; l < 2; ++l) {      // the sparse segments of an iteration; those selected again
+            EG_ALLOC(c->tk.list[l].plan, 1);
+            EG_ALLOC(c->tk.list[l].sp_seg, S);
+            EG_ALLOC(c->tk.list[l].sp_begin, S + 1);
+            EG_ALLOC(c->tk.list[l].cta_q, (size_t)c->topk_grid * kFine);
+        }
+        EG_ALLOC(c->tk.offcnt, S * kOffBins);
+        EG_ALLOC(c->tk.offsel, S);
+        EG_ALLOC(c->tk.redo, S);
+        EG_ALLOC(c->tk.redo_count, 1);
+        EG_ALLOC(c->tk.redo_total, 1);
         EG_ALLOC(c->tk.outbox, (size_t)P * c->out_stride);
         {
             // one cooperative launch needs all its CTAs resident at the same time
@@ -520,6 +532,13 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
         }
         c->tk.out_off = c->d_out_off;
         c->tk.count = c->d_kcount;
+        c->tk.numel = c->d_numel;
+        {
+            // safety margin of the guessed bin, in standard deviations of the sampled count; a
+            // negative value makes the guess fail on purpose (exercises the exact repeat)
+            const char* e = getenv("EG_TOPK_GUESS_MARGIN");
+            c->tk.guess_margin = e && *e ? (float)atof(e) : 5.0f;
+        }
         c->tk.out_stride = c->out_stride;
     }
 #undef EG_ALLOC
@@ -601,6 +620,18 @@ eg_status eg_layout(const eg_ctx* c, int64_t* tensor_offset_host, int64_t* repli
 eg_status eg_topk_count(const eg_ctx* c, int t, int64_t* k_t_host) {
     if (!c || t < 0 || t >= c->T || !k_t_host) return EG_ERR_INVALID;
     *k_t_host = c->kcount[t];
+    return EG_OK;
+}
+
+eg_status eg_topk_repeat_count(eg_ctx* c, uint64_t* repeats_host) {
+    if (!c || !repeats_host) return EG_ERR_INVALID;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    unsigned long long v = 0;
+    if (c->topk.enabled)
+        EG_CUDA(c, cudaMemcpy(&v, c->tk.redo_total, sizeof(v), cudaMemcpyDeviceToHost));
+    *repeats_host = v;
     return EG_OK;
 }
 
@@ -718,21 +749,29 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                                                    dim3(kThreads), args, 0, stream));
             launches += 1;
         } else {
-            // Nine launches.  They can be started as dependent launches (each waits on the device,
-            // first thing it does, for the kernel before it), but measured on 64 x 25.6 M elements
-            // that made the sequence 30 % slower, so it is only done on request (EG_TOPK_PDL).
+            // Fourteen launches, five of which (the exact repeat for segments whose guessed bin
+            // did not work out) leave at once in an ordinary iteration.  They can be started as
+            // dependent launches (each waits on the device, first thing it does, for the kernel
+            // before it), but measured on 64 x 25.6 M elements that made the sequence 30 % slower,
+            // so it is only done on request (EG_TOPK_PDL).
             const bool pdl = !c->timing && !c->no_pdl && c->topk_pdl;
-            const dim3 tile_blocks(tile_grid), entry_blocks(tile_grid / kEntryShares), seg_blocks(seg_grid);
-            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, dim3(1), dim3(kThreads), 0, stream, ta));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, dim3(kThreads), 0, stream, ta));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, dim3(kThreads), 0, stream, ta, 0));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, tile_blocks, dim3(kThreads), 0, stream, ta));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, dim3(kThreads), 0, stream, ta, 1));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_digit2, entry_blocks, dim3(kThreads), 0, stream, ta));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, dim3(kThreads), 0, stream, ta, 2));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_scan, seg_blocks, dim3(kThreads), 0, stream, ta));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_write, entry_blocks, dim3(kThreads), 0, stream, ta));
-            launches += 9;
+            const dim3 one(1), tile_blocks(tile_grid), entry_blocks(tile_grid / kEntryShares), seg_blocks(seg_grid);
+            const dim3 threads(kThreads);
+            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, threads, 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, threads, 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_guess, seg_blocks, threads, 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, tile_blocks, threads, 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_resolve, seg_blocks, threads, 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, threads, 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, threads, 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, threads, 0, stream, ta, 1, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, tile_blocks, threads, 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_resolve, seg_blocks, threads, 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_digit2, entry_blocks, threads, 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, threads, 0, stream, ta, 0, 2));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_scan, seg_blocks, threads, 0, stream, ta));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_write, entry_blocks, threads, 0, stream, ta));
+            launches += 14;
         }
     }
     // a3 + a5: dense snapshot, consensus average, SGD

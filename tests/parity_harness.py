@@ -48,6 +48,7 @@ class Report:
     max_norm_rel: float = 0.0
     params_bit_exact: bool = True
     launches: int = 0
+    topk_repeats: int = 0
     seconds: dict = field(default_factory=lambda: {"inputs": 0.0, "oracle": 0.0, "compare": 0.0})
 
 
@@ -324,6 +325,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
                 assert arrivals == o.arrivals, f"arrivals, step {k}"
         lap("compare")
 
+    rep.topk_repeats = eg.topk_repeat_count()
     eg.close()
     o.close()
     return rep

@@ -357,12 +357,32 @@ def test_topk_degenerate_all_keys_equal(separate, monkeypatch):
 
 
 def test_topk_with_separate_launches(monkeypatch):
-    """The nine single-phase Top-K launches (fallback where a cooperative launch is unavailable)."""
+    """The single-phase Top-K launches (fallback where a cooperative launch is unavailable)."""
     monkeypatch.setenv("EG_TOPK_SEPARATE_LAUNCHES", "1")
     wl = W.synthetic(3, RAGGED, steps=10, lr=0.1, grad_sigma=0.01, topk=(10, 100))
     rep = lockstep(wl, init="distinct", outbox_samples=64)
     assert rep.params_bit_exact and rep.sparse_checked > 5
-    assert rep.launches == 10 * 12
+    assert rep.launches == 10 * 17
+
+
+@pytest.mark.parametrize("separate", [False, True])
+@pytest.mark.parametrize("margin", ["-8", "0", "5"])
+def test_topk_guess_and_exact_repeat(separate, margin, monkeypatch):
+    """Tensors large enough to be sampled (2^20 + 1 and 300,000 elements at 1 % and 7 %).  A negative
+    margin makes every guessed bin too high, so every such message takes the exact repeat; margin 0
+    fails about every other time; the default margin practically never.  The messages are the
+    oracle's in all three cases."""
+    monkeypatch.setenv("EG_TOPK_GUESS_MARGIN", margin)
+    if separate:
+        monkeypatch.setenv("EG_TOPK_SEPARATE_LAUNCHES", "1")
+    for frac in ((1, 100), (7, 100)):
+        wl = W.synthetic(3, [5, 300000, 4097, (1 << 20) + 1, 70000], steps=8, lr=0.1, grad_sigma=0.01, topk=frac)
+        rep = lockstep(wl, init="distinct", outbox_samples=10 ** 6, carry=True)
+        assert rep.params_bit_exact and rep.sparse_checked > 10
+        if margin == "-8":
+            assert rep.topk_repeats >= 6          # the two sampled tensors of three replicas, several iterations
+        if margin == "5":
+            assert rep.topk_repeats <= 1
 
 
 @pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_REGISTER])
@@ -467,6 +487,7 @@ def test_config2_resnet20(carry, kernel):
 def _report(name, rep):
     """What a configured run did, on the test log (shown with -s or on failure)."""
     print(f"{name}: steps {rep.steps}, events {rep.events}, sparse messages checked {rep.sparse_checked}, "
+          f"Top-K messages selected again exactly {rep.topk_repeats}, "
           f"largest norm error {rep.max_norm_rel:.2e} of its tolerance, parameters bit-exact {rep.params_bit_exact}, "
           f"decisions within 1e-6 of the threshold that differed {rep.near_threshold}; seconds spent on "
           + ", ".join(f"{k} {v:.1f}" for k, v in rep.seconds.items()))
