@@ -36,14 +36,15 @@ constexpr int kTopkCtasPerSm = 8;      // CTAs per multiprocessor of the tile ke
 constexpr int kTopkSegCtasPerSm = 4;   // ... of the per-segment kernels
 
 // The work tiles of a list are cut into chunks of equal size, kFine of them for every CTA of the
-// tile phases: a phase whose tiles all cost the same gives a CTA kFine consecutive chunks, the
-// sampling phase (whose tiles do not) deals the chunks out round-robin.
-constexpr int kFine = 8;
+// tile phases: a phase whose tiles all cost the same gives a CTA kFine consecutive chunks, in the
+// sampling phase (whose tiles do not) a CTA takes the next chunk whenever it has finished one.
+constexpr int kFine = 16;
 struct TopkPlan {
     int n_sparse;       // segments on the list
     int total_tiles;    // their tiles
     int chunk;          // work tiles per chunk
     int n_chunks;       // chunks planned
+    int ticket;         // next chunk to hand out in the sampling phase
 };
 
 // A list of segments to select from and of their tiles.  List 0: the segments that send a sparse
@@ -118,7 +119,7 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
     // its first tile falls into, so that no phase has to search for it
     n_cta *= kFine;
     const int chunk = max(1, (s_tiles[kThreads - 1] + n_cta - 1) / n_cta);
-    if (threadIdx.x == 0) { wl.plan->chunk = chunk; wl.plan->n_chunks = n_cta; }
+    if (threadIdx.x == 0) { wl.plan->chunk = chunk; wl.plan->n_chunks = n_cta; wl.plan->ticket = 0; }
     int q = s_cnt[threadIdx.x] - cnt, w = s_tiles[threadIdx.x] - tiles;
     for (int s = lo; s < hi; ++s)
         if (flagged[s]) {
@@ -215,11 +216,19 @@ topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable
     __shared__ unsigned int s_hist[kMaxBins];
     for (int b = threadIdx.x; b < kMaxBins; b += kThreads) s_hist[b] = 0;
     __syncthreads();
-    // every tile costs the same when all are read: one contiguous share; sampled: the chunks are
-    // dealt out round-robin, because the fraction that is read differs from tensor to tensor
+    // every tile costs the same when all are read: one contiguous share; sampled: chunk after
+    // chunk as handed out by a counter, because the fraction that is read differs from tensor to
+    // tensor
+    __shared__ int s_ticket;
     const int n_chunks = wl.plan->n_chunks;
-    const int step = sampled ? (int)gridDim.x : n_chunks;
-    for (int first = sampled ? (int)blockIdx.x : (int)blockIdx.x * kFine; first < n_chunks; first += step) {
+    for (int first = (int)blockIdx.x * kFine;;) {
+        if (sampled) {
+            __syncthreads();                  // everybody has read the previous ticket
+            if (threadIdx.x == 0) s_ticket = atomicAdd(&wl.plan->ticket, 1);
+            __syncthreads();
+            first = s_ticket;
+        }
+        if (first >= n_chunks) break;
         const WorkRange r = chunk_range(wl, first, sampled ? 1 : kFine);
         if (r.w0 >= r.w1) break;
         WorkCursor cur;
@@ -256,6 +265,7 @@ topk_hist(const float* __restrict__ x, const float* __restrict__ xhat, TileTable
                 any = false;
             }
         }
+        if (!sampled) break;
     }
 }
 
@@ -403,9 +413,14 @@ __device__ __forceinline__ int sub_offset(int len, int w) { return min(len, w * 
 // sub-slice (the later phases rely on that order: concatenating the sub-slices of a tensor's
 // tiles lists its entries by index).  The entries are counted per top digit and digit 1 of those
 // in the two lowest bins is histogrammed on the way.  Nothing is shared between warps except
-// these counters: a lane marks its elements in four 4-bit masks, one warp scan of the four
-// packed 8-bit counts (a chunk holds 128 elements, so a field cannot overflow) gives every lane
-// its first slot in each chunk.
+// these counters.  Entries are few, so the work is split: every lane MARKS its sixteen elements
+// in four 4-bit masks (one floating-point comparison per element: non-negative floats order
+// like their bit patterns, so |x - x_hat| >= the float whose bits are b' << 20 says the same as
+// the comparison of the top digits); one warp scan of the four packed 8-bit counts (a chunk
+// holds 128 elements, so a field cannot overflow) gives every lane its first slot in each chunk;
+// the marked elements go to a small per-warp staging area in slot order, and the warp then
+// turns them into entries side by side, one per lane, with coalesced stores.
+constexpr int kStage = 128;     // staged elements per warp and tile; fuller sub-slices are written directly
 __device__ __forceinline__ void
 topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
              long long stride, const TopkState& tk, const WorkList& wl) {
@@ -413,6 +428,8 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
     static_assert(kOffHist * kBins1 == kMaxBins, "the digit-1 histograms of two bins share the segment's histogram");
     __shared__ unsigned int s_hist[kOffHist * kBins1];
     __shared__ unsigned int s_off[kOffBins];
+    __shared__ float2 s_pair[kWarps][kStage];             // (x, x_hat) of a marked element
+    __shared__ unsigned short s_where[kWarps][kStage];    // its position inside the warp's 512 elements
     WorkRange r = work_range(wl);
     if (r.w0 >= r.w1) return;
     for (int b = threadIdx.x; b < kOffHist * kBins1; b += kThreads) s_hist[b] = 0;
@@ -423,31 +440,59 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
     WorkCursor cur;
     cur.init(r.q);
     unsigned int b0 = 0;
+    float thr = 0.f;
+    // one entry from an element: counted, digit 1 histogrammed, stored at slot `pos`
+    auto emit = [&](uint2* ent, int room, float xv, float hv, unsigned int pos, unsigned int where) {
+        const unsigned int k = rank_key(xv, hv);
+        const unsigned int off = min((k >> 20) - b0, (unsigned int)(kOffBins - 1));
+        if (!EG_INDEX_OK(tt.err, pos, room)) return;
+        ent[pos] = make_uint2((off << 29) | ((k & 0xfffffu) << 9) | where, __float_as_uint(xv));
+        atomicAdd(&s_off[off], 1u);
+        if (off < (unsigned int)kOffHist) atomicAdd(&s_hist[off * kBins1 + ((k >> 10) & (kBins1 - 1))], 1u);
+    };
     for (int w = r.w0; w < r.w1; ++w) {
         bool changed;
         const int tile = cur.advance(wl, tt, T, w, changed);
-        if (changed) b0 = tk.prefix[cur.s];
+        if (changed) { b0 = tk.prefix[cur.s]; thr = __uint_as_float(b0 << 20); }
         const int i = cur.i;
         const int len = tt.length[tile];
         const long long base = (long long)i * stride + tt.offset[tile];
         float4 a[kSubChunks], b[kSubChunks];
-#pragma unroll
-        for (int j = 0; j < kSubChunks; ++j) {
-            const int local = mine + j * 128;
-            a[j] = b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (local < len) { a[j] = ld_stream(x + base + local); b[j] = ld_stream(xhat + base + local); }
-        }
         unsigned int mask = 0, packed = 0;      // bit 4j+c: element c of chunk j is an entry
+        if (len == kNormTile) {                 // a whole tile: no element needs a length test
 #pragma unroll
-        for (int j = 0; j < kSubChunks; ++j) {
-            const int nel = len - (mine + j * 128);   // live elements of this float4 (<= 0: none)
-            unsigned int m = 0;
-            m |= (0 < nel && (rank_key(a[j].x, b[j].x) >> 20) >= b0) ? 1u : 0u;
-            m |= (1 < nel && (rank_key(a[j].y, b[j].y) >> 20) >= b0) ? 2u : 0u;
-            m |= (2 < nel && (rank_key(a[j].z, b[j].z) >> 20) >= b0) ? 4u : 0u;
-            m |= (3 < nel && (rank_key(a[j].w, b[j].w) >> 20) >= b0) ? 8u : 0u;
-            mask |= m << (4 * j);
-            packed |= (unsigned int)__popc(m) << (8 * j);
+            for (int j = 0; j < kSubChunks; ++j) {
+                a[j] = ld_stream(x + base + mine + j * 128);
+                b[j] = ld_stream(xhat + base + mine + j * 128);
+            }
+#pragma unroll
+            for (int j = 0; j < kSubChunks; ++j) {
+                unsigned int m = 0;
+                m |= !(fabsf(__fsub_rn(a[j].x, b[j].x)) < thr) ? 1u : 0u;
+                m |= !(fabsf(__fsub_rn(a[j].y, b[j].y)) < thr) ? 2u : 0u;
+                m |= !(fabsf(__fsub_rn(a[j].z, b[j].z)) < thr) ? 4u : 0u;
+                m |= !(fabsf(__fsub_rn(a[j].w, b[j].w)) < thr) ? 8u : 0u;
+                mask |= m << (4 * j);
+                packed |= (unsigned int)__popc(m) << (8 * j);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kSubChunks; ++j) {
+                const int local = mine + j * 128;
+                a[j] = b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (local < len) { a[j] = ld_stream(x + base + local); b[j] = ld_stream(xhat + base + local); }
+            }
+#pragma unroll
+            for (int j = 0; j < kSubChunks; ++j) {
+                const int nel = len - (mine + j * 128);   // live elements of this float4 (<= 0: none)
+                unsigned int m = 0;
+                m |= (0 < nel && !(fabsf(__fsub_rn(a[j].x, b[j].x)) < thr)) ? 1u : 0u;
+                m |= (1 < nel && !(fabsf(__fsub_rn(a[j].y, b[j].y)) < thr)) ? 2u : 0u;
+                m |= (2 < nel && !(fabsf(__fsub_rn(a[j].z, b[j].z)) < thr)) ? 4u : 0u;
+                m |= (3 < nel && !(fabsf(__fsub_rn(a[j].w, b[j].w)) < thr)) ? 8u : 0u;
+                mask |= m << (4 * j);
+                packed |= (unsigned int)__popc(m) << (8 * j);
+            }
         }
         unsigned int inc = packed;
 #pragma unroll
@@ -457,31 +502,47 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
         }
         const unsigned int tot = __shfl_sync(0xffffffffu, inc, 31);
         const unsigned int excl = inc - packed;
+        const unsigned int total = (tot & 0xffu) + ((tot >> 8) & 0xffu) + ((tot >> 16) & 0xffu) + (tot >> 24);
         uint2* ent = tk.ent + base + sub_offset(len, warp);
         const int room = len - sub_offset(len, warp);      // slots of this sub-slice (bounds-checked build)
-        unsigned int chunk_first = 0;
-        auto emit = [&](float xv, float hv, unsigned int pos, unsigned int where) {
-            const unsigned int k = rank_key(xv, hv);
-            const unsigned int off = min((k >> 20) - b0, (unsigned int)(kOffBins - 1));
-            if (!EG_INDEX_OK(tt.err, pos, room)) return;
-            ent[pos] = make_uint2((off << 29) | ((k & 0xfffffu) << 9) | where, __float_as_uint(xv));
-            atomicAdd(&s_off[off], 1u);
-            if (off < (unsigned int)kOffHist) atomicAdd(&s_hist[off * kBins1 + ((k >> 10) & (kBins1 - 1))], 1u);
-        };
+        if (total <= (unsigned int)kStage) {
+            unsigned int chunk_first = 0;
 #pragma unroll
-        for (int j = 0; j < kSubChunks; ++j) {
-            const unsigned int m = (mask >> (4 * j)) & 0xfu;
-            if (m) {                                         // few lanes hold an entry in a given chunk
-                unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
-                const unsigned int where = (unsigned int)(j * 128 + lane * 4);
-                if (m & 1u) emit(a[j].x, b[j].x, pos++, where);
-                if (m & 2u) emit(a[j].y, b[j].y, pos++, where + 1);
-                if (m & 4u) emit(a[j].z, b[j].z, pos++, where + 2);
-                if (m & 8u) emit(a[j].w, b[j].w, pos++, where + 3);
+            for (int j = 0; j < kSubChunks; ++j) {
+                const unsigned int m = (mask >> (4 * j)) & 0xfu;
+                if (m) {                                         // few lanes hold an entry in a given chunk
+                    unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
+                    const unsigned short where = (unsigned short)(j * 128 + lane * 4);
+                    if (m & 1u) { s_pair[warp][pos] = make_float2(a[j].x, b[j].x); s_where[warp][pos++] = where; }
+                    if (m & 2u) { s_pair[warp][pos] = make_float2(a[j].y, b[j].y); s_where[warp][pos++] = where + 1; }
+                    if (m & 4u) { s_pair[warp][pos] = make_float2(a[j].z, b[j].z); s_where[warp][pos++] = where + 2; }
+                    if (m & 8u) { s_pair[warp][pos] = make_float2(a[j].w, b[j].w); s_where[warp][pos++] = where + 3; }
+                }
+                chunk_first += (tot >> (8 * j)) & 0xffu;
             }
-            chunk_first += (tot >> (8 * j)) & 0xffu;
+            __syncwarp();
+            for (unsigned int e = lane; e < total; e += 32) {
+                const float2 v = s_pair[warp][e];
+                emit(ent, room, v.x, v.y, e, s_where[warp][e]);
+            }
+            __syncwarp();
+        } else {
+            unsigned int chunk_first = 0;
+#pragma unroll
+            for (int j = 0; j < kSubChunks; ++j) {
+                const unsigned int m = (mask >> (4 * j)) & 0xfu;
+                if (m) {
+                    unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
+                    const unsigned int where = (unsigned int)(j * 128 + lane * 4);
+                    if (m & 1u) emit(ent, room, a[j].x, b[j].x, pos++, where);
+                    if (m & 2u) emit(ent, room, a[j].y, b[j].y, pos++, where + 1);
+                    if (m & 4u) emit(ent, room, a[j].z, b[j].z, pos++, where + 2);
+                    if (m & 8u) emit(ent, room, a[j].w, b[j].w, pos++, where + 3);
+                }
+                chunk_first += (tot >> (8 * j)) & 0xffu;
+            }
         }
-        if (lane == 0) tk.tile_cand[((long long)i * tt.n_tiles + tile) * kSubSlices + warp] = (int)chunk_first;
+        if (lane == 0) tk.tile_cand[((long long)i * tt.n_tiles + tile) * kSubSlices + warp] = (int)total;
         if (w + 1 == r.w1 || w + 1 >= cur.end) {   // last tile of this segment here
             __syncthreads();
             unsigned int* gh = tk.hist + (long long)cur.s * kMaxBins;
@@ -763,6 +824,10 @@ topk_scan(TileTable tt, int T, long long stride, const TopkState& tk, const Work
 // (index, value) pairs are written into the mailbox x_hat, which is what the receivers hold
 // once the message has arrived.  Works from the entries alone (a few percent of the tensor);
 // x and x_hat are not read again.
+// (Delivering from the averaging kernel that runs next -- it reads x and x_hat anyway and can
+// tell the entries greater than tau by one comparison -- was built and measured: the scattered
+// words here cost as much as the comparisons there, and the quiet iterations paid for the
+// larger kernel, so the delivery stayed here.)
 // An entry is selected if key > tau, or key == tau and fewer than `remaining` equal keys
 // precede it in the tensor.  Its slot is (#greater before it) + min(#equal before it, remaining).
 // One warp per tile; within a sub-slice the entries are taken in index order, four at a time by
@@ -936,9 +1001,15 @@ __global__ void __launch_bounds__(kThreads) k_topk_resolve(TopkArgs a, int which
     if (!topk_enter(a, which)) return;
     topk_resolve(a.T, a.tk, a.tk.list[which], which != 0, a.err);
 }
-// The phases that work from the entries run half the planned CTAs, each taking two planned shares.
-constexpr int kEntryShares = 2;
-__global__ void __launch_bounds__(kThreads, 4) k_topk_digit2(TopkArgs a) {
+// The phases that work from the entries: planned shares per CTA and CTAs per multiprocessor.
+#ifndef EG_ENTRY_SHARES
+#define EG_ENTRY_SHARES 2
+#endif
+#ifndef EG_ENTRY_MINB
+#define EG_ENTRY_MINB 4
+#endif
+constexpr int kEntryShares = EG_ENTRY_SHARES;
+__global__ void __launch_bounds__(kThreads, EG_ENTRY_MINB) k_topk_digit2(TopkArgs a) {
     if (!topk_enter(a, 0)) return;
     topk_digit2(a.tt, a.T, a.stride, a.tk, a.tk.list[0], kEntryShares);
 }
@@ -946,7 +1017,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) {
     if (!topk_enter(a, 0)) return;
     topk_scan(a.tt, a.T, a.stride, a.tk, a.tk.list[0]);
 }
-__global__ void __launch_bounds__(kThreads, 4) k_topk_write(TopkArgs a) {
+__global__ void __launch_bounds__(kThreads, EG_ENTRY_MINB) k_topk_write(TopkArgs a) {
     if (!topk_enter(a, 0)) return;
     topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, a.tk.list[0], a.err, kEntryShares);
 }

@@ -224,6 +224,7 @@ eg_status init_state(eg_ctx* c) {
         EG_CUDA(c, cudaMemset(c->tk.redo, 0, S));
         EG_CUDA(c, cudaMemset(c->tk.redo_count, 0, sizeof(unsigned int)));
         EG_CUDA(c, cudaMemset(c->tk.redo_total, 0, sizeof(unsigned long long)));
+        for (int l = 0; l < 2; ++l) EG_CUDA(c, cudaMemset(c->tk.list[l].plan, 0, sizeof(TopkPlan)));
     }
     if (c->async) {
         EG_CUDA(c, cudaMemset(c->mailbox, 0, (size_t)c->P * c->stride * sizeof(float)));
