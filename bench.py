@@ -46,19 +46,57 @@ FUSED_BYTES_PER_ELEMENT = 16       # fused kernel: reads x, g, touches x_hat onc
 MOMENTUM_BYTES_PER_ELEMENT = 8     # --momentum: the velocity is read and written once more
 
 # DRAM traffic of the fused kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum per launch on the default workload), keyed by the hash of the kernel
-# sources it was taken with; reported as null once the sources change.
+# dram__bytes_write.sum per launch, captured on a prefix of the default workload), keyed by the
+# hash of the kernel sources the timed configuration launches.  Once any of those sources has
+# changed the figure is reported as null, together with what it was captured with.
 FUSED_TRAFFIC_ELEMENTS = 16 * 11173962     # element-replicas of one launch on the default workload
-FUSED_TRAFFIC = {"bd6fa63752f4": 2.636e9}   # profiles/k_fused_pipe_resnet18_first45tensors.md
+FUSED_TRAFFIC = {
+    # sources of a dense run: hash -> (bytes per launch of the default workload, where the counters are)
+    "dense": {"bd6fa63752f4": (2.636e9, "profiles/k_fused_pipe_resnet18_first45tensors.md")},
+}
+DENSE_SOURCES = ("eg_common.cuh", "eg_norm.cuh", "eg_fused.cuh", "eg_fused_pipe.cuh")
 
 
-def kernel_source_hash() -> str:
+def kernel_sources(wl) -> tuple:
+    """The kernel sources a run of this workload launches from (the single-launch kernel serves
+    the small dense configurations, the Top-K kernels the Top-K ones)."""
+    names = list(DENSE_SOURCES)
+    if wl.topk:
+        names.append("eg_topk.cuh")
+    elif wl.P <= 16 and wl.N <= 300000:
+        names.append("eg_step_small.cuh")
+    return tuple(names)
+
+
+def kernel_source_hash(names=DENSE_SOURCES) -> str:
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2103_07454_b200", "csrc")
-    for name in ("eg_common.cuh", "eg_norm.cuh", "eg_fused.cuh", "eg_fused_pipe.cuh"):
+    for name in names:
         with open(os.path.join(d, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:12]
+
+
+def fused_traffic(wl, elems: int, momentum) -> dict:
+    """`traffic` of the roofline object, and what to say when the counters are out of date."""
+    names = kernel_sources(wl)
+    current = kernel_source_hash(names)
+    if momentum is not None or names != DENSE_SOURCES:
+        # counters exist for the default kernel on dense runs only
+        return {"traffic": None, "traffic_note": "no capture for this configuration's kernels",
+                "traffic_sources": list(names), "traffic_sources_hash": current}
+    known = FUSED_TRAFFIC["dense"]
+    if current in known:
+        per_launch, where = known[current]
+        # the capture was taken on a prefix of the default workload; a streaming kernel's traffic
+        # grows with the elements, so it is scaled to the elements of one launch of this run
+        return {"traffic": per_launch * elems / FUSED_TRAFFIC_ELEMENTS, "traffic_from": where,
+                "traffic_sources": list(names), "traffic_sources_hash": current}
+    captured, (_, where) = next(iter(known.items()))
+    return {"traffic": None,
+            "traffic_stale_since": f"kernel sources changed after the capture in {where} "
+                                   f"(captured with sources hash {captured}, now {current})",
+            "traffic_sources": list(names), "traffic_sources_hash": current}
 
 
 # ----------------------------------------------------------------------------------------
@@ -470,16 +508,12 @@ def run_native(args):
 
     fused_ms = main["kernel_ms"]["fused"]
     achieved = elems * (FUSED_BYTES_PER_ELEMENT + extra) / fused_ms / 1e6 if fused_ms else None
-    # the capture was taken on a prefix of the default workload; a streaming kernel's traffic
-    # grows with the elements, so it is scaled to the elements of one launch of this run
-    traffic = FUSED_TRAFFIC.get(kernel_source_hash()) if args.momentum is None else None
-    if traffic is not None:
-        traffic *= elems / FUSED_TRAFFIC_ELEMENTS
+    traffic = fused_traffic(wl, elems, args.momentum)
     roofline = {"bound": "hbm", "kernel": "k_fused_pipe" if args.momentum is None else "k_fused_pipe_momentum",
                 "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
-                "traffic": traffic,
+                **traffic,
                 "algorithmic_bytes_per_launch": elems * (FUSED_BYTES_PER_ELEMENT + extra),
                 "kernel_ms": fused_ms,
                 "kernel_timed_in": "a second pass over the same K steps with CUDA events around every kernel "

@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_the_requested_build():
+    """A run that was asked to use the bounds-checked library (EG_EXPECT_DEBUG) must not fall back
+    silently to the ordinary one."""
+    if os.environ.get("EG_EXPECT_DEBUG"):
+        from paper_2103_07454_b200 import binding
+        assert binding.load_library().eg_debug_build() == 1, "EG_LIBRARY does not name the bounds-checked build"
+    yield

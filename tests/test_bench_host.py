@@ -50,3 +50,28 @@ def test_reference_arm_prints_one_json_line():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["config"]["workload"] == "mlp_p4_dense"
+
+
+def test_captured_traffic_is_tied_to_the_kernel_sources(monkeypatch):
+    """`roofline.traffic` comes from an ncu capture: it is reported only while the sources of the
+    kernels the configuration launches are the ones the capture was taken with, and says so
+    otherwise instead of going silently null."""
+    import types
+
+    import bench
+    dense = types.SimpleNamespace(topk=None, P=16, N=11173962)
+    small = types.SimpleNamespace(topk=None, P=8, N=269722)
+    sparse = types.SimpleNamespace(topk=(1, 100), P=8, N=11173962)
+    assert bench.kernel_sources(dense) == bench.DENSE_SOURCES
+    assert "eg_step_small.cuh" in bench.kernel_sources(small) and "eg_topk.cuh" in bench.kernel_sources(sparse)
+    now = bench.kernel_source_hash(bench.DENSE_SOURCES)
+    monkeypatch.setitem(bench.FUSED_TRAFFIC, "dense", {now: (2.0e9, "profiles/somewhere.md")})
+    got = bench.fused_traffic(dense, 2 * bench.FUSED_TRAFFIC_ELEMENTS, None)
+    assert got["traffic"] == 4.0e9 and got["traffic_from"] == "profiles/somewhere.md"
+    monkeypatch.setitem(bench.FUSED_TRAFFIC, "dense", {"0" * 12: (2.0e9, "profiles/somewhere.md")})
+    stale = bench.fused_traffic(dense, bench.FUSED_TRAFFIC_ELEMENTS, None)
+    assert stale["traffic"] is None and "0" * 12 in stale["traffic_stale_since"] and now in stale["traffic_stale_since"]
+    for wl in (small, sparse):
+        other = bench.fused_traffic(wl, 1000, None)
+        assert other["traffic"] is None and "traffic_note" in other
+    assert bench.fused_traffic(dense, 1000, 0.9)["traffic"] is None

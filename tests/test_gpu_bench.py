@@ -43,6 +43,9 @@ def test_bench_line_has_the_agreed_keys(config, variant):
     roof = line["roofline"]
     assert roof["bound"] == "hbm" and roof["unit"] == "GB/s" and roof["peak"] > 0
     assert roof["frac"] is None or abs(roof["frac"] - roof["achieved"] / roof["peak"]) < 1e-9
+    # the captured DRAM traffic, or null together with the reason
+    assert "traffic" in roof and roof["traffic_sources_hash"]
+    assert roof["traffic"] is not None or "traffic_stale_since" in roof or "traffic_note" in roof
     cpu = line["cpu_baseline"]
     assert cpu["kind"] == "oracle" and cpu["cores"] >= 1 and cpu["value"] > 0 and cpu["sample"]
     assert set(line["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
