@@ -10,6 +10,8 @@
 // (replica P-1 for replica 0, replica 0 for replica P-1) live in two extra shared buffers
 // that are private per column.
 //
+// A CTA works through several tiles, one after the other, and keeps the ring full across them.
+//
 // Every mbarrier wait is bounded: when the limit is hit the CTA raises an abort flag, sets a
 // bit in the context's error word, lets its copies land and returns.
 #pragma once
@@ -103,26 +105,38 @@ struct PipeCfg {
 };
 
 // Shared-memory layout (dynamic), all offsets multiples of 16.
-template <int TILE, int STAGES, int ARRAYS = 3>
+// RUNS: a CTA may take several tiles (two wrap-around buffers, two mode tables).
+template <int TILE, int STAGES, int ARRAYS = 3, bool RUNS = true>
 struct PipeSmem {
     static constexpr int kTileBytes = TILE * 4;
     static constexpr int kStageBytes = ARRAYS * kTileBytes;       // x, g, x_hat (, velocity)
-    static constexpr int kWrapL = STAGES * kStageBytes;
-    static constexpr int kWrapR = kWrapL + kTileBytes;
-    static constexpr int kBars = kWrapR + kTileBytes;             // full[S], empty[S], wrap
-    static constexpr int kFlags = kBars + 8 * (2 * STAGES + 1) + 8;
-    // carried norm: per stage one slot of 8 doubles per consumer warp (see the consumers' end of
-    // a replica and the producer warp's reduce_slot)
+    static constexpr int kWrapL = STAGES * kStageBytes;           // two buffers: consecutive tiles alternate
+    static constexpr int kWrapR = kWrapL + (RUNS ? 2 : 1) * kTileBytes;
+    static constexpr int kBars = kWrapR + kTileBytes;             // full[S], empty[S], wrap[2]
+    static constexpr int kFlags = kBars + 8 * (2 * STAGES + 2);
+    // then 16 bytes of flags, two tables of per-replica modes (consecutive tiles alternate) and,
+    // for the carried norm, per stage one slot of 8 doubles per consumer warp (see the consumers'
+    // end of a replica and the producer warp's reduce_slot)
+    __host__ __device__ static size_t mode_bytes(int P) { return ((size_t)P + 15) & ~(size_t)15; }
     __host__ __device__ static size_t bytes(int P, bool carry, int consumer_warps) {
-        size_t b = kFlags + 16 + (((size_t)P + 15) & ~(size_t)15);
+        size_t b = kFlags + 16 + (RUNS ? 2 : 1) * mode_bytes(P);
         if (carry) b += (size_t)STAGES * consumer_warps * 8 * sizeof(double);
         return b;
     }
 };
 
-// Body of the kernels below.  grid n_tiles (tile table with TILE elements per tile),
-// CONSUMERS + 32 threads.
-// COLS = TILE / (4 * CONSUMERS) float4 columns per consumer thread.
+// Body of the kernels below.  The launch covers `n_launch` tiles of the tile table (TILE elements
+// per tile); CTA b takes the tiles b, b + gridDim.x, b + 2 gridDim.x, ... one after the other (so
+// that the CTAs running at any moment work on neighbouring tiles, as they would with one tile
+// per CTA: runs of consecutive tiles per CTA measured 5-10 % slower at 16 and 64 replicas), and
+// keeps its ring of stages full across them: the producer warp starts on the replicas of the
+// next tile while the consumers still work on the current one, so that a CTA pays for filling
+// and draining the ring once, not once per tile (with few replicas that was a large part of a
+// CTA's life).  What belongs to a tile and not to a stage -- the per-replica modes and the
+// wrap-around contribution of replica P-1 -- exists twice and consecutive tiles alternate; this
+// is safe when P >= STAGES (the producer is then never more than one tile ahead of the
+// consumers), which the host guarantees by launching one CTA per tile otherwise.
+// CONSUMERS + 32 threads; COLS = TILE / (4 * CONSUMERS) float4 columns per consumer thread.
 //
 // ASYNC (intermittent delivery): x_hat is what a replica has SENT, `mailbox` what its
 // neighbours have RECEIVED, `arrive` says whose outstanding messages arrive in this step and
@@ -135,76 +149,72 @@ struct PipeSmem {
 // MOM (heavy-ball momentum, an extension to another training algorithm): every replica owns a
 // velocity `vel` laid out like x; a stage carries a fourth tile (v), the consumers form
 // v <- fp32(mu * v + g) in fp64, write it back and use it in place of the gradient.
-template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC, bool PLAIN, bool MOM = false>
+// RUNS = false (the momentum kernel, whose four tiles per stage leave no room for the second
+// wrap-around buffer at three CTAs per multiprocessor): one tile per CTA.
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC, bool PLAIN, bool MOM = false,
+          bool RUNS = !MOM>
 __device__ __forceinline__ void
 fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
                 const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, const TileTable& tt,
                 int P, int T, long long stride, float lr, double* __restrict__ partials,
                 long long* step_k, unsigned int* __restrict__ err, int variant_arg,
-                float* mailbox, const uint8_t* __restrict__ arrive, float* __restrict__ vel = nullptr,
-                double mu = 0.0) {
+                float* mailbox, const uint8_t* __restrict__ arrive, int n_launch,
+                float* __restrict__ vel = nullptr, double mu = 0.0) {
     static_assert(!(MOM && ASYNC), "momentum is not combined with intermittent delivery");
     constexpr int kArr = MOM ? 4 : 3;              // tiles per stage
     static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
     const int variant = PLAIN ? 0 : variant_arg;
     // mode bit that says "contributes its own x": the dense-message bit itself unless ASYNC
     constexpr unsigned kCx = ASYNC ? 4u : 1u;
-    static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
-    using L = PipeSmem<TILE, STAGES, kArr>;
+    using L = PipeSmem<TILE, STAGES, kArr, RUNS>;
     constexpr int COLS = TILE / (4 * CONSUMERS);
     constexpr int CWARPS = CONSUMERS / 32;
     static_assert(COLS * 4 * CONSUMERS == TILE, "tile must be covered exactly");
     extern __shared__ __align__(128) unsigned char smem[];
     float* stages = reinterpret_cast<float*>(smem);
-    float* wrap_l = reinterpret_cast<float*>(smem + L::kWrapL);   // contribution of replica P-1
+    float* wrap_l2 = reinterpret_cast<float*>(smem + L::kWrapL);  // [2][TILE] contribution of replica P-1
     float* wrap_r = reinterpret_cast<float*>(smem + L::kWrapR);   // contribution of replica 0
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBars);
     uint64_t* empty = full + STAGES;
-    uint64_t* wrap_bar = empty + STAGES;
+    uint64_t* wrap_bar2 = empty + STAGES;                          // [2]
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kFlags);
     // bit 0: dense message, bit 1: valid, bit 2: contributes its own x, bit 3: arrives now
-    uint8_t* s_mode = smem + L::kFlags + 16;
-    double* s_part = reinterpret_cast<double*>(s_mode + ((P + 15) & ~15));   // [STAGES][CWARPS * 8]
+    uint8_t* s_mode2 = smem + L::kFlags + 16;                      // [2][mode_bytes(P)]
+    const int mode_stride = (int)L::mode_bytes(P);
+    double* s_part = reinterpret_cast<double*>(s_mode2 + (RUNS ? 2 : 1) * mode_stride);   // [STAGES][CWARPS * 8]
 
-    const int tile = blockIdx.x, tid = threadIdx.x;
-    if (!tile_ok(tt, tile, T, stride, TILE)) return;       // bounds-checked build only; the same in every thread
-    const int t = tt.tensor[tile];
-    const int len = tt.length[tile];
-    const long long off = tt.offset[tile];
-    const uint32_t copy_bytes = (uint32_t)(((len + 3) & ~3) * 4);
+    const int tid = threadIdx.x;
+    // tiles of this CTA: first, first + hop, ... below last (RUNS = false: the first one only)
+    const int first = (int)blockIdx.x, hop = (int)gridDim.x;
+    const int last = RUNS ? n_launch : min(n_launch, first + 1);
+    if (first >= last) return;                   // the same in every thread
 
-    // up to here only the tile table, which no kernel writes, has been read
-    pdl_release();
+    // up to here nothing that a kernel writes has been read.  The kernel after this one is let
+    // in when every CTA has begun its LAST tile (below): released at the start of a kernel that
+    // goes on for long, it made this kernel up to 45 % slower (measured).
     pdl_wait();
-    for (int j = tid; j < P; j += CONSUMERS + 32) {
-        const bool sn = snap[(long long)j * T + t] != 0;
-        const bool ar = ASYNC ? (arrive[(long long)j * T + t] != 0) : sn;
-        s_mode[j] = (uint8_t)((sn ? 1 : 0) | (valid[(long long)j * T + t] ? 2 : 0) |
-                              ((sn && ar) ? 4 : 0) | (ar ? 8 : 0));
-    }
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], CWARPS);
         }
-        mbar_init(wrap_bar, 1);
+        mbar_init(&wrap_bar2[0], 1);
+        mbar_init(&wrap_bar2[1], 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (blockIdx.x == 0 && step_k) *step_k += 1;   // nothing in this launch reads it
     }
     __syncthreads();
-
-    const bool cx_last = (s_mode[P - 1] & kCx) != 0;
-    // Replica P-1 contributes wrap_l; its own stage then only needs what wrap_l does not hold.
-    const bool last_opt = P >= 2;
+    const bool last_opt = P >= 2;   // replica P-1 contributes wrap_l; its own stage then only needs what wrap_l does not hold
 
     if (tid >= CONSUMERS) {
-        // ------------------------------------------------------------------ producer
-        // CARRY: the whole warp walks the loop, because it also finishes the sums of squares that
-        // the consumers leave behind (8 values per consumer warp and replica, in the slot of the
+        // ------------------------------------------------------------------ producer warp
+        // All 32 lanes walk the loop: they fill in the per-replica modes of a tile together, lane 0
+        // issues the copies, and with CARRY the warp also finishes the sums of squares that the
+        // consumers leave behind (8 values per consumer warp and replica, in the slot of the
         // replica's stage): once a stage has been released, its slot is complete.
         const int pl = tid - CONSUMERS;
-        auto reduce_slot = [&](int slot, int j) {
+        auto reduce_slot = [&](int slot, int tile, int j) {
             static_assert(CWARPS == 8 || CWARPS == 4 || CWARPS == 2, "a slot holds 64, 32 or 16 values");
             const double* sp = s_part + slot * (CWARPS * 8);
             double r = (CWARPS == 8) ? __dadd_rn(sp[pl], sp[32 + pl])
@@ -215,31 +225,92 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
             if (pl == 0 && EG_INDEX_OK(err, j, P) && EG_INDEX_OK(err, slot, STAGES))
                 partials[(long long)j * tt.n_tiles + tile] = r;
         };
-        if (CARRY || tid == CONSUMERS) {
-            const float* xp = x + off;
-            const float* gp = g + off;
-            const float* hp = xhat + off;
-            const float* mp = ASYNC ? mailbox + off : hp;
-            const float* vp = MOM ? vel + off : nullptr;
-            if (pl == 0) {
-                mbar_expect_tx(wrap_bar, copy_bytes);
-                bulk_g2s(wrap_l,
-                         (cx_last ? xp : ((s_mode[P - 1] & 8) ? hp : mp)) + (long long)(P - 1) * stride,
-                         copy_bytes, wrap_bar);
+        // Items are (tile, replica) pairs in the order they go through the ring; item m uses
+        // stage m % STAGES in its (m / STAGES)-th filling.  retire(m): wait until the consumers
+        // have released item m, then (CARRY) finish its sum of squares.
+        int retired = 0, r_tile = first, r_j = 0;     // next item to retire and what it is
+        auto retire = [&]() -> bool {
+            const int sm = retired % STAGES;
+            bool alive = mbar_wait_bounded(&empty[sm], (uint32_t)((retired / STAGES) & 1), s_abort, err);
+            alive = __all_sync(0xffffffffu, alive);
+            if (!alive) return false;
+            if (CARRY) reduce_slot(sm, r_tile, r_j);
+            ++retired;
+            if (++r_j == P) { r_j = 0; r_tile += hop; }
+            return true;
+        };
+        // the record of a tile: lane-uniform
+        struct Rec { int t, len; long long off; };
+        auto load_rec = [&](int tile) {
+            Rec r;
+            r.t = tt.tensor[tile]; r.len = tt.length[tile]; r.off = tt.offset[tile];
+            return r;
+        };
+        // the per-replica flags of a tile: read one tile ahead, two replicas per lane, and kept
+        // as they come (the first use of a loaded value would make the warp wait for it) --
+        // rings of up to 64 replicas; larger ones read their flags when the tile begins
+        constexpr int kPre = 2;
+        const bool prefetch = P <= 32 * kPre;
+        uint8_t pre_sn[kPre], pre_va[kPre], pre_ar[kPre];
+        auto mode_of = [&](uint8_t sn_b, uint8_t va_b, uint8_t ar_b) -> uint8_t {
+            const bool sn = sn_b != 0;
+            const bool ar = ASYNC ? (ar_b != 0) : sn;
+            return (uint8_t)((sn ? 1u : 0u) | (va_b ? 2u : 0u) | ((sn && ar) ? 4u : 0u) | (ar ? 8u : 0u));
+        };
+        auto fetch_flags = [&](int t) {
+#pragma unroll
+            for (int q = 0; q < kPre; ++q) {
+                const long long at = (long long)min(pl + 32 * q, P - 1) * T + t;
+                pre_sn[q] = snap[at];
+                pre_va[q] = valid[at];
+                pre_ar[q] = ASYNC ? arrive[at] : (uint8_t)0;
             }
-            int s = 0;
-            uint32_t wait_parity = 1;     // parity of the phase before the one to wait for
-            bool alive = true;
-            for (int j = 0; j < P; ++j) {
-                if (j >= STAGES) {
-                    alive = mbar_wait_bounded(&empty[s], wait_parity, s_abort, err);
-                    if (CARRY) alive = __all_sync(0xffffffffu, alive);
-                    if (!alive) break;
-                    if (CARRY) reduce_slot(s, j - STAGES);     // before the stage is filled again
+        };
+        int issued = 0, s = 0;
+        bool alive = true;
+        Rec rec = load_rec(first);
+        Rec rec_next = (first + hop < last) ? load_rec(first + hop) : rec;
+        if (prefetch) fetch_flags(rec.t);
+        int it = 0;                                 // how many tiles this CTA has begun
+        for (int tile = first; tile < last && alive; tile += hop, ++it) {
+            if (!tile_ok(tt, tile, T, stride, TILE)) break;      // bounds-checked build only (the consumers leave too)
+            if (tile + hop >= last) pdl_release();
+            const int buf = RUNS ? (it & 1) : 0;
+            uint8_t* sm = s_mode2 + buf * mode_stride;
+            // modes of this tile (its flags were read one tile ago), then the flags of the next
+            if (prefetch) {
+#pragma unroll
+                for (int q = 0; q < kPre; ++q)
+                    if (pl + 32 * q < P) sm[pl + 32 * q] = mode_of(pre_sn[q], pre_va[q], pre_ar[q]);
+            } else {
+                for (int j = pl; j < P; j += 32) {
+                    const long long at = (long long)j * T + rec.t;
+                    sm[j] = mode_of(snap[at], valid[at], ASYNC ? arrive[at] : (uint8_t)0);
                 }
-                if (pl == 0 && EG_INDEX_OK(err, s, STAGES) && EG_INDEX_OK(err, j, P)) {
+            }
+            __syncwarp();
+            const Rec cur = rec;
+            rec = rec_next;
+            if (tile + 2 * hop < last) rec_next = load_rec(tile + 2 * hop);
+            if (prefetch && tile + hop < last) fetch_flags(rec.t);
+            const uint32_t copy_bytes = (uint32_t)(((cur.len + 3) & ~3) * 4);
+            const float* xp = x + cur.off;
+            const float* gp = g + cur.off;
+            const float* hp = xhat + cur.off;
+            const float* mp = ASYNC ? mailbox + cur.off : hp;
+            const float* vp = MOM ? vel + cur.off : nullptr;
+            if (pl == 0) {
+                const bool cx_last = (sm[P - 1] & kCx) != 0;
+                mbar_expect_tx(&wrap_bar2[buf], copy_bytes);
+                bulk_g2s(wrap_l2 + buf * TILE,
+                         (cx_last ? xp : ((sm[P - 1] & 8) ? hp : mp)) + (long long)(P - 1) * stride,
+                         copy_bytes, &wrap_bar2[buf]);
+            }
+            for (int j = 0; j < P; ++j) {
+                if (issued >= STAGES && !retire()) { alive = false; break; }   // before the stage is filled again
+                if (pl == 0 && EG_INDEX_OK(err, s, STAGES)) {
                     float* st = stages + s * (kArr * TILE);
-                    const bool cx = (s_mode[j] & kCx) != 0;
+                    const bool cx = (sm[j] & kCx) != 0;
                     const bool is_last = last_opt && (j == P - 1);
                     const bool need_x = !(is_last && cx);
                     const bool need_h = !cx && !is_last;
@@ -248,189 +319,202 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     bulk_g2s(st + TILE, gp, copy_bytes, &full[s]);
                     if (MOM) { bulk_g2s(st + 3 * TILE, vp, copy_bytes, &full[s]); vp += stride; }
                     if (need_x) bulk_g2s(st, xp, copy_bytes, &full[s]);
-                    if (need_h) bulk_g2s(st + 2 * TILE, (s_mode[j] & 8) ? hp : mp, copy_bytes, &full[s]);
+                    if (need_h) bulk_g2s(st + 2 * TILE, (sm[j] & 8) ? hp : mp, copy_bytes, &full[s]);
                     xp += stride; gp += stride; hp += stride; mp += stride;
                 }
-                if (++s == STAGES) { s = 0; wait_parity ^= 1u; }
+                ++issued;
+                if (++s == STAGES) s = 0;
             }
-            if (CARRY && alive) {
-                // the replicas whose stages are not filled again
-                for (int j = max(0, P - STAGES); j < P; ++j) {
-                    const int sj = j % STAGES;
-                    alive = __all_sync(0xffffffffu,
-                                       mbar_wait_bounded(&empty[sj], (uint32_t)((j / STAGES) & 1), s_abort, err));
-                    if (!alive) break;
-                    reduce_slot(sj, j);
-                }
-            }
+        }
+        if (CARRY) {
+            // the items whose stages are not filled again
+            while (alive && retired < issued) alive = retire();
         }
     } else {
         // ------------------------------------------------------------------ consumers
         const int lane = tid & 31, warp = tid >> 5;
-        int nel[COLS];
-#pragma unroll
-        for (int v = 0; v < COLS; ++v) nel[v] = min(4, max(0, len - (v * CONSUMERS + tid) * 4));
         const int c0 = tid * 4;                      // column v starts at c0 + v * 4 * CONSUMERS
         const double neg_lr = -(double)lr;
         const double w_one = 1.0, w_half = 0.5, w_third = __ddiv_rn(1.0, 3.0);
         const bool has_left = P >= 2, has_right = P >= 3;
-        // contributions of replica j-1 and j to their neighbours, for this thread's columns,
-        // kept as doubles so that every value is converted once
-        double hp[COLS][4], hc[COLS][4];
-        bool ok = mbar_wait_bounded(wrap_bar, 0, s_abort, err) &&
-                  mbar_wait_bounded(&full[0], 0, s_abort, err);
-        unsigned mode_prev = s_mode[P - 1], mode_cur = s_mode[0];
-#pragma unroll
-        for (int v = 0; v < COLS; ++v) {
-            const int c = c0 + v * 4 * CONSUMERS;
-            const float4 a = ok ? *reinterpret_cast<const float4*>(wrap_l + c) : make_float4(0, 0, 0, 0);
-            const float4 b = ok ? *reinterpret_cast<const float4*>(((mode_cur & kCx) ? stages : stages + 2 * TILE) + c)
-                                : make_float4(0, 0, 0, 0);
-            hp[v][0] = a.x; hp[v][1] = a.y; hp[v][2] = a.z; hp[v][3] = a.w;
-            hc[v][0] = b.x; hc[v][1] = b.y; hc[v][2] = b.z; hc[v][3] = b.w;
-        }
+        // the ring position of the next item: stage s in a filling of parity par_s, and the one after it
         int s = 0, s1 = (STAGES > 1) ? 1 : 0;
-        uint32_t parity1 = (STAGES > 1) ? 0u : 1u;   // phase parity of the fill of stage s1 for j+1
-        float* xo = x + off + c0;                    // output pointers of replica j
-        float* ho = xhat + off + c0;
-        float* mo = ASYNC ? mailbox + off + c0 : nullptr;
-        float* vo = MOM ? vel + off + c0 : nullptr;
-        // One replica.  A = contributions of replica j-1, B = of replica j, C receives those of
-        // replica j+1.  The three arrays swap roles from one replica to the next (see the loop
-        // below), so nothing is copied between them.
-        auto one_replica = [&](const int j, double (&hA)[COLS][4], double (&hB)[COLS][4],
-                               double (&hC)[COLS][4]) -> bool {
-            const bool more = j + 1 < P;
-            if (!EG_INDEX_OK(err, s, STAGES) || !EG_INDEX_OK(err, s1, STAGES) || !EG_INDEX_OK(err, j, P)) return false;
-            if (more) {
-                ok = mbar_wait_bounded(&full[s1], parity1, s_abort, err);
-                if (!ok) return false;
-            }
-            const unsigned mode_next = s_mode[more ? j + 1 : 0];
-            const float* st = stages + s * (kArr * TILE);
-            const bool sn = (mode_cur & 1) != 0;
-            const bool cx = (mode_cur & kCx) != 0;     // == sn unless ASYNC
-            const bool is_last = last_opt && !more;
-            // fp32 copy of this replica's contribution (its old x when a dense message arrives)
-            const float* hs = is_last ? wrap_l : (cx ? st : st + 2 * TILE);
-            // contribution of replica j+1
-            const float* sq = stages + s1 * (kArr * TILE);
-            const float* hn_s = !more ? wrap_r
-                                      : ((last_opt && j + 2 == P) ? wrap_l
-                                                                  : ((mode_next & kCx) ? sq : sq + 2 * TILE));
-            const bool ul = has_left && (mode_prev & 2) != 0;
-            const bool ur = has_right && (mode_next & 2) != 0;
-            const double w = (ul && ur) ? w_third : ((ul || ur) ? w_half : w_one);
-            double acc = 0.0;
+        uint32_t par_s = 0u, parity1 = (STAGES > 1) ? 0u : 1u;
+        bool ok = true;
+        int len = tt.length[first];
+        long long off = tt.offset[first];
+        int it = 0;
+        for (int tile = first; tile < last && ok; tile += hop, ++it) {
+            if (!tile_ok(tt, tile, T, stride, TILE)) break;      // bounds-checked build only (the producer leaves too)
+            if (tile + hop >= last) pdl_release();
+            const int buf = RUNS ? (it & 1) : 0;
+            const uint8_t* s_mode = s_mode2 + buf * mode_stride;
+            const float* wrap_l = wrap_l2 + buf * TILE;
+            uint64_t* wrap_bar = &wrap_bar2[buf];
+            const int len_now = len;
+            const long long off_now = off;
+            if (tile + hop < last) { len = tt.length[tile + hop]; off = tt.offset[tile + hop]; }   // used one tile later
+            int nel[COLS];
+#pragma unroll
+            for (int v = 0; v < COLS; ++v) nel[v] = min(4, max(0, len_now - (v * CONSUMERS + tid) * 4));
+            // contributions of replica j-1 and j to their neighbours, for this thread's columns,
+            // kept as doubles so that every value is converted once
+            double hp[COLS][4], hc[COLS][4];
+            ok = mbar_wait_bounded(wrap_bar, (uint32_t)((it >> (RUNS ? 1 : 0)) & 1), s_abort, err) &&
+                 mbar_wait_bounded(&full[s], par_s, s_abort, err);
+            if (!ok) break;
+            unsigned mode_prev = s_mode[P - 1], mode_cur = s_mode[0];
 #pragma unroll
             for (int v = 0; v < COLS; ++v) {
-                if (PLAIN && !ASYNC && !MOM && nel[v] == 4 && ul && ur) {
-                    // The common case -- a full float4, both neighbours heard from, default
-                    // readings -- as straight-line code: the same operations in the same order
-                    // as the general form below, without its per-element conditions.
-                    const int c = c0 + v * 4 * CONSUMERS;
-                    const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
-                    const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
-                    const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
-                    if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;
-                    hC[v][0] = (double)hnf.x; hC[v][1] = (double)hnf.y; hC[v][2] = (double)hnf.z; hC[v][3] = (double)hnf.w;
-                    double xd[4];
-                    if (cx) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) xd[q] = hB[v][q];
-                    } else {
-                        const float4 xf = *reinterpret_cast<const float4*>(st + c);
-                        xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
-                    }
-                    float4 xn4;
-                    xn4.x = __double2float_rn(__fma_rn(neg_lr, (double)gf.x,
-                                __dmul_rn(__dadd_rn(__dadd_rn(xd[0], hA[v][0]), hC[v][0]), w_third)));
-                    xn4.y = __double2float_rn(__fma_rn(neg_lr, (double)gf.y,
-                                __dmul_rn(__dadd_rn(__dadd_rn(xd[1], hA[v][1]), hC[v][1]), w_third)));
-                    xn4.z = __double2float_rn(__fma_rn(neg_lr, (double)gf.z,
-                                __dmul_rn(__dadd_rn(__dadd_rn(xd[2], hA[v][2]), hC[v][2]), w_third)));
-                    xn4.w = __double2float_rn(__fma_rn(neg_lr, (double)gf.w,
-                                __dmul_rn(__dadd_rn(__dadd_rn(xd[3], hA[v][3]), hC[v][3]), w_third)));
-                    st_stream(xo + v * 4 * CONSUMERS, xn4);
-                    if (sn) st_stream(ho + v * 4 * CONSUMERS, hcf);
-                    if (CARRY) {
-                        const float d0 = __fsub_rn(xn4.x, hcf.x), d1 = __fsub_rn(xn4.y, hcf.y);
-                        const float d2 = __fsub_rn(xn4.z, hcf.z), d3 = __fsub_rn(xn4.w, hcf.w);
-                        acc = __fma_rn((double)d0, (double)d0, acc);
-                        acc = __fma_rn((double)d1, (double)d1, acc);
-                        acc = __fma_rn((double)d2, (double)d2, acc);
-                        acc = __fma_rn((double)d3, (double)d3, acc);
-                    }
-                } else if (nel[v] > 0) {
-                    const int c = c0 + v * 4 * CONSUMERS;
-                    const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
-                    const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
-                    const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
-                    if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;   // private to this thread
-                    hC[v][0] = (double)hnf.x; hC[v][1] = (double)hnf.y; hC[v][2] = (double)hnf.z; hC[v][3] = (double)hnf.w;
-                    double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
-                    if (MOM) {      // v <- mu * v + g, kept in fp32; the update then uses gamma * v
-                        const float4 vf = *reinterpret_cast<const float4*>(st + 3 * TILE + c);
-                        const float vn[4] = {__double2float_rn(__fma_rn(mu, (double)vf.x, gd[0])),
-                                             __double2float_rn(__fma_rn(mu, (double)vf.y, gd[1])),
-                                             __double2float_rn(__fma_rn(mu, (double)vf.z, gd[2])),
-                                             __double2float_rn(__fma_rn(mu, (double)vf.w, gd[3]))};
-                        store_masked(vo + v * 4 * CONSUMERS, make_float4(vn[0], vn[1], vn[2], vn[3]), nel[v]);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) gd[q] = (double)vn[q];
-                    }
-                    double xd[4];
-                    float4 x_old = make_float4(0.f, 0.f, 0.f, 0.f);   // only needed under ASYNC
-                    if (cx || (variant & kOwnLastSent)) {   // own term = this replica's contribution
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) xd[q] = hB[v][q];
-                        if (ASYNC) x_old = hcf;
-                    } else {
-                        const float4 xf = *reinterpret_cast<const float4*>(st + c);
-                        xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
-                        if (ASYNC) x_old = xf;
-                    }
-                    float xn[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        double sum = xd[q];
-                        if (ul) sum = __dadd_rn(sum, hA[v][q]);
-                        if (ur) sum = __dadd_rn(sum, hC[v][q]);
-                        xn[q] = __double2float_rn(__fma_rn(neg_lr, gd[q], __dmul_rn(sum, w)));
-                    }
-                    const float4 xn4 = make_float4(xn[0], xn[1], xn[2], xn[3]);
-                    store_masked(xo + v * 4 * CONSUMERS, xn4, nel[v]);
-                    // a dense message: the sender's record becomes its old x (== hcf unless ASYNC)
-                    if (sn) store_masked(ho + v * 4 * CONSUMERS, ASYNC ? x_old : hcf, nel[v]);
-                    if (ASYNC && (mode_cur & 8)) store_masked(mo + v * 4 * CONSUMERS, hcf, nel[v]);
-                    if (CARRY)
-                        acc = sq_diff4(xn4, (variant & kChangeOfNorm) ? make_float4(0.f, 0.f, 0.f, 0.f) : hcf,
-                                       nel[v], acc);
+                const int c = c0 + v * 4 * CONSUMERS;
+                const float* st0 = stages + s * (kArr * TILE);
+                const float4 a = *reinterpret_cast<const float4*>(wrap_l + c);
+                const float4 b = *reinterpret_cast<const float4*>(((mode_cur & kCx) ? st0 : st0 + 2 * TILE) + c);
+                hp[v][0] = a.x; hp[v][1] = a.y; hp[v][2] = a.z; hp[v][3] = a.w;
+                hc[v][0] = b.x; hc[v][1] = b.y; hc[v][2] = b.z; hc[v][3] = b.w;
+            }
+            float* xo = x + off_now + c0;                // output pointers of replica j
+            float* ho = xhat + off_now + c0;
+            float* mo = ASYNC ? mailbox + off_now + c0 : nullptr;
+            float* vo = MOM ? vel + off_now + c0 : nullptr;
+            // One replica.  A = contributions of replica j-1, B = of replica j, C receives those of
+            // replica j+1.  The three arrays swap roles from one replica to the next (see the loop
+            // below), so nothing is copied between them.
+            auto one_replica = [&](const int j, double (&hA)[COLS][4], double (&hB)[COLS][4],
+                                   double (&hC)[COLS][4]) -> bool {
+                const bool more = j + 1 < P;
+                if (!EG_INDEX_OK(err, s, STAGES) || !EG_INDEX_OK(err, s1, STAGES) || !EG_INDEX_OK(err, j, P)) return false;
+                if (more) {
+                    ok = mbar_wait_bounded(&full[s1], parity1, s_abort, err);
+                    if (!ok) return false;
                 }
+                const unsigned mode_next = s_mode[more ? j + 1 : 0];
+                const float* st = stages + s * (kArr * TILE);
+                const bool sn = (mode_cur & 1) != 0;
+                const bool cx = (mode_cur & kCx) != 0;     // == sn unless ASYNC
+                const bool is_last = last_opt && !more;
+                // fp32 copy of this replica's contribution (its old x when a dense message arrives)
+                const float* hs = is_last ? wrap_l : (cx ? st : st + 2 * TILE);
+                // contribution of replica j+1
+                const float* sq = stages + s1 * (kArr * TILE);
+                const float* hn_s = !more ? wrap_r
+                                          : ((last_opt && j + 2 == P) ? wrap_l
+                                                                      : ((mode_next & kCx) ? sq : sq + 2 * TILE));
+                const bool ul = has_left && (mode_prev & 2) != 0;
+                const bool ur = has_right && (mode_next & 2) != 0;
+                const double w = (ul && ur) ? w_third : ((ul || ur) ? w_half : w_one);
+                double acc = 0.0;
+    #pragma unroll
+                for (int v = 0; v < COLS; ++v) {
+                    if (PLAIN && !ASYNC && !MOM && nel[v] == 4 && ul && ur) {
+                        // The common case -- a full float4, both neighbours heard from, default
+                        // readings -- as straight-line code: the same operations in the same order
+                        // as the general form below, without its per-element conditions.
+                        const int c = c0 + v * 4 * CONSUMERS;
+                        const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
+                        const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
+                        const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
+                        if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;
+                        hC[v][0] = (double)hnf.x; hC[v][1] = (double)hnf.y; hC[v][2] = (double)hnf.z; hC[v][3] = (double)hnf.w;
+                        double xd[4];
+                        if (cx) {
+    #pragma unroll
+                            for (int q = 0; q < 4; ++q) xd[q] = hB[v][q];
+                        } else {
+                            const float4 xf = *reinterpret_cast<const float4*>(st + c);
+                            xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
+                        }
+                        float4 xn4;
+                        xn4.x = __double2float_rn(__fma_rn(neg_lr, (double)gf.x,
+                                    __dmul_rn(__dadd_rn(__dadd_rn(xd[0], hA[v][0]), hC[v][0]), w_third)));
+                        xn4.y = __double2float_rn(__fma_rn(neg_lr, (double)gf.y,
+                                    __dmul_rn(__dadd_rn(__dadd_rn(xd[1], hA[v][1]), hC[v][1]), w_third)));
+                        xn4.z = __double2float_rn(__fma_rn(neg_lr, (double)gf.z,
+                                    __dmul_rn(__dadd_rn(__dadd_rn(xd[2], hA[v][2]), hC[v][2]), w_third)));
+                        xn4.w = __double2float_rn(__fma_rn(neg_lr, (double)gf.w,
+                                    __dmul_rn(__dadd_rn(__dadd_rn(xd[3], hA[v][3]), hC[v][3]), w_third)));
+                        st_stream(xo + v * 4 * CONSUMERS, xn4);
+                        if (sn) st_stream(ho + v * 4 * CONSUMERS, hcf);
+                        if (CARRY) {
+                            const float d0 = __fsub_rn(xn4.x, hcf.x), d1 = __fsub_rn(xn4.y, hcf.y);
+                            const float d2 = __fsub_rn(xn4.z, hcf.z), d3 = __fsub_rn(xn4.w, hcf.w);
+                            acc = __fma_rn((double)d0, (double)d0, acc);
+                            acc = __fma_rn((double)d1, (double)d1, acc);
+                            acc = __fma_rn((double)d2, (double)d2, acc);
+                            acc = __fma_rn((double)d3, (double)d3, acc);
+                        }
+                    } else if (nel[v] > 0) {
+                        const int c = c0 + v * 4 * CONSUMERS;
+                        const float4 hcf = *reinterpret_cast<const float4*>(hs + c);
+                        const float4 hnf = *reinterpret_cast<const float4*>(hn_s + c);
+                        const float4 gf = *reinterpret_cast<const float4*>(st + TILE + c);
+                        if (j == 0) *reinterpret_cast<float4*>(wrap_r + c) = hcf;   // private to this thread
+                        hC[v][0] = (double)hnf.x; hC[v][1] = (double)hnf.y; hC[v][2] = (double)hnf.z; hC[v][3] = (double)hnf.w;
+                        double gd[4] = {(double)gf.x, (double)gf.y, (double)gf.z, (double)gf.w};
+                        if (MOM) {      // v <- mu * v + g, kept in fp32; the update then uses gamma * v
+                            const float4 vf = *reinterpret_cast<const float4*>(st + 3 * TILE + c);
+                            const float vn[4] = {__double2float_rn(__fma_rn(mu, (double)vf.x, gd[0])),
+                                                 __double2float_rn(__fma_rn(mu, (double)vf.y, gd[1])),
+                                                 __double2float_rn(__fma_rn(mu, (double)vf.z, gd[2])),
+                                                 __double2float_rn(__fma_rn(mu, (double)vf.w, gd[3]))};
+                            store_masked(vo + v * 4 * CONSUMERS, make_float4(vn[0], vn[1], vn[2], vn[3]), nel[v]);
+    #pragma unroll
+                            for (int q = 0; q < 4; ++q) gd[q] = (double)vn[q];
+                        }
+                        double xd[4];
+                        float4 x_old = make_float4(0.f, 0.f, 0.f, 0.f);   // only needed under ASYNC
+                        if (cx || (variant & kOwnLastSent)) {   // own term = this replica's contribution
+    #pragma unroll
+                            for (int q = 0; q < 4; ++q) xd[q] = hB[v][q];
+                            if (ASYNC) x_old = hcf;
+                        } else {
+                            const float4 xf = *reinterpret_cast<const float4*>(st + c);
+                            xd[0] = (double)xf.x; xd[1] = (double)xf.y; xd[2] = (double)xf.z; xd[3] = (double)xf.w;
+                            if (ASYNC) x_old = xf;
+                        }
+                        float xn[4];
+    #pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            double sum = xd[q];
+                            if (ul) sum = __dadd_rn(sum, hA[v][q]);
+                            if (ur) sum = __dadd_rn(sum, hC[v][q]);
+                            xn[q] = __double2float_rn(__fma_rn(neg_lr, gd[q], __dmul_rn(sum, w)));
+                        }
+                        const float4 xn4 = make_float4(xn[0], xn[1], xn[2], xn[3]);
+                        store_masked(xo + v * 4 * CONSUMERS, xn4, nel[v]);
+                        // a dense message: the sender's record becomes its old x (== hcf unless ASYNC)
+                        if (sn) store_masked(ho + v * 4 * CONSUMERS, ASYNC ? x_old : hcf, nel[v]);
+                        if (ASYNC && (mode_cur & 8)) store_masked(mo + v * 4 * CONSUMERS, hcf, nel[v]);
+                        if (CARRY)
+                            acc = sq_diff4(xn4, (variant & kChangeOfNorm) ? make_float4(0.f, 0.f, 0.f, 0.f) : hcf,
+                                           nel[v], acc);
+                    }
+                }
+                if (CARRY) {
+                    // two of the five rounds of the warp sum; the producer warp does the rest once
+                    // this stage has been released by all consumer warps
+                    acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, 16));
+                    acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, 8));
+                    if (lane < 8) s_part[s * (CWARPS * 8) + warp * 8 + lane] = acc;
+                }
+                // everything later iterations need from this stage now sits in registers
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[s]);
+                xo += stride; ho += stride;
+                if (ASYNC) mo += stride;
+                if (MOM) vo += stride;
+                mode_prev = mode_cur; mode_cur = mode_next;
+                s = s1;
+                par_s = parity1;
+                if (++s1 == STAGES) { s1 = 0; parity1 ^= 1u; }
+                return true;
+            };
+            double hn[COLS][4];
+            for (int j = 0; ok && j < P; j += 3) {
+                if (!one_replica(j, hp, hc, hn)) { ok = false; break; }
+                if (j + 1 < P && !one_replica(j + 1, hc, hn, hp)) { ok = false; break; }
+                if (j + 2 < P && !one_replica(j + 2, hn, hp, hc)) { ok = false; break; }
             }
-            if (CARRY) {
-                // two of the five rounds of the warp sum; the producer warp does the rest once
-                // this stage has been released by all consumer warps
-                acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, 16));
-                acc = __dadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, 8));
-                if (lane < 8) s_part[s * (CWARPS * 8) + warp * 8 + lane] = acc;
-            }
-            // everything later iterations need from this stage now sits in registers
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[s]);
-            xo += stride; ho += stride;
-            if (ASYNC) mo += stride;
-            if (MOM) vo += stride;
-            mode_prev = mode_cur; mode_cur = mode_next;
-            s = s1;
-            if (++s1 == STAGES) { s1 = 0; parity1 ^= 1u; }
-            return true;
-        };
-        double hn[COLS][4];
-        for (int j = 0; ok && j < P; j += 3) {
-            if (!one_replica(j, hp, hc, hn)) break;
-            if (j + 1 < P && !one_replica(j + 1, hc, hn, hp)) break;
-            if (j + 2 < P && !one_replica(j + 2, hn, hp, hc)) break;
         }
     }
     if (*s_abort) {
@@ -447,9 +531,10 @@ __global__ void __launch_bounds__(CONSUMERS + 32, 3)
 k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
-             long long* step_k, unsigned int* __restrict__ err) {
+             long long* step_k, unsigned int* __restrict__ err, int n_launch) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true>(x, g, xhat, snap, valid, tt, P, T, stride, lr,
-                                                                partials, step_k, err, 0, nullptr, nullptr);
+                                                                partials, step_k, err, 0, nullptr, nullptr,
+                                                                n_launch);
 }
 
 // Heavy-ball momentum on the default readings (eg_set_momentum): four tiles per stage.
@@ -458,10 +543,11 @@ __global__ void __launch_bounds__(CONSUMERS + 32)
 k_fused_pipe_momentum(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
                       const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
                       int P, int T, long long stride, float lr, double* __restrict__ partials,
-                      long long* step_k, unsigned int* __restrict__ err, float* __restrict__ vel, double mu) {
+                      long long* step_k, unsigned int* __restrict__ err, int n_launch,
+                      float* __restrict__ vel, double mu) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true, true>(x, g, xhat, snap, valid, tt, P, T, stride,
                                                                       lr, partials, step_k, err, 0, nullptr,
-                                                                      nullptr, vel, mu);
+                                                                      nullptr, n_launch, vel, mu);
 }
 
 // Variants (eg_set_variant) and intermittent delivery; bounded to 72 registers for 3 CTAs per SM.
@@ -470,11 +556,11 @@ __global__ void __launch_bounds__(CONSUMERS + 32, 3)
 k_fused_pipe_general(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
                      const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
                      int P, int T, long long stride, float lr, double* __restrict__ partials,
-                     long long* step_k, unsigned int* __restrict__ err, int variant, float* mailbox,
-                     const uint8_t* __restrict__ arrive) {
+                     long long* step_k, unsigned int* __restrict__ err, int n_launch, int variant,
+                     float* mailbox, const uint8_t* __restrict__ arrive) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, ASYNC, false>(x, g, xhat, snap, valid, tt, P, T, stride,
                                                                  lr, partials, step_k, err, variant, mailbox,
-                                                                 arrive);
+                                                                 arrive, n_launch);
 }
 
 // Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes.  The

@@ -964,13 +964,12 @@ __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, all, a.err);
 }
 
-// Every single-phase kernel can be launched while the kernel before it drains (programmatic
-// dependent launch): it lets its own successor do the same and then waits for its predecessor
-// before it reads anything.  `which` names the work list: 0 for this iteration's sparse
+// Every single-phase kernel can be launched as a dependent launch: it waits for its predecessor
+// before it reads anything.  None of them lets its successor in before it ends: a successor let
+// in at the start of a kernel that goes on for a millisecond made that kernel much slower.  `which` names the work list: 0 for this iteration's sparse
 // segments, 1 for the exact repeat; the kernels of the repeat leave at once when no segment
 // asked for it.
 __device__ __forceinline__ bool topk_enter(const TopkArgs& a, int which) {
-    pdl_release();
     pdl_wait();
     return which == 0 || *a.tk.redo_count != 0u;
 }

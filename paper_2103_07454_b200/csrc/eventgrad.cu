@@ -27,7 +27,7 @@ constexpr int kFusedVpt = EG_FUSED_VPT;               // float4 columns per thre
 constexpr int kFusedTile = kThreads * 4 * kFusedVpt;  // elements per CTA of the fused kernel
 using PipeLayout = PipeSmem<kPipeTile, kPipeStages>;
 constexpr int kMomStages = 4;                         // four tiles per stage: same footprint as 5 x 3
-using MomLayout = PipeSmem<kPipeTile, kMomStages, 4>;
+using MomLayout = PipeSmem<kPipeTile, kMomStages, 4, false>;
 static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
 constexpr uint64_t kStateMagic = 0x4547535441544533ull;  // "EGSTATE3"
 
@@ -109,7 +109,9 @@ struct eg_ctx {
     // optional per-kernel timing (events on the launching stream)
     bool timing = false;
     bool nvtx = false;      // EG_NVTX in the environment at eg_create: named ranges around the kernel groups
-    bool topk_pdl = false;  // EG_TOPK_PDL in the environment at eg_create: dependent launches inside the Top-K sequence too
+    int fused_waves = 1;    // EG_FUSED_WAVES in the environment at eg_create: CTAs of a walking pipelined kernel per resident slot
+    int fused_walk_max_p = 12;   // EG_FUSED_WALK_MAX_P: rings of up to this many replicas use the walking form
+    bool topk_pdl = true;   // EG_TOPK_PDL=0 in the environment at eg_create: no dependent launches inside the Top-K sequence
     bool no_pdl = false;    // EG_NO_PDL in the environment at eg_create: every kernel starts after its predecessor has ended
     std::vector<cudaEvent_t> ev_pool;      // pairs
     std::vector<int> ev_kind;              // kernel group of every recorded pair
@@ -445,7 +447,9 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     if (cudaGetDevice(&c->device) != cudaSuccess) return fail(EG_ERR_CUDA);
     { const char* e = getenv("EG_NVTX"); c->nvtx = e && *e && *e != '0'; }
     { const char* e = getenv("EG_NO_PDL"); c->no_pdl = e && *e && *e != '0'; }
-    { const char* e = getenv("EG_TOPK_PDL"); c->topk_pdl = e && *e && *e != '0'; }
+    { const char* e = getenv("EG_TOPK_PDL"); c->topk_pdl = !(e && *e == '0'); }
+    { const char* e = getenv("EG_FUSED_WAVES"); if (e && atoi(e) > 0) c->fused_waves = atoi(e); }
+    { const char* e = getenv("EG_FUSED_WALK_MAX_P"); if (e && *e) c->fused_walk_max_p = atoi(e); }
     c->P = P; c->T = T; c->H = thr->history_len; c->thr = *thr;
     if (topk) c->topk = *topk;
     if (cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->sms < 1)
@@ -751,10 +755,9 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
             launches += 1;
         } else {
             // Fourteen launches, five of which (the exact repeat for segments whose guessed bin
-            // did not work out) leave at once in an ordinary iteration.  They can be started as
-            // dependent launches (each waits on the device, first thing it does, for the kernel
-            // before it), but measured on 64 x 25.6 M elements that made the sequence 30 % slower,
-            // so it is only done on request (EG_TOPK_PDL).
+            // did not work out) leave at once in an ordinary iteration.  They are dependent launches:
+            // each waits on the device, first thing it does, for the kernel before it, and none
+            // lets its successor in before it ends.
             const bool pdl = !c->timing && !c->no_pdl && c->topk_pdl;
             const dim3 one(1), tile_blocks(tile_grid), entry_blocks(tile_grid / kEntryShares), seg_blocks(seg_grid);
             const dim3 threads(kThreads);
@@ -779,6 +782,15 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     if (!small) {
         TimedSection ts(c, stream, EG_KERNEL_FUSED);
         const uint8_t* valid = c->async ? c->recv_valid : c->st.valid;   // whom the neighbours have heard from
+        // Rings of few replicas: a CTA of the pipelined kernels lives for P replicas only, and filling
+        // and draining its ring of stages is a large part of that (8 replicas: 6.0 TB/s against
+        // 6.7 at 16 and 64).  There the kernels are launched as one CTA per resident slot, each
+        // walking the tiles b, b + grid, ... with its ring kept full across them (8 replicas:
+        // 6.5 TB/s).  From 16 replicas on one CTA per tile is faster (measured: 2 % at 16, 8 % at
+        // 64 replicas -- the hardware hands tiles out in order, CTAs that walk drift apart).
+        const int pipe_stages = c->momentum ? kMomStages : kPipeStages;
+        const bool walk = c->P >= pipe_stages && c->P <= c->fused_walk_max_p && !c->momentum;
+        const int grid_pipe = walk ? std::min(grid_fused, c->sms * 3 * c->fused_waves) : grid_fused;
         if (c->hops > 1 && c->hops <= kMaxStagedHops && c->P >= 2 * c->hops + 1 &&
             c->fused_kind != EG_FUSED_REGISTER) {
             // rows staged through shared memory; the register kernel choice keeps the plain form
@@ -795,41 +807,41 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                     c->async ? c->mailbox : nullptr, c->async ? c->arrive : nullptr);
         } else if (c->async) {
             k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>
-                <<<grid_fused, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
+                <<<grid_pipe, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                 params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                partials_fused, step_k, c->err, c->variant, c->mailbox, c->arrive);
+                partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive);
         } else if (c->momentum) {
             const size_t smem = MomLayout::bytes(c->P, carry, kPipeConsumers / 32);
             if (carry)
                 k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, true>
-                    <<<grid_fused, kPipeThreads, smem, stream>>>(
+                    <<<grid_pipe, kPipeThreads, smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->err, c->vel, c->mu);
+                    partials_fused, step_k, c->err, grid_fused, c->vel, c->mu);
             else
                 k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, false>
-                    <<<grid_fused, kPipeThreads, smem, stream>>>(
+                    <<<grid_pipe, kPipeThreads, smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->err, c->vel, c->mu);
+                    partials_fused, step_k, c->err, grid_fused, c->vel, c->mu);
         } else if (c->fused_kind != EG_FUSED_REGISTER) {
             const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
 #define EG_PIPE_ARGS params, grads, c->xhat, (const uint8_t*)c->st.snap, valid, tf, c->P, c->T, \
-                     (long long)c->stride, lr, partials_fused, step_k, c->err
+                     (long long)c->stride, lr, partials_fused, step_k, c->err, grid_fused
             if (c->variant == 0) {
                 // started while the kernel before it (the decision kernel, or the Top-K sequence)
                 // drains: it waits on the device before it reads anything that kernel writes
                 if (carry)
                     EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
-                                          dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
+                                          dim3(grid_pipe), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
                 else
                     EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
-                                          dim3(grid_fused), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
+                                          dim3(grid_pipe), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
             } else {
                 if (carry)
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, true, false>
-                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                        <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
                 else
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, false>
-                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                        <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
             }
 #undef EG_PIPE_ARGS
         } else if (carry)
