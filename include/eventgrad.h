@@ -151,8 +151,9 @@ eg_status eg_set_variant(eg_ctx* ctx, int own_term, int trigger_metric);
  * one in flight, as a later put into the same window does).  deliver_dev == NULL (and plain
  * eg_step) delivers everything outstanding.  eg_enable_delivery_masks allocates the second
  * copy (P*replica_stride floats) and synchronises; everything sent until then counts as
- * arrived.  Not available together with EG_OWN_LAST_SENT, the carried norm is not used while
- * it is on.
+ * arrived.  Not available together with EG_OWN_LAST_SENT (that reading has no received copy to
+ * average with).  The carried norm, momentum, more neighbours and Top-K all work with it; the
+ * carried norms are taken against what a replica has SENT.
  * eg_read_received copies the received copies to the host ([P][replica_stride] fp32; equal to
  * eg_read_mailboxes under synchronous delivery); eg_delivery_status returns the per-(replica,
  * tensor) "in flight" flags (host, P*T bytes) and the number of arrivals so far. */
@@ -180,10 +181,10 @@ eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
  * like params, owned by the context (allocated and zeroed by the first enabling call, zeroed
  * again by eg_reset); mu * v + g is one fp64 fused multiply-add rounded to fp32, and the update
  * uses that rounded value.  mu = 0 reproduces the plain update bit for bit.  0 <= mu < 1
- * (EG_ERR_INVALID otherwise).  Available with the default readings on the nearest-neighbour ring
- * and the default kernel choice, dense or Top-K (EG_ERR_STATE with eg_set_variant choices,
- * EG_TOPO_RING_HOPS(m > 1), intermittent delivery or EG_FUSED_REGISTER).  enabled = 0 returns to
- * the plain update and keeps the buffer.  The velocities are part of eg_export_state once the
+ * (EG_ERR_INVALID otherwise).  Works with every other option (readings, more neighbours,
+ * intermittent delivery, Top-K, either kernel choice); the default readings on the
+ * nearest-neighbour ring have the fastest kernel.  enabled = 0 returns to the plain update and
+ * keeps the buffer.  The velocities are part of eg_export_state once the
  * buffer exists; eg_read_velocity / eg_write_velocity copy them to / from a host buffer of
  * P*replica_stride floats (both synchronise; EG_ERR_STATE before the first enabling call). */
 eg_status eg_set_momentum(eg_ctx* ctx, int enabled, double mu);

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kThreads)
 k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
         const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
         int P, int T, long long stride, float lr, double* __restrict__ partials,
-        long long* step_k, int variant) {
+        long long* step_k, int variant, float* vel = nullptr, double mu = 0.0) {
     extern __shared__ __align__(128) unsigned char smem[];
     uint8_t* s_snap = smem;
     uint8_t* s_valid = smem + P;
@@ -133,6 +133,16 @@ k_fused(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ 
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             if (nel[v] > 0) {
+                if (vel) {   // heavy-ball momentum: v <- fp32(mu * v + g), used in place of g
+                    float* vc = vel + rb + e[v];
+                    const float4 vj = *reinterpret_cast<const float4*>(vc);
+                    const float4 gj = g_cur[v];
+                    g_cur[v] = make_float4(__double2float_rn(__fma_rn(mu, (double)vj.x, (double)gj.x)),
+                                           __double2float_rn(__fma_rn(mu, (double)vj.y, (double)gj.y)),
+                                           __double2float_rn(__fma_rn(mu, (double)vj.z, (double)gj.z)),
+                                           __double2float_rn(__fma_rn(mu, (double)vj.w, (double)gj.w)));
+                    store_masked(vc, g_cur[v], nel[v]);
+                }
                 const float4 own = (variant & kOwnLastSent) ? h_cur[v] : x_cur[v];
                 const float4 xn = upd4(own, g_cur[v], h_prev[v], h_nxt[v], ul, ur, w, neg_lr);
                 store_masked(x + rb + e[v], xn, nel[v]);

@@ -23,9 +23,10 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
              long long* step_k, int variant, int hops, float* mailbox = nullptr,
-             const uint8_t* __restrict__ arrive = nullptr) {
+             const uint8_t* __restrict__ arrive = nullptr, float* vel = nullptr, double mu = 0.0) {
     // Intermittent delivery (arrive != nullptr): x_hat is the SENT copy, `mailbox` the RECEIVED
     // one, `valid` means "received at least once"; otherwise both copies are x_hat.
+    // Heavy-ball momentum (vel != nullptr): v <- fp32(mu * v + g) per replica, used in place of g.
     extern __shared__ __align__(128) unsigned char smem[];
     uint8_t* s_mode = smem;   // bit 0: dense message, bit 1: valid, bit 2: contributes own x, bit 3: arrives
     double* s_red = reinterpret_cast<double*>(smem + ((P + 15) & ~15));
@@ -78,7 +79,16 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
         if (nel > 0) {
             const long long rb = (long long)j * stride;
             const float4 xj = *reinterpret_cast<const float4*>(xc + rb);
-            const float4 gj = ld_stream(gc + rb);
+            float4 gj = ld_stream(gc + rb);
+            if (vel) {
+                float* vc = vel + off + c + rb;
+                const float4 vj = *reinterpret_cast<const float4*>(vc);
+                gj = make_float4(__double2float_rn(__fma_rn(mu, (double)vj.x, (double)gj.x)),
+                                 __double2float_rn(__fma_rn(mu, (double)vj.y, (double)gj.y)),
+                                 __double2float_rn(__fma_rn(mu, (double)vj.z, (double)gj.z)),
+                                 __double2float_rn(__fma_rn(mu, (double)vj.w, (double)gj.w)));
+                store_masked(vc, gj, nel);
+            }
             const unsigned mj = s_mode[j];
             // what this replica contributes to its neighbours in this step
             const float4 hj = (mj & 4) ? xj
@@ -108,7 +118,15 @@ k_fused_hops(float* x, const float* __restrict__ g, float* xhat,
             if (sn) store_masked(hc + rb, xj, nel);
             if (async && (mj & 8)) store_masked(mc + rb, hj, nel);
             store_masked(xc + rb, xn, nel);
-            if (CARRY) acc = sq_diff4(xn, (variant & kChangeOfNorm) ? zero4 : hj, nel, acc);
+            if (CARRY) {
+                // the next trigger test compares with what this replica has SENT: its x of this
+                // step after a dense message, else the sent copy -- which is what it contributes
+                // unless its neighbours still hold an older copy (a message in flight)
+                float4 ref = hj;
+                if (async && !sn && !(mj & 8)) ref = *reinterpret_cast<const float4*>(hc + rb);
+                if (async && sn) ref = xj;
+                acc = sq_diff4(xn, (variant & kChangeOfNorm) ? zero4 : ref, nel, acc);
+            }
         }
         if (CARRY) {
 #pragma unroll

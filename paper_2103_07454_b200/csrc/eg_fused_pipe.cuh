@@ -160,7 +160,6 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                 long long* step_k, unsigned int* __restrict__ err, int variant_arg,
                 float* mailbox, const uint8_t* __restrict__ arrive, int n_launch,
                 float* __restrict__ vel = nullptr, double mu = 0.0) {
-    static_assert(!(MOM && ASYNC), "momentum is not combined with intermittent delivery");
     constexpr int kArr = MOM ? 4 : 3;              // tiles per stage
     static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
     const int variant = PLAIN ? 0 : variant_arg;
@@ -551,16 +550,18 @@ k_fused_pipe_momentum(float* __restrict__ x, const float* __restrict__ g, float*
 }
 
 // Variants (eg_set_variant) and intermittent delivery; bounded to 72 registers for 3 CTAs per SM.
-template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC>
+// MOM: with heavy-ball momentum (four tiles per stage, one tile per CTA).
+template <int TILE, int STAGES, int CONSUMERS, bool CARRY, bool ASYNC, bool MOM = false>
 __global__ void __launch_bounds__(CONSUMERS + 32, 3)
 k_fused_pipe_general(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
                      const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
                      int P, int T, long long stride, float lr, double* __restrict__ partials,
                      long long* step_k, unsigned int* __restrict__ err, int n_launch, int variant,
-                     float* mailbox, const uint8_t* __restrict__ arrive) {
-    fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, ASYNC, false>(x, g, xhat, snap, valid, tt, P, T, stride,
-                                                                 lr, partials, step_k, err, variant, mailbox,
-                                                                 arrive, n_launch);
+                     float* mailbox, const uint8_t* __restrict__ arrive, float* __restrict__ vel = nullptr,
+                     double mu = 0.0) {
+    fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, ASYNC, false, MOM>(x, g, xhat, snap, valid, tt, P, T, stride,
+                                                                      lr, partials, step_k, err, variant, mailbox,
+                                                                      arrive, n_launch, vel, mu);
 }
 
 // Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes.  The

@@ -656,8 +656,6 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     if (!c || !params || !grads) return EG_ERR_INVALID;
     if (deliver_dev && !c->async) return EG_ERR_STATE;     // eg_enable_delivery_masks first
     if (c->async && (c->variant & kOwnLastSent)) return EG_ERR_STATE;
-    if (c->momentum && (c->async || c->variant != 0 || c->hops > 1 || c->fused_kind == EG_FUSED_REGISTER))
-        return EG_ERR_STATE;
     if (((uintptr_t)params & 15u) || ((uintptr_t)grads & 15u)) return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
     if (!guard.ok) return EG_ERR_CUDA;
@@ -700,7 +698,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         return EG_ERR_STATE;
 
     // a1: || x - x_hat || partial sums, unless the previous step carried them over
-    const bool carry = c->carry && !c->async;   // no carried norm under intermittent delivery
+    const bool carry = c->carry;
     const bool use_carried = carry && c->carried_valid && c->carried_params == params;
     if (!use_carried) {
         TimedSection ts(c, stream, EG_KERNEL_NORM);
@@ -791,38 +789,68 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         const int pipe_stages = c->momentum ? kMomStages : kPipeStages;
         const bool walk = c->P >= pipe_stages && c->P <= c->fused_walk_max_p && !c->momentum;
         const int grid_pipe = walk ? std::min(grid_fused, c->sms * 3 * c->fused_waves) : grid_fused;
-        if (c->hops > 1 && c->hops <= kMaxStagedHops && c->P >= 2 * c->hops + 1 &&
-            c->fused_kind != EG_FUSED_REGISTER) {
+        float* vel = c->momentum ? c->vel : nullptr;
+        float* mailbox = c->async ? c->mailbox : nullptr;
+        const uint8_t* arrive = c->async ? c->arrive : nullptr;
+        // The plain general kernel serves what the specialised ones leave out: more neighbours on
+        // small rings or with momentum, and the carried norm under intermittent delivery.
+        const bool staged = c->hops > 1 && c->hops <= kMaxStagedHops && c->P >= 2 * c->hops + 1 &&
+                            c->fused_kind != EG_FUSED_REGISTER && !c->momentum && !(c->async && carry);
+        if (staged) {
             // rows staged through shared memory; the register kernel choice keeps the plain form
             launch_hops_staged(c, carry, grid_fused, stream, params, grads, valid, tf, lr, partials_fused, step_k);
-        } else if (c->hops > 1) {
+        } else if (c->hops > 1 || (c->async && carry)) {
             if (carry)
                 k_fused_hops<true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->variant, c->hops);
+                    partials_fused, step_k, c->variant, c->hops, mailbox, arrive, vel, c->mu);
             else
                 k_fused_hops<false><<<grid_fused, kThreads, c->fused_smem, stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->variant, c->hops,
-                    c->async ? c->mailbox : nullptr, c->async ? c->arrive : nullptr);
+                    partials_fused, step_k, c->variant, c->hops, mailbox, arrive, vel, c->mu);
         } else if (c->async) {
-            k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>
-                <<<grid_pipe, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
-                params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive);
+            if (c->momentum)
+                k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, false, true, true>
+                    <<<grid_fused, kPipeThreads, MomLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive, vel, c->mu);
+            else
+                k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>
+                    <<<grid_pipe, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive);
+        } else if (c->fused_kind == EG_FUSED_REGISTER) {
+            if (carry)
+                k_fused<kFusedVpt, true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    partials_fused, step_k, c->variant, vel, c->mu);
+            else
+                k_fused<kFusedVpt, false><<<grid_fused, kThreads, c->fused_smem, stream>>>(
+                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
+                    partials_fused, step_k, c->variant, vel, c->mu);
         } else if (c->momentum) {
             const size_t smem = MomLayout::bytes(c->P, carry, kPipeConsumers / 32);
-            if (carry)
-                k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, true>
-                    <<<grid_pipe, kPipeThreads, smem, stream>>>(
-                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->err, grid_fused, c->vel, c->mu);
-            else
-                k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, false>
-                    <<<grid_pipe, kPipeThreads, smem, stream>>>(
-                    params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->err, grid_fused, c->vel, c->mu);
-        } else if (c->fused_kind != EG_FUSED_REGISTER) {
+#define EG_MOM_ARGS params, grads, c->xhat, (const uint8_t*)c->st.snap, valid, tf, c->P, c->T, \
+                    (long long)c->stride, lr, partials_fused, step_k, c->err, grid_fused
+            if (c->variant == 0) {
+                if (carry)
+                    k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, true>
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_MOM_ARGS, c->vel, c->mu);
+                else
+                    k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, false>
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_MOM_ARGS, c->vel, c->mu);
+            } else {
+                if (carry)
+                    k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, true, false, true>
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_MOM_ARGS, c->variant, nullptr, nullptr,
+                                                                      c->vel, c->mu);
+                else
+                    k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, false, false, true>
+                        <<<grid_fused, kPipeThreads, smem, stream>>>(EG_MOM_ARGS, c->variant, nullptr, nullptr,
+                                                                      c->vel, c->mu);
+            }
+#undef EG_MOM_ARGS
+        } else {
             const size_t smem = PipeLayout::bytes(c->P, carry, kPipeConsumers / 32);
 #define EG_PIPE_ARGS params, grads, c->xhat, (const uint8_t*)c->st.snap, valid, tf, c->P, c->T, \
                      (long long)c->stride, lr, partials_fused, step_k, c->err, grid_fused
@@ -844,14 +872,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                         <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
             }
 #undef EG_PIPE_ARGS
-        } else if (carry)
-            k_fused<kFusedVpt, true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
-                params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                partials_fused, step_k, c->variant);
-        else
-            k_fused<kFusedVpt, false><<<grid_fused, kThreads, c->fused_smem, stream>>>(
-                params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                partials_fused, step_k, c->variant);
+        }
         ++launches;
     }
     c->carried_valid = carry && whole;
@@ -1154,7 +1175,6 @@ eg_status eg_set_momentum(eg_ctx* c, int enabled, double mu) {
     if (!c) return EG_ERR_INVALID;
     if (!enabled) { c->momentum = false; c->carried_valid = false; return EG_OK; }
     if (!(mu >= 0.0 && mu < 1.0)) return EG_ERR_INVALID;
-    if (c->async || c->variant != 0 || c->hops > 1) return EG_ERR_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return EG_ERR_CUDA;
     if (!c->vel) {
@@ -1165,6 +1185,12 @@ eg_status eg_set_momentum(eg_ctx* c, int enabled, double mu) {
         EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, true>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_momentum<kPipeTile, kMomStages, kPipeConsumers, false>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, true, false, true>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, false, false, true>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        EG_CUDA(c, cudaFuncSetAttribute(k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, false, true, true>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         EG_CUDA(c, cudaDeviceSynchronize());
         c->vel = v;

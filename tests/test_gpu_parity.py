@@ -82,17 +82,21 @@ def _random_links(P, T, p_up, seed):
 
 @pytest.mark.parametrize("P,hops", [(1, 1), (2, 1), (3, 1), (5, 1), (16, 1), (5, 2), (9, 3), (4, 2), (12, 4)])
 @pytest.mark.parametrize("p_up", [0.0, 0.5, 1.0])
-def test_intermittent_delivery_dense(P, hops, p_up):
+@pytest.mark.parametrize("carry", [False, True])
+def test_intermittent_delivery_dense(P, hops, p_up, carry):
+    """With the carried norm the averaging kernel also leaves the next change norms, taken
+    against what every replica has SENT (not what its neighbours hold)."""
     wl = W.synthetic(P, RAGGED[:-1], steps=16, lr=0.1, grad_sigma=0.01)
-    rep = lockstep(wl, init="distinct", oracle_kw=dict(hops=hops),
+    rep = lockstep(wl, init="distinct", oracle_kw=dict(hops=hops), carry=carry,
                    deliver_fn=_random_links(P, wl.T, p_up, seed=P * 10 + hops))
     assert rep.params_bit_exact and not rep.near_threshold
+    assert rep.launches == (wl.steps * 2 + 1 if carry else wl.steps * 3)
 
 
 @pytest.mark.parametrize("con", [False, True])
 def test_intermittent_delivery_topk(con):
     wl = W.synthetic(6, RAGGED[:-1], steps=16, lr=0.1, grad_sigma=0.01, topk=(5, 100))
-    rep = lockstep(wl, init="distinct", outbox_samples=32, carry=True,     # carry is ignored here
+    rep = lockstep(wl, init="distinct", outbox_samples=32, carry=True,
                    oracle_kw=dict(change_of_norm=con), deliver_fn=_random_links(6, wl.T, 0.4, seed=3))
     assert rep.params_bit_exact
 
@@ -113,12 +117,14 @@ def _random_case(seed):
         okw["threshold_cap"] = (1e-3, 0.8)
     if rng.integers(0, 5) == 0:
         okw.update(mode=1, delta_fixed=float(rng.choice([0.0, 0.01])), force_first_event=bool(rng.integers(0, 2)))
+    if rng.integers(0, 3) == 0:
+        okw["momentum"] = float(rng.choice([0.0, 0.5, 0.9]))
     return dict(P=P, sizes=sizes, topk=topk, okw=okw, carry=bool(rng.integers(0, 2)),
                 kernel=[B.FUSED_PIPELINED, B.FUSED_REGISTER][int(rng.integers(0, 2))],
                 deliver=_random_links(P, len(sizes), float(rng.choice([0.3, 0.8])), seed) if deliver else None)
 
 
-@pytest.mark.parametrize("seed", range(32))
+@pytest.mark.parametrize("seed", range(48))
 def test_random_option_combinations(seed):
     case = _random_case(seed)
     wl = W.synthetic(case["P"], case["sizes"], steps=14, lr=0.1, grad_sigma=0.01, topk=case["topk"],
@@ -442,18 +448,39 @@ def test_momentum_zero_reset_roundtrip_and_refusals():
     for bad in (-0.5, 1.0, float("nan")):
         with pytest.raises(B.EventGradError):
             mom.set_momentum(bad)
-    # combinations that have no momentum kernel are refused, not silently computed without it
-    mom.set_momentum(0.9)
-    mom.set_fused_kernel(B.FUSED_REGISTER)
-    with pytest.raises(B.EventGradError):
-        mom.step(xb, g, wl.lr)
-    mom.set_fused_kernel(B.FUSED_PIPELINED)
-    mom.step(xb, g, wl.lr)
-    wide = B.from_workload(wl, hops=2)
-    with pytest.raises(B.EventGradError):
-        wide.set_momentum(0.9)
-    for e in (plain, mom, wide):
+    for e in (plain, mom):
         e.close()
+
+
+@pytest.mark.parametrize("what", ["hops2", "hops3_small_ring", "own_last_sent", "change_of_norm", "delivery",
+                                  "delivery_hops", "register", "topk_hops", "everything"])
+@pytest.mark.parametrize("carry", [False, True])
+def test_momentum_with_every_other_option(what, carry):
+    """Heavy-ball momentum next to more neighbours, the other readings, intermittent delivery, the
+    register kernel and Top-K: velocities, parameters, mailboxes and counters are the oracle's."""
+    okw, kw, topk, P = dict(momentum=0.9), {}, None, 7
+    if what == "hops2":
+        okw.update(hops=2)
+    elif what == "hops3_small_ring":
+        okw.update(hops=3); P = 4
+    elif what == "own_last_sent":
+        okw.update(own_last_sent=True)
+    elif what == "change_of_norm":
+        okw.update(change_of_norm=True)
+    elif what == "delivery":
+        kw.update(deliver_fn=_random_links(P, len(RAGGED) - 1, 0.5, seed=5))
+    elif what == "delivery_hops":
+        okw.update(hops=2); kw.update(deliver_fn=_random_links(P, len(RAGGED) - 1, 0.5, seed=6))
+    elif what == "register":
+        kw.update(fused_kernel=B.FUSED_REGISTER)
+    elif what == "topk_hops":
+        okw.update(hops=2); topk = (5, 100)
+    else:
+        okw.update(hops=2, change_of_norm=True, history_len=3, threshold_cap=(1e-3, 0.8)); topk = (5, 100)
+        kw.update(deliver_fn=_random_links(P, len(RAGGED) - 1, 0.6, seed=7))
+    wl = W.synthetic(P, RAGGED[:-1], steps=12, lr=0.1, grad_sigma=0.01, topk=topk)
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=okw, outbox_samples=16, **kw)
+    assert rep.params_bit_exact and not rep.near_threshold
 
 
 def test_momentum_resnet18_shapes_p16():
