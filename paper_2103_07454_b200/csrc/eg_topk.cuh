@@ -29,6 +29,7 @@
 #include <cooperative_groups.h>
 
 #include "eg_common.cuh"
+#include "eg_fused_pipe.cuh"
 
 namespace eg {
 
@@ -559,6 +560,183 @@ topk_collect(const float* __restrict__ x, const float* __restrict__ xhat, TileTa
     }
 }
 
+// The collecting pass with the tiles staged through shared memory (the form the single-phase
+// launch uses; needs eg_fused_pipe.cuh's barrier and bulk-copy wrappers).  Same entries, counts
+// and histograms as topk_collect.  One producer warp walks the CTA's share of the work list and
+// brings tile after tile -- 16 KB of x and 16 KB of x_hat, two bulk asynchronous copies -- into a
+// ring of kCollectStages stages together with a small header (segment, bin, length, where the
+// entries go), so that the bytes in flight do not depend on what the eight consumer warps are
+// doing; the consumers read their 512 elements from shared memory, mark them, and since the
+// tile stays where it is they build the entries from it by position afterwards.
+constexpr int kCollectStages = 3;
+constexpr int kCollectThreads = kThreads + 32;
+struct CollectHeader {
+    int len, i, tile, s;        // elements of the tile, replica, tile id, segment id
+    unsigned int b0;            // the bin b' of the segment
+    int last_of_segment;        // flush the counters after this tile
+    int pad[2];
+};
+struct CollectSmem {
+    static constexpr int kStageBytes = 2 * kNormTile * 4;                       // x, x_hat
+    static constexpr int kHeaders = kCollectStages * kStageBytes;
+    static constexpr int kBars = kHeaders + kCollectStages * (int)sizeof(CollectHeader);
+    static constexpr int kHist = kBars + 8 * 2 * kCollectStages + 16;             // full[S], empty[S], abort flag
+    static constexpr int kOff = kHist + kMaxBins * 4;
+    static constexpr int kWhere = kOff + kOffBins * 4 + 32;
+    static constexpr int kBytes = kWhere + kWarps * kWarpSpan * 2;                // a position per possible entry
+};
+
+__device__ __forceinline__ void
+topk_collect_staged(const float* __restrict__ x, const float* __restrict__ xhat, TileTable tt, int T,
+                    long long stride, const TopkState& tk, const WorkList& wl, unsigned int* __restrict__ err,
+                    int shares) {
+    constexpr int kBins1 = 1 << kDigitBits1;
+    extern __shared__ __align__(128) unsigned char smem[];
+    CollectHeader* headers = reinterpret_cast<CollectHeader*>(smem + CollectSmem::kHeaders);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + CollectSmem::kBars);
+    uint64_t* empty = full + kCollectStages;
+    volatile int* s_abort = reinterpret_cast<volatile int*>(empty + kCollectStages);
+    unsigned int* s_hist = reinterpret_cast<unsigned int*>(smem + CollectSmem::kHist);
+    unsigned int* s_off = reinterpret_cast<unsigned int*>(smem + CollectSmem::kOff);
+    unsigned short* s_where = reinterpret_cast<unsigned short*>(smem + CollectSmem::kWhere);
+    const WorkRange r = work_range(wl, shares);
+    if (r.w0 >= r.w1) return;                   // the same in every thread
+    const int tid = threadIdx.x;
+    for (int b = tid; b < kMaxBins; b += kCollectThreads) s_hist[b] = 0;
+    if (tid < kOffBins) s_off[tid] = 0;
+    if (tid == 0) {
+        for (int s = 0; s < kCollectStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWarps); }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid >= kThreads) {
+        // ------------------------------------------------------------------ producer (one lane)
+        if (tid == kThreads) {
+            WorkCursor cur;
+            cur.init(r.q);
+            unsigned int b0 = 0;
+            int s = 0;
+            for (int w = r.w0, n = 0; w < r.w1; ++w, ++n) {
+                bool changed;
+                const int tile = cur.advance(wl, tt, T, w, changed);
+                if (changed) b0 = tk.prefix[cur.s];
+                const int len = tt.length[tile];
+                const long long base = (long long)cur.i * stride + tt.offset[tile];
+                if (n >= kCollectStages &&
+                    !mbar_wait_bounded(&empty[s], (uint32_t)((n / kCollectStages - 1) & 1), s_abort, err))
+                    break;
+                CollectHeader h;
+                h.len = len; h.i = cur.i; h.tile = tile; h.s = cur.s; h.b0 = b0;
+                h.last_of_segment = (w + 1 == r.w1 || w + 1 >= cur.end) ? 1 : 0;
+                h.pad[0] = h.pad[1] = 0;
+                headers[s] = h;
+                const uint32_t bytes = (uint32_t)(((len + 3) & ~3) * 4);
+                float* st = reinterpret_cast<float*>(smem + s * CollectSmem::kStageBytes);
+                mbar_expect_tx(&full[s], 2u * bytes);      // (a release: the header is visible with the data)
+                bulk_g2s(st, x + base, bytes, &full[s]);
+                bulk_g2s(st + kNormTile, xhat + base, bytes, &full[s]);
+                if (++s == kCollectStages) s = 0;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumers
+        const int lane = tid & 31, warp = tid >> 5;
+        const int mine = warp * kWarpSpan + lane * 4;      // this lane's first element of the tile
+        unsigned short* my_where = s_where + warp * kWarpSpan;
+        int s = 0;
+        for (int w = r.w0, n = 0; w < r.w1; ++w, ++n) {
+            if (!mbar_wait_bounded(&full[s], (uint32_t)((n / kCollectStages) & 1), s_abort, err)) break;
+            const CollectHeader h = headers[s];
+            const float* sx = reinterpret_cast<const float*>(smem + s * CollectSmem::kStageBytes);
+            const float* sh = sx + kNormTile;
+            const unsigned int b0 = h.b0;
+            const float thr = __uint_as_float(b0 << 20);
+            const int len = h.len;
+            unsigned int mask = 0, packed = 0;      // bit 4j+c: element c of chunk j is an entry
+#pragma unroll
+            for (int j = 0; j < kSubChunks; ++j) {
+                const int local = mine + j * 128;
+                const int nel = len - local;          // live elements of this float4 (<= 0: none)
+                unsigned int m = 0;
+                if (nel > 0) {
+                    const float4 a = *reinterpret_cast<const float4*>(sx + local);
+                    const float4 b = *reinterpret_cast<const float4*>(sh + local);
+                    m |= !(fabsf(__fsub_rn(a.x, b.x)) < thr) ? 1u : 0u;
+                    m |= (1 < nel && !(fabsf(__fsub_rn(a.y, b.y)) < thr)) ? 2u : 0u;
+                    m |= (2 < nel && !(fabsf(__fsub_rn(a.z, b.z)) < thr)) ? 4u : 0u;
+                    m |= (3 < nel && !(fabsf(__fsub_rn(a.w, b.w)) < thr)) ? 8u : 0u;
+                }
+                mask |= m << (4 * j);
+                packed |= (unsigned int)__popc(m) << (8 * j);
+            }
+            unsigned int inc = packed;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int u = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += u;
+            }
+            const unsigned int tot = __shfl_sync(0xffffffffu, inc, 31);
+            const unsigned int excl = inc - packed;
+            const unsigned int total = (tot & 0xffu) + ((tot >> 8) & 0xffu) + ((tot >> 16) & 0xffu) + (tot >> 24);
+            // positions of the marked elements, in slot order
+            unsigned int chunk_first = 0;
+#pragma unroll
+            for (int j = 0; j < kSubChunks; ++j) {
+                const unsigned int m = (mask >> (4 * j)) & 0xfu;
+                if (m) {                                         // few lanes hold an entry in a given chunk
+                    unsigned int pos = chunk_first + ((excl >> (8 * j)) & 0xffu);
+                    const unsigned short where = (unsigned short)(j * 128 + lane * 4);
+                    if (m & 1u) my_where[pos++] = where;
+                    if (m & 2u) my_where[pos++] = where + 1;
+                    if (m & 4u) my_where[pos++] = where + 2;
+                    if (m & 8u) my_where[pos++] = where + 3;
+                }
+                chunk_first += (tot >> (8 * j)) & 0xffu;
+            }
+            __syncwarp();
+            // the entries, one per lane, from the tile in shared memory
+            const long long base = (long long)h.i * stride + tt.offset[h.tile];
+            uint2* ent = tk.ent + base + sub_offset(len, warp);
+            const int room = len - sub_offset(len, warp);      // slots of this sub-slice (bounds-checked build)
+            for (unsigned int e = lane; e < total; e += 32) {
+                const unsigned int where = my_where[e];
+                const float xv = sx[warp * kWarpSpan + where];
+                const unsigned int k = rank_key(xv, sh[warp * kWarpSpan + where]);
+                const unsigned int off = min((k >> 20) - b0, (unsigned int)(kOffBins - 1));
+                if (!EG_INDEX_OK(tt.err, e, room)) continue;
+                ent[e] = make_uint2((off << 29) | ((k & 0xfffffu) << 9) | where, __float_as_uint(xv));
+                atomicAdd(&s_off[off], 1u);
+                if (off < (unsigned int)kOffHist) atomicAdd(&s_hist[off * kBins1 + ((k >> 10) & (kBins1 - 1))], 1u);
+            }
+            if (lane == 0) tk.tile_cand[((long long)h.i * tt.n_tiles + h.tile) * kSubSlices + warp] = (int)total;
+            // everything this warp needs from the stage has been read
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+            if (h.last_of_segment) {
+                // the eight consumer warps meet (the producer does not take part)
+                asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+                unsigned int* gh = tk.hist + (long long)h.s * kMaxBins;
+                for (int b = tid; b < kMaxBins; b += kThreads) {
+                    const unsigned int v = s_hist[b];
+                    if (v) { atomicAdd(&gh[b], v); s_hist[b] = 0; }
+                }
+                if (tid < kOffBins) {
+                    const unsigned int v = s_off[tid];
+                    if (v) { atomicAdd(&tk.offcnt[(long long)h.s * kOffBins + tid], v); s_off[tid] = 0; }
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+            }
+            if (++s == kCollectStages) s = 0;
+        }
+    }
+    if (*s_abort) {
+        // failure path only: give copies in flight time to land before the CTA retires
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) {}
+    }
+}
+
 // One warp per listed segment, after the collecting pass: the exact counts of the collected bins
 // place tau's top digit (counting K_t entries down from the highest bin) and the rank left
 // inside that bin; digit 1 then comes from the bin's digit-1 histogram.  A segment whose guess
@@ -989,12 +1167,12 @@ __global__ void __launch_bounds__(kThreads) k_topk_pick(TopkArgs a, int which, i
     if (!topk_enter(a, which)) return;
     topk_pick(a.T, a.tk, a.tk.list[which], digit);
 }
-#ifndef EG_COLLECT_MINB
-#define EG_COLLECT_MINB 4
-#endif
-__global__ void __launch_bounds__(kThreads, EG_COLLECT_MINB) k_topk_collect(TopkArgs a, int which) {
+// The collecting pass runs kCollectShares planned shares per CTA (two CTAs of 288 threads and
+// 107 KB of shared memory fit a multiprocessor).
+constexpr int kCollectShares = 4;
+__global__ void __launch_bounds__(kCollectThreads, 2) k_topk_collect(TopkArgs a, int which) {
     if (!topk_enter(a, which)) return;
-    topk_collect(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.tk.list[which]);
+    topk_collect_staged(a.x, a.xhat, a.tt, a.T, a.stride, a.tk, a.tk.list[which], a.err, kCollectShares);
 }
 __global__ void __launch_bounds__(kThreads) k_topk_resolve(TopkArgs a, int which) {
     if (!topk_enter(a, which)) return;

@@ -535,6 +535,11 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
             if ((long long)P * c->tiles_norm.n_tiles > 65536 || getenv("EG_TOPK_SEPARATE_LAUNCHES"))
                 c->topk_coop_grid = 0;
         }
+        {
+            const cudaError_t e = cudaFuncSetAttribute(k_topk_collect, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                       (int)CollectSmem::kBytes);
+            if (e != cudaSuccess) { c->last_cuda_error = (int)e; return fail(EG_ERR_CUDA); }
+        }
         c->tk.out_off = c->d_out_off;
         c->tk.count = c->d_kcount;
         c->tk.numel = c->d_numel;
@@ -758,16 +763,17 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
             // lets its successor in before it ends.
             const bool pdl = !c->timing && !c->no_pdl && c->topk_pdl;
             const dim3 one(1), tile_blocks(tile_grid), entry_blocks(tile_grid / kEntryShares), seg_blocks(seg_grid);
+            const dim3 collect_blocks(tile_grid / kCollectShares);
             const dim3 threads(kThreads);
             EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, threads, 0, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, threads, 0, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_guess, seg_blocks, threads, 0, stream, ta));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, tile_blocks, threads, 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, collect_blocks, dim3(kCollectThreads), (size_t)CollectSmem::kBytes, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_resolve, seg_blocks, threads, 0, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, threads, 0, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, threads, 0, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, threads, 0, stream, ta, 1, 0));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, tile_blocks, threads, 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_collect, collect_blocks, dim3(kCollectThreads), (size_t)CollectSmem::kBytes, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_resolve, seg_blocks, threads, 0, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_digit2, entry_blocks, threads, 0, stream, ta));
             EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, threads, 0, stream, ta, 0, 2));
