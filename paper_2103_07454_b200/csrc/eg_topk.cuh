@@ -881,7 +881,7 @@ store_tile_counts(const TopkState& tk, long long slot, long long tile_index, uns
 // decides).  Open entries -- about one in a thousand -- go into the digit-2 histogram.  Per
 // sub-slice and per tile the kernel stores (greater for sure, open); for a tile without open
 // entries these are already its final (greater than tau, equal to tau) counts, the few tiles
-// that have some are counted again once tau is complete (topk_scan).
+// that have some are counted again once tau is complete (topk_recount).
 __device__ __forceinline__ void
 topk_digit2(TileTable tt, int T, long long stride, const TopkState& tk, const WorkList& wl, int shares = 1) {
     const int lane = threadIdx.x & 31, u = lane / kGroupLanes, r = lane % kGroupLanes;
@@ -944,9 +944,24 @@ count_tile_exact(const TileTable& tt, long long stride, const TopkState& tk, int
     store_tile_counts(tk, index * kSubSlices, index, gt, eq);
 }
 
-// One CTA per sparse segment.  First the tiles that held open entries are counted again, now
-// that tau is complete (a handful per tensor, unless many keys tie); then the exclusive prefix
-// of the tile counts, in tile order.
+// Once tau is complete: the tiles that held open entries are counted again (a handful per tensor
+// unless many keys tie).  One warp per tile of the work list; a tile without open entries costs
+// one 8-byte read.
+__device__ __forceinline__ void
+topk_recount(TileTable tt, int T, long long stride, const TopkState& tk, const WorkList& wl, int shares = 1) {
+    WarpWalk walk;
+    walk.init(wl, shares);
+    WarpTile z;
+    int s_now = -1;
+    unsigned int tau20 = 0, sel = 0;
+    while (walk.next(wl, tt, T, z)) {
+        if (tk.tile_count[(long long)z.i * tt.n_tiles + z.tile].y == 0u) continue;     // the same in every lane
+        if (z.s != s_now) { s_now = z.s; tau20 = tk.prefix[z.s] & 0xfffffu; sel = tk.offsel[z.s]; }
+        count_tile_exact(tt, stride, tk, z.i, z.tile, sel, tau20);
+    }
+}
+
+// One CTA per sparse segment: the exclusive prefix of the tile counts, in tile order.
 __device__ __forceinline__ void
 topk_scan(TileTable tt, int T, long long stride, const TopkState& tk, const WorkList& wl) {
     __shared__ unsigned int s_gt[kWarps], s_eq[kWarps];
@@ -958,19 +973,8 @@ topk_scan(TileTable tt, int T, long long stride, const TopkState& tk, const Work
         const int i = s / T, t = s - i * T;
         const int q0 = tt.seg_begin[t], q1 = tt.seg_begin[t + 1];
         uint2* tc = tk.tile_count + (long long)i * tt.n_tiles;
-        const unsigned int tau20 = tk.prefix[s] & 0xfffffu, sel = tk.offsel[s];
-        for (int c0 = q0; c0 < q1; c0 += 32 * kWarps) {
-            // a lane looks at one tile; the warp then counts the marked ones together, one by one
-            const int z = c0 + warp * 32 + lane;
-            unsigned int marked = __ballot_sync(0xffffffffu, z < q1 && tc[z].y != 0u);
-            while (marked) {
-                const int l = __ffs(marked) - 1;
-                marked &= marked - 1u;
-                count_tile_exact(tt, stride, tk, i, c0 + warp * 32 + l, sel, tau20);
-            }
-        }
         if (threadIdx.x == 0) s_run[0] = s_run[1] = 0;
-        __syncthreads();            // the recounted pairs are visible to the whole CTA
+        __syncthreads();
         for (int c0 = q0; c0 < q1; c0 += kThreads) {
             const int z = c0 + threadIdx.x;
             uint2 v = make_uint2(0, 0);
@@ -1137,6 +1141,8 @@ __global__ void __launch_bounds__(kThreads, 4) k_topk_all(TopkArgs a) {
     grid.sync();
     topk_pick(a.T, a.tk, all, 2);
     grid.sync();
+    topk_recount(a.tt, a.T, a.stride, a.tk, all);
+    grid.sync();
     topk_scan(a.tt, a.T, a.stride, a.tk, all);
     grid.sync();
     topk_write(a.xhat, a.tt, a.T, a.stride, a.tk, all, a.err);
@@ -1189,6 +1195,10 @@ constexpr int kEntryShares = EG_ENTRY_SHARES;
 __global__ void __launch_bounds__(kThreads, EG_ENTRY_MINB) k_topk_digit2(TopkArgs a) {
     if (!topk_enter(a, 0)) return;
     topk_digit2(a.tt, a.T, a.stride, a.tk, a.tk.list[0], kEntryShares);
+}
+__global__ void __launch_bounds__(kThreads, EG_ENTRY_MINB) k_topk_recount(TopkArgs a) {
+    if (!topk_enter(a, 0)) return;
+    topk_recount(a.tt, a.T, a.stride, a.tk, a.tk.list[0], kEntryShares);
 }
 __global__ void __launch_bounds__(kThreads) k_topk_scan(TopkArgs a) {
     if (!topk_enter(a, 0)) return;

@@ -757,7 +757,7 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                                                    dim3(kThreads), args, 0, stream));
             launches += 1;
         } else {
-            // Fourteen launches, five of which (the exact repeat for segments whose guessed bin
+            // Fifteen launches, five of which (the exact repeat for segments whose guessed bin
             // did not work out) leave at once in an ordinary iteration.  They are dependent launches:
             // each waits on the device, first thing it does, for the kernel before it, and none
             // lets its successor in before it ends.
@@ -777,9 +777,10 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
             EG_CUDA(c, launch_pdl(pdl, k_topk_resolve, seg_blocks, threads, 0, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_digit2, entry_blocks, threads, 0, stream, ta));
             EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, threads, 0, stream, ta, 0, 2));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_recount, entry_blocks, threads, 0, stream, ta));
             EG_CUDA(c, launch_pdl(pdl, k_topk_scan, seg_blocks, threads, 0, stream, ta));
             EG_CUDA(c, launch_pdl(pdl, k_topk_write, entry_blocks, threads, 0, stream, ta));
-            launches += 14;
+            launches += 15;
         }
     }
     // a3 + a5: dense snapshot, consensus average, SGD
