@@ -114,28 +114,34 @@ struct PipeSmem {
     static constexpr int kWrapR = kWrapL + (RUNS ? 2 : 1) * kTileBytes;
     static constexpr int kBars = kWrapR + kTileBytes;             // full[S], empty[S], wrap[2]
     static constexpr int kFlags = kBars + 8 * (2 * STAGES + 2);
-    // then 16 bytes of flags, two tables of per-replica modes (consecutive tiles alternate) and,
+    static constexpr int kModes = kFlags + 16 + 2 * 32;           // after the flags: two tile headers of 32 bytes
+    // then 16 bytes of flags, two tile headers, two tables of per-replica modes (consecutive tiles alternate) and,
     // for the carried norm, per stage one slot of 8 doubles per consumer warp (see the consumers'
     // end of a replica and the producer warp's reduce_slot)
     __host__ __device__ static size_t mode_bytes(int P) { return ((size_t)P + 15) & ~(size_t)15; }
     __host__ __device__ static size_t bytes(int P, bool carry, int consumer_warps) {
-        size_t b = kFlags + 16 + (RUNS ? 2 : 1) * mode_bytes(P);
+        size_t b = kModes + (RUNS ? 2 : 1) * mode_bytes(P);
         if (carry) b += (size_t)STAGES * consumer_warps * 8 * sizeof(double);
         return b;
     }
 };
 
 // Body of the kernels below.  The launch covers `n_launch` tiles of the tile table (TILE elements
-// per tile); CTA b takes the tiles b, b + gridDim.x, b + 2 gridDim.x, ... one after the other (so
-// that the CTAs running at any moment work on neighbouring tiles, as they would with one tile
-// per CTA: runs of consecutive tiles per CTA measured 5-10 % slower at 16 and 64 replicas), and
-// keeps its ring of stages full across them: the producer warp starts on the replicas of the
-// next tile while the consumers still work on the current one, so that a CTA pays for filling
-// and draining the ring once, not once per tile (with few replicas that was a large part of a
-// CTA's life).  What belongs to a tile and not to a stage -- the per-replica modes and the
-// wrap-around contribution of replica P-1 -- exists twice and consecutive tiles alternate; this
-// is safe when P >= STAGES (the producer is then never more than one tile ahead of the
-// consumers), which the host guarantees by launching one CTA per tile otherwise.
+// per tile).  CTA b begins with tile b; launched with fewer CTAs than tiles and a `ticket`
+// counter (zeroed by the decision kernel before it), a CTA goes on with tile gridDim.x + the
+// counter's next value, and so on until the tiles are used up.  The CTAs running at any moment
+// then work on neighbouring tiles, as they would with one tile per CTA, however far they drift
+// apart (runs of consecutive tiles per CTA measured 5-10 % slower at 16 and 64 replicas, the
+// fixed stride b, b + gridDim.x, ... 2-10 % slower from 16 replicas on).  A walking CTA keeps
+// its ring of stages full across tiles: the producer warp starts on the replicas of the next
+// tile while the consumers still work on the current one, so that a CTA pays for filling and
+// draining the ring once, not once per tile (with few replicas that was a large part of a
+// CTA's life).  The producer knows its tiles three ahead (number, then record, then flags, each
+// fetched a tile before it is needed) and tells the consumers about each through a header in
+// shared memory.  What belongs to a tile and not to a stage -- the header, the per-replica
+// modes and the wrap-around contribution of replica P-1 -- exists twice and consecutive tiles
+// alternate; this is safe when P >= STAGES (the producer is then never more than one tile
+// ahead of the consumers), which the host guarantees by launching one CTA per tile otherwise.
 // CONSUMERS + 32 threads; COLS = TILE / (4 * CONSUMERS) float4 columns per consumer thread.
 //
 // ASYNC (intermittent delivery): x_hat is what a replica has SENT, `mailbox` what its
@@ -158,7 +164,7 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                 const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, const TileTable& tt,
                 int P, int T, long long stride, float lr, double* __restrict__ partials,
                 long long* step_k, unsigned int* __restrict__ err, int variant_arg,
-                float* mailbox, const uint8_t* __restrict__ arrive, int n_launch,
+                float* mailbox, const uint8_t* __restrict__ arrive, int n_launch, int* ticket,
                 float* __restrict__ vel = nullptr, double mu = 0.0) {
     constexpr int kArr = MOM ? 4 : 3;              // tiles per stage
     static_assert(!(ASYNC && CARRY), "the carried norm is not produced under intermittent delivery");
@@ -178,12 +184,19 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
     uint64_t* wrap_bar2 = empty + STAGES;                          // [2]
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kFlags);
     // bit 0: dense message, bit 1: valid, bit 2: contributes its own x, bit 3: arrives now
-    uint8_t* s_mode2 = smem + L::kFlags + 16;                      // [2][mode_bytes(P)]
+    // what the producer tells the consumers about a tile: which one, its length and place, and
+    // whether this CTA has another tile after it
+    struct TileHeader { int tile, len; long long off; int has_next; int pad[3]; };
+    static_assert(sizeof(TileHeader) == 32, "two headers sit between the flags and the mode tables");
+    TileHeader* s_hdr = reinterpret_cast<TileHeader*>(smem + L::kFlags + 16);   // [2]
+    uint8_t* s_mode2 = smem + L::kModes;                           // [2][mode_bytes(P)]
     const int mode_stride = (int)L::mode_bytes(P);
     double* s_part = reinterpret_cast<double*>(s_mode2 + (RUNS ? 2 : 1) * mode_stride);   // [STAGES][CWARPS * 8]
 
     const int tid = threadIdx.x;
-    // tiles of this CTA: first, first + hop, ... below last (RUNS = false: the first one only)
+    // Tiles of this CTA: the first is its own number; with RUNS further ones follow -- first + hop,
+    // first + 2 hop, ... below last, or (`ticket` given) whatever a counter shared by the CTAs
+    // hands out next, so that tiles are begun in order however unevenly the CTAs advance.
     const int first = (int)blockIdx.x, hop = (int)gridDim.x;
     const int last = RUNS ? n_launch : min(n_launch, first + 1);
     if (first >= last) return;                   // the same in every thread
@@ -227,15 +240,15 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         // Items are (tile, replica) pairs in the order they go through the ring; item m uses
         // stage m % STAGES in its (m / STAGES)-th filling.  retire(m): wait until the consumers
         // have released item m, then (CARRY) finish its sum of squares.
-        int retired = 0, r_tile = first, r_j = 0;     // next item to retire and what it is
+        int retired = 0, r_buf = 0, r_j = 0;          // next item to retire: replica r_j of the tile of header r_buf
         auto retire = [&]() -> bool {
             const int sm = retired % STAGES;
             bool alive = mbar_wait_bounded(&empty[sm], (uint32_t)((retired / STAGES) & 1), s_abort, err);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) return false;
-            if (CARRY) reduce_slot(sm, r_tile, r_j);
+            if (CARRY) reduce_slot(sm, s_hdr[r_buf].tile, r_j);
             ++retired;
-            if (++r_j == P) { r_j = 0; r_tile += hop; }
+            if (++r_j == P) { r_j = 0; r_buf = RUNS ? (r_buf ^ 1) : 0; }
             return true;
         };
         // the record of a tile: lane-uniform
@@ -265,15 +278,32 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                 pre_ar[q] = ASYNC ? arrive[at] : (uint8_t)0;
             }
         };
+        // The tiles to come, known three ahead: the number of tile it + 3 is asked for when tile it
+        // begins (lane 0 holds the counter's answer; it is passed round one tile later, when it has
+        // long arrived), the record of tile it + 2 is read then, and the flags of tile it + 1.
+        int seq = first;                              // fixed stride: the last number formed
+        auto ask = [&]() -> int {
+            if (ticket) return (pl == 0) ? hop + atomicAdd(ticket, 1) : 0;
+            seq += hop;
+            return seq;
+        };
+        auto told = [&](int raw) -> int {             // the answer, in every lane; none left: last
+            const int id = ticket ? __shfl_sync(0xffffffffu, raw, 0) : raw;
+            return (id >= 0 && id < last) ? id : last;
+        };
         int issued = 0, s = 0;
         bool alive = true;
-        Rec rec = load_rec(first);
-        Rec rec_next = (first + hop < last) ? load_rec(first + hop) : rec;
+        const int raw1 = RUNS ? ask() : last, raw2 = RUNS ? ask() : last;
+        int raw3 = RUNS ? ask() : last;               // three requests on their way together
+        int id0 = first, id1 = RUNS ? told(raw1) : last, id2 = RUNS ? told(raw2) : last;
+        Rec rec = load_rec(id0);
+        Rec rec1 = (id1 < last) ? load_rec(id1) : rec;
+        Rec rec2 = (id2 < last) ? load_rec(id2) : rec;
         if (prefetch) fetch_flags(rec.t);
-        int it = 0;                                 // how many tiles this CTA has begun
-        for (int tile = first; tile < last && alive; tile += hop, ++it) {
+        for (int it = 0; id0 < last && alive; ++it) {
+            const int tile = id0;
             if (!tile_ok(tt, tile, T, stride, TILE)) break;      // bounds-checked build only (the consumers leave too)
-            if (tile + hop >= last) pdl_release();
+            if (id1 >= last) pdl_release();
             const int buf = RUNS ? (it & 1) : 0;
             uint8_t* sm = s_mode2 + buf * mode_stride;
             // modes of this tile (its flags were read one tile ago), then the flags of the next
@@ -287,11 +317,20 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
                     sm[j] = mode_of(snap[at], valid[at], ASYNC ? arrive[at] : (uint8_t)0);
                 }
             }
-            __syncwarp();
             const Rec cur = rec;
-            rec = rec_next;
-            if (tile + 2 * hop < last) rec_next = load_rec(tile + 2 * hop);
-            if (prefetch && tile + hop < last) fetch_flags(rec.t);
+            if (pl == 0) {
+                TileHeader h;
+                h.tile = tile; h.len = cur.len; h.off = cur.off; h.has_next = id1 < last ? 1 : 0;
+                h.pad[0] = h.pad[1] = h.pad[2] = 0;
+                s_hdr[buf] = h;
+            }
+            __syncwarp();
+            // move on by one tile: numbers, records, flags
+            id0 = id1; id1 = id2; id2 = RUNS ? told(raw3) : last;
+            rec = rec1; rec1 = rec2;
+            if (RUNS) raw3 = ask();
+            if (id2 < last) rec2 = load_rec(id2);
+            if (prefetch && id0 < last) fetch_flags(rec.t);
             const uint32_t copy_bytes = (uint32_t)(((cur.len + 3) & ~3) * 4);
             const float* xp = x + cur.off;
             const float* gp = g + cur.off;
@@ -340,28 +379,28 @@ fused_pipe_body(float* __restrict__ x, const float* __restrict__ g, float* __res
         int s = 0, s1 = (STAGES > 1) ? 1 : 0;
         uint32_t par_s = 0u, parity1 = (STAGES > 1) ? 0u : 1u;
         bool ok = true;
-        int len = tt.length[first];
-        long long off = tt.offset[first];
-        int it = 0;
-        for (int tile = first; tile < last && ok; tile += hop, ++it) {
-            if (!tile_ok(tt, tile, T, stride, TILE)) break;      // bounds-checked build only (the producer leaves too)
-            if (tile + hop >= last) pdl_release();
+        bool more_tiles = true;
+        for (int it = 0; more_tiles && ok; ++it) {
             const int buf = RUNS ? (it & 1) : 0;
             const uint8_t* s_mode = s_mode2 + buf * mode_stride;
             const float* wrap_l = wrap_l2 + buf * TILE;
             uint64_t* wrap_bar = &wrap_bar2[buf];
-            const int len_now = len;
-            const long long off_now = off;
-            if (tile + hop < last) { len = tt.length[tile + hop]; off = tt.offset[tile + hop]; }   // used one tile later
-            int nel[COLS];
-#pragma unroll
-            for (int v = 0; v < COLS; ++v) nel[v] = min(4, max(0, len_now - (v * CONSUMERS + tid) * 4));
             // contributions of replica j-1 and j to their neighbours, for this thread's columns,
             // kept as doubles so that every value is converted once
             double hp[COLS][4], hc[COLS][4];
             ok = mbar_wait_bounded(wrap_bar, (uint32_t)((it >> (RUNS ? 1 : 0)) & 1), s_abort, err) &&
                  mbar_wait_bounded(&full[s], par_s, s_abort, err);
             if (!ok) break;
+            // (the header and the mode table were written before the tile's first copies were started)
+            const int tile = s_hdr[buf].tile;
+            const int len_now = s_hdr[buf].len;
+            const long long off_now = s_hdr[buf].off;
+            more_tiles = s_hdr[buf].has_next != 0;
+            if (!tile_ok(tt, tile, T, stride, TILE)) break;      // bounds-checked build only (the producer leaves too)
+            if (!more_tiles) pdl_release();
+            int nel[COLS];
+#pragma unroll
+            for (int v = 0; v < COLS; ++v) nel[v] = min(4, max(0, len_now - (v * CONSUMERS + tid) * 4));
             unsigned mode_prev = s_mode[P - 1], mode_cur = s_mode[0];
 #pragma unroll
             for (int v = 0; v < COLS; ++v) {
@@ -530,10 +569,10 @@ __global__ void __launch_bounds__(CONSUMERS + 32, 3)
 k_fused_pipe(float* __restrict__ x, const float* __restrict__ g, float* __restrict__ xhat,
              const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
              int P, int T, long long stride, float lr, double* __restrict__ partials,
-             long long* step_k, unsigned int* __restrict__ err, int n_launch) {
+             long long* step_k, unsigned int* __restrict__ err, int n_launch, int* ticket) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true>(x, g, xhat, snap, valid, tt, P, T, stride, lr,
                                                                 partials, step_k, err, 0, nullptr, nullptr,
-                                                                n_launch);
+                                                                n_launch, ticket);
 }
 
 // Heavy-ball momentum on the default readings (eg_set_momentum): four tiles per stage.
@@ -546,7 +585,7 @@ k_fused_pipe_momentum(float* __restrict__ x, const float* __restrict__ g, float*
                       float* __restrict__ vel, double mu) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, false, true, true>(x, g, xhat, snap, valid, tt, P, T, stride,
                                                                       lr, partials, step_k, err, 0, nullptr,
-                                                                      nullptr, n_launch, vel, mu);
+                                                                      nullptr, n_launch, nullptr, vel, mu);
 }
 
 // Variants (eg_set_variant) and intermittent delivery; bounded to 72 registers for 3 CTAs per SM.
@@ -557,11 +596,11 @@ k_fused_pipe_general(float* __restrict__ x, const float* __restrict__ g, float* 
                      const uint8_t* __restrict__ snap, const uint8_t* __restrict__ valid, TileTable tt,
                      int P, int T, long long stride, float lr, double* __restrict__ partials,
                      long long* step_k, unsigned int* __restrict__ err, int n_launch, int variant,
-                     float* mailbox, const uint8_t* __restrict__ arrive, float* __restrict__ vel = nullptr,
-                     double mu = 0.0) {
+                     float* mailbox, const uint8_t* __restrict__ arrive, int* ticket,
+                     float* __restrict__ vel = nullptr, double mu = 0.0) {
     fused_pipe_body<TILE, STAGES, CONSUMERS, CARRY, ASYNC, false, MOM>(x, g, xhat, snap, valid, tt, P, T, stride,
                                                                       lr, partials, step_k, err, variant, mailbox,
-                                                                      arrive, n_launch, vel, mu);
+                                                                      arrive, n_launch, ticket, vel, mu);
 }
 
 // Self-test of the bounded wait: one warp waits on a barrier that nothing ever completes.  The

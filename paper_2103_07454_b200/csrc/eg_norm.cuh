@@ -70,6 +70,7 @@ struct DecideParams {
     double cap_beta;
     int t0, tn;               // tensors [t0, t0 + tn) are decided by this launch
     unsigned int* err;        // the context's error word (bounds-checked build)
+    int* ticket;              // tile counter of the walking fused kernel that follows: set to zero (nullptr: none)
 };
 
 // Intermittent delivery: which outstanding messages arrive in this step.
@@ -195,6 +196,7 @@ k_decide(const double* __restrict__ partials, const int* __restrict__ seg_begin,
     if (lane != 0) return;
     const long long k = *step_k;
     if (w == 0 && st.sparse_steps) st.sparse_steps[(k + 1) & 1] = 0;   // the next iteration's count starts at zero
+    if (w == 0 && dp.ticket) *dp.ticket = 0;
     const double cap = iteration_cap(dp, k);
     // next term of the sequence, once per iteration (the launch that holds tensor 0)
     if (w == 0 && dp.t0 == 0 && dp.cap_g) dp.cap_g[(k + 1) & 1] = __dmul_rn(dp.cap_g[k & 1], dp.cap_beta);

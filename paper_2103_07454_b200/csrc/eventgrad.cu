@@ -110,7 +110,8 @@ struct eg_ctx {
     bool timing = false;
     bool nvtx = false;      // EG_NVTX in the environment at eg_create: named ranges around the kernel groups
     int fused_waves = 1;    // EG_FUSED_WAVES in the environment at eg_create: CTAs of a walking pipelined kernel per resident slot
-    int fused_walk_max_p = 12;   // EG_FUSED_WALK_MAX_P: rings of up to this many replicas use the walking form
+    int* ticket = nullptr;       // device: tile counter of the walking fused kernel
+    int fused_walk_max_p = 24;   // EG_FUSED_WALK_MAX_P: rings of up to this many replicas use the walking form
     bool topk_pdl = true;   // EG_TOPK_PDL=0 in the environment at eg_create: no dependent launches inside the Top-K sequence
     bool no_pdl = false;    // EG_NO_PDL in the environment at eg_create: every kernel starts after its predecessor has ended
     std::vector<cudaEvent_t> ev_pool;      // pairs
@@ -497,7 +498,7 @@ eg_status eg_create(eg_ctx** out, int topology, int P, const int64_t* layer_nume
     EG_ALLOC(c->st.hist_len, S); EG_ALLOC(c->st.valid, S); EG_ALLOC(c->st.flag, S);
     EG_ALLOC(c->st.snap, S); EG_ALLOC(c->st.sparse, S); EG_ALLOC(c->st.norm, S);
     EG_ALLOC(c->st.thr_used, S); EG_ALLOC(c->st.events, S); EG_ALLOC(c->st.sent_norm, S);
-    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 2); EG_ALLOC(c->cap_g, 2);
+    EG_ALLOC(c->ctr, 1); EG_ALLOC(c->step_k, 1); EG_ALLOC(c->err, 2); EG_ALLOC(c->cap_g, 2); EG_ALLOC(c->ticket, 1);
     EG_ALLOC(c->outbox_count, S);
     if (c->topk.enabled) EG_ALLOC(c->st.sparse_steps, 2);
     EG_ALLOC(c->cons_partials, (size_t)c->tiles_fused.n_tiles + 1);
@@ -716,7 +717,8 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     // a2 + a6: decision, threshold update, counters
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
                     c->topk.enabled, c->degree, c->variant,
-                    c->cap_alpha > 0.0 ? c->cap_g : nullptr, c->cap_beta, t0, tcount, c->err};
+                    c->cap_alpha > 0.0 ? c->cap_g : nullptr, c->cap_beta, t0, tcount, c->err,
+                    c->ticket};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf_all : tn_all;
     if (small) {
@@ -789,13 +791,15 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         const uint8_t* valid = c->async ? c->recv_valid : c->st.valid;   // whom the neighbours have heard from
         // Rings of few replicas: a CTA of the pipelined kernels lives for P replicas only, and filling
         // and draining its ring of stages is a large part of that (8 replicas: 6.0 TB/s against
-        // 6.7 at 16 and 64).  There the kernels are launched as one CTA per resident slot, each
-        // walking the tiles b, b + grid, ... with its ring kept full across them (8 replicas:
-        // 6.5 TB/s).  From 16 replicas on one CTA per tile is faster (measured: 2 % at 16, 8 % at
-        // 64 replicas -- the hardware hands tiles out in order, CTAs that walk drift apart).
+        // 6.7 at 64).  There the kernels are launched as one CTA per resident slot, each walking
+        // from tile to tile with its ring kept full across them; after its first tile a CTA takes
+        // whatever tile a counter hands out next, so that tiles are begun in address order however
+        // the CTAs drift (measured against one CTA per tile on ResNet-18: 8 replicas 6.0 -> 6.7
+        // TB/s, 12 replicas -6 % time, 16 replicas -2.5 %, 24 equal, 32 and 48 replicas +1-2 %).
         const int pipe_stages = c->momentum ? kMomStages : kPipeStages;
         const bool walk = c->P >= pipe_stages && c->P <= c->fused_walk_max_p && !c->momentum;
         const int grid_pipe = walk ? std::min(grid_fused, c->sms * 3 * c->fused_waves) : grid_fused;
+        int* ticket = walk ? c->ticket : nullptr;
         float* vel = c->momentum ? c->vel : nullptr;
         float* mailbox = c->async ? c->mailbox : nullptr;
         const uint8_t* arrive = c->async ? c->arrive : nullptr;
@@ -820,12 +824,12 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                 k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, false, true, true>
                     <<<grid_fused, kPipeThreads, MomLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive, vel, c->mu);
+                    partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive, nullptr, vel, c->mu);
             else
                 k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, true>
                     <<<grid_pipe, kPipeThreads, PipeLayout::bytes(c->P, false, kPipeConsumers / 32), stream>>>(
                     params, grads, c->xhat, c->st.snap, valid, tf, c->P, c->T, c->stride, lr,
-                    partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive);
+                    partials_fused, step_k, c->err, grid_fused, c->variant, c->mailbox, c->arrive, ticket);
         } else if (c->fused_kind == EG_FUSED_REGISTER) {
             if (carry)
                 k_fused<kFusedVpt, true><<<grid_fused, kThreads, c->fused_smem, stream>>>(
@@ -850,11 +854,11 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                 if (carry)
                     k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, true, false, true>
                         <<<grid_fused, kPipeThreads, smem, stream>>>(EG_MOM_ARGS, c->variant, nullptr, nullptr,
-                                                                      c->vel, c->mu);
+                                                                      nullptr, c->vel, c->mu);
                 else
                     k_fused_pipe_general<kPipeTile, kMomStages, kPipeConsumers, false, false, true>
                         <<<grid_fused, kPipeThreads, smem, stream>>>(EG_MOM_ARGS, c->variant, nullptr, nullptr,
-                                                                      c->vel, c->mu);
+                                                                      nullptr, c->vel, c->mu);
             }
 #undef EG_MOM_ARGS
         } else {
@@ -866,17 +870,17 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                 // drains: it waits on the device before it reads anything that kernel writes
                 if (carry)
                     EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, true>,
-                                          dim3(grid_pipe), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
+                                          dim3(grid_pipe), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS, ticket));
                 else
                     EG_CUDA(c, launch_pdl(!c->timing && !c->no_pdl, k_fused_pipe<kPipeTile, kPipeStages, kPipeConsumers, false>,
-                                          dim3(grid_pipe), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS));
+                                          dim3(grid_pipe), dim3(kPipeThreads), smem, stream, EG_PIPE_ARGS, ticket));
             } else {
                 if (carry)
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, true, false>
-                        <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                        <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr, ticket);
                 else
                     k_fused_pipe_general<kPipeTile, kPipeStages, kPipeConsumers, false, false>
-                        <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr);
+                        <<<grid_pipe, kPipeThreads, smem, stream>>>(EG_PIPE_ARGS, c->variant, nullptr, nullptr, ticket);
             }
 #undef EG_PIPE_ARGS
         }
