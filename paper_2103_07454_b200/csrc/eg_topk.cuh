@@ -90,13 +90,16 @@ __device__ __forceinline__ unsigned int rank_key(float a, float b) {
 // digit 0: bits 30..20, digit 1: bits 19..10, digit 2: bits 9..0
 __device__ __forceinline__ int digit_bits(int digit) { return digit == 0 ? kDigitBits0 : kDigitBits1; }
 
-// One CTA (of kThreads threads): compact list of the flagged segments and of their tiles, in
-// segment order.  `main_list`: also forget the previous iteration's repeat requests.
+// One CTA (of up to kPlanThreads threads; the more, the shorter each thread's run of segments):
+// compact list of the flagged segments and of their tiles, in segment order.  `main_list`: also
+// forget the previous iteration's repeat requests.
+constexpr int kPlanThreads = 1024;
 __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restrict__ flagged,
                                           const int* __restrict__ seg_begin, const TopkState& tk,
                                           const WorkList& wl, int n_cta, bool main_list) {
-    __shared__ int s_cnt[kThreads], s_tiles[kThreads];
-    const int per = (S + kThreads - 1) / kThreads;
+    __shared__ int s_cnt[kPlanThreads], s_tiles[kPlanThreads];
+    const int nt = (int)blockDim.x;
+    const int per = (S + nt - 1) / nt;
     const int lo = threadIdx.x * per, hi = min(S, lo + per);
     int cnt = 0, tiles = 0;
     for (int s = lo; s < hi; ++s) {
@@ -108,7 +111,7 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
     s_tiles[threadIdx.x] = tiles;
     __syncthreads();
     // inclusive scan (Hillis-Steele) over the per-thread totals
-    for (int o = 1; o < kThreads; o <<= 1) {
+    for (int o = 1; o < nt; o <<= 1) {
         int a = 0, b = 0;
         if (threadIdx.x >= o) { a = s_cnt[threadIdx.x - o]; b = s_tiles[threadIdx.x - o]; }
         __syncthreads();
@@ -119,7 +122,7 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
     // chunk c holds the work tiles [c * chunk, (c + 1) * chunk): note for every c the list slot
     // its first tile falls into, so that no phase has to search for it
     n_cta *= kFine;
-    const int chunk = max(1, (s_tiles[kThreads - 1] + n_cta - 1) / n_cta);
+    const int chunk = max(1, (s_tiles[nt - 1] + n_cta - 1) / n_cta);
     if (threadIdx.x == 0) { wl.plan->chunk = chunk; wl.plan->n_chunks = n_cta; wl.plan->ticket = 0; }
     int q = s_cnt[threadIdx.x] - cnt, w = s_tiles[threadIdx.x] - tiles;
     for (int s = lo; s < hi; ++s)
@@ -132,7 +135,7 @@ __device__ __forceinline__ void topk_plan(int S, int T, const uint8_t* __restric
             ++q;
             w = w_end;
         }
-    if (threadIdx.x == kThreads - 1) {
+    if (threadIdx.x == nt - 1) {
         wl.plan->n_sparse = s_cnt[threadIdx.x];
         wl.plan->total_tiles = s_tiles[threadIdx.x];
         wl.sp_begin[s_cnt[threadIdx.x]] = s_tiles[threadIdx.x];
@@ -1157,7 +1160,7 @@ __device__ __forceinline__ bool topk_enter(const TopkArgs& a, int which) {
     pdl_wait();
     return which == 0 || *a.tk.redo_count != 0u;
 }
-__global__ void __launch_bounds__(kThreads) k_topk_plan(TopkArgs a, int which) {
+__global__ void __launch_bounds__(kPlanThreads) k_topk_plan(TopkArgs a, int which) {
     if (!topk_enter(a, which)) return;
     topk_plan(a.S, a.T, which ? a.tk.redo : a.sparse, a.tt.seg_begin, a.tk, a.tk.list[which], a.plan_ctas, which == 0);
 }

@@ -767,12 +767,12 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
             const dim3 one(1), tile_blocks(tile_grid), entry_blocks(tile_grid / kEntryShares), seg_blocks(seg_grid);
             const dim3 collect_blocks(tile_grid / kCollectShares);
             const dim3 threads(kThreads);
-            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, threads, 0, stream, ta, 0));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, dim3(kPlanThreads), 0, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, threads, 0, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_guess, seg_blocks, threads, 0, stream, ta));
             EG_CUDA(c, launch_pdl(pdl, k_topk_collect, collect_blocks, dim3(kCollectThreads), (size_t)CollectSmem::kBytes, stream, ta, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_resolve, seg_blocks, threads, 0, stream, ta, 0));
-            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, threads, 0, stream, ta, 1));
+            EG_CUDA(c, launch_pdl(pdl, k_topk_plan, one, dim3(kPlanThreads), 0, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_hist, tile_blocks, threads, 0, stream, ta, 1));
             EG_CUDA(c, launch_pdl(pdl, k_topk_pick, seg_blocks, threads, 0, stream, ta, 1, 0));
             EG_CUDA(c, launch_pdl(pdl, k_topk_collect, collect_blocks, dim3(kCollectThreads), (size_t)CollectSmem::kBytes, stream, ta, 1));
