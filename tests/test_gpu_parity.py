@@ -677,15 +677,20 @@ def test_steps_replayed_from_a_cuda_graph_match_direct_calls():
     assert all(np.array_equal(a, b) for a, b in zip(outs[0][2], outs[1][2]))
 
 
-@pytest.mark.parametrize("what", ["pipelined_carry_cap", "small_cap", "topk_cap", "two_pass"])
+@pytest.mark.parametrize("what", ["pipelined_carry_cap", "small_cap", "topk_cap", "two_pass", "walking_cap"])
 def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(what):
     """Replays of one captured eg_step against direct calls and the oracle, for the launch forms a
     step can take: decision + pipelined kernel started as dependent launches (carried norm), the
-    single-launch kernel, norm + decision + pipelined kernel, and the cooperative Top-K launch;
-    with a geometric bound on the thresholds, whose sequence advances on the device."""
+    single-launch kernel, norm + decision + pipelined kernel, the cooperative Top-K launch, and the
+    pipelined kernel walking more tiles than it has CTAs (their order comes from a counter that
+    every replay has to find at zero); with a geometric bound on the thresholds, whose sequence
+    advances on the device."""
     from oracle import eg_oracle as eo
     topk = (10, 100) if what == "topk_cap" else None
-    wl = W.synthetic(4, [5, 1000, 4097, 70000], steps=9, lr=0.1, grad_sigma=0.01, topk=topk)
+    if what == "walking_cap":       # 6 replicas, 680 tiles of 1024 elements for 444 CTAs
+        wl = W.synthetic(6, [5, 4097, 690000], steps=9, lr=0.1, grad_sigma=0.01)
+    else:
+        wl = W.synthetic(4, [5, 1000, 4097, 70000], steps=9, lr=0.1, grad_sigma=0.01, topk=topk)
     kernel = B.FUSED_AUTO if what == "small_cap" else B.FUSED_PIPELINED
     cap = None if what == "two_pass" else (4e-3, 0.6)
     carry = what != "two_pass"
@@ -731,7 +736,7 @@ def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(w
     assert outs[1][1] == o.stats()
     assert np.array_equal(outs[1][2][0], o.flags())
     if cap:
-        assert 0 < outs[1][1]["events"] < 9 * 4 * wl.T
+        assert 0 < outs[1][1]["events"] < 9 * wl.P * wl.T
     eg.close()
 
 
