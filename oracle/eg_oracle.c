@@ -53,7 +53,20 @@
  *    giving one): heavy-ball momentum (ego_set_momentum), off by default.  Every replica keeps
  *    a velocity v of its own, never communicated, v <- mu * v + g, and the gradient term of
  *    Eq. (dist_sgd_event) becomes gamma * v.  Pinned against torch.optim.SGD(momentum=mu), a
- *    closed-form geometric series, mu = 0 == the plain update, and the dense X W - gamma V.
+ *    closed-form geometric series, mu = 0 == the plain update, and the dense X W - gamma V;
+ *  - a second compression on top of the events (Section 7 says quantization can be applied on
+ *    top of event-triggered communication and gives no scheme): uniform b-bit quantisation of
+ *    the CHANGE since the last message (ego_set_quantisation), off by default.  On an event of
+ *    a tensor that has been sent before, with d[e] = x[e] - x_hat[e] (fp32) and L = 2^(b-1) - 1:
+ *    the scale is the power of two 2^E with the smallest integer E such that L 2^E >= max|d|,
+ *    the codes are q[e] = d[e] / 2^E rounded to the nearest integer (ties to even; |q| <= L by
+ *    the choice of E), the message is E and the n codes (4 + ceil(n b / 8) bytes), and sender and
+ *    receivers alike set x_hat[e] <- fp32(fp64(x_hat[e]) + q[e] 2^E).  What was not sent,
+ *    x - x_hat, stays in the difference and enters the next test and the next message.  The
+ *    first message of a tensor is sent in full (as with Top-K), a change that is not finite
+ *    too, and b = 32 means no quantisation.  Pinned against exact rational arithmetic on small
+ *    inputs, the round-trip bound |x - x_hat| <= 2^E / 2 (+ rounding), changes that lie on the
+ *    grid (reproduced exactly, E as constructed), b = 32 == dense, and the payload count.
  */
 #include <float.h>
 #include <math.h>
@@ -128,6 +141,10 @@ typedef struct ego_ctx {
     /* heavy-ball momentum (an extension to another training algorithm, Introduction) */
     float *vel;           /* [P][N] velocity of every replica, fp32 like the parameters; NULL: off */
     double mu;            /* momentum coefficient */
+    /* quantised messages (a second compression on top of the events, Section 7) */
+    int quant_bits;       /* 0: off; 2..16: bits per code */
+    int32_t *qexp;        /* [P*T] scale exponent E of the last step's quantised message */
+    uint8_t *quantised;   /* [P*T] the last step's message of this segment was quantised */
 } ego_ctx;
 
 void ego_destroy(ego_ctx *c) {
@@ -137,6 +154,7 @@ void ego_destroy(ego_ctx *c) {
     free(c->flag); free(c->norm); free(c->thr_used); free(c->out_idx); free(c->out_val);
     free(c->out_count); free(c->seg_events); free(c->seg_payload); free(c->sent_norm);
     free(c->mailbox); free(c->pending); free(c->recv_valid); free(c->vel);
+    free(c->qexp); free(c->quantised);
     free(c);
 }
 
@@ -257,6 +275,23 @@ int ego_set_momentum(ego_ctx *c, double mu) {
 }
 float *ego_velocity(ego_ctx *c) { return c->vel; }
 
+/* bits per code of a quantised message: 2..16; 0 or 32: messages in full precision.  Not
+ * together with Top-K messages (one compression at a time). */
+int ego_set_quantisation(ego_ctx *c, int bits) {
+    if (bits == 32) bits = 0;
+    if (bits != 0 && (bits < 2 || bits > 16)) return -1;
+    if (bits != 0 && c->topk) return -1;
+    if (bits != 0 && !c->qexp) {
+        c->qexp = (int32_t *)calloc((size_t)c->P * c->T, sizeof(int32_t));
+        c->quantised = (uint8_t *)calloc((size_t)c->P * c->T, 1);
+        if (!c->qexp || !c->quantised) return -1;
+    }
+    c->quant_bits = bits;
+    return 0;
+}
+const int32_t *ego_quant_exponents(const ego_ctx *c) { return c->qexp; }
+const uint8_t *ego_quantised(const ego_ctx *c) { return c->quantised; }
+
 void ego_set_threads(ego_ctx *c, int threads) { c->threads = threads < 1 ? 1 : threads; }
 
 int ego_threads_available(void) {
@@ -365,7 +400,35 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
 
     /* 4b: the message */
     uint64_t payload;
-    if (!c->topk || !c->valid[s]) {
+    int quantise = c->quant_bits != 0 && c->valid[s];
+    float dmax = 0.0f;
+    if (quantise) { /* the largest change; a change that is not finite is sent in full */
+        for (int64_t e = 0; e < n; ++e) {
+            const float a = fabsf(xs[e] - hs[e]);
+            if (!(a <= FLT_MAX)) quantise = 0;
+            if (a > dmax) dmax = a;
+        }
+    }
+    if (c->qexp) { c->qexp[s] = 0; c->quantised[s] = (uint8_t)quantise; }
+    if (quantise) {
+        const int b = c->quant_bits;
+        const double L = (double)((1 << (b - 1)) - 1);
+        int E = 0;
+        if (dmax > 0.0f) { /* the smallest E with L 2^E >= max|d| */
+            E = -400;
+            while (ldexp(L, E) < (double)dmax) ++E;
+        }
+        for (int64_t e = 0; e < n; ++e) {
+            const float d32 = xs[e] - hs[e];
+            double q = rint((double)d32 * ldexp(1.0, -E)); /* exact scaling, ties to even */
+            if (q > L) q = L;
+            if (q < -L) q = -L;
+            const double r = (double)hs[e] + q * ldexp(1.0, E);
+            hs[e] = (float)r;
+        }
+        c->qexp[s] = E;
+        payload = 4u + ((uint64_t)n * (uint64_t)b + 7u) / 8u;
+    } else if (!c->topk || !c->valid[s]) {
         for (int64_t e = 0; e < n; ++e) hs[e] = xs[e];
         payload = 4u * (uint64_t)n;
     } else {

@@ -51,6 +51,11 @@ def _load():
         lib.ego_set_momentum.argtypes = [C.c_void_p, C.c_double]
         lib.ego_velocity.restype = C.c_void_p
         lib.ego_velocity.argtypes = [C.c_void_p]
+        lib.ego_set_quantisation.restype = C.c_int
+        lib.ego_set_quantisation.argtypes = [C.c_void_p, C.c_int]
+        for name in ("ego_quant_exponents", "ego_quantised"):
+            getattr(lib, name).restype = C.c_void_p
+            getattr(lib, name).argtypes = [C.c_void_p]
         lib.ego_threads_available.restype = C.c_int
         lib.ego_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
         lib.ego_step_masked.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
@@ -103,7 +108,8 @@ class Oracle:
                  delta_fixed: float = 0.0, force_first_event: bool = True,
                  topk: Optional[tuple] = None, threads: int = 1,
                  own_last_sent: bool = False, change_of_norm: bool = False, hops: int = 1,
-                 threshold_cap: Optional[tuple] = None, momentum: Optional[float] = None):
+                 threshold_cap: Optional[tuple] = None, momentum: Optional[float] = None,
+                 quant_bits: Optional[int] = None):
         lib = _load()
         self._lib = lib
         self.P, self.T = int(P), len(numel)
@@ -124,6 +130,8 @@ class Oracle:
             lib.ego_set_threshold_cap(self._h, float(threshold_cap[0]), float(threshold_cap[1]))
         if momentum is not None and lib.ego_set_momentum(self._h, float(momentum)):
             raise ValueError("momentum must be in [0, 1)")
+        if quant_bits is not None and lib.ego_set_quantisation(self._h, int(quant_bits)):
+            raise ValueError("quantisation: 2..16 bits (or 32 for none), and not together with Top-K")
         self.S = self.P * self.T
         self.history_len = int(history_len)
 
@@ -236,6 +244,21 @@ class Oracle:
         if not p:
             return None
         return _view(p, np.float32, self.P * self.N).reshape(self.P, self.N).copy()
+
+    def quant_exponents(self) -> Optional[np.ndarray]:
+        """Scale exponents E of the last step's quantised messages, ``[P, T]`` int32 (None when
+        quantisation is off); only meaningful where ``quantised()`` is set."""
+        p = self._lib.ego_quant_exponents(self._h)
+        if not p:
+            return None
+        return _view(p, np.int32, self.S).reshape(self.P, self.T).copy()
+
+    def quantised(self) -> Optional[np.ndarray]:
+        """Which (replica, tensor) pairs sent a quantised message in the last step."""
+        p = self._lib.ego_quantised(self._h)
+        if not p:
+            return None
+        return _view(p, np.uint8, self.S).reshape(self.P, self.T).copy()
 
     def topk_count(self, t: int) -> int:
         return int(self._lib.ego_topk_count(self._h, t))

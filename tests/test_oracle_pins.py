@@ -687,6 +687,138 @@ def test_momentum_reset_clears_the_velocity_and_range_is_checked():
 # ---------------------------------------------------------------------------------------
 # after training: averaged model (last line of Algorithms A and B)
 # ---------------------------------------------------------------------------------------
+# ---------------------------------------------------------------------------------------
+# Quantised messages (Section 7: quantization can be applied on top of the events; the scheme is
+# this build's reading, stated in the oracle's header)
+# ---------------------------------------------------------------------------------------
+def _exact_quantised_message(x_row, h_row, bits):
+    """The reading restated with exact rational arithmetic: (E, new x_hat) of one tensor."""
+    from fractions import Fraction
+    L = (1 << (bits - 1)) - 1
+    d = (x_row - h_row).astype(np.float32)                 # the fp32 differences the method ranks
+    dmax = max((abs(Fraction(float(v))) for v in d), default=Fraction(0))
+    E = 0
+    if dmax > 0:
+        E = -400
+        while L * Fraction(2) ** E < dmax:
+            E += 1
+    out = np.empty_like(h_row)
+    for e in range(len(d)):
+        r = Fraction(float(d[e])) / Fraction(2) ** E
+        lo = r.numerator // r.denominator                  # floor
+        frac = r - lo
+        q = lo + (1 if frac > Fraction(1, 2) or (frac == Fraction(1, 2) and lo % 2 == 1) else 0)   # ties to even
+        assert abs(q) <= L
+        exact = Fraction(float(h_row[e])) + q * Fraction(2) ** E
+        out[e] = np.float32(float(exact))                  # to fp64 (correctly rounded), then to fp32
+    return E, out
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8, 16])
+def test_quantised_messages_against_exact_rational_arithmetic(bits):
+    wl = small(P=4, numel=(1, 9, 64, 257), steps=6, lr=0.1, grad_sigma=0.02)
+    o = eo.from_workload(wl, mode=eo.FIXED, delta_fixed=0.0, quant_bits=bits)      # every tensor sends every step
+    x = W.distinct_init_params(wl).numpy().copy()
+    off = np.concatenate([[0], np.cumsum(wl.numel)])
+    L = (1 << (bits - 1)) - 1
+    bytes_before = 0
+    for k in range(wl.steps):
+        h_before = o.xhat().copy()
+        x_before = x.copy()
+        o.step(x, wl.grads(k).numpy(), wl.lr)
+        h_after, qe, qd = o.xhat(), o.quant_exponents(), o.quantised()
+        payload = 0
+        for i in range(wl.P):
+            for t in range(wl.T):
+                a, b = off[t], off[t + 1]
+                if k == 0:
+                    # the first message of a tensor goes out in full
+                    assert qd[i, t] == 0 and np.array_equal(h_after[i, a:b], x_before[i, a:b])
+                    payload += 4 * wl.numel[t]
+                    continue
+                assert qd[i, t] == 1
+                E, want = _exact_quantised_message(x_before[i, a:b], h_before[i, a:b], bits)
+                assert qe[i, t] == E
+                assert np.array_equal(h_after[i, a:b], want)
+                # round trip: what the receivers hold is within half a step of x (plus the two
+                # roundings to fp32, of the difference and of the sum)
+                err = np.abs(x_before[i, a:b].astype(np.float64) - h_after[i, a:b])
+                slack = ulp32(x_before[i, a:b] - h_before[i, a:b]) / 2 + ulp32(h_after[i, a:b]) / 2
+                assert np.all(err <= 2.0 ** E / 2 + slack)
+                # E is the smallest exponent whose grid reaches the largest change
+                dmax = float(np.abs((x_before[i, a:b] - h_before[i, a:b]).astype(np.float32)).max())
+                assert L * 2.0 ** E >= dmax and (dmax == 0 or L * 2.0 ** (E - 1) < dmax)
+                payload += 4 + (wl.numel[t] * bits + 7) // 8
+        deg = 2
+        assert o.stats()["bytes"] - bytes_before == deg * payload
+        bytes_before = o.stats()["bytes"]
+
+
+def test_quantised_changes_on_the_grid_are_reproduced_exactly():
+    """Changes that are integer multiples of 2^e with the largest equal to L 2^e: E = e, every code
+    is the multiple itself, and the receivers end up with x exactly."""
+    bits, e = 6, -7
+    L = (1 << (bits - 1)) - 1
+    n = 50
+    wl = W.synthetic(3, [n], steps=2, lr=0.0, grad_sigma=0.0)
+    o = eo.from_workload(wl, mode=eo.FIXED, delta_fixed=0.0, quant_bits=bits)
+    rng = np.random.default_rng(5)
+    x = (rng.integers(-1000, 1000, size=(3, n)) * 2.0 ** -4).astype(np.float32)
+    g = np.zeros_like(x)
+    o.step(x, g, 0.0)                                   # first messages, in full: x_hat == x
+    sent = o.xhat().copy()
+    # lr = 0 and identical mailboxes: the average moves x; put it back on a chosen grid
+    mult = rng.integers(-L, L + 1, size=(3, n))
+    mult[:, 0] = L                                      # the largest change sits on the end of the grid
+    x[:] = (sent.astype(np.float64) + mult * 2.0 ** e).astype(np.float32)
+    assert np.array_equal((x - sent).astype(np.float32), (mult * 2.0 ** e).astype(np.float32))   # representable
+    x_sent = x.copy()
+    o.step(x, g, 0.0)
+    assert np.all(o.quantised() == 1) and np.all(o.quant_exponents() == e)
+    assert np.array_equal(o.xhat(), x_sent)
+
+
+def test_thirty_two_bits_and_the_first_message_are_full_precision():
+    wl = small(P=5, steps=8, lr=0.1, grad_sigma=0.01)
+    a, b = eo.from_workload(wl), eo.from_workload(wl, quant_bits=32)
+    xa = W.distinct_init_params(wl).numpy().copy()
+    xb = xa.copy()
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        a.step(xa, g, wl.lr)
+        b.step(xb, g, wl.lr)
+        assert np.array_equal(xa, xb) and np.array_equal(a.xhat(), b.xhat())
+    assert a.stats() == b.stats() and a.stats()["events"] > wl.P * wl.T
+    assert b.quantised() is None
+    with pytest.raises(ValueError):
+        eo.from_workload(wl, quant_bits=1)
+    with pytest.raises(ValueError):
+        eo.from_workload(wl, quant_bits=17)
+    with pytest.raises(ValueError):
+        eo.Oracle(3, [10, 20], topk=(1, 10), quant_bits=8)      # one compression at a time
+
+
+def test_quantised_run_keeps_the_error_bound_and_saves_bytes():
+    """With the adaptive threshold the trigger still bounds what the neighbours are missing:
+    after every step ||x_before - x_hat|| of a tensor that did not fire is below the threshold it
+    was tested against (Section 5), quantised or not -- the un-sent remainder is part of the tested
+    norm -- and the run sends fewer bytes than the same run in full precision."""
+    wl = small(P=4, numel=(40, 300, 1000), steps=30, lr=0.1, grad_sigma=0.02)
+    full, q8 = eo.from_workload(wl), eo.from_workload(wl, quant_bits=8)
+    xf = W.distinct_init_params(wl).numpy().copy()
+    xq = xf.copy()
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        full.step(xf, g, wl.lr)
+        before = xq.copy()
+        q8.step(xq, g, wl.lr)
+        fl, nr, th = q8.flags(), q8.norms(), q8.thresholds_used()
+        assert np.all(nr[fl == 0] < th[fl == 0])
+        assert np.all(np.isfinite(before)) and np.all(np.isfinite(q8.xhat()))
+    assert 0 < q8.stats()["bytes"] < full.stats()["bytes"]
+    assert np.any(q8.quantised() == 1) or q8.stats()["events"] > wl.P * wl.T
+
+
 def test_average_model_and_consensus_distance():
     wl = small(P=5)
     o = eo.from_workload(wl)
