@@ -188,6 +188,30 @@ eg_status eg_set_threshold_cap(eg_ctx* ctx, double alpha, double beta);
  * buffer exists; eg_read_velocity / eg_write_velocity copy them to / from a host buffer of
  * P*replica_stride floats (both synchronise; EG_ERR_STATE before the first enabling call). */
 eg_status eg_set_momentum(eg_ctx* ctx, int enabled, double mu);
+
+/* Quantised messages: a second compression on top of the events.  Section 7 says that
+ * quantization can be applied on top of event-triggered communication and gives no scheme; the
+ * one built here quantises the CHANGE since the last message.  On an event of a tensor that has
+ * been sent before, with d[e] = x[e] - x_hat[e] (one fp32 subtraction) and L = 2^(bits-1) - 1:
+ *   scale    2^E, E the smallest integer with L * 2^E >= max_e |d[e]|   (E = 0 if all d are 0)
+ *   codes    q[e] = d[e] / 2^E rounded to the nearest integer, ties to even (so |q[e]| <= L)
+ *   message  E and the n codes: 4 + ceil(n * bits / 8) bytes per neighbour
+ *   receipt  x_hat[e] <- fp32( fp64(x_hat[e]) + q[e] * 2^E ), at the sender too, so that x_hat
+ *            stays what the receivers hold.
+ * What was not sent, x - x_hat, remains part of the difference: it enters the next trigger test
+ * and the next message (nothing is dropped for good).  The first message of a tensor is sent in
+ * full precision (x_hat <- x, 4 n bytes), as with Top-K messages; so is a message whose change
+ * holds an infinity or a NaN.  bits: 2..16; 0 or 32 switches quantisation off.  Not available
+ * in a context created with Top-K messages (one compression at a time: EG_ERR_STATE), and only
+ * before the first step or after eg_reset (EG_ERR_STATE otherwise).  Works with every other
+ * option: the messages are delivered into x_hat by kernels of their own before the averaging
+ * kernel runs, the way Top-K messages are.
+ * eg_last_quantised copies, for the last step, which (replica, tensor) pairs sent a quantised
+ * message (1; 2: the change was not finite and the message went out in full; 0: none) and the
+ * exponents E of those messages to host arrays of P*T entries; EG_ERR_STATE when quantisation
+ * was never switched on.  Synchronises. */
+eg_status eg_set_quantisation(eg_ctx* ctx, int bits);
+eg_status eg_last_quantised(eg_ctx* ctx, uint8_t* quantised_host, int32_t* exponents_host);
 eg_status eg_read_velocity(eg_ctx* ctx, float* velocity_host);
 eg_status eg_write_velocity(eg_ctx* ctx, const float* velocity_host);
 

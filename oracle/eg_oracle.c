@@ -382,6 +382,7 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
     c->flag[s] = (uint8_t)fire;
     c->out_count[s] = 0;
     c->seg_payload[s] = 0;
+    if (c->qexp) { c->qexp[s] = 0; c->quantised[s] = 0; }
     if (!fire) return;
 
     /* 4a: new threshold from the slope between this event and the previous one */

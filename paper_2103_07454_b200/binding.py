@@ -31,6 +31,8 @@ EXPORTS = [
     "eg_selftest_wait_timeout", "eg_set_momentum", "eg_read_velocity", "eg_write_velocity",
     "eg_debug_fail_allocation", "eg_status_of_error_word", "eg_debug_build",
     "eg_topk_repeat_count",
+    "eg_set_quantisation",
+    "eg_last_quantised",
 ]
 STATIC_MAX_TENSORS = 192
 STATIC_MAX_PARTIALS = 524288
@@ -110,6 +112,8 @@ def load_library() -> C.CDLL:
     lib.eg_status_of_error_word.argtypes = [C.c_uint]
     lib.eg_debug_build.argtypes = []
     lib.eg_topk_repeat_count.argtypes = [vp, u64p]
+    lib.eg_set_quantisation.argtypes = [vp, C.c_int]
+    lib.eg_last_quantised.argtypes = [vp, vp, vp]
     lib.eg_last_cuda_error.argtypes = [vp]
     lib.eg_last_launch_count.argtypes = [vp]
     _lib = lib
@@ -275,6 +279,18 @@ class EventGrad:
         n = C.c_uint64()
         _check(self._lib, self._lib.eg_topk_repeat_count(self._h, C.byref(n)), self._h, "eg_topk_repeat_count")
         return int(n.value)
+
+    def set_quantisation(self, bits: int):
+        """Quantised messages of ``bits`` bits per element (2..16; 0 or 32: full precision)."""
+        _check(self._lib, self._lib.eg_set_quantisation(self._h, int(bits)), self._h, "eg_set_quantisation")
+
+    def last_quantised(self):
+        """(which, exponents) of the last step, ``[P, T]`` uint8 / int32 host arrays."""
+        q = np.zeros((self.P, self.T), dtype=np.uint8)
+        e = np.zeros((self.P, self.T), dtype=np.int32)
+        _check(self._lib, self._lib.eg_last_quantised(self._h, q.ctypes.data, e.ctypes.data), self._h,
+               "eg_last_quantised")
+        return q, e
 
     def last_outbox(self, i: int, t: int):
         cap = max(1, self.topk_count(t))

@@ -72,6 +72,8 @@ struct SegState {
     unsigned long long* events;  // events so far
     double* sent_norm;           // ||x|| at the last event (change-of-norm variant)
     unsigned int* sparse_steps;  // [2] Top-K messages decided in the iteration of this parity (nullptr: dense)
+    uint8_t* quant;              // event whose message is quantised and delivered into x_hat by the
+                                 // quantising kernels before the averaging kernel runs (nullptr: never)
 };
 
 // Variants of the method that the paper's text also admits (kernel argument `variant`).

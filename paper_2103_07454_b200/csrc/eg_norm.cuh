@@ -71,6 +71,7 @@ struct DecideParams {
     int t0, tn;               // tensors [t0, t0 + tn) are decided by this launch
     unsigned int* err;        // the context's error word (bounds-checked build)
     int* ticket;              // tile counter of the walking fused kernel that follows: set to zero (nullptr: none)
+    int quant_bits;           // bits per code of a quantised message (0: messages in full precision)
 };
 
 // Intermittent delivery: which outstanding messages arrive in this step.
@@ -120,7 +121,7 @@ decide_segment(double acc, long long s, int t, long long k, double cap, const De
     st.thr_used[s] = thr;
     const bool fire = (dp.force_first && k == 0) || (d >= thr);
     const bool was_valid = st.valid[s] != 0;
-    uint8_t snap = 0, sparse = 0;
+    uint8_t snap = 0, sparse = 0, quant = 0;
     int out_count = 0;
     if (fire) {
         if (dp.mode == 0 && was_valid) {
@@ -140,7 +141,11 @@ decide_segment(double acc, long long s, int t, long long k, double cap, const De
             st.delta[s] = __dmul_rn(dp.horizon, __ddiv_rn(sum, (double)n));
         }
         unsigned long long payload;
-        if (!dp.topk || !was_valid) {   // the first message of a tensor is always dense
+        if (dp.quant_bits && was_valid) {
+            // b-bit codes of the change since the last message and the exponent of their scale
+            quant = 1;
+            payload = 4ull + ((unsigned long long)numel[t] * (unsigned long long)dp.quant_bits + 7ull) / 8ull;
+        } else if (!dp.topk || !was_valid) {   // the first message of a tensor is always dense
             snap = 1;
             payload = 4ull * (unsigned long long)numel[t];
         } else {
@@ -172,6 +177,7 @@ decide_segment(double acc, long long s, int t, long long k, double cap, const De
     st.flag[s] = fire ? 1 : 0;
     st.snap[s] = snap;
     st.sparse[s] = sparse;
+    if (st.quant) st.quant[s] = quant;
     if (outbox_count) outbox_count[s] = out_count;
 }
 

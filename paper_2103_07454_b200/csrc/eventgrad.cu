@@ -16,6 +16,7 @@
 #include "eg_fused_hops.cuh"
 #include "eg_fused_pipe.cuh"
 #include "eg_norm.cuh"
+#include "eg_quant.cuh"
 #include "eg_step_small.cuh"
 #include "eg_topk.cuh"
 
@@ -29,7 +30,7 @@ using PipeLayout = PipeSmem<kPipeTile, kPipeStages>;
 constexpr int kMomStages = 4;                         // four tiles per stage: same footprint as 5 x 3
 using MomLayout = PipeSmem<kPipeTile, kMomStages, 4, false>;
 static_assert(kFusedTile == kPipeTile, "both fused kernels share one tile table");
-constexpr uint64_t kStateMagic = 0x4547535441544533ull;  // "EGSTATE3"
+constexpr uint64_t kStateMagic = 0x4547535441544534ull;  // "EGSTATE4"
 
 struct HostTiles {
     std::vector<int> tensor, length, seg_begin;
@@ -111,6 +112,10 @@ struct eg_ctx {
     bool nvtx = false;      // EG_NVTX in the environment at eg_create: named ranges around the kernel groups
     int fused_waves = 1;    // EG_FUSED_WAVES in the environment at eg_create: CTAs of a walking pipelined kernel per resident slot
     int* ticket = nullptr;       // device: tile counter of the walking fused kernel
+    // quantised messages (eg_set_quantisation)
+    int quant_bits = 0;                  // 0: messages in full precision
+    float* quant_tile_max = nullptr;     // [P][norm tiles]
+    int* quant_exp = nullptr;            // [P*T] scale exponent of the last quantised message
     int fused_walk_max_p = 24;   // EG_FUSED_WALK_MAX_P: rings of up to this many replicas use the walking form
     bool topk_pdl = true;   // EG_TOPK_PDL=0 in the environment at eg_create: no dependent launches inside the Top-K sequence
     bool no_pdl = false;    // EG_NO_PDL in the environment at eg_create: every kernel starts after its predecessor has ended
@@ -209,6 +214,10 @@ eg_status init_state(eg_ctx* c) {
     EG_CUDA(c, cudaMemset(c->st.flag, 0, S));
     EG_CUDA(c, cudaMemset(c->st.snap, 0, S));
     EG_CUDA(c, cudaMemset(c->st.sparse, 0, S));
+    if (c->st.quant) {
+        EG_CUDA(c, cudaMemset(c->st.quant, 0, S));
+        EG_CUDA(c, cudaMemset(c->quant_exp, 0, S * sizeof(int)));
+    }
     EG_CUDA(c, cudaMemset(c->st.norm, 0, S * sizeof(double)));
     EG_CUDA(c, cudaMemset(c->st.events, 0, S * sizeof(unsigned long long)));
     EG_CUDA(c, cudaMemset(c->st.sent_norm, 0, S * sizeof(double)));
@@ -700,7 +709,8 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     double* partials_norm = c->partials_norm + nb;
     double* partials_fused = c->partials_fused + fb;
     long long* step_k = c->range_last ? c->step_k : nullptr;
-    if (!whole && (c->topk.enabled || c->async || c->hops > 1 || c->fused_kind == EG_FUSED_REGISTER))
+    if (!whole && (c->topk.enabled || c->async || c->hops > 1 || c->fused_kind == EG_FUSED_REGISTER ||
+                   c->quant_bits != 0))
         return EG_ERR_STATE;
 
     // a1: || x - x_hat || partial sums, unless the previous step carried them over
@@ -713,12 +723,12 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
         ++launches;
     }
     const bool small = c->fused_kind == EG_FUSED_AUTO && c->small_eligible && whole && !c->async &&
-                       c->variant == 0 && !c->momentum;
+                       c->variant == 0 && !c->momentum && c->quant_bits == 0;
     // a2 + a6: decision, threshold update, counters
     DecideParams dp{c->P, c->T, c->H, c->thr.mode, c->thr.horizon, c->thr.force_first_event,
                     c->topk.enabled, c->degree, c->variant,
                     c->cap_alpha > 0.0 ? c->cap_g : nullptr, c->cap_beta, t0, tcount, c->err,
-                    c->ticket};
+                    c->ticket, c->quant_bits};
     const double* partials = use_carried ? c->partials_fused : c->partials_norm;
     const TileTable& tp = use_carried ? tf_all : tn_all;
     if (small) {
@@ -746,6 +756,17 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
                               DeliveryState{deliver_dev, c->pending, c->recv_valid, c->arrive, c->arrivals,
                                             c->async ? 1 : 0}));
         ++launches;
+    }
+    // quantised messages: delivered into x_hat before the averaging kernel, like Top-K messages
+    if (c->quant_bits != 0 && !small) {
+        TimedSection ts(c, stream, EG_KERNEL_TOPK);
+        QuantArgs qa{params, c->xhat, tn_all, c->P, c->T, c->stride, c->st.quant, c->quant_tile_max, c->quant_exp,
+                     c->d_numel, c->quant_bits, c->degree, c->ctr};
+        const int walk_grid = c->sms * 8;
+        k_quant_max<<<walk_grid, kThreads, 0, stream>>>(qa);
+        k_quant_scale<<<(int)((S + kWarps - 1) / kWarps), kThreads, 0, stream>>>(qa);
+        k_quant_apply<<<walk_grid, kThreads, 0, stream>>>(qa);
+        launches += 3;
     }
     // a4: Top-K select / pack / deliver for the segments that send a sparse message
     if (c->topk.enabled && !small) {
@@ -1182,6 +1203,38 @@ eg_status eg_kernel_times(eg_ctx* c, double* ms_host, uint64_t* sections_host) {
     return EG_OK;
 }
 
+eg_status eg_set_quantisation(eg_ctx* c, int bits) {
+    if (!c) return EG_ERR_INVALID;
+    if (bits == 32) bits = 0;
+    if (bits != 0 && (bits < 2 || bits > 16)) return EG_ERR_INVALID;
+    if (c->stepped) return EG_ERR_STATE;            // only before the first step (or after eg_reset)
+    if (bits != 0 && c->topk.enabled) return EG_ERR_STATE;   // one compression at a time
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return EG_ERR_CUDA;
+    if (bits != 0 && !c->st.quant) {
+        const size_t S = (size_t)c->P * c->T;
+        eg_status s;
+        if ((s = dev_alloc(c, &c->st.quant, S)) != EG_OK) return s;
+        if ((s = dev_alloc(c, &c->quant_exp, S)) != EG_OK) return s;
+        if ((s = dev_alloc(c, &c->quant_tile_max, (size_t)c->P * c->tiles_norm.n_tiles)) != EG_OK) return s;
+    }
+    c->quant_bits = bits;
+    c->carried_valid = false;
+    return EG_OK;
+}
+
+eg_status eg_last_quantised(eg_ctx* c, uint8_t* quantised_host, int32_t* exponents_host) {
+    if (!c || !quantised_host || !exponents_host) return EG_ERR_INVALID;
+    if (!c->st.quant) return EG_ERR_STATE;
+    DeviceGuard guard(c->device);
+    eg_status s = sync_and_check(c);
+    if (s != EG_OK) return s;
+    const size_t S = (size_t)c->P * c->T;
+    EG_CUDA(c, cudaMemcpy(quantised_host, c->st.quant, S, cudaMemcpyDeviceToHost));
+    EG_CUDA(c, cudaMemcpy(exponents_host, c->quant_exp, S * sizeof(int), cudaMemcpyDeviceToHost));
+    return EG_OK;
+}
+
 eg_status eg_set_momentum(eg_ctx* c, int enabled, double mu) {
     if (!c) return EG_ERR_INVALID;
     if (!enabled) { c->momentum = false; c->carried_valid = false; return EG_OK; }
@@ -1363,6 +1416,7 @@ struct StateHeader {
     int64_t hops, mode, force_first, delivery, velocity;
     double horizon, delta_init, delta_fixed, cap_alpha, cap_beta, mu;
     uint64_t arrivals;
+    int64_t quant_bits;
 };
 
 static size_t state_bytes(const eg_ctx* c) {
@@ -1383,6 +1437,7 @@ static StateHeader state_header(const eg_ctx* c) {
     h.delivery = c->async ? 1 : 0; h.velocity = c->vel ? 1 : 0;
     h.horizon = c->thr.horizon; h.delta_init = c->thr.delta_init; h.delta_fixed = c->thr.delta_fixed;
     h.cap_alpha = c->cap_alpha; h.cap_beta = c->cap_beta; h.mu = c->momentum ? c->mu : 0.0;
+    h.quant_bits = c->quant_bits;
     return h;
 }
 
@@ -1441,7 +1496,8 @@ eg_status eg_import_state(eg_ctx* c, const void* host_buf, size_t bytes) {
         (h.topk && (h.k_num != w.k_num || h.k_den != w.k_den)) || h.hops != w.hops || h.mode != w.mode ||
         h.force_first != w.force_first || h.delivery != w.delivery || h.velocity != w.velocity ||
         !same(h.horizon, w.horizon) || !same(h.delta_init, w.delta_init) || !same(h.delta_fixed, w.delta_fixed) ||
-        !same(h.cap_alpha, w.cap_alpha) || !same(h.cap_beta, w.cap_beta) || !same(h.mu, w.mu) || h.step < 0)
+        !same(h.cap_alpha, w.cap_alpha) || !same(h.cap_beta, w.cap_beta) || !same(h.mu, w.mu) ||
+        h.quant_bits != w.quant_bits || h.step < 0)
         return EG_ERR_INVALID;
     DeviceGuard guard(c->device);
     EG_CUDA(c, cudaStreamSynchronize(c->last_stream));

@@ -49,6 +49,7 @@ class Report:
     params_bit_exact: bool = True
     launches: int = 0
     topk_repeats: int = 0
+    quantised_checked: int = 0
     seconds: dict = field(default_factory=lambda: {"inputs": 0.0, "oracle": 0.0, "compare": 0.0})
 
 
@@ -77,8 +78,8 @@ def _counters_from_events(events: np.ndarray, numel, k_t, degree: int) -> dict:
 
 # Checkpoint header, 8-byte words: magic, P, T, H, stride, N, topk, k_num, k_den, variant, step,
 # 3 counters, hops, mode, force_first, delivery, velocity, 6 doubles (horizon, delta_init,
-# delta_fixed, bound alpha / beta, mu), arrivals.
-HEADER_WORDS = 26
+# delta_fixed, bound alpha / beta, mu), arrivals, bits of a quantised message.
+HEADER_WORDS = 27
 
 
 def resynchronise(eg: B.EventGrad, o: eo.Oracle, x_dev: torch.Tensor, x_host: np.ndarray, delivery: bool = False):
@@ -149,6 +150,7 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
     ekw.pop("own_last_sent", None)
     ekw.pop("change_of_norm", None)
     ekw.pop("momentum", None)
+    ekw.pop("quant_bits", None)
     for key in ("mode", "delta_fixed", "force_first_event", "horizon", "history_len", "delta_init"):
         if key in okw and key not in ekw:
             ekw[key] = okw[key]
@@ -163,6 +165,8 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
         eg.set_threshold_cap(*cap)
     if okw.get("momentum") is not None:
         eg.set_momentum(okw["momentum"])
+    if okw.get("quant_bits") is not None:
+        eg.set_quantisation(okw["quant_bits"])
 
     x0 = (W.distinct_init_params(wl, gen_device) if init == "distinct" else wl.init_params(gen_device)).to(dev)
     x_dev = eg.to_layout(x0)
@@ -313,6 +317,14 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             assert np.array_equal(xh_g.view(np.uint32), o.xhat().view(np.uint32)), f"mailboxes, step {k}"
         else:
             assert host_sub(eg.mailboxes(out=box_pin).numpy(), o.xhat()), f"mailboxes, step {k}"
+        if okw.get("quant_bits") not in (None, 0, 32):
+            q_g, e_g = eg.last_quantised()
+            q_o, e_o = o.quantised(), o.quant_exponents()
+            # (the library tells a message that went out in full because its change was not finite
+            #  from one that was never a candidate; the oracle marks both 0)
+            assert np.array_equal(q_g[:, tensors] == 1, q_o == 1), f"which messages are quantised, step {k}"
+            assert np.array_equal(e_g[:, tensors][q_o == 1], e_o[q_o == 1]), f"scale exponents, step {k}"
+            rep.quantised_checked += int((q_o == 1).sum())
         if okw.get("momentum") is not None:
             v_g = gpu_sub(eg.velocity().to(dev))
             assert np.array_equal(v_g.view(np.uint32), o.velocity().view(np.uint32)), f"velocity, step {k}"

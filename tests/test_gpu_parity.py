@@ -740,6 +740,131 @@ def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(w
     eg.close()
 
 
+# ---------------------------------------------------------------------------------------
+# quantised messages (Section 7: quantization on top of the events; the reading is in the header)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("carry", [False, True])
+@pytest.mark.parametrize("bits", [2, 5, 8, 16])
+def test_quantised_messages_ragged(bits, carry):
+    """Every element of x_hat after a quantised message, the scale exponents, which messages were
+    quantised and the byte counter equal the oracle's; ragged sizes over several tiles."""
+    wl = W.synthetic(5, RAGGED, steps=10, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=carry, oracle_kw=dict(quant_bits=bits))
+    assert rep.params_bit_exact and rep.quantised_checked > 20
+    # every tensor sends every step: nothing but quantised messages after the first
+    rep = lockstep(wl, init="distinct", carry=carry, steps=5,
+                   oracle_kw=dict(quant_bits=bits, mode=1, delta_fixed=0.0))
+    assert rep.params_bit_exact and rep.quantised_checked == 4 * wl.P * wl.T
+
+
+def test_quantised_messages_large_tensor_and_many_replicas():
+    wl = W.synthetic(7, [3, (1 << 20) + 1, 4096, 70001], steps=6, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=True, oracle_kw=dict(quant_bits=8))
+    assert rep.params_bit_exact and rep.quantised_checked > 10
+    wl = W.synthetic(64, [5, 1000, 4097], steps=6, lr=0.1, grad_sigma=0.01)
+    rep = lockstep(wl, init="distinct", carry=True, oracle_kw=dict(quant_bits=4))
+    assert rep.params_bit_exact and rep.quantised_checked > 100
+
+
+@pytest.mark.parametrize("what", ["momentum", "hops", "own_last_sent", "change_of_norm", "register", "history_cap",
+                                  "delivery"])
+def test_quantised_messages_with_every_other_option(what):
+    wl = W.synthetic(6, [5, 1000, 4097, 30000], steps=12, lr=0.1, grad_sigma=0.01, history_len=3)
+    okw = dict(quant_bits=6)
+    kw = dict(init="distinct", carry=what not in ("delivery",))
+    if what == "momentum":
+        okw["momentum"] = 0.9
+    elif what == "hops":
+        okw["hops"] = 2
+    elif what == "own_last_sent":
+        okw["own_last_sent"] = True
+    elif what == "change_of_norm":
+        okw["change_of_norm"] = True
+    elif what == "register":
+        kw["fused_kernel"] = B.FUSED_REGISTER
+    elif what == "history_cap":
+        okw["threshold_cap"] = (4e-3, 0.8)
+    elif what == "delivery":
+        rng = np.random.default_rng(3)
+        kw["deliver_fn"] = lambda k: (rng.random((wl.P, wl.T)) < 0.6).astype(np.uint8)
+    rep = lockstep(wl, oracle_kw=okw, **kw)
+    assert rep.params_bit_exact and rep.quantised_checked > 10
+
+
+def test_quantised_messages_small_problem_and_zero_change():
+    """A problem small enough for the single-launch kernel takes the other path when messages are
+    quantised; a tensor whose change is zero sends codes that are all zero (E = 0)."""
+    wl = W.synthetic(4, [7, 300, 2000], steps=6, lr=0.0, grad_sigma=0.0)
+
+    def no_gradient(k, g):
+        return torch.zeros_like(g)
+
+    # identical replicas, no gradient, every tensor sends every step: x never moves, the change is zero
+    rep = lockstep(wl, oracle_kw=dict(quant_bits=8, mode=1, delta_fixed=0.0), grad_hook=no_gradient,
+                   fused_kernel=B.FUSED_AUTO)
+    assert rep.params_bit_exact and rep.quantised_checked == 5 * wl.P * wl.T
+
+
+def test_quantised_message_with_a_change_that_is_not_finite_goes_out_in_full():
+    from oracle import eg_oracle as eo
+    wl = W.synthetic(3, [10, 5000], steps=3, lr=0.1, grad_sigma=0.01)
+    eg = B.from_workload(wl, mode=B.THRESH_FIXED, delta_fixed=0.0)
+    eg.set_quantisation(8)
+    o = eo.from_workload(wl, mode=eo.FIXED, delta_fixed=0.0, quant_bits=8)
+    x = W.distinct_init_params(wl)
+    xh = x.numpy().copy()
+    xd = eg.to_layout(x.cuda())
+    for k in range(3):
+        g = wl.grads(k)
+        if k == 1:                                  # an infinity in tensor 1 of replica 2
+            xh[2, 10 + 4321] = np.inf
+            xd[2, eg.tensor_offset[1] + 4321] = float("inf")
+        eg.step(xd, eg.to_layout(g.cuda()), wl.lr)
+        o.step(xh, g.numpy(), wl.lr)
+        q, _ = eg.last_quantised()
+        if k == 1:
+            assert q[2, 1] == 2 and o.quantised()[2, 1] == 0
+            assert np.array_equal((q == 1), (o.quantised() == 1))
+        assert eg.stats() == o.stats()
+        got = eg.from_layout(eg.mailboxes()).numpy()
+        assert np.array_equal(got.view(np.uint32), o.xhat().view(np.uint32))
+    eg.close()
+
+
+def test_quantisation_refusals_and_checkpoint():
+    wl = W.synthetic(3, [7, 3000], steps=3, lr=0.1, grad_sigma=0.01)
+    eg = B.from_workload(wl)
+    for bad in (1, 17, -3, 33):
+        with pytest.raises(B.EventGradError):
+            eg.set_quantisation(bad)
+    with pytest.raises(B.EventGradError):
+        eg.last_quantised()                         # never switched on
+    eg.set_quantisation(8)
+    eg.set_quantisation(32)                         # off again
+    eg.set_quantisation(8)
+    x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
+    eg.step(x, eg.to_layout(wl.grads(0, "cuda")), wl.lr)
+    with pytest.raises(B.EventGradError, match="not allowed"):
+        eg.set_quantisation(4)                      # only before the first step
+    blob = eg.export_state()
+    other = B.from_workload(wl)                     # full precision: another set of rules
+    with pytest.raises(B.EventGradError):
+        other.import_state(blob)
+    other.set_quantisation(8)
+    other.import_state(blob)
+    y = x.clone()
+    g = eg.to_layout(wl.grads(1, "cuda"))
+    eg.step(x, g, wl.lr)
+    other.step(y, g, wl.lr)
+    assert torch.equal(x, y) and eg.stats() == other.stats()
+    assert torch.equal(eg.mailboxes(), other.mailboxes())
+    topk = B.from_workload(W.synthetic(3, [7, 3000], topk=(10, 100)))
+    with pytest.raises(B.EventGradError, match="not allowed"):
+        topk.set_quantisation(8)
+    for c in (eg, other, topk):
+        c.close()
+
+
 def test_one_stream_at_a_time():
     """A context moves to another stream only once the stream of its previous step has run dry."""
     wl = W.synthetic(3, [7, 3000], steps=3, lr=0.1, grad_sigma=0.01)
