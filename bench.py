@@ -77,11 +77,11 @@ def kernel_source_hash(names=DENSE_SOURCES) -> str:
     return h.hexdigest()[:12]
 
 
-def fused_traffic(wl, elems: int, momentum) -> dict:
+def fused_traffic(wl, elems: int, momentum, quant_bits=None) -> dict:
     """`traffic` of the roofline object, and what to say when the counters are out of date."""
     names = kernel_sources(wl)
     current = kernel_source_hash(names)
-    if momentum is not None or names != DENSE_SOURCES:
+    if momentum is not None or quant_bits is not None or names != DENSE_SOURCES:
         # counters exist for the default kernel on dense runs only
         return {"traffic": None, "traffic_note": "no capture for this configuration's kernels",
                 "traffic_sources": list(names), "traffic_sources_hash": current}
@@ -345,11 +345,13 @@ def time_steps(eg, x, grads, lr, steps, sampler=None):
 
 
 def measure_workload(B, wl, K, Wm, dev, world, variants, sampler, sampled_variant, graph_steps=0,
-                     momentum=None):
+                     momentum=None, quant_bits=None):
     """Times K steps of `wl` for every variant; returns ({variant: figures}, context)."""
     eg = B.from_workload(wl)
     if momentum is not None:      # heavy-ball update: the velocity is read and written as well
         eg.set_momentum(momentum)
+    if quant_bits is not None:    # quantised messages: delivered by kernels of their own, on events only
+        eg.set_quantisation(quant_bits)
     extra = MOMENTUM_BYTES_PER_ELEMENT if momentum is not None else 0
     buf_bytes = wl.P * eg.replica_stride * 4
     free, _ = torch.cuda.mem_get_info()
@@ -478,7 +480,7 @@ def run_native(args):
         return
     results, ctx = measure_workload(B, wl, K, Wm, dev, world,
                                     [args.variant] + [v for v in ("carry", "two_pass") if v != args.variant],
-                                    sampler, args.variant, momentum=args.momentum)
+                                    sampler, args.variant, momentum=args.momentum, quant_bits=args.quant_bits)
     eg, x0, grads, n_buf, buf_bytes = ctx
     extra = MOMENTUM_BYTES_PER_ELEMENT if args.momentum is not None else 0
     clocks = sampler.summary()
@@ -508,7 +510,7 @@ def run_native(args):
 
     fused_ms = main["kernel_ms"]["fused"]
     achieved = elems * (FUSED_BYTES_PER_ELEMENT + extra) / fused_ms / 1e6 if fused_ms else None
-    traffic = fused_traffic(wl, elems, args.momentum)
+    traffic = fused_traffic(wl, elems, args.momentum, args.quant_bits)
     roofline = {"bound": "hbm", "kernel": "k_fused_pipe" if args.momentum is None else "k_fused_pipe_momentum",
                 "achieved": achieved, "peak": peak,
                 "peak_kind": f"of {peak_kind}", "unit": "GB/s",
@@ -540,7 +542,7 @@ def run_native(args):
                 "config": {"workload": wl.name, "P": wl.P, "tensors": wl.T, "elements": wl.N,
                            "variant": args.variant,
                            "bytes_per_element_step": BYTES_PER_ELEMENT[args.variant] + extra,
-                           "momentum": args.momentum,
+                           "momentum": args.momentum, "quant_bits": args.quant_bits,
                            "l2": "inputs larger than L2 (no flush needed)",
                            "gradient_buffers": n_buf, "multi_gpu": "replicas only"},
                 "pct_of_peak": 100.0 * main["gbs"] / peak,
@@ -569,6 +571,8 @@ def main():
                     help="time all five configurations (their own step counts) instead of the default one")
     ap.add_argument("--momentum", type=float, default=None,
                     help="heavy-ball momentum coefficient (default: plain SGD update, the paper's)")
+    ap.add_argument("--quant-bits", type=int, default=None,
+                    help="bits per element of quantised messages (default: messages in full precision, the paper's)")
     ap.add_argument("--max-elements", type=int, default=0,
                     help="keep only the leading tensors of the workload up to this many elements")
     args = ap.parse_args()

@@ -15,8 +15,10 @@
 //   k_quant_scale  per marked segment: E from the largest change; a change that is not finite
 //                  turns the message into a full-precision one (and corrects the byte counter)
 //   k_quant_apply  per tile of a marked segment: the update of x_hat above (or x_hat <- x)
-// The kernels walk all (replica, tile) pairs with a fixed grid and skip the unmarked ones, so an
-// iteration without quantised messages costs three short launches.
+// The kernels walk all (replica, tile) pairs with a fixed grid: the threads of a CTA first look,
+// each at a pair of its own, for the marked ones (one round of loads for 256 pairs), then the CTA
+// works through those it found.  An iteration without quantised messages costs three launches of
+// a few microseconds.
 #pragma once
 #include "eg_common.cuh"
 #include "eg_norm.cuh"
@@ -41,6 +43,21 @@ struct QuantArgs {
     Counters* ctr;
 };
 
+// The marked pairs among the kThreads pairs `first + (j * gridDim.x + blockIdx.x)`, j = 0 ..
+// kThreads - 1, into `list` (any order); returns how many.  All threads of the CTA call it.
+__device__ __forceinline__ int quant_marked_pairs(const QuantArgs& a, long long first, long long pairs, int* list,
+                                                  int* count) {
+    if (threadIdx.x == 0) *count = 0;
+    __syncthreads();
+    const long long w = first + (long long)threadIdx.x * gridDim.x + blockIdx.x;
+    if (w < pairs) {
+        const int i = (int)(w / a.tt.n_tiles), tile = (int)(w % a.tt.n_tiles);
+        if (a.quant[(long long)i * a.T + a.tt.tensor[tile]] != 0) list[atomicAdd(count, 1)] = (int)(w - first);
+    }
+    __syncthreads();
+    return *count;
+}
+
 // 2^k as a double, -1022 <= k <= 1023
 __device__ __forceinline__ double pow2_double(int k) {
     return __longlong_as_double((long long)(k + 1023) << 52);
@@ -49,11 +66,13 @@ __device__ __forceinline__ double pow2_double(int k) {
 // grid: any; CTA b takes the (replica, tile) pairs b, b + grid, ...
 __global__ void __launch_bounds__(kThreads) k_quant_max(QuantArgs a) {
     __shared__ float s_warp[kWarps];
+    __shared__ int s_list[kThreads], s_count;
     const long long pairs = (long long)a.P * a.tt.n_tiles;
-    for (long long w = blockIdx.x; w < pairs; w += gridDim.x) {
+    for (long long first = 0; first < pairs; first += (long long)gridDim.x * kThreads) {
+      const int found = quant_marked_pairs(a, first, pairs, s_list, &s_count);
+      for (int f = 0; f < found; ++f) {
+        const long long w = first + s_list[f];
         const int i = (int)(w / a.tt.n_tiles), tile = (int)(w % a.tt.n_tiles);
-        const int t = a.tt.tensor[tile];
-        if (a.quant[(long long)i * a.T + t] == 0) continue;          // the same in every thread
         if (!tile_ok(a.tt, tile, a.T, a.stride, kNormTile)) continue;  // bounds-checked build only
         const int len = a.tt.length[tile];
         const long long base = (long long)i * a.stride + a.tt.offset[tile];
@@ -83,6 +102,7 @@ __global__ void __launch_bounds__(kThreads) k_quant_max(QuantArgs a) {
             for (int q = 1; q < kWarps; ++q) all = fmaxf(all, s_warp[q]);
             a.tile_max[w] = all;
         }
+      }
     }
 }
 
@@ -127,15 +147,18 @@ __global__ void __launch_bounds__(kThreads) k_quant_scale(QuantArgs a) {
 
 // grid: any; CTA b takes the (replica, tile) pairs b, b + grid, ...
 __global__ void __launch_bounds__(kThreads) k_quant_apply(QuantArgs a) {
+    __shared__ int s_list[kThreads], s_count;
     const long long pairs = (long long)a.P * a.tt.n_tiles;
     const double L = (double)((1 << (a.bits - 1)) - 1);
-    for (long long w = blockIdx.x; w < pairs; w += gridDim.x) {
+    for (long long first = 0; first < pairs; first += (long long)gridDim.x * kThreads) {
+      const int found = quant_marked_pairs(a, first, pairs, s_list, &s_count);
+      for (int f = 0; f < found; ++f) {
+        const long long w = first + s_list[f];
         const int i = (int)(w / a.tt.n_tiles), tile = (int)(w % a.tt.n_tiles);
+        if (!tile_ok(a.tt, tile, a.T, a.stride, kNormTile)) continue;  // bounds-checked build only
         const int t = a.tt.tensor[tile];
         const long long s = (long long)i * a.T + t;
         const uint8_t kind = a.quant[s];
-        if (kind == 0) continue;
-        if (!tile_ok(a.tt, tile, a.T, a.stride, kNormTile)) continue;  // bounds-checked build only
         const int len = a.tt.length[tile];
         const long long base = (long long)i * a.stride + a.tt.offset[tile];
         const int E = a.qexp[s];
@@ -167,6 +190,7 @@ __global__ void __launch_bounds__(kThreads) k_quant_apply(QuantArgs a) {
                 if (nel > 2) out[2] = hv.z;
             }
         }
+      }
     }
 }
 

@@ -927,7 +927,7 @@ eg_status eg_step_host(eg_ctx* c, float* params_host, const float* grads_host, f
     }
     cudaStream_t stream = c->last_stream;
     c->carried_valid = false;  // the parameters come from outside
-    const bool pipelined = !c->topk.enabled && !c->async && c->hops == 1 &&
+    const bool pipelined = !c->topk.enabled && !c->async && c->hops == 1 && c->quant_bits == 0 &&
                            c->fused_kind != EG_FUSED_REGISTER && c->T >= 2;
     if (!pipelined) {
         EG_CUDA(c, cudaMemcpyAsync(c->stage_x, params_host, bytes, cudaMemcpyHostToDevice, stream));

@@ -62,13 +62,16 @@ def _columns(numel: Sequence[int], tensors: Sequence[int]) -> np.ndarray:
     return np.concatenate([np.arange(off[t], off[t] + numel[t]) for t in tensors])
 
 
-def _counters_from_events(events: np.ndarray, numel, k_t, degree: int) -> dict:
+def _counters_from_events(events: np.ndarray, numel, k_t, degree: int, quant_bits: int = 0) -> dict:
     """Message, byte and event totals implied by the number of events of every (replica,
     tensor): `degree` messages per event, 4 n_t bytes for a dense message, 8 K_t for a Top-K
-    message, the first message of a tensor always being dense."""
+    message, 4 + ceil(n_t b / 8) for a quantised one (finite changes), the first message of a
+    tensor always being dense."""
     ev = np.asarray(events, dtype=np.int64)
     n = np.asarray(numel, dtype=np.int64)[None, :]
-    if k_t is None:
+    if quant_bits:
+        payload = np.where(ev > 0, 4 * n + (4 + (n * quant_bits + 7) // 8) * (ev - 1), 0)
+    elif k_t is None:
         payload = 4 * n * ev
     else:
         kt = np.asarray(k_t, dtype=np.int64)[None, :]
@@ -287,8 +290,10 @@ def lockstep(wl: W.Workload, *, steps: Optional[int] = None, init: str = "worklo
             # the oracle's counters must equal that sum over its tensors and the library's the
             # same sum over all tensors, the per-tensor events of the sample being equal.
             so, sg = o.stats(), eg.stats()
-            assert so == _counters_from_events(o.segment_events(), sub_numel, sub_kt, degree), f"step {k}"
-            assert sg == _counters_from_events(ev_g, wl.numel, all_kt, degree), f"counters, step {k}"
+            qb = okw.get("quant_bits") or 0
+            qb = 0 if qb == 32 else qb
+            assert so == _counters_from_events(o.segment_events(), sub_numel, sub_kt, degree, qb), f"step {k}"
+            assert sg == _counters_from_events(ev_g, wl.numel, all_kt, degree, qb), f"counters, step {k}"
         dl_g, _ = eg.thresholds()
         dl_g, dl_o = dl_g[:, tensors], o.thresholds()
         fin = np.isfinite(dl_o)

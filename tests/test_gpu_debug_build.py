@@ -6,7 +6,7 @@ modes, pipeline stages, partial sums, entry slots) is compared with the table's 
 miss sets a bit of the context's error word -- which the next synchronising call reports as an
 error -- and the access is skipped.  Here a slice of the parity suite (ragged sizes, dense and
 Top-K, the guessed and the repeated Top-K route, the single-launch kernel, more neighbours,
-intermittent delivery, momentum, the pipelined kernel walking tiles handed out by a counter) runs against that build in a child process: it must pass, which
+intermittent delivery, momentum, the pipelined kernel walking tiles handed out by a counter, quantised messages) runs against that build in a child process: it must pass, which
 includes every eg_stats / eg_last_decisions call returning EG_OK, i.e. the error word staying 0.
 """
 import os
@@ -24,7 +24,7 @@ SLICE = ("test_ragged_dense and (True-7 or False-64 or True-3 or False-5) or tes
          "or test_topk_guess_and_exact_repeat and (5-True or -8-False) or test_topk_degenerate "
          "or test_more_neighbours_per_side and (9-4 or 16-8) or test_intermittent_delivery_topk "
          "or test_momentum_with_topk_and_history or test_history_and_horizon and 4-1.0 "
-         "or test_graph_replay and walking_cap")
+         "or test_graph_replay and walking_cap or test_quantised_messages_ragged and 5-True")
 
 
 def test_parity_slice_under_the_bounds_checked_build():

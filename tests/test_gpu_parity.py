@@ -103,7 +103,7 @@ def test_intermittent_delivery_topk(con):
 
 def _random_case(seed):
     """One seeded draw over the options of a context; combinations the library documents as
-    unavailable (delivery masks with the own-term variant) are not drawn."""
+    unavailable (delivery masks with the own-term variant, quantised Top-K messages) are not drawn."""
     rng = np.random.default_rng(1000 + seed)
     P = int(rng.integers(1, 12))
     sizes = [int(v) for v in rng.choice(RAGGED[:-1], size=int(rng.integers(1, 6)), replace=False)]
@@ -119,6 +119,8 @@ def _random_case(seed):
         okw.update(mode=1, delta_fixed=float(rng.choice([0.0, 0.01])), force_first_event=bool(rng.integers(0, 2)))
     if rng.integers(0, 3) == 0:
         okw["momentum"] = float(rng.choice([0.0, 0.5, 0.9]))
+    if topk is None and rng.integers(0, 2) == 0:
+        okw["quant_bits"] = int(rng.choice([3, 8, 12]))
     return dict(P=P, sizes=sizes, topk=topk, okw=okw, carry=bool(rng.integers(0, 2)),
                 kernel=[B.FUSED_PIPELINED, B.FUSED_REGISTER][int(rng.integers(0, 2))],
                 deliver=_random_links(P, len(sizes), float(rng.choice([0.3, 0.8])), seed) if deliver else None)
@@ -491,6 +493,15 @@ def test_momentum_resnet18_shapes_p16():
     assert rep.params_bit_exact
 
 
+def test_quantised_resnet18_shapes_p16():
+    """The 16-replica ResNet-18 ring with 8-bit messages: many tiles per tensor, the walking form of
+    the averaging kernel, carried norm; the oracle follows a sample of the tensors."""
+    (wl,) = W.config(3)
+    rep = lockstep(wl, steps=12, tensors=_sample_tensors(wl), carry=True, check_every=3,
+                   oracle_kw=dict(quant_bits=8))
+    assert rep.params_bit_exact and rep.quantised_checked > 50
+
+
 @pytest.mark.parametrize("carry", [False, True])
 @pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_AUTO])
 def test_config1_mlp(carry, kernel):
@@ -829,6 +840,26 @@ def test_quantised_message_with_a_change_that_is_not_finite_goes_out_in_full():
         got = eg.from_layout(eg.mailboxes()).numpy()
         assert np.array_equal(got.view(np.uint32), o.xhat().view(np.uint32))
     eg.close()
+
+
+def test_quantised_messages_through_host_buffers():
+    """eg_step_host with quantised messages (whole-step form: the messages need every tensor's
+    decision before the averaging kernel) against eg_step on device buffers."""
+    wl = W.synthetic(4, [5, 1000, 4097, 30000], steps=6, lr=0.1, grad_sigma=0.01)
+    a, b = B.from_workload(wl), B.from_workload(wl)
+    a.set_quantisation(8)
+    b.set_quantisation(8)
+    x = a.to_layout(W.distinct_init_params(wl, "cuda"))
+    xh = x.cpu().pin_memory()
+    for k in range(wl.steps):
+        g = a.to_layout(wl.grads(k, "cuda"))
+        a.step(x, g, wl.lr)
+        b.step_host(xh, g.cpu().pin_memory(), wl.lr)
+    torch.cuda.synchronize()
+    assert torch.equal(x.cpu(), xh) and a.stats() == b.stats()
+    assert torch.equal(a.mailboxes(), b.mailboxes())
+    a.close()
+    b.close()
 
 
 def test_quantisation_refusals_and_checkpoint():
