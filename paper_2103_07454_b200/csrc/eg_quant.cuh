@@ -163,9 +163,24 @@ __global__ void __launch_bounds__(kThreads) k_quant_apply(QuantArgs a) {
         const long long base = (long long)i * a.stride + a.tt.offset[tile];
         const int E = a.qexp[s];
         const double up = pow2_double(E), down = pow2_double(-E);
-        for (int local = threadIdx.x * 4; local < len; local += kThreads * 4) {
-            const float4 xv = ld_stream(a.x + base + local);
-            float4 hv = *reinterpret_cast<const float4*>(a.xhat + base + local);
+        constexpr int kIter = kNormTile / (kThreads * 4);
+        float4 xq[kIter], hq[kIter];
+#pragma unroll
+        for (int q = 0; q < kIter; ++q) {       // all eight loads of the tile before the first use
+            const int local = (q * kThreads + threadIdx.x) * 4;
+            if (local < len) {
+                xq[q] = ld_stream(a.x + base + local);
+                hq[q] = *reinterpret_cast<const float4*>(a.xhat + base + local);
+            } else {
+                xq[q] = hq[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kIter; ++q) {
+            const int local = (q * kThreads + threadIdx.x) * 4;
+            if (local >= len) continue;
+            const float4 xv = xq[q];
+            float4 hv = hq[q];
             const int nel = min(4, len - local);
             if (kind == kQuantFull) {
                 hv = xv;
