@@ -688,7 +688,8 @@ def test_steps_replayed_from_a_cuda_graph_match_direct_calls():
     assert all(np.array_equal(a, b) for a, b in zip(outs[0][2], outs[1][2]))
 
 
-@pytest.mark.parametrize("what", ["pipelined_carry_cap", "small_cap", "topk_cap", "two_pass", "walking_cap"])
+@pytest.mark.parametrize("what", ["pipelined_carry_cap", "small_cap", "topk_cap", "two_pass", "walking_cap",
+                                  "quantised_cap"])
 def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(what):
     """Replays of one captured eg_step against direct calls and the oracle, for the launch forms a
     step can take: decision + pipelined kernel started as dependent launches (carried norm), the
@@ -712,6 +713,8 @@ def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(w
         eg.set_fused_kernel(kernel)
         if cap:
             eg.set_threshold_cap(*cap)
+        if what == "quantised_cap":
+            eg.set_quantisation(6)
         x = eg.to_layout(W.distinct_init_params(wl, "cuda"))
         grad = eg.to_layout(wl.grads(0, "cuda"))
         eg.step(x, grad, wl.lr)
@@ -737,13 +740,17 @@ def test_graph_replay_of_every_launch_form_matches_direct_calls_and_the_oracle(w
     assert torch.equal(outs[0][3], outs[1][3])
     assert all(np.array_equal(a, b) for a, b in zip(outs[0][2], outs[1][2]))
     # and the oracle, fed the same gradient nine times
-    o = eo.from_workload(wl, threshold_cap=cap) if cap else eo.from_workload(wl)
+    okw = dict(threshold_cap=cap) if cap else {}
+    if what == "quantised_cap":
+        okw["quant_bits"] = 6
+    o = eo.from_workload(wl, **okw)
     xh = W.distinct_init_params(wl).numpy().copy()
     gh = wl.grads(0).numpy()
     for _ in range(9):
         o.step(xh, gh, wl.lr)
     eg = B.from_workload(wl)
     assert np.array_equal(eg.from_layout(outs[1][0]).cpu().numpy(), xh)
+    assert np.array_equal(eg.from_layout(outs[1][3]).numpy().view(np.uint32), o.xhat().view(np.uint32))
     assert outs[1][1] == o.stats()
     assert np.array_equal(outs[1][2][0], o.flags())
     if cap:
