@@ -689,7 +689,7 @@ def test_momentum_reset_clears_the_velocity_and_range_is_checked():
 # ---------------------------------------------------------------------------------------
 # ---------------------------------------------------------------------------------------
 # Quantised messages (Section 7: quantization can be applied on top of the events; the scheme is
-# this build's reading, stated in the oracle's header)
+# the reading taken here, stated in the oracle's header)
 # ---------------------------------------------------------------------------------------
 def _exact_quantised_message(x_row, h_row, bits):
     """The reading restated with exact rational arithmetic: (E, new x_hat) of one tensor."""
