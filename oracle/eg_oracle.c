@@ -64,7 +64,10 @@
  *    receivers alike set x_hat[e] <- fp32(fp64(x_hat[e]) + q[e] 2^E).  What was not sent,
  *    x - x_hat, stays in the difference and enters the next test and the next message.  The
  *    first message of a tensor is sent in full (as with Top-K), a change that is not finite
- *    too, and b = 32 means no quantisation.  Pinned against exact rational arithmetic on small
+ *    too, and b = 32 means no quantisation.  Together with Top-K messages ("quantization and
+ *    sparsification on top"): the K_t entries are selected as before, E comes from the largest
+ *    change (which is among them), and the message holds E, the K_t indices and the K_t codes
+ *    (4 + 4 K_t + ceil(K_t b / 8) bytes); x_hat is updated at the selected entries only.  Pinned against exact rational arithmetic on small
  *    inputs, the round-trip bound |x - x_hat| <= 2^E / 2 (+ rounding), changes that lie on the
  *    grid (reproduced exactly, E as constructed), b = 32 == dense, and the payload count.
  */
@@ -275,12 +278,10 @@ int ego_set_momentum(ego_ctx *c, double mu) {
 }
 float *ego_velocity(ego_ctx *c) { return c->vel; }
 
-/* bits per code of a quantised message: 2..16; 0 or 32: messages in full precision.  Not
- * together with Top-K messages (one compression at a time). */
+/* bits per code of a quantised message: 2..16; 0 or 32: messages in full precision. */
 int ego_set_quantisation(ego_ctx *c, int bits) {
     if (bits == 32) bits = 0;
     if (bits != 0 && (bits < 2 || bits > 16)) return -1;
-    if (bits != 0 && c->topk) return -1;
     if (bits != 0 && !c->qexp) {
         c->qexp = (int32_t *)calloc((size_t)c->P * c->T, sizeof(int32_t));
         c->quantised = (uint8_t *)calloc((size_t)c->P * c->T, 1);
@@ -402,6 +403,7 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
     /* 4b: the message */
     uint64_t payload;
     int quantise = c->quant_bits != 0 && c->valid[s];
+    const int sparse_route = c->topk && c->valid[s];
     float dmax = 0.0f;
     if (quantise) { /* the largest change; a change that is not finite is sent in full */
         for (int64_t e = 0; e < n; ++e) {
@@ -411,14 +413,17 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
         }
     }
     if (c->qexp) { c->qexp[s] = 0; c->quantised[s] = (uint8_t)quantise; }
+    int E = 0;
+    const double L = c->quant_bits ? (double)((1 << (c->quant_bits - 1)) - 1) : 0.0;
     if (quantise) {
-        const int b = c->quant_bits;
-        const double L = (double)((1 << (b - 1)) - 1);
-        int E = 0;
         if (dmax > 0.0f) { /* the smallest E with L 2^E >= max|d| */
             E = -400;
             while (ldexp(L, E) < (double)dmax) ++E;
         }
+        c->qexp[s] = E;
+    }
+    if (quantise && !sparse_route) {
+        const int b = c->quant_bits;
         for (int64_t e = 0; e < n; ++e) {
             const float d32 = xs[e] - hs[e];
             double q = rint((double)d32 * ldexp(1.0, -E)); /* exact scaling, ties to even */
@@ -427,7 +432,6 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
             const double r = (double)hs[e] + q * ldexp(1.0, E);
             hs[e] = (float)r;
         }
-        c->qexp[s] = E;
         payload = 4u + ((uint64_t)n * (uint64_t)b + 7u) / 8u;
     } else if (!c->topk || !c->valid[s]) {
         for (int64_t e = 0; e < n; ++e) hs[e] = xs[e];
@@ -448,9 +452,19 @@ static void phase_a_segment(ego_ctx *c, const float *x, int i, int t) {
             oi[q] = r[q].idx;
             ov[q] = xs[r[q].idx];
         }
+        if (quantise) { /* the values go out as codes of the change: what arrives is x_hat + q 2^E */
+            for (int64_t q = 0; q < K; ++q) {
+                const float d32 = xs[oi[q]] - hs[oi[q]];
+                double code = rint((double)d32 * ldexp(1.0, -E));
+                if (code > L) code = L;
+                if (code < -L) code = -L;
+                ov[q] = (float)((double)hs[oi[q]] + code * ldexp(1.0, E));
+            }
+        }
         for (int64_t q = 0; q < K; ++q) hs[oi[q]] = ov[q]; /* scatter on receipt */
         c->out_count[s] = (int32_t)K;
-        payload = 8u * (uint64_t)K;
+        payload = quantise ? 4u + 4u * (uint64_t)K + ((uint64_t)K * (uint64_t)c->quant_bits + 7u) / 8u
+                           : 8u * (uint64_t)K;
         free(r);
     }
     c->seg_payload[s] = payload;

@@ -794,8 +794,76 @@ def test_thirty_two_bits_and_the_first_message_are_full_precision():
         eo.from_workload(wl, quant_bits=1)
     with pytest.raises(ValueError):
         eo.from_workload(wl, quant_bits=17)
-    with pytest.raises(ValueError):
-        eo.Oracle(3, [10, 20], topk=(1, 10), quant_bits=8)      # one compression at a time
+
+
+@pytest.mark.parametrize("bits", [3, 8])
+def test_quantised_topk_messages_against_brute_force_and_exact_arithmetic(bits):
+    """Both compressions together: the K_t entries of largest |x - x_hat| (brute-force lexsort, ties
+    to the lower index), their values sent as codes of the change on the grid of the largest change
+    (exact rational arithmetic), x_hat untouched elsewhere, 4 + 4 K + ceil(K b / 8) bytes."""
+    from fractions import Fraction
+    wl = small(P=3, numel=(1, 40, 257), steps=5, lr=0.1, grad_sigma=0.02, topk=(10, 100))
+    o = eo.from_workload(wl, mode=eo.FIXED, delta_fixed=0.0, quant_bits=bits)
+    x = W.distinct_init_params(wl).numpy().copy()
+    off = np.concatenate([[0], np.cumsum(wl.numel)])
+    L = (1 << (bits - 1)) - 1
+    bytes_before = 0
+    for k in range(wl.steps):
+        h_before, x_before = o.xhat().copy(), x.copy()
+        o.step(x, wl.grads(k).numpy(), wl.lr)
+        h_after = o.xhat()
+        payload = 0
+        for i in range(wl.P):
+            for t in range(wl.T):
+                a, b = off[t], off[t + 1]
+                n = wl.numel[t]
+                if k == 0:
+                    assert np.array_equal(h_after[i, a:b], x_before[i, a:b])
+                    payload += 4 * n
+                    continue
+                K = o.topk_count(t)
+                d = (x_before[i, a:b] - h_before[i, a:b]).astype(np.float32)
+                keys = np.abs(d).view(np.uint32)
+                order = np.lexsort((np.arange(n), -keys.astype(np.int64)))      # key descending, index ascending
+                chosen = np.sort(order[:K])
+                idx, val = o.outbox(i, t)
+                assert np.array_equal(idx, chosen)
+                dmax = max(abs(Fraction(float(v))) for v in d)
+                E = 0
+                if dmax > 0:
+                    E = -400
+                    while L * Fraction(2) ** E < dmax:
+                        E += 1
+                assert o.quant_exponents()[i, t] == E and o.quantised()[i, t] == 1
+                want = h_before[i, a:b].copy()
+                for e in chosen:
+                    r = Fraction(float(d[e])) / Fraction(2) ** E
+                    lo = r.numerator // r.denominator
+                    frac = r - lo
+                    q = lo + (1 if frac > Fraction(1, 2) or (frac == Fraction(1, 2) and lo % 2 == 1) else 0)
+                    want[e] = np.float32(float(Fraction(float(h_before[i, a + e])) + q * Fraction(2) ** E))
+                assert np.array_equal(h_after[i, a:b], want)
+                assert np.array_equal(val, want[chosen])            # the message's values: what arrives
+                payload += 4 + 4 * K + (K * bits + 7) // 8
+        assert o.stats()["bytes"] - bytes_before == 2 * payload
+        bytes_before = o.stats()["bytes"]
+
+
+def test_quantised_topk_with_every_entry_selected_is_the_quantised_dense_message():
+    wl = small(P=4, numel=(9, 64, 300), steps=8, lr=0.1, grad_sigma=0.02)
+    dense = eo.from_workload(wl, quant_bits=6)
+    wl_all = small(P=4, numel=(9, 64, 300), steps=8, lr=0.1, grad_sigma=0.02, topk=(1, 1))
+    sparse = eo.from_workload(wl_all, quant_bits=6)
+    xa = W.distinct_init_params(wl).numpy().copy()
+    xb = xa.copy()
+    for k in range(wl.steps):
+        g = wl.grads(k).numpy()
+        dense.step(xa, g, wl.lr)
+        sparse.step(xb, g, wl.lr)
+        assert np.array_equal(xa, xb) and np.array_equal(dense.xhat(), sparse.xhat())
+        assert np.array_equal(dense.flags(), sparse.flags())
+        assert np.array_equal(dense.quant_exponents(), sparse.quant_exponents())
+    assert dense.stats()["events"] == sparse.stats()["events"] > wl.P * wl.T
 
 
 def test_quantised_run_keeps_the_error_bound_and_saves_bytes():
