@@ -201,11 +201,16 @@ eg_status eg_set_momentum(eg_ctx* ctx, int enabled, double mu);
  * What was not sent, x - x_hat, remains part of the difference: it enters the next trigger test
  * and the next message (nothing is dropped for good).  The first message of a tensor is sent in
  * full precision (x_hat <- x, 4 n bytes), as with Top-K messages; so is a message whose change
- * holds an infinity or a NaN.  bits: 2..16; 0 or 32 switches quantisation off.  Not available
- * in a context created with Top-K messages (one compression at a time: EG_ERR_STATE), and only
- * before the first step or after eg_reset (EG_ERR_STATE otherwise).  Works with every other
- * option: the messages are delivered into x_hat by kernels of their own before the averaging
- * kernel runs, the way Top-K messages are.
+ * holds an infinity or a NaN.  bits: 2..16; 0 or 32 switches quantisation off.  Only before the
+ * first step or after eg_reset (EG_ERR_STATE otherwise).  Works with every other option: the
+ * messages are delivered into x_hat by kernels of their own before the averaging kernel runs,
+ * the way Top-K messages are.
+ * In a context with Top-K messages both compressions apply ("quantization and sparsification on
+ * top of event-triggered communication", Section 7): the K_t entries are selected as without
+ * quantisation, E comes from the largest change of the tensor (which is among them), the message
+ * holds E, the K_t indices and the K_t codes (4 + 4 K_t + ceil(K_t * bits / 8) bytes), and x_hat is
+ * updated at the selected entries only; eg_last_outbox then returns, as values, what the
+ * receivers hold at those entries after the message.
  * eg_last_quantised copies, for the last step, which (replica, tensor) pairs sent a quantised
  * message (1; 2: the change was not finite and the message went out in full; 0: none) and the
  * exponents E of those messages to host arrays of P*T entries; EG_ERR_STATE when quantisation

@@ -57,6 +57,11 @@ __device__ __forceinline__ bool tile_ok(const TileTable& tt, int tile, int T, lo
 #endif
 }
 
+// 2^k as a double, -1022 <= k <= 1023
+__device__ __forceinline__ double pow2_double(int k) {
+    return __longlong_as_double((long long)(k + 1023) << 52);
+}
+
 // Per-(replica, tensor) trigger state and the decisions of the current step, all [P*T].
 struct SegState {
     double* delta;               // threshold in force

@@ -141,7 +141,7 @@ decide_segment(double acc, long long s, int t, long long k, double cap, const De
             st.delta[s] = __dmul_rn(dp.horizon, __ddiv_rn(sum, (double)n));
         }
         unsigned long long payload;
-        if (dp.quant_bits && was_valid) {
+        if (dp.quant_bits && was_valid && !dp.topk) {
             // b-bit codes of the change since the last message and the exponent of their scale
             quant = 1;
             payload = 4ull + ((unsigned long long)numel[t] * (unsigned long long)dp.quant_bits + 7ull) / 8ull;
@@ -153,6 +153,11 @@ decide_segment(double acc, long long s, int t, long long k, double cap, const De
             if (st.sparse_steps) atomicAdd(&st.sparse_steps[k & 1], 1u);   // tells the Top-K launch there is work
             out_count = (int)topk_count[t];
             payload = 8ull * (unsigned long long)topk_count[t];
+            if (dp.quant_bits) {   // the K_t values as codes: exponent, indices, codes
+                quant = 1;
+                payload = 4ull + 4ull * (unsigned long long)topk_count[t] +
+                          ((unsigned long long)topk_count[t] * (unsigned long long)dp.quant_bits + 7ull) / 8ull;
+            }
         }
         if (dp.variant & kChangeOfNorm) st.sent_norm[s] = root;
         st.khat[s] = k;

@@ -38,6 +38,9 @@ struct QuantArgs {
     float* tile_max;           // [P][n_tiles]
     int* qexp;                 // [P*T] E of the segment's message
     const long long* numel;    // [T]
+    const uint8_t* sparse;     // [P*T] SegState::sparse: the message is a Top-K message; its values are
+                               //       quantised by the Top-K packing kernel (which needs E from here)
+    const long long* topk_count;   // [T] K_t (nullptr without Top-K)
     int bits;
     int degree;                // distinct ring neighbours of a replica
     Counters* ctr;
@@ -56,11 +59,6 @@ __device__ __forceinline__ int quant_marked_pairs(const QuantArgs& a, long long 
     }
     __syncthreads();
     return *count;
-}
-
-// 2^k as a double, -1022 <= k <= 1023
-__device__ __forceinline__ double pow2_double(int k) {
-    return __longlong_as_double((long long)(k + 1023) << 52);
 }
 
 // grid: any; CTA b takes the (replica, tile) pairs b, b + grid, ...
@@ -124,10 +122,15 @@ __global__ void __launch_bounds__(kThreads) k_quant_scale(QuantArgs a) {
         a.quant[s] = kQuantFull;
         a.qexp[s] = 0;
         const unsigned long long n = (unsigned long long)a.numel[t];
-        const unsigned long long coded = 4ull + (n * (unsigned long long)a.bits + 7ull) / 8ull;
+        unsigned long long coded = 4ull + (n * (unsigned long long)a.bits + 7ull) / 8ull, full = 4ull * n;
+        if (a.sparse && a.sparse[s]) {      // a Top-K message: 8 K_t bytes in full, E + indices + codes otherwise
+            const unsigned long long K = (unsigned long long)a.topk_count[t];
+            coded = 4ull + 4ull * K + (K * (unsigned long long)a.bits + 7ull) / 8ull;
+            full = 8ull * K;
+        }
         if (a.degree > 0) {
-            // (unsigned arithmetic: the two updates together add degree * (4 n - coded))
-            atomicAdd(&a.ctr->bytes, (unsigned long long)a.degree * 4ull * n);
+            // (unsigned arithmetic: the two updates together add degree * (full - coded))
+            atomicAdd(&a.ctr->bytes, (unsigned long long)a.degree * full);
             atomicAdd(&a.ctr->bytes, 0ull - (unsigned long long)a.degree * coded);
         }
         return;
@@ -159,6 +162,7 @@ __global__ void __launch_bounds__(kThreads) k_quant_apply(QuantArgs a) {
         const int t = a.tt.tensor[tile];
         const long long s = (long long)i * a.T + t;
         const uint8_t kind = a.quant[s];
+        if (a.sparse && a.sparse[s]) continue;      // a Top-K message: delivered by the Top-K packing kernel
         const int len = a.tt.length[tile];
         const long long base = (long long)i * a.stride + a.tt.offset[tile];
         const int E = a.qexp[s];

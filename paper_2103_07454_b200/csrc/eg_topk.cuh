@@ -81,6 +81,12 @@ struct TopkState {
     const long long* numel;    // [T] n_t
     long long out_stride;      // sum K_t
     float guess_margin;        // safety margin of the guess, in standard deviations of the sampled count
+    // quantised Top-K messages (eg_set_quantisation in a Top-K context): which segments' values go
+    // out as codes (SegState::quant == 1) and the exponent of their scale (found by the quantising
+    // kernels before the select runs); nullptr: values in full precision
+    const uint8_t* quant;      // [P*T]
+    const int* qexp;           // [P*T]
+    int quant_bits;
 };
 
 __device__ __forceinline__ unsigned int rank_key(float a, float b) {
@@ -1031,6 +1037,8 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, const TopkState& 
     int s_now = -1;
     unsigned int tau20 = 0, take = 0, K = 0, sel = 0;
     int2* out = nullptr;
+    bool coded = false;            // the segment's values go out as codes of the change
+    double up = 1.0, down = 1.0, qmax = 0.0;
     while (feed.next(tk, wl, tt, T, z, n)) {
         if (z.s != s_now) {
             s_now = z.s;
@@ -1039,6 +1047,12 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, const TopkState& 
             take = tk.remaining[z.s];
             K = (unsigned int)tk.count[z.t];
             out = tk.outbox + (long long)z.i * tk.out_stride + tk.out_off[z.t];
+            coded = tk.quant != nullptr && tk.quant[z.s] == 1;
+            if (coded) {
+                const int E = tk.qexp[z.s];
+                up = pow2_double(E); down = pow2_double(-E);
+                qmax = (double)((1 << (tk.quant_bits - 1)) - 1);
+            }
         }
         const long long index = (long long)z.i * tt.n_tiles + z.tile;
         const uint2 before = tk.tile_count[index];
@@ -1076,8 +1090,17 @@ topk_write(float* xhat, TileTable tt, int T, long long stride, const TopkState& 
                     const unsigned int slot = my_gt + min(my_eq, take);
                     const int local = u * kWarpSpan + (int)(e[q].x & 0x1ffu);
                     if (slot < K && local < len) {
-                        out[slot] = make_int2(first + local, (int)e[q].y);
-                        xhat[base + local] = __uint_as_float(e[q].y);
+                        unsigned int bits = e[q].y;          // x at the entry: what a plain message delivers
+                        if (coded) {
+                            // the change as a code on the segment's grid; what arrives is x_hat + code * 2^E
+                            const float had = xhat[base + local];
+                            const float d = __fsub_rn(__uint_as_float(bits), had);
+                            double code = rint(__dmul_rn((double)d, down));
+                            code = fmin(fmax(code, -qmax), qmax);
+                            bits = __float_as_uint(__double2float_rn(__dadd_rn((double)had, __dmul_rn(code, up))));
+                        }
+                        out[slot] = make_int2(first + local, (int)bits);
+                        xhat[base + local] = __uint_as_float(bits);
                     } else {
                         atomicOr(err, kErrTopkSlot);
                     }

@@ -761,7 +761,8 @@ eg_status eg_step_masked(eg_ctx* c, float* params, const float* grads, float lr,
     if (c->quant_bits != 0 && !small) {
         TimedSection ts(c, stream, EG_KERNEL_TOPK);
         QuantArgs qa{params, c->xhat, tn_all, c->P, c->T, c->stride, c->st.quant, c->quant_tile_max, c->quant_exp,
-                     c->d_numel, c->quant_bits, c->degree, c->ctr};
+                     c->d_numel, c->topk.enabled ? c->st.sparse : nullptr,
+                     c->topk.enabled ? c->d_kcount : nullptr, c->quant_bits, c->degree, c->ctr};
         const int walk_grid = c->sms * 8;
         k_quant_max<<<walk_grid, kThreads, 0, stream>>>(qa);
         k_quant_scale<<<(int)((S + kWarps - 1) / kWarps), kThreads, 0, stream>>>(qa);
@@ -1208,7 +1209,6 @@ eg_status eg_set_quantisation(eg_ctx* c, int bits) {
     if (bits == 32) bits = 0;
     if (bits != 0 && (bits < 2 || bits > 16)) return EG_ERR_INVALID;
     if (c->stepped) return EG_ERR_STATE;            // only before the first step (or after eg_reset)
-    if (bits != 0 && c->topk.enabled) return EG_ERR_STATE;   // one compression at a time
     DeviceGuard guard(c->device);
     if (!guard.ok) return EG_ERR_CUDA;
     if (bits != 0 && !c->st.quant) {
@@ -1219,6 +1219,10 @@ eg_status eg_set_quantisation(eg_ctx* c, int bits) {
         if ((s = dev_alloc(c, &c->quant_tile_max, (size_t)c->P * c->tiles_norm.n_tiles)) != EG_OK) return s;
     }
     c->quant_bits = bits;
+    // in a Top-K context the packing kernel turns the selected values into codes
+    c->tk.quant = bits != 0 ? c->st.quant : nullptr;
+    c->tk.qexp = bits != 0 ? c->quant_exp : nullptr;
+    c->tk.quant_bits = bits;
     c->carried_valid = false;
     return EG_OK;
 }

@@ -65,11 +65,14 @@ def _columns(numel: Sequence[int], tensors: Sequence[int]) -> np.ndarray:
 def _counters_from_events(events: np.ndarray, numel, k_t, degree: int, quant_bits: int = 0) -> dict:
     """Message, byte and event totals implied by the number of events of every (replica,
     tensor): `degree` messages per event, 4 n_t bytes for a dense message, 8 K_t for a Top-K
-    message, 4 + ceil(n_t b / 8) for a quantised one (finite changes), the first message of a
-    tensor always being dense."""
+    message, 4 + ceil(n_t b / 8) for a quantised one and 4 + 4 K_t + ceil(K_t b / 8) for a quantised
+    Top-K one (finite changes), the first message of a tensor always being dense."""
     ev = np.asarray(events, dtype=np.int64)
     n = np.asarray(numel, dtype=np.int64)[None, :]
-    if quant_bits:
+    if quant_bits and k_t is not None:
+        kt = np.asarray(k_t, dtype=np.int64)[None, :]
+        payload = np.where(ev > 0, 4 * n + (4 + 4 * kt + (kt * quant_bits + 7) // 8) * (ev - 1), 0)
+    elif quant_bits:
         payload = np.where(ev > 0, 4 * n + (4 + (n * quant_bits + 7) // 8) * (ev - 1), 0)
     elif k_t is None:
         payload = 4 * n * ev
