@@ -52,7 +52,7 @@ MOMENTUM_BYTES_PER_ELEMENT = 8     # --momentum: the velocity is read and writte
 FUSED_TRAFFIC_ELEMENTS = 16 * 11173962     # element-replicas of one launch on the default workload
 FUSED_TRAFFIC = {
     # sources of a dense run: hash -> (bytes per launch of the default workload, where the counters are)
-    "dense": {"e831c0c65719": (2.634e9, "profiles/k_fused_pipe_resnet18_first45tensors.md")},
+    "dense": {"244492e95c38": (2.634e9, "profiles/k_fused_pipe_resnet18_first45tensors.md")},
 }
 DENSE_SOURCES = ("eg_common.cuh", "eg_norm.cuh", "eg_fused.cuh", "eg_fused_pipe.cuh")
 

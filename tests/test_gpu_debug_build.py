@@ -24,7 +24,8 @@ SLICE = ("test_ragged_dense and (True-7 or False-64 or True-3 or False-5) or tes
          "or test_topk_guess_and_exact_repeat and (5-True or -8-False) or test_topk_degenerate "
          "or test_more_neighbours_per_side and (9-4 or 16-8) or test_intermittent_delivery_topk "
          "or test_momentum_with_topk_and_history or test_history_and_horizon and 4-1.0 "
-         "or test_graph_replay and walking_cap or test_quantised_messages_ragged and 5-True")
+         "or test_graph_replay and walking_cap or test_quantised_messages_ragged and 5-True "
+         "or test_quantised_topk_messages and 8-True")
 
 
 def test_parity_slice_under_the_bounds_checked_build():
