@@ -502,6 +502,14 @@ def test_quantised_resnet18_shapes_p16():
     assert rep.params_bit_exact and rep.quantised_checked > 50
 
 
+def test_quantised_topk_resnet18_shapes_p8():
+    """The 8-replica ResNet-18 ring with Top-K 1 % messages whose values go out as 4-bit codes."""
+    wl = W.config(4)[0]
+    rep = lockstep(wl, steps=40, tensors=_sample_tensors(wl), carry=True, check_every=5,
+                   oracle_kw=dict(quant_bits=4), outbox_samples=16)
+    assert rep.params_bit_exact and rep.quantised_checked > 50 and rep.sparse_checked > 10
+
+
 @pytest.mark.parametrize("carry", [False, True])
 @pytest.mark.parametrize("kernel", [B.FUSED_PIPELINED, B.FUSED_AUTO])
 def test_config1_mlp(carry, kernel):
