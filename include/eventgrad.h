@@ -300,7 +300,8 @@ eg_status eg_average_model(eg_ctx* ctx, const float* params, float* avg_dev,
  * the velocities.  eg_import_state restores it into a context created with the same arguments
  * and configured alike -- ring size, tensors, neighbourhood, threshold parameters, Top-K
  * fraction, readings (eg_set_variant), threshold bound, delivery masks enabled or not,
- * momentum buffer and coefficient -- and returns EG_ERR_INVALID otherwise. */
+ * momentum buffer and coefficient, bits of a quantised message -- and returns EG_ERR_INVALID
+ * otherwise. */
 eg_status eg_export_state(eg_ctx* ctx, void* host_buf, size_t* bytes);
 eg_status eg_import_state(eg_ctx* ctx, const void* host_buf, size_t bytes);
 
